@@ -1,0 +1,235 @@
+"""CPU oracle for the CompAct compressed linear layer (test infrastructure).
+
+A plain, slow, fp64 restatement of what the layer computes, written from the
+paper's Algorithms 1-3 (forward, backward, Adam update step with CompAct) and
+Section 3.3 (random projection matrix).  It exists only to check the CUDA
+path: tests, the smoke check and the benchmark's CPU-baseline leg may import
+it; the product path never does.  It shares no code with the CUDA sources.
+
+Every floating-point step is fp64.  Matrix products call numpy's fp64 matmul
+(a library primitive standing for the sum in the definition); there is no
+blocking, fusion or reordering beyond what the algorithms state.
+
+Two modes:
+  * "exact": no storage rounding anywhere (comparison target for fp32 runs);
+  * "bf16" : tensors that the method stores in bfloat16 are rounded to
+             nearest-even at exactly these points: P, Y, Z, dX, N, W.
+
+Readings of the paper taken here (the paper is silent or inconsistent):
+  * P_ij ~ N(0, 1/r) means variance 1/r (only this gives E[P P^T] = I).
+  * P is n x r (it multiplies x of shape bl x n on the right).
+  * Adam follows Algorithm 3 (bias correction, sqrt(V)+eps); the bias-corrected
+    moments are temporaries and the stored moments are the uncorrected ones;
+    the step count used for bias correction is 1-based.
+  * The generator behind "set_random_seed(s); P <- N(0,1/r)" is Philox4x32-10
+    keyed by the 64-bit seed with counter (j>>2, i, layer, epoch), followed by
+    Box-Muller; the seed bump "s <- s+1" is the epoch word.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass
+
+import numpy as np
+
+# ----------------------------------------------------------------------------
+# Philox4x32-10 (Salmon et al., SC'11).  Integer-only; results are exact.
+# ----------------------------------------------------------------------------
+_PHILOX_M0 = np.uint64(0xD2511F53)
+_PHILOX_M1 = np.uint64(0xCD9E8D57)
+_PHILOX_W0 = 0x9E3779B9
+_PHILOX_W1 = 0xBB67AE85
+_MASK32 = np.uint64(0xFFFFFFFF)
+
+
+def philox4x32_10(ctr, key):
+    """Ten-round Philox on arrays of counters.
+
+    ctr: integer array (..., 4), key: integer array broadcastable to (..., 2).
+    Returns uint32 array (..., 4).
+    """
+    ctr = np.asarray(ctr, dtype=np.uint64)
+    key = np.asarray(key, dtype=np.uint64)
+    c0, c1, c2, c3 = (ctr[..., i] & _MASK32 for i in range(4))
+    k0 = key[..., 0] & _MASK32
+    k1 = key[..., 1] & _MASK32
+    for rnd in range(10):
+        p0 = _PHILOX_M0 * c0            # 32x32 -> 64 bit product
+        p1 = _PHILOX_M1 * c2
+        hi0, lo0 = p0 >> np.uint64(32), p0 & _MASK32
+        hi1, lo1 = p1 >> np.uint64(32), p1 & _MASK32
+        c0, c1, c2, c3 = hi1 ^ c1 ^ k0, lo1, hi0 ^ c3 ^ k1, lo0
+        k0 = (k0 + np.uint64(_PHILOX_W0)) & _MASK32
+        k1 = (k1 + np.uint64(_PHILOX_W1)) & _MASK32
+    return np.stack([c0, c1, c2, c3], axis=-1).astype(np.uint32)
+
+
+def projection_words(seed: int, layer_id: int, epoch: int, n: int, r: int) -> np.ndarray:
+    """The raw Philox stream behind P: uint32 array (n, 4*ceil(r/4)).
+
+    Word (i, 4*q + w) is output word w of the call with counter
+    (q, i, layer_id, epoch) and key (seed low half, seed high half).
+    """
+    groups = (r + 3) // 4
+    i = np.arange(n, dtype=np.uint64)[:, None]
+    q = np.arange(groups, dtype=np.uint64)[None, :]
+    ctr = np.empty((n, groups, 4), dtype=np.uint64)
+    ctr[..., 0] = q
+    ctr[..., 1] = i
+    ctr[..., 2] = np.uint64(layer_id & 0xFFFFFFFF)
+    ctr[..., 3] = np.uint64(epoch & 0xFFFFFFFF)
+    key = np.array([seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF], dtype=np.uint64)
+    return philox4x32_10(ctr, key).reshape(n, groups * 4)
+
+
+def box_muller_from_words(words: np.ndarray) -> np.ndarray:
+    """Standard normals from a (..., 4q) uint32 stream, four per Philox call.
+
+    Within a call, words (0,1) make the pair (cos, sin) for lanes 0,1 and words
+    (2,3) for lanes 2,3.  u1 = ((x>>9)+0.5)/2^23 lies in (0,1); u2 = (x>>8)/2^24
+    lies in [0,1).
+    """
+    w = np.asarray(words, dtype=np.uint32)
+    shp = w.shape
+    w = w.reshape(shp[:-1] + (shp[-1] // 2, 2))
+    u1 = ((w[..., 0] >> np.uint32(9)).astype(np.float64) + 0.5) * 2.0 ** -23
+    u2 = (w[..., 1] >> np.uint32(8)).astype(np.float64) * 2.0 ** -24
+    rad = np.sqrt(-2.0 * np.log(u1))
+    ang = 2.0 * np.pi * u2
+    out = np.stack([rad * np.cos(ang), rad * np.sin(ang)], axis=-1)
+    return out.reshape(shp)
+
+
+def projection(seed: int, layer_id: int, epoch: int, n: int, r: int, mode: str = "exact") -> np.ndarray:
+    """P (n x r), entries N(0, 1/r): Algorithm 1 lines 1-2, Algorithm 3 lines 6-7."""
+    g = box_muller_from_words(projection_words(seed, layer_id, epoch, n, r))[:, :r]
+    P = g / math.sqrt(r)
+    return round_bf16(P) if mode == "bf16" else P
+
+
+# ----------------------------------------------------------------------------
+# bfloat16 storage rounding (round-to-nearest-even straight from fp64)
+# ----------------------------------------------------------------------------
+_BF16_MAX = float((2.0 - 2.0 ** -7) * 2.0 ** 127)
+
+
+def round_bf16(x) -> np.ndarray:
+    """Nearest bfloat16 value (ties to even) of each fp64 entry, returned as fp64."""
+    x = np.asarray(x, dtype=np.float64)
+    out = x.copy()
+    fin = np.isfinite(x) & (x != 0.0)
+    if not fin.any():
+        return out
+    xf = x[fin]
+    _, e = np.frexp(xf)                       # xf = mant * 2^e, mant in [0.5, 1)
+    q = np.maximum(e - 8, -133)               # 8 significant bits; subnormal quantum 2^-133
+    y = np.ldexp(np.rint(np.ldexp(xf, -q)), q)
+    y = np.where(np.abs(y) > _BF16_MAX, np.copysign(np.inf, y), y)
+    out[fin] = y
+    return out
+
+
+def _store(x: np.ndarray, mode: str) -> np.ndarray:
+    return round_bf16(x) if mode == "bf16" else x
+
+
+# ----------------------------------------------------------------------------
+# Algorithms 1-3
+# ----------------------------------------------------------------------------
+def linear_fwd(X: np.ndarray, W: np.ndarray, P: np.ndarray, mode: str = "exact"):
+    """Algorithm 1: o = x W and z = x P.  Returns (Y, Z); row t of Z is token t."""
+    X = np.asarray(X, dtype=np.float64)
+    Y = X @ np.asarray(W, dtype=np.float64)
+    Z = X @ np.asarray(P, dtype=np.float64)
+    return _store(Y, mode), _store(Z, mode)
+
+
+def linear_bwd(dY: np.ndarray, Z: np.ndarray, W: np.ndarray, mode: str = "exact"):
+    """Algorithm 2: G_hat = z^T dL/do (r x m, never rounded) and dL/dx = dL/do W^T."""
+    dY = np.asarray(dY, dtype=np.float64)
+    Gc = np.asarray(Z, dtype=np.float64).T @ dY
+    dX = dY @ np.asarray(W, dtype=np.float64).T
+    return _store(dX, mode), Gc
+
+
+def adam_update(W, Gc, M, V, t: int, P, lr: float, beta1: float, beta2: float, eps: float,
+                alpha: float = 1.0, mode: str = "exact"):
+    """Algorithm 3 lines 1-9 for the update whose 1-based count is t.
+
+    Returns (W_next, M_next, V_next); the returned moments are the uncorrected
+    running averages.
+    """
+    Gc = np.asarray(Gc, dtype=np.float64)
+    M = beta1 * np.asarray(M, dtype=np.float64) + (1.0 - beta1) * Gc
+    V = beta2 * np.asarray(V, dtype=np.float64) + (1.0 - beta2) * Gc * Gc
+    M_hat = M / (1.0 - beta1 ** t)
+    V_hat = V / (1.0 - beta2 ** t)
+    N = _store(M_hat / (np.sqrt(V_hat) + eps), mode)
+    G_tilde = alpha * (np.asarray(P, dtype=np.float64) @ N)
+    W_next = np.asarray(W, dtype=np.float64) - lr * G_tilde
+    return _store(W_next, mode), M, V
+
+
+@dataclass
+class LayerState:
+    """Seed, step and refresh bookkeeping of one layer (Algorithm 3 lines 10-13)."""
+    seed: int
+    layer_id: int
+    refresh_T: int          # 0: never refresh
+    epoch: int = 0
+    step: int = 0
+
+    def advance(self) -> None:
+        """t <- t+1; every T-th update bumps the seed (here: the epoch word)."""
+        self.step += 1
+        if self.refresh_T > 0 and self.step % self.refresh_T == 0:
+            self.epoch += 1
+
+
+class CompActLayerOracle:
+    """One layer's W, M, V and schedule, stepping through Algorithms 1-3."""
+
+    def __init__(self, W0, n: int, m: int, r: int, seed: int, layer_id: int, refresh_T: int,
+                 lr: float, beta1: float, beta2: float, eps: float, alpha: float = 1.0,
+                 mode: str = "exact", P_override=None):
+        self.n, self.m, self.r = n, m, r
+        self.W = np.array(W0, dtype=np.float64)
+        self.M = np.zeros((r, m))
+        self.V = np.zeros((r, m))
+        self.state = LayerState(seed, layer_id, refresh_T)
+        self.lr, self.beta1, self.beta2, self.eps, self.alpha = lr, beta1, beta2, eps, alpha
+        self.mode = mode
+        self.P_override = P_override      # explicit P for algebraic pins (orthonormal, identity)
+
+    def P(self, epoch: int | None = None) -> np.ndarray:
+        if self.P_override is not None:
+            return np.asarray(self.P_override, dtype=np.float64)
+        ep = self.state.epoch if epoch is None else epoch
+        return projection(self.state.seed, self.state.layer_id, ep, self.n, self.r, self.mode)
+
+    def forward(self, X):
+        return linear_fwd(X, self.W, self.P(), self.mode)
+
+    def backward(self, dY, Z):
+        return linear_bwd(dY, Z, self.W, self.mode)
+
+    def update(self, Gc, lr: float | None = None) -> None:
+        t = self.state.step + 1
+        self.W, self.M, self.V = adam_update(
+            self.W, Gc, self.M, self.V, t, self.P(), self.lr if lr is None else lr,
+            self.beta1, self.beta2, self.eps, self.alpha, self.mode)
+        self.state.advance()
+
+
+def saved_elements(tokens: int, r: int) -> int:
+    """Elements kept for backward per compressed linear (Table 1: b l n -> b l r)."""
+    return tokens * r
+
+
+def rel_frobenius(a, b) -> float:
+    """||a - b||_F / ||b||_F with b the oracle's tensor."""
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    den = np.linalg.norm(b)
+    num = np.linalg.norm(a - b)
+    return float(num / den) if den > 0 else float(num)

@@ -1,0 +1,356 @@
+"""Pins for the CPU oracle: each checks it against something other than itself
+(published vectors, closed forms, algebraic identities, library routines,
+brute-force loops), chosen so a dropped term, wrong sign/index or transposed
+operand fails at least one of them."""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+from scipy import stats
+
+from oracle import compact_oracle as co
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# --- Philox integer stream vs published known-answer vectors ------------------
+def _kat_rows():
+    rows = []
+    with open(os.path.join(GOLDEN, "philox4x32_10_kat.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            v = [int(x, 16) for x in line.split()]
+            rows.append((v[:4], v[4:6], v[6:]))
+    return rows
+
+
+def test_philox_known_answers():
+    rows = _kat_rows()
+    assert len(rows) == 3
+    for ctr, key, want in rows:
+        got = co.philox4x32_10(np.array(ctr), np.array(key))
+        assert [int(x) for x in got] == want
+
+
+def test_philox_vectorised_equals_scalar_calls():
+    ctr = np.array([[0, 0, 0, 0], [0xFFFFFFFF] * 4, [0x243F6A88, 0x85A308D3, 0x13198A2E, 0x03707344]])
+    key = np.array([[0, 0], [0xFFFFFFFF] * 2, [0xA4093822, 0x299F31D0]])
+    got = co.philox4x32_10(ctr, key)
+    for row, (_, _, want) in zip(got, _kat_rows()):
+        assert [int(x) for x in row] == want
+
+
+def test_projection_words_counter_layout():
+    # word (i, 4q+w) is word w of philox(ctr=(q, i, layer, epoch), key=(seed_lo, seed_hi))
+    seed, layer, epoch = (0x1234 << 32) | 0x89ABCDEF, 5, 3
+    words = co.projection_words(seed, layer, epoch, 9, 10)
+    assert words.shape == (9, 12)
+    for i, q in [(0, 0), (8, 2), (4, 1)]:
+        ref = co.philox4x32_10(np.array([q, i, layer, epoch]), np.array([0x89ABCDEF, 0x1234]))
+        assert (words[i, 4 * q:4 * q + 4] == ref).all()
+    # the all-zero call is the first published vector
+    w0 = co.projection_words(0, 0, 0, 1, 4)
+    assert [int(x) for x in w0[0]] == _kat_rows()[0][2]
+
+
+# --- Box-Muller closed forms and distribution -----------------------------------
+def test_box_muller_closed_forms():
+    # u2 = 0 -> (rad, 0); u2 = 1/4 -> (0, rad)
+    w = np.array([[0x80000000, 0, 0x80000000, 1 << 30]], dtype=np.uint32)
+    g = co.box_muller_from_words(w)[0]
+    u1 = ((0x80000000 >> 9) + 0.5) * 2.0 ** -23
+    rad = math.sqrt(-2 * math.log(u1))
+    assert g[0] == pytest.approx(rad, rel=1e-15) and g[1] == 0.0
+    assert abs(g[2]) < 1e-15 and g[3] == pytest.approx(rad, rel=1e-15)
+    # extreme radii: u1 = 1 - 2^-24 and u1 = 2^-24
+    w = np.array([[0xFFFFFFFF, 0, 0x00000000, 0]], dtype=np.uint32)
+    g = co.box_muller_from_words(w)[0]
+    assert g[0] == pytest.approx(math.sqrt(-2 * math.log1p(-2.0 ** -24)), rel=1e-9)
+    assert g[0] == pytest.approx(3.4527e-4, rel=1e-4)
+    assert g[2] == pytest.approx(math.sqrt(48 * math.log(2)), rel=1e-15)
+    # u2 = 1/2 -> (-rad, ~0): sign of cos
+    w = np.array([[0, 1 << 31, 0, 3 << 30]], dtype=np.uint32)
+    g = co.box_muller_from_words(w)[0]
+    assert g[0] == pytest.approx(-math.sqrt(48 * math.log(2)), rel=1e-15)
+    assert g[3] == pytest.approx(-math.sqrt(48 * math.log(2)), rel=1e-15)  # sin(3pi/2) = -1
+
+
+def test_projection_distribution():
+    r = 64
+    P = co.projection(seed=7, layer_id=1, epoch=0, n=40000, r=r)
+    x = (P * math.sqrt(r)).ravel()
+    N = x.size
+    assert abs(x.mean()) < 5 / math.sqrt(N)
+    assert abs(x.var() - 1.0) < 5 * math.sqrt(2.0 / N)
+    assert abs(stats.kurtosis(x, fisher=False) - 3.0) < 5 * math.sqrt(24.0 / N)
+    assert abs(stats.skew(x)) < 5 * math.sqrt(6.0 / N)
+    assert stats.kstest(x[:500000], "norm").pvalue > 1e-3
+    # cos lanes and sin lanes are uncorrelated; columns are uncorrelated
+    assert abs(np.corrcoef(P[:, 0], P[:, 1])[0, 1]) < 5 / math.sqrt(P.shape[0])
+    assert abs(np.corrcoef(P[:, 1], P[:, 2])[0, 1]) < 5 / math.sqrt(P.shape[0])
+
+
+def test_projection_scale_gives_identity():
+    # E[P P^T] = I_n when the variance is 1/r (Section 3.3)
+    n, r, S = 12, 8, 4000
+    acc = np.zeros((n, n))
+    for s in range(S):
+        P = co.projection(seed=s, layer_id=0, epoch=0, n=n, r=r)
+        acc += P @ P.T
+    acc /= S
+    d = np.diag(acc)
+    off = acc - np.diag(d)
+    assert np.all(np.abs(d - 1.0) < 5 * math.sqrt(2.0 / (r * S)))
+    assert np.all(np.abs(off) < 5 * math.sqrt(1.0 / (r * S)))
+
+
+def test_projection_depends_on_each_counter_word():
+    base = co.projection(1, 2, 3, 6, 8)
+    assert not np.array_equal(base, co.projection(2, 2, 3, 6, 8))
+    assert not np.array_equal(base, co.projection(1 + (1 << 32), 2, 3, 6, 8))
+    assert not np.array_equal(base, co.projection(1, 3, 3, 6, 8))
+    assert not np.array_equal(base, co.projection(1, 2, 4, 6, 8))
+    # a taller P with the same r shares the row prefix; ragged r is a column prefix
+    assert np.array_equal(base, co.projection(1, 2, 3, 9, 8)[:6])
+    assert np.allclose(co.projection(1, 2, 3, 6, 7) * math.sqrt(7), base[:, :7] * math.sqrt(8), rtol=1e-15)
+
+
+# --- bf16 storage rounding --------------------------------------------------------
+def _f32_from_bits(b):
+    return float(np.array([b], dtype=np.uint32).view(np.float32)[0])
+
+
+def test_round_bf16_bit_patterns():
+    cases = {
+        0x3F808000: 0x3F80,  # tie -> even (down)
+        0x3F818000: 0x3F82,  # tie -> even (up)
+        0x3F808001: 0x3F81,  # just above the tie
+        0x3F807FFF: 0x3F80,
+        0xBF818000: 0xBF82,
+        0x00000000: 0x0000,
+        0x00400000: 0x0040,  # bf16 subnormal kept
+        0x00008000: 0x0000,  # half of the smallest subnormal: tie -> even (0)
+        0x00018000: 0x0002,
+        0x7F7FFFFF: 0x7F80,  # rounds up to +inf
+    }
+    for bits32, want16 in cases.items():
+        y = co.round_bf16(np.array([_f32_from_bits(bits32)]))[0]
+        got = int(np.array([y], dtype=np.float32).view(np.uint32)[0])
+        assert got == want16 << 16, hex(bits32)
+    assert np.isnan(co.round_bf16(np.array([np.nan]))[0])
+    assert co.round_bf16(np.array([-np.inf]))[0] == -np.inf
+
+
+def test_round_bf16_matches_torch_conversion():
+    rng = np.random.default_rng(0)
+    bits = rng.integers(0, 2 ** 32, size=200000, dtype=np.uint64).astype(np.uint32)
+    x = bits.view(np.float32)
+    x = x[np.isfinite(x)]
+    want = torch.from_numpy(x.copy()).to(torch.bfloat16).to(torch.float64).numpy()
+    got = co.round_bf16(x.astype(np.float64))
+    assert np.array_equal(got, want)
+
+
+# --- GEMM definitions: brute force on tiny shapes -------------------------------
+def _brute_fwd(X, W, P):
+    bl, n = len(X), len(W)
+    m, r = len(W[0]), len(P[0])
+    Y = [[sum(X[t][k] * W[k][c] for k in range(n)) for c in range(m)] for t in range(bl)]
+    Z = [[sum(X[t][k] * P[k][j] for k in range(n)) for j in range(r)] for t in range(bl)]
+    return Y, Z
+
+
+def _brute_bwd(dY, Z, W):
+    bl, m = len(dY), len(dY[0])
+    n, r = len(W), len(Z[0])
+    Gc = [[sum(Z[t][j] * dY[t][c] for t in range(bl)) for c in range(m)] for j in range(r)]
+    dX = [[sum(dY[t][c] * W[k][c] for c in range(m)) for k in range(n)] for t in range(bl)]
+    return dX, Gc
+
+
+@pytest.mark.parametrize("bl,n,m,r", [(5, 7, 3, 4), (3, 6, 5, 5), (1, 2, 2, 1)])
+def test_fwd_bwd_brute_force(bl, n, m, r):
+    rng = np.random.default_rng(bl * 100 + r)
+    X, W, dY = rng.standard_normal((bl, n)), rng.standard_normal((n, m)), rng.standard_normal((bl, m))
+    P = co.projection(3, 1, 0, n, r)
+    Y, Z = co.linear_fwd(X, W, P)
+    Yb, Zb = _brute_fwd(X.tolist(), W.tolist(), P.tolist())
+    assert np.allclose(Y, Yb, rtol=1e-13, atol=1e-13) and np.allclose(Z, Zb, rtol=1e-13, atol=1e-13)
+    dX, Gc = co.linear_bwd(dY, Z, W)
+    dXb, Gcb = _brute_bwd(dY.tolist(), Z.tolist(), W.tolist())
+    assert np.allclose(dX, dXb, rtol=1e-13, atol=1e-13) and np.allclose(Gc, Gcb, rtol=1e-13, atol=1e-13)
+    assert Y.shape == (bl, m) and Z.shape == (bl, r) and dX.shape == (bl, n) and Gc.shape == (r, m)
+
+
+def test_update_brute_force():
+    rng = np.random.default_rng(5)
+    n, m, r = 4, 3, 2
+    W, Gc = rng.standard_normal((n, m)), rng.standard_normal((r, m))
+    M0, V0 = rng.standard_normal((r, m)), rng.random((r, m))
+    P = co.projection(0, 0, 0, n, r)
+    b1, b2, eps, lr, alpha, t = 0.8, 0.95, 1e-6, 0.01, 0.25, 3
+    Wn, Mn, Vn = co.adam_update(W, Gc, M0, V0, t, P, lr, b1, b2, eps, alpha)
+    for i in range(n):
+        for c in range(m):
+            acc = 0.0
+            for j in range(r):
+                mm = b1 * M0[j, c] + (1 - b1) * Gc[j, c]
+                vv = b2 * V0[j, c] + (1 - b2) * Gc[j, c] ** 2
+                assert Mn[j, c] == pytest.approx(mm, rel=1e-14)
+                assert Vn[j, c] == pytest.approx(vv, rel=1e-14)
+                nn = (mm / (1 - b1 ** t)) / (math.sqrt(vv / (1 - b2 ** t)) + eps)
+                acc += P[i, j] * nn
+            assert Wn[i, c] == pytest.approx(W[i, c] - lr * alpha * acc, rel=1e-13)
+
+
+# --- Algebraic identities ----------------------------------------------------------
+def test_compressed_gradient_is_projected_gradient():
+    # (X P)^T dY = P^T (X^T dY): CompAct is GaLore with Q = I (Section 3.2)
+    rng = np.random.default_rng(1)
+    bl, n, m, r = 40, 24, 10, 6
+    X, W, dY = rng.standard_normal((bl, n)), rng.standard_normal((n, m)), rng.standard_normal((bl, m))
+    P = co.projection(11, 0, 0, n, r)
+    _, Z = co.linear_fwd(X, W, P)
+    _, Gc = co.linear_bwd(dY, Z, W)
+    G = X.T @ dY
+    assert np.allclose(Gc, P.T @ G, rtol=1e-12, atol=1e-12)
+
+
+def test_orthonormal_full_rank_projection_recovers_gradient():
+    # r = n and P orthonormal: P Gc = X^T dY exactly
+    rng = np.random.default_rng(2)
+    bl, n, m = 30, 16, 9
+    X, W, dY = rng.standard_normal((bl, n)), rng.standard_normal((n, m)), rng.standard_normal((bl, m))
+    Q, _ = np.linalg.qr(co.projection(4, 0, 0, n, n))
+    _, Z = co.linear_fwd(X, W, Q)
+    _, Gc = co.linear_bwd(dY, Z, W)
+    assert np.allclose(Q @ Gc, X.T @ dY, rtol=1e-12, atol=1e-12)
+
+
+def test_dx_is_gradient_of_inner_product():
+    # d/dX <X W, dY> = dY W^T : finite difference on one entry
+    rng = np.random.default_rng(3)
+    X, W, dY = rng.standard_normal((4, 5)), rng.standard_normal((5, 3)), rng.standard_normal((4, 3))
+    P = co.projection(0, 0, 0, 5, 2)
+    dX, _ = co.linear_bwd(dY, co.linear_fwd(X, W, P)[1], W)
+    h = 1e-6
+    for (t, k) in [(0, 0), (3, 4), (2, 1)]:
+        Xp = X.copy(); Xp[t, k] += h
+        Xm = X.copy(); Xm[t, k] -= h
+        fd = (np.sum(co.linear_fwd(Xp, W, P)[0] * dY) - np.sum(co.linear_fwd(Xm, W, P)[0] * dY)) / (2 * h)
+        assert dX[t, k] == pytest.approx(fd, rel=1e-7)
+
+
+# --- Adam ----------------------------------------------------------------------------
+def test_adam_constant_gradient_closed_form():
+    rng = np.random.default_rng(4)
+    n, m, r, k = 10, 6, 4, 7
+    g = rng.standard_normal((r, m))
+    W0 = rng.standard_normal((n, m))
+    lr, alpha, eps = 3e-3, 0.25, 1e-8
+    lay = co.CompActLayerOracle(W0, n, m, r, seed=9, layer_id=2, refresh_T=0, lr=lr,
+                                beta1=0.7, beta2=0.93, eps=eps, alpha=alpha)
+    for _ in range(k):
+        lay.update(g)
+    N = g / (np.abs(g) + eps)
+    want = W0 - k * lr * alpha * (lay.P() @ N)
+    assert np.allclose(lay.W, want, rtol=1e-12, atol=1e-12)
+
+
+def test_adam_identity_projection_equals_torch_adam():
+    # r = n, P = I, alpha = 1: CompAct is plain Adam on W with gradient X^T dY
+    rng = np.random.default_rng(6)
+    bl, n, m, steps = 12, 5, 4, 5
+    W0 = rng.standard_normal((n, m))
+    lay = co.CompActLayerOracle(W0, n, m, n, seed=0, layer_id=0, refresh_T=2, lr=1e-2,
+                                beta1=0.9, beta2=0.999, eps=1e-8, P_override=np.eye(n))
+    Wt = torch.tensor(W0, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.Adam([Wt], lr=1e-2, betas=(0.9, 0.999), eps=1e-8, weight_decay=0.0)
+    for s in range(steps):
+        X, dY = rng.standard_normal((bl, n)), rng.standard_normal((bl, m))
+        Y, Z = lay.forward(X)
+        _, Gc = lay.backward(dY, Z)
+        lay.update(Gc)
+        opt.zero_grad()
+        Wt.grad = torch.tensor(X.T @ dY)
+        opt.step()
+        assert np.allclose(lay.W, Wt.detach().numpy(), rtol=1e-10, atol=1e-12), s
+    assert lay.state.step == steps
+
+
+def test_zero_inputs_change_nothing():
+    rng = np.random.default_rng(8)
+    n, m, r, bl = 6, 5, 3, 4
+    W0 = rng.standard_normal((n, m))
+    lay = co.CompActLayerOracle(W0, n, m, r, 1, 0, 0, 1e-2, 0.9, 0.999, 1e-8)
+    Y, Z = lay.forward(np.zeros((bl, n)))
+    assert not Y.any() and not Z.any()
+    dX, Gc = lay.backward(rng.standard_normal((bl, m)), Z)
+    assert not Gc.any()
+    lay.update(Gc)
+    assert np.array_equal(lay.W, W0) and not lay.M.any() and not lay.V.any()
+    dX, Gc = lay.backward(np.zeros((bl, m)), rng.standard_normal((bl, r)))
+    assert not dX.any() and not Gc.any()
+
+
+# --- Refresh schedule (Algorithm 3 lines 10-13) -------------------------------------
+def test_refresh_schedule():
+    st = co.LayerState(seed=0, layer_id=0, refresh_T=2)
+    used = []
+    for _ in range(3):
+        used.append(st.epoch)
+        st.advance()
+    assert used == [0, 0, 1] and st.epoch == 1 and st.step == 3
+    st = co.LayerState(seed=0, layer_id=0, refresh_T=0)
+    for _ in range(10):
+        st.advance()
+    assert st.epoch == 0
+    st = co.LayerState(seed=0, layer_id=0, refresh_T=10)
+    eps = []
+    for _ in range(20):
+        eps.append(st.epoch)
+        st.advance()
+    assert eps == [0] * 10 + [1] * 10 and st.epoch == 2
+    assert not np.array_equal(co.projection(0, 0, 0, 8, 4), co.projection(0, 0, 1, 8, 4))
+
+
+def test_layer_uses_refreshed_projection():
+    rng = np.random.default_rng(10)
+    n, m, r = 6, 4, 2
+    lay = co.CompActLayerOracle(rng.standard_normal((n, m)), n, m, r, 5, 1, 1, 1e-2, 0.9, 0.999, 1e-8)
+    P0 = lay.P()
+    lay.update(rng.standard_normal((r, m)))
+    assert lay.state.epoch == 1
+    assert np.array_equal(lay.P(), co.projection(5, 1, 1, n, r)) and not np.array_equal(lay.P(), P0)
+
+
+# --- bf16 storage mode: rounding happens at the stated points only --------------------
+def test_bf16_mode_rounding_points():
+    rng = np.random.default_rng(12)
+    bl, n, m, r = 9, 8, 6, 4
+    rb = co.round_bf16
+    X, W, dY = rb(rng.standard_normal((bl, n))), rb(rng.standard_normal((n, m))), rb(rng.standard_normal((bl, m)))
+    P = co.projection(2, 0, 0, n, r, mode="bf16")
+    assert np.array_equal(P, rb(co.projection(2, 0, 0, n, r)))
+    Y, Z = co.linear_fwd(X, W, P, mode="bf16")
+    assert np.array_equal(Y, rb(X @ W)) and np.array_equal(Z, rb(X @ P))
+    dX, Gc = co.linear_bwd(dY, Z, W, mode="bf16")
+    assert np.array_equal(dX, rb(dY @ W.T)) and np.array_equal(Gc, Z.T @ dY)
+    Wn, Mn, Vn = co.adam_update(W, Gc, np.zeros((r, m)), np.zeros((r, m)), 1, P, 1e-3, 0.9, 0.999, 1e-8, mode="bf16")
+    N = rb((0.1 * Gc / 0.1) / (np.sqrt(0.001 * Gc * Gc / 0.001) + 1e-8))
+    assert np.allclose(Wn, rb(W - 1e-3 * (P @ N)), rtol=0, atol=1e-2 * np.abs(W).max() * 2 ** -8)
+    assert np.array_equal(Wn, rb(Wn))
+
+
+# --- Memory accounting (Table 1, Table 3 with Appendix E) ----------------------------
+def test_saved_activation_accounting():
+    bl = 64 * 256
+    assert co.saved_elements(bl, 256) == bl * 256
+    n, m = 1024, 2736
+    dense = bl * (2 * n + m)                         # x2 (shared by q,k,v), x6 (gate, up), x7 (down)
+    comp = 3 * co.saved_elements(bl, n // 4) + 2 * co.saved_elements(bl, n // 4) + co.saved_elements(bl, m // 4)
+    assert comp / dense == pytest.approx(1964 / 4784)
+    assert 7.0 * comp / dense == pytest.approx(2.87, abs=0.005)   # Table 3 activation row at r = n/4
