@@ -1,0 +1,164 @@
+/*
+ * compact.h -- C ABI of the CompAct compressed linear layer for NVIDIA B200 (sm_100a).
+ *
+ * The layer follows "CompAct: Compressed Activations for Memory-Efficient LLM
+ * Training": the forward computes o = x W and keeps only z = x P for the
+ * backward (Algorithm 1); the backward computes the compressed weight gradient
+ * G_hat = z^T dL/do and the input gradient dL/dx = dL/do W^T (Algorithm 2); the
+ * update runs Adam on G_hat with r x m moments and applies
+ * W <- W - eta * alpha * P N (Algorithm 3).  P (n x r, entries N(0, 1/r),
+ * Section 3.3) is never stored: every kernel regenerates the entries it needs
+ * from (seed, layer_id, epoch) with Philox4x32-10 and Box-Muller.
+ *
+ * Conventions that hold for every entry point
+ *   - Matrices are row-major with an explicit leading dimension in ELEMENTS.
+ *     W is n x m as in the paper's Section 3.1 (not [out, in]).
+ *   - All tensor pointers are DEVICE pointers owned by the caller.  The library
+ *     allocates no tensor memory and keeps no pointer after a call returns.
+ *   - Element type of X, W, Y, dY, dX, Z is the layer's dtype; Gc, M, V are
+ *     always fp32.
+ *   - `stream` is a cudaStream_t passed as void*.  Compute calls are asynchronous
+ *     on it and never synchronise the host.
+ *   - Base pointers must be 16-byte aligned and every leading dimension times
+ *     the element size a multiple of 16 bytes.
+ *   - Every function returns a compact_status_t; nothing throws or aborts.
+ *     Argument checks happen on the host before any launch.
+ *   - A layer handle must not be used from two threads at once.
+ *   - Only compute capability 10.x devices are supported; there is no fallback.
+ */
+#ifndef COMPACT_H_
+#define COMPACT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct compact_layer compact_layer_t; /* opaque, host side */
+
+typedef enum {
+  COMPACT_OK = 0,
+  COMPACT_ERR_INVALID_ARG = 1,
+  COMPACT_ERR_SHAPE = 2,
+  COMPACT_ERR_ALIGNMENT = 3,
+  COMPACT_ERR_DTYPE = 4,
+  COMPACT_ERR_EPOCH_MISMATCH = 5,
+  COMPACT_ERR_WORKSPACE = 6,
+  COMPACT_ERR_UNSUPPORTED_ARCH = 7,
+  COMPACT_ERR_CUDA = 8,
+  COMPACT_ERR_DEVICE_TIMEOUT = 9
+} compact_status_t;
+
+typedef enum { COMPACT_F32 = 0, COMPACT_BF16 = 1 } compact_dtype_t;
+
+/* Inputs of Algorithms 1 and 3: rank r, seed s, Adam decay rates, scale alpha,
+ * learning rate eta, projection update gap T (refresh_T == 0: never refresh). */
+typedef struct {
+  int32_t n, m, r;
+  int32_t dtype;      /* compact_dtype_t */
+  uint64_t seed;
+  uint32_t layer_id;
+  uint32_t refresh_T;
+  float lr, beta1, beta2, eps, alpha;
+} compact_layer_config_t;
+
+typedef struct {
+  uint64_t seed;
+  uint32_t layer_id;
+  uint32_t epoch;     /* number of refreshes so far: the "s <- s + 1" of Algorithm 3 line 12 */
+  uint64_t step;      /* t of Algorithm 3: number of completed updates */
+} compact_layer_state_t;
+
+/* Creates a layer (host bookkeeping only; touches no device).  Fails with
+ * SHAPE unless 1 <= r <= n, m >= 1, n and m multiples of 8 (bf16) or 4 (f32). */
+compact_status_t compact_layer_create(const compact_layer_config_t* cfg, compact_layer_t** out);
+compact_status_t compact_layer_destroy(compact_layer_t* layer);
+
+/* Row pitch of Z in elements: r rounded up to a multiple of 16.  Columns
+ * r..ldz-1 of Z are written as exact zeros by the forward. */
+int64_t compact_z_ld(const compact_layer_t* layer);
+
+/* Bytes of device scratch that compact_linear_bwd / compact_adam_update need
+ * for `tokens` rows (split-K partials of Gc; the normalised step N). */
+size_t compact_workspace_bytes(const compact_layer_t* layer, int64_t tokens);
+
+/* Bytes kept for the backward by one forward: tokens * ldz * sizeof(element)
+ * (Table 1: b l n -> b l r). */
+size_t compact_saved_bytes(const compact_layer_t* layer, int64_t tokens);
+
+/* Algorithm 1.  Y[tokens x m] = X W and Z[tokens x ldz] = X P, both rounded once
+ * from fp32 accumulators.  Row t of Z belongs to row t of X.  *epoch_used
+ * (host pointer, may be NULL) receives the epoch P was generated with. */
+compact_status_t compact_linear_fwd(compact_layer_t* layer, int64_t tokens,
+                                    const void* X, int64_t ldx,
+                                    const void* W, int64_t ldw,
+                                    void* Y, int64_t ldy,
+                                    void* Z, int64_t ldz,
+                                    uint32_t* epoch_used, void* stream);
+
+/* Algorithm 2.  Gc[r x m] (fp32) = Z^T dY summed over all tokens, and
+ * dX[tokens x n] = dY W^T.  dX may be NULL (skip it).  accumulate != 0 adds to
+ * Gc instead of overwriting it (micro-batches of one step).  The reduction
+ * order over tokens is fixed, so results are bitwise reproducible. */
+compact_status_t compact_linear_bwd(compact_layer_t* layer, int64_t tokens,
+                                    const void* dY, int64_t lddy,
+                                    const void* Z, int64_t ldz,
+                                    const void* W, int64_t ldw,
+                                    void* dX, int64_t lddx,
+                                    float* Gc, int64_t ldg, int accumulate,
+                                    void* workspace, size_t workspace_bytes, void* stream);
+
+/* Algorithm 3 lines 1-10.  In place on W, M, V (M, V: r x m fp32, pitch ldg);
+ * stored moments are the uncorrected running averages and the bias correction
+ * uses the 1-based count of this update.  epoch_of_Gc must equal the layer's
+ * current epoch (the one the forward reported).  lr = NaN uses the config's.
+ * Increments the layer's step. */
+compact_status_t compact_adam_update(compact_layer_t* layer,
+                                     void* W, int64_t ldw,
+                                     const float* Gc, int64_t ldg,
+                                     float* M, float* V,
+                                     uint32_t epoch_of_Gc, float lr,
+                                     void* workspace, size_t workspace_bytes, void* stream);
+
+/* Algorithm 3 lines 11-13 and Section 3.3: changing the projection only
+ * replaces the seed.  If force != 0, or refresh_T > 0 and the step count is a
+ * positive multiple of refresh_T not yet refreshed at, epoch <- epoch + 1.
+ * Host only: launches nothing and moves no memory.  *new_epoch may be NULL. */
+compact_status_t compact_refresh_projection(compact_layer_t* layer, int force, uint32_t* new_epoch);
+
+/* Checkpoint / resume: P is never stored, so (W, M, V) plus this state is a
+ * complete checkpoint of a layer. */
+compact_status_t compact_layer_get_state(const compact_layer_t* layer, compact_layer_state_t* out);
+compact_status_t compact_layer_set_state(compact_layer_t* layer, const compact_layer_state_t* in);
+
+/* Reads and clears the layer's device status word (synchronises the device).
+ * Returns DEVICE_TIMEOUT if a kernel gave up on a bounded wait since the last
+ * call, OK otherwise. */
+compact_status_t compact_layer_status(compact_layer_t* layer);
+
+/* Test hooks that make the in-kernel generator observable.
+ * compact_debug_philox_u32: out_dev[n x 4*ceil(r/4)] receives the raw Philox
+ * words behind P (Algorithm 1 lines 1-2).
+ * compact_debug_projection: P_dev[n x r] (layer dtype, pitch r) receives P at
+ * `epoch`, produced by the same device function the GEMM kernels call. */
+compact_status_t compact_debug_philox_u32(uint64_t seed, uint32_t layer_id, uint32_t epoch,
+                                          int32_t n, int32_t r, uint32_t* out_dev, void* stream);
+compact_status_t compact_debug_projection(const compact_layer_t* layer, uint32_t epoch,
+                                          void* P_dev, void* stream);
+
+/* Selects the kernel family: 0 = automatic (tensor-core kernels for bf16 where
+ * the shape allows, SIMT otherwise), 1 = force the SIMT kernels (used by the
+ * tests as an on-device cross-check).  Returns the previous value. */
+int compact_set_kernel_family(int family);
+
+/* Number of kernels this library has launched since it was loaded. */
+uint64_t compact_kernel_launch_count(void);
+
+const char* compact_status_string(compact_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COMPACT_H_ */

@@ -1,0 +1,393 @@
+// C ABI of the CompAct compressed linear layer (see include/compact.h).
+// Host-side bookkeeping, argument validation and kernel dispatch.
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <atomic>
+#include <new>
+
+#include "../../include/compact.h"
+#include "philox.cuh"
+#include "simt_kernels.cuh"
+#include "tc_kernels.cuh"
+
+using namespace compact;
+
+struct compact_layer {
+  compact_layer_config_t cfg;
+  uint32_t epoch;
+  uint64_t step;
+  uint64_t last_refresh_step;
+  int status_slot;
+  int device_checked;   // -1: unsupported, 0: not yet, 1: ok
+};
+
+namespace {
+
+std::atomic<uint64_t> g_launches{0};
+std::atomic<int> g_family{0};
+std::atomic<int> g_next_slot{0};
+
+constexpr int kStatusSlots = 256;
+__device__ unsigned int g_status_words[kStatusSlots];
+
+inline size_t elem_size(int dtype) { return dtype == COMPACT_BF16 ? 2 : 4; }
+inline int64_t round_up(int64_t a, int64_t b) { return (a + b - 1) / b * b; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+compact_status_t check_device(compact_layer_t* L) {
+  if (L->device_checked == 1) return COMPACT_OK;
+  if (L->device_checked == -1) return COMPACT_ERR_UNSUPPORTED_ARCH;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return COMPACT_ERR_CUDA; }
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+    cudaGetLastError();
+    return COMPACT_ERR_CUDA;
+  }
+  if (major != 10) { L->device_checked = -1; return COMPACT_ERR_UNSUPPORTED_ARCH; }
+  L->device_checked = 1;
+  return COMPACT_OK;
+}
+
+unsigned int* status_word(const compact_layer_t* L) {
+  unsigned int* base = nullptr;
+  if (cudaGetSymbolAddress((void**)&base, g_status_words) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+  return base + L->status_slot;
+}
+
+ProjectionParams make_pp(const compact_layer_t* L, uint32_t epoch) {
+  ProjectionParams pp;
+  pp.key = make_philox_key(L->cfg.seed);
+  pp.layer_id = L->cfg.layer_id;
+  pp.epoch = epoch;
+  pp.n = L->cfg.n;
+  pp.r = L->cfg.r;
+  pp.inv_sqrt_r = (float)(1.0 / sqrt((double)L->cfg.r));
+  return pp;
+}
+
+compact_status_t launch_result() {
+  return cudaGetLastError() == cudaSuccess ? COMPACT_OK : COMPACT_ERR_CUDA;
+}
+
+template <class AF, class BF, class EP>
+void simt_gemm(int M, int N, int K, AF a, BF b, EP ep, cudaStream_t st) {
+  dim3 grid((N + 63) / 64, (M + 63) / 64);
+  simt::gemm_kernel<AF, BF, EP><<<grid, 256, 0, st>>>(M, N, K, a, b, ep);
+  g_launches++;
+}
+
+inline bool pitch_ok(int64_t ld, int64_t min_cols, size_t es) { return ld >= min_cols && (ld * (int64_t)es) % 16 == 0; }
+
+// ---- forward ---------------------------------------------------------------------------
+template <typename T>
+compact_status_t fwd_simt(compact_layer_t* L, int64_t tokens, const T* X, int64_t ldx, const T* W, int64_t ldw,
+                          T* Y, int64_t ldy, T* Z, int64_t ldz, cudaStream_t st) {
+  constexpr bool kBf16 = sizeof(T) == 2;
+  const int n = L->cfg.n, m = L->cfg.m, r = L->cfg.r;
+  simt_gemm((int)tokens, m, n, simt::RowMajor<T>{X, ldx}, simt::Transposed<T>{W, ldw}, simt::StoreAs<T>{Y, ldy}, st);
+  simt::GeneratedP<kBf16, true> gp{make_pp(L, L->epoch)};
+  simt_gemm((int)tokens, r, n, simt::RowMajor<T>{X, ldx}, gp, simt::StoreAs<T>{Z, ldz}, st);
+  const int zc = (int)compact_z_ld(L);
+  if (zc > r) {
+    const int64_t cnt = tokens * (zc - r);
+    simt::zero_pad_columns<T><<<(unsigned)((cnt + 255) / 256), 256, 0, st>>>(Z, ldz, tokens, r, zc);
+    g_launches++;
+  }
+  return launch_result();
+}
+
+template <typename T>
+compact_status_t bwd_simt(compact_layer_t* L, int64_t tokens, const T* dY, int64_t lddy, const T* Z, int64_t ldz,
+                          const T* W, int64_t ldw, T* dX, int64_t lddx, float* Gc, int64_t ldg, int accumulate,
+                          cudaStream_t st) {
+  const int n = L->cfg.n, m = L->cfg.m, r = L->cfg.r;
+  simt_gemm(r, m, (int)tokens, simt::Transposed<T>{Z, ldz}, simt::Transposed<T>{dY, lddy},
+            simt::StoreF32{Gc, ldg, accumulate}, st);
+  if (dX)
+    simt_gemm((int)tokens, n, m, simt::RowMajor<T>{dY, lddy}, simt::RowMajor<T>{W, ldw}, simt::StoreAs<T>{dX, lddx}, st);
+  return launch_result();
+}
+
+simt::AdamScalars adam_scalars(const compact_layer_t* L, uint64_t t) {
+  simt::AdamScalars s;
+  const double b1 = (double)L->cfg.beta1, b2 = (double)L->cfg.beta2;
+  s.beta1 = L->cfg.beta1;
+  s.beta2 = L->cfg.beta2;
+  s.one_minus_beta1 = (float)(1.0 - b1);
+  s.one_minus_beta2 = (float)(1.0 - b2);
+  s.inv_bias1 = (float)(1.0 / (1.0 - pow(b1, (double)t)));
+  s.inv_bias2 = (float)(1.0 / (1.0 - pow(b2, (double)t)));
+  s.eps = L->cfg.eps;
+  return s;
+}
+
+template <typename T>
+compact_status_t update_simt(compact_layer_t* L, T* W, int64_t ldw, const float* Gc, int64_t ldg, float* M, float* V,
+                             float lr, float* Nbuf, cudaStream_t st) {
+  constexpr bool kBf16 = sizeof(T) == 2;
+  const int n = L->cfg.n, m = L->cfg.m, r = L->cfg.r;
+  const simt::AdamScalars s = adam_scalars(L, L->step + 1);
+  const int64_t cnt = (int64_t)r * m;
+  simt::adam_moments_kernel<kBf16><<<(unsigned)((cnt + 255) / 256), 256, 0, st>>>(Gc, ldg, M, V, Nbuf, m, r, m, s);
+  g_launches++;
+  simt::GeneratedP<kBf16, false> gp{make_pp(L, L->epoch)};
+  simt_gemm(n, m, r, gp, simt::Transposed<float>{Nbuf, m}, simt::ApplyUpdate<T>{W, ldw, lr * L->cfg.alpha}, st);
+  return launch_result();
+}
+
+}  // namespace
+
+// =========================================================================================
+extern "C" {
+
+compact_status_t compact_layer_create(const compact_layer_config_t* cfg, compact_layer_t** out) {
+  if (!cfg || !out) return COMPACT_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (cfg->dtype != COMPACT_F32 && cfg->dtype != COMPACT_BF16) return COMPACT_ERR_DTYPE;
+  const int mult = cfg->dtype == COMPACT_BF16 ? 8 : 4;
+  if (cfg->n < 1 || cfg->m < 1 || cfg->r < 1 || cfg->r > cfg->n) return COMPACT_ERR_SHAPE;
+  if (cfg->n % mult || cfg->m % mult) return COMPACT_ERR_SHAPE;
+  if (!(cfg->beta1 >= 0.f && cfg->beta1 < 1.f) || !(cfg->beta2 >= 0.f && cfg->beta2 < 1.f)) return COMPACT_ERR_INVALID_ARG;
+  if (!(cfg->eps >= 0.f) || isnan(cfg->lr) || isnan(cfg->alpha)) return COMPACT_ERR_INVALID_ARG;
+  compact_layer_t* L = new (std::nothrow) compact_layer_t;
+  if (!L) return COMPACT_ERR_INVALID_ARG;
+  L->cfg = *cfg;
+  L->epoch = 0;
+  L->step = 0;
+  L->last_refresh_step = 0;
+  L->status_slot = g_next_slot.fetch_add(1) % kStatusSlots;
+  L->device_checked = 0;
+  *out = L;
+  return COMPACT_OK;
+}
+
+compact_status_t compact_layer_destroy(compact_layer_t* layer) {
+  if (!layer) return COMPACT_ERR_INVALID_ARG;
+  delete layer;
+  return COMPACT_OK;
+}
+
+int64_t compact_z_ld(const compact_layer_t* layer) { return layer ? round_up(layer->cfg.r, 16) : -1; }
+
+size_t compact_workspace_bytes(const compact_layer_t* layer, int64_t tokens) {
+  if (!layer || tokens < 0) return 0;
+  const int m = layer->cfg.m, r = layer->cfg.r;
+  // update: N as fp32 r x m (SIMT) or bf16 (tensor-core kernels); backward: split-K partials.
+  size_t upd = (size_t)r * m * sizeof(float);
+  size_t bwd = tc::gc_workspace_bytes(tokens, r, m);
+  size_t need = upd > bwd ? upd : bwd;
+  return (size_t)round_up((int64_t)need, 256);
+}
+
+size_t compact_saved_bytes(const compact_layer_t* layer, int64_t tokens) {
+  if (!layer || tokens < 0) return 0;
+  return (size_t)tokens * (size_t)compact_z_ld(layer) * elem_size(layer->cfg.dtype);
+}
+
+compact_status_t compact_linear_fwd(compact_layer_t* L, int64_t tokens, const void* X, int64_t ldx, const void* W,
+                                    int64_t ldw, void* Y, int64_t ldy, void* Z, int64_t ldz, uint32_t* epoch_used,
+                                    void* stream) {
+  if (!L || tokens < 0 || tokens > 0x7fffffff) return COMPACT_ERR_INVALID_ARG;
+  if (epoch_used) *epoch_used = L->epoch;
+  if (tokens == 0) return COMPACT_OK;
+  if (!X || !W || !Y || !Z) return COMPACT_ERR_INVALID_ARG;
+  const size_t es = elem_size(L->cfg.dtype);
+  if (!aligned16(X) || !aligned16(W) || !aligned16(Y) || !aligned16(Z)) return COMPACT_ERR_ALIGNMENT;
+  if (!pitch_ok(ldx, L->cfg.n, es) || !pitch_ok(ldw, L->cfg.m, es) || !pitch_ok(ldy, L->cfg.m, es) ||
+      !pitch_ok(ldz, compact_z_ld(L), es))
+    return COMPACT_ERR_ALIGNMENT;
+  compact_status_t s = check_device(L);
+  if (s != COMPACT_OK) return s;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (L->cfg.dtype == COMPACT_BF16) {
+    typedef __nv_bfloat16 T;
+    if (g_family.load() == 0) {
+      tc::LaunchInfo li{st, status_word(L), &g_launches};
+      s = tc::forward(li, make_pp(L, L->epoch), tokens, (const T*)X, ldx, (const T*)W, ldw, (T*)Y, ldy, (T*)Z, ldz,
+                      (int)compact_z_ld(L));
+      if (s != COMPACT_ERR_SHAPE) return s;   // SHAPE: the tensor-core kernel does not take it
+    }
+    return fwd_simt<T>(L, tokens, (const T*)X, ldx, (const T*)W, ldw, (T*)Y, ldy, (T*)Z, ldz, st);
+  }
+  return fwd_simt<float>(L, tokens, (const float*)X, ldx, (const float*)W, ldw, (float*)Y, ldy, (float*)Z, ldz, st);
+}
+
+compact_status_t compact_linear_bwd(compact_layer_t* L, int64_t tokens, const void* dY, int64_t lddy, const void* Z,
+                                    int64_t ldz, const void* W, int64_t ldw, void* dX, int64_t lddx, float* Gc,
+                                    int64_t ldg, int accumulate, void* workspace, size_t workspace_bytes,
+                                    void* stream) {
+  if (!L || tokens < 0 || tokens > 0x7fffffff) return COMPACT_ERR_INVALID_ARG;
+  if (!Gc) return COMPACT_ERR_INVALID_ARG;
+  const size_t es = elem_size(L->cfg.dtype);
+  if (!aligned16(Gc) || !pitch_ok(ldg, L->cfg.m, 4)) return COMPACT_ERR_ALIGNMENT;
+  compact_status_t s = check_device(L);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (tokens == 0) {
+    // An empty micro-batch contributes nothing: Gc is zeroed unless accumulating.
+    if (accumulate) return COMPACT_OK;
+    if (s != COMPACT_OK) return s;
+    if (cudaMemset2DAsync(Gc, (size_t)ldg * 4, 0, (size_t)L->cfg.m * 4, (size_t)L->cfg.r, st) != cudaSuccess) {
+      cudaGetLastError();
+      return COMPACT_ERR_CUDA;
+    }
+    return COMPACT_OK;
+  }
+  if (!dY || !Z || !W) return COMPACT_ERR_INVALID_ARG;
+  if (!aligned16(dY) || !aligned16(Z) || !aligned16(W) || (dX && !aligned16(dX))) return COMPACT_ERR_ALIGNMENT;
+  if (!pitch_ok(lddy, L->cfg.m, es) || !pitch_ok(ldz, compact_z_ld(L), es) || !pitch_ok(ldw, L->cfg.m, es) ||
+      (dX && !pitch_ok(lddx, L->cfg.n, es)))
+    return COMPACT_ERR_ALIGNMENT;
+  if (workspace_bytes < compact_workspace_bytes(L, tokens) || (!workspace && compact_workspace_bytes(L, tokens)))
+    return COMPACT_ERR_WORKSPACE;
+  if (workspace && !aligned16(workspace)) return COMPACT_ERR_ALIGNMENT;
+  if (s != COMPACT_OK) return s;
+  if (L->cfg.dtype == COMPACT_BF16) {
+    typedef __nv_bfloat16 T;
+    if (g_family.load() == 0) {
+      tc::LaunchInfo li{st, status_word(L), &g_launches};
+      s = tc::backward(li, tokens, L->cfg.n, L->cfg.m, L->cfg.r, (const T*)dY, lddy, (const T*)Z, ldz, (const T*)W,
+                       ldw, (T*)dX, lddx, Gc, ldg, accumulate, workspace, workspace_bytes);
+      if (s != COMPACT_ERR_SHAPE) return s;
+    }
+    return bwd_simt<T>(L, tokens, (const T*)dY, lddy, (const T*)Z, ldz, (const T*)W, ldw, (T*)dX, lddx, Gc, ldg,
+                       accumulate, st);
+  }
+  return bwd_simt<float>(L, tokens, (const float*)dY, lddy, (const float*)Z, ldz, (const float*)W, ldw, (float*)dX,
+                         lddx, Gc, ldg, accumulate, st);
+}
+
+compact_status_t compact_adam_update(compact_layer_t* L, void* W, int64_t ldw, const float* Gc, int64_t ldg, float* M,
+                                     float* V, uint32_t epoch_of_Gc, float lr, void* workspace, size_t workspace_bytes,
+                                     void* stream) {
+  if (!L || !W || !Gc || !M || !V) return COMPACT_ERR_INVALID_ARG;
+  if (epoch_of_Gc != L->epoch) return COMPACT_ERR_EPOCH_MISMATCH;
+  const size_t es = elem_size(L->cfg.dtype);
+  if (!aligned16(W) || !aligned16(Gc) || !aligned16(M) || !aligned16(V)) return COMPACT_ERR_ALIGNMENT;
+  if (!pitch_ok(ldw, L->cfg.m, es) || !pitch_ok(ldg, L->cfg.m, 4)) return COMPACT_ERR_ALIGNMENT;
+  if (!workspace || workspace_bytes < compact_workspace_bytes(L, 0)) return COMPACT_ERR_WORKSPACE;
+  if (!aligned16(workspace)) return COMPACT_ERR_ALIGNMENT;
+  compact_status_t s = check_device(L);
+  if (s != COMPACT_OK) return s;
+  if (isnan(lr)) lr = L->cfg.lr;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (L->cfg.dtype == COMPACT_BF16) {
+    typedef __nv_bfloat16 T;
+    s = COMPACT_ERR_SHAPE;
+    if (g_family.load() == 0) {
+      tc::LaunchInfo li{st, status_word(L), &g_launches};
+      s = tc::update(li, make_pp(L, L->epoch), adam_scalars(L, L->step + 1), L->cfg.n, L->cfg.m, L->cfg.r, (T*)W, ldw,
+                     Gc, ldg, M, V, lr * L->cfg.alpha, workspace, workspace_bytes);
+    }
+    if (s == COMPACT_ERR_SHAPE) s = update_simt<T>(L, (T*)W, ldw, Gc, ldg, M, V, lr, (float*)workspace, st);
+  } else {
+    s = update_simt<float>(L, (float*)W, ldw, Gc, ldg, M, V, lr, (float*)workspace, st);
+  }
+  if (s == COMPACT_OK) L->step += 1;
+  return s;
+}
+
+compact_status_t compact_refresh_projection(compact_layer_t* L, int force, uint32_t* new_epoch) {
+  if (!L) return COMPACT_ERR_INVALID_ARG;
+  const uint32_t T = L->cfg.refresh_T;
+  if (force) {
+    L->epoch += 1;
+  } else if (T > 0 && L->step > 0 && L->step % T == 0 && L->last_refresh_step != L->step) {
+    L->epoch += 1;
+    L->last_refresh_step = L->step;
+  }
+  if (new_epoch) *new_epoch = L->epoch;
+  return COMPACT_OK;
+}
+
+compact_status_t compact_layer_get_state(const compact_layer_t* L, compact_layer_state_t* out) {
+  if (!L || !out) return COMPACT_ERR_INVALID_ARG;
+  out->seed = L->cfg.seed;
+  out->layer_id = L->cfg.layer_id;
+  out->epoch = L->epoch;
+  out->step = L->step;
+  return COMPACT_OK;
+}
+
+compact_status_t compact_layer_set_state(compact_layer_t* L, const compact_layer_state_t* in) {
+  if (!L || !in) return COMPACT_ERR_INVALID_ARG;
+  L->cfg.seed = in->seed;
+  L->cfg.layer_id = in->layer_id;
+  L->epoch = in->epoch;
+  L->step = in->step;
+  // A restored step that is a multiple of T has already been refreshed at if
+  // the restored epoch accounts for it; the caller restores what get_state gave.
+  const uint32_t T = L->cfg.refresh_T;
+  L->last_refresh_step = (T > 0 && in->step > 0 && in->step % T == 0 && in->epoch >= in->step / T) ? in->step : 0;
+  return COMPACT_OK;
+}
+
+compact_status_t compact_layer_status(compact_layer_t* L) {
+  if (!L) return COMPACT_ERR_INVALID_ARG;
+  compact_status_t s = check_device(L);
+  if (s != COMPACT_OK) return s;
+  unsigned int* w = status_word(L);
+  if (!w) return COMPACT_ERR_CUDA;
+  unsigned int v = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return COMPACT_ERR_CUDA; }
+  if (cudaMemcpy(&v, w, 4, cudaMemcpyDeviceToHost) != cudaSuccess) { cudaGetLastError(); return COMPACT_ERR_CUDA; }
+  if (v) {
+    unsigned int z = 0;
+    cudaMemcpy(w, &z, 4, cudaMemcpyHostToDevice);
+    return COMPACT_ERR_DEVICE_TIMEOUT;
+  }
+  return COMPACT_OK;
+}
+
+compact_status_t compact_debug_philox_u32(uint64_t seed, uint32_t layer_id, uint32_t epoch, int32_t n, int32_t r,
+                                          uint32_t* out_dev, void* stream) {
+  if (n < 1 || r < 1 || !out_dev) return COMPACT_ERR_INVALID_ARG;
+  if (!aligned16(out_dev)) return COMPACT_ERR_ALIGNMENT;
+  const int groups = (r + 3) / 4;
+  const int64_t cnt = (int64_t)n * groups;
+  debug_philox_words_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
+      make_philox_key(seed), layer_id, epoch, n, groups, out_dev);
+  g_launches++;
+  return launch_result();
+}
+
+compact_status_t compact_debug_projection(const compact_layer_t* L, uint32_t epoch, void* P_dev, void* stream) {
+  if (!L || !P_dev) return COMPACT_ERR_INVALID_ARG;
+  const ProjectionParams pp = make_pp(L, epoch);
+  const int64_t cnt = (int64_t)pp.n * ((pp.r + 3) / 4);
+  const unsigned blocks = (unsigned)((cnt + 255) / 256);
+  if (L->cfg.dtype == COMPACT_BF16)
+    debug_projection_kernel<__nv_bfloat16><<<blocks, 256, 0, (cudaStream_t)stream>>>(pp, (__nv_bfloat16*)P_dev);
+  else
+    debug_projection_kernel<float><<<blocks, 256, 0, (cudaStream_t)stream>>>(pp, (float*)P_dev);
+  g_launches++;
+  return launch_result();
+}
+
+int compact_set_kernel_family(int family) {
+  if (family != 0 && family != 1) return g_family.load();
+  return g_family.exchange(family);
+}
+
+uint64_t compact_kernel_launch_count(void) { return g_launches.load(); }
+
+const char* compact_status_string(compact_status_t s) {
+  switch (s) {
+    case COMPACT_OK: return "ok";
+    case COMPACT_ERR_INVALID_ARG: return "invalid argument";
+    case COMPACT_ERR_SHAPE: return "unsupported shape";
+    case COMPACT_ERR_ALIGNMENT: return "pointer or pitch not 16-byte aligned";
+    case COMPACT_ERR_DTYPE: return "unsupported dtype";
+    case COMPACT_ERR_EPOCH_MISMATCH: return "gradient was produced under another projection epoch";
+    case COMPACT_ERR_WORKSPACE: return "workspace missing or too small";
+    case COMPACT_ERR_UNSUPPORTED_ARCH: return "device is not compute capability 10.x";
+    case COMPACT_ERR_CUDA: return "CUDA runtime error";
+    case COMPACT_ERR_DEVICE_TIMEOUT: return "a kernel gave up on a bounded wait";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"

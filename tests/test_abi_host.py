@@ -1,0 +1,120 @@
+"""Host-only checks of the C-ABI library: it loads without a GPU, exports every
+symbol the header declares, and its host logic (schedule, accounting, argument
+validation) behaves as documented.  No compute call is made."""
+import ctypes as C
+import os
+import re
+
+import pytest
+import torch
+
+from paper_2410_15352_b200 import binding as cb
+from paper_2410_15352_b200.build import build_library
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build_library()
+
+
+def _declared_functions():
+    src = open(os.path.join(ROOT, "include", "compact.h")).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(compact_[a-z0-9_]+)\s*\(", src)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = _declared_functions()
+    assert len(names) >= 17 and set(cb.EXPORTS) == set(names)
+    L = cb.lib()
+    for nm in names:
+        assert hasattr(L, nm), nm
+
+
+def test_status_strings():
+    assert cb.status_string(cb.OK) == "ok"
+    for code in range(1, 10):
+        assert cb.status_string(code) not in ("ok", "unknown status")
+
+
+def test_create_validation():
+    with pytest.raises(cb.CompactError) as e:
+        cb.CompactLinear(128, 512, 256)            # r > n
+    assert e.value.code == cb.ERR_SHAPE
+    with pytest.raises(cb.CompactError) as e:
+        cb.CompactLinear(130, 512, 16)             # n not a multiple of 8 in bf16
+    assert e.value.code == cb.ERR_SHAPE
+    with pytest.raises(cb.CompactError) as e:
+        cb.CompactLinear(128, 512, 16, dtype=torch.float16)
+    assert e.value.code == cb.ERR_DTYPE
+    with pytest.raises(cb.CompactError) as e:
+        cb.CompactLinear(128, 512, 16, beta1=1.0)
+    assert e.value.code == cb.ERR_INVALID_ARG
+    assert cb.lib().compact_layer_create(None, None) == cb.ERR_INVALID_ARG
+
+
+def test_z_pitch_and_saved_bytes():
+    # Table 1: b l n -> b l r; Z rows are padded to a multiple of 16 columns
+    for r, ld in ((16, 16), (342, 352), (344, 352), (684, 688), (1376, 1376), (1, 16)):
+        lay = cb.CompactLinear(2736, 1024, r)
+        assert lay.ldz == ld
+        assert lay.saved_bytes(16384) == 16384 * ld * 2
+    lay = cb.CompactLinear(128, 512, 16, dtype=torch.float32)
+    assert lay.saved_bytes(256) == 256 * 16 * 4
+    # Table 3 / Appendix E ratio at r = n/4 for the LLaMA-350M block (n=1024, m=2736)
+    bl = 64 * 256
+    comp = 5 * cb.CompactLinear(1024, 1024, 256).saved_bytes(bl) + cb.CompactLinear(2736, 1024, 684).saved_bytes(bl)
+    dense = bl * (2 * 1024 + 2736) * 2
+    assert abs(comp / dense - 1964 / 4784) < 2e-3   # the 684 -> 688 pad shifts it slightly
+
+
+def test_refresh_schedule_is_host_only():
+    lay = cb.CompactLinear(128, 512, 16, dtype=torch.float32, refresh_T=2)
+    before = cb.kernel_launch_count()
+    assert lay.refresh_projection() == 0            # step 0: nothing to refresh
+    lay.set_state(0, 0, 0, 1)
+    assert lay.refresh_projection() == 0
+    lay.set_state(0, 0, 0, 2)
+    assert lay.refresh_projection() == 1            # t mod T == 0 -> epoch + 1
+    assert lay.refresh_projection() == 1            # idempotent within a step
+    lay.set_state(0, 0, 1, 3)
+    assert lay.refresh_projection() == 1
+    assert lay.refresh_projection(force=True) == 2
+    never = cb.CompactLinear(128, 512, 16, dtype=torch.float32, refresh_T=0)
+    never.set_state(0, 0, 0, 1000)
+    assert never.refresh_projection() == 0
+    assert cb.kernel_launch_count() == before       # Section 3.3: a refresh only replaces the seed
+
+
+def test_state_round_trip():
+    lay = cb.CompactLinear(128, 512, 16, seed=(7 << 32) | 5, layer_id=3, refresh_T=10)
+    st = lay.state()
+    assert (st.seed, st.layer_id, st.epoch, st.step) == ((7 << 32) | 5, 3, 0, 0)
+    lay.set_state(11, 4, 2, 20)
+    st = lay.state()
+    assert (st.seed, st.layer_id, st.epoch, st.step) == (11, 4, 2, 20)
+    assert lay.refresh_projection() == 2            # restored epoch already accounts for step 20
+
+
+def test_argument_errors_before_any_launch():
+    lay = cb.CompactLinear(128, 512, 16, dtype=torch.float32)
+    L = cb.lib()
+    before = cb.kernel_launch_count()
+    assert L.compact_linear_fwd(lay._h, 4, None, 128, None, 512, None, 512, None, 16, None, None) == cb.ERR_INVALID_ARG
+    assert L.compact_linear_fwd(lay._h, -1, None, 128, None, 512, None, 512, None, 16, None, None) == cb.ERR_INVALID_ARG
+    buf = C.c_void_p(0x1000)
+    odd = C.c_void_p(0x1004)
+    assert L.compact_linear_fwd(lay._h, 4, odd, 128, buf, 512, buf, 512, buf, 16, None, None) == cb.ERR_ALIGNMENT
+    assert L.compact_linear_fwd(lay._h, 4, buf, 126, buf, 512, buf, 512, buf, 16, None, None) == cb.ERR_ALIGNMENT
+    assert L.compact_linear_fwd(lay._h, 4, buf, 128, buf, 512, buf, 512, buf, 8, None, None) == cb.ERR_ALIGNMENT
+    assert L.compact_linear_bwd(lay._h, 4, buf, 512, buf, 16, buf, 512, buf, 128, buf, 512, 0, None, 0, None) \
+        == cb.ERR_WORKSPACE
+    assert L.compact_adam_update(lay._h, buf, 512, buf, 512, buf, buf, 1, 1e-3, buf, 1 << 20, None) \
+        == cb.ERR_EPOCH_MISMATCH
+    assert L.compact_adam_update(lay._h, buf, 512, buf, 512, buf, buf, 0, 1e-3, None, 0, None) == cb.ERR_WORKSPACE
+    ep = C.c_uint32(99)
+    assert L.compact_linear_fwd(lay._h, 0, None, 128, None, 512, None, 512, None, 16, C.byref(ep), None) == cb.OK
+    assert ep.value == 0                            # empty batch: no launch, epoch still reported
+    assert cb.kernel_launch_count() == before

@@ -1,0 +1,198 @@
+"""GPU parity tests: the CUDA path, called through the C ABI, against the CPU
+oracle on the same seeded inputs.  Integer streams must match bit for bit;
+floating-point tensors within the stated relative Frobenius tolerance
+(1e-5 in fp32, 2e-2 in bf16 with fp32 accumulation)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import compact_oracle as co
+from paper_2410_15352_b200 import binding as cb
+from paper_2410_15352_b200 import workloads as wlm
+from paper_2410_15352_b200.build import build_library
+from tests._harness import TOL, f32, make_pair, run_layer_trajectory, to64
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build_library()
+    cb.set_kernel_family(0)
+    yield
+    cb.set_kernel_family(0)
+
+
+@pytest.fixture(params=[0, 1], ids=["auto", "simt"])
+def family(request):
+    cb.set_kernel_family(request.param)
+    yield request.param
+    cb.set_kernel_family(0)
+
+
+# ---- F0: the generator -----------------------------------------------------------------
+@pytest.mark.parametrize("seed,layer,epoch,n,r", [
+    (0, 0, 0, 128, 16), ((5 << 32) | 0xDEADBEEF, 6, 3, 300, 342), (2 ** 64 - 1, 0xFFFFFFFF, 0xFFFFFFFF, 64, 7),
+    (1, 2, 1, 1376, 344)])
+def test_philox_words_bit_exact(seed, layer, epoch, n, r):
+    got = cb.debug_philox_u32(seed, layer, epoch, n, r).cpu().numpy().view(np.uint32)
+    want = co.projection_words(seed, layer, epoch, n, r)
+    assert got.shape == want.shape and np.array_equal(got, want)
+
+
+def test_philox_known_answer_on_device():
+    got = cb.debug_philox_u32(0, 0, 0, 1, 4).cpu().numpy().view(np.uint32)[0]
+    assert [int(x) for x in got] == [0x6627E8D5, 0xE169C58D, 0xBC57AC4C, 0x9B00DBD8]
+
+
+def test_projection_fp32_entries():
+    lay = cb.CompactLinear(512, 64, 100, dtype=torch.float32, seed=3, layer_id=2)
+    P = to64(lay.debug_projection(epoch=1))
+    want = co.projection(3, 2, 1, 512, 100)
+    assert np.max(np.abs(P - want)) <= 4e-7 * np.max(np.abs(want)) + 1e-9
+    assert co.rel_frobenius(P, want) < 2e-7
+
+
+def test_projection_bf16_entries():
+    lay = cb.CompactLinear(1376, 64, 344, dtype=torch.bfloat16, seed=9, layer_id=1)
+    P = to64(lay.debug_projection(epoch=0))
+    want = co.projection(9, 1, 0, 1376, 344, mode="bf16")
+    diff = P != want
+    # fp32 Box-Muller then one rounding vs fp64 then one rounding: rare one-ulp differences only
+    assert diff.mean() < 5e-3
+    ulp = np.maximum(np.abs(want), 2.0 ** -126) * 2.0 ** -7
+    assert np.all(np.abs(P - want) <= ulp * 1.001)
+
+
+# ---- config 1: fp32, full trajectory with refresh -------------------------------------
+def test_config1_fp32_trajectory():
+    wl = wlm.config1()
+    errs, epochs, dW = run_layer_trajectory(wl, 0, wl.steps)
+    assert epochs == [0, 0, 1]
+    for k, v in errs.items():
+        assert v <= TOL["f32"], (k, v)
+    assert dW <= 1e-4
+
+
+# ---- small bf16 shapes spanning tiles and ragged tails, both kernel families ------------
+SMALL = [
+    # tokens, n, m, r
+    (256, 128, 512, 16),
+    (384, 512, 512, 128),
+    (300, 1376, 512, 344),       # ragged tokens, ragged r (ldz 352)
+    (1000, 512, 1376, 128),      # ragged m tile
+    (130, 264, 72, 50),          # everything ragged
+]
+
+
+@pytest.mark.parametrize("tokens,n,m,r", SMALL)
+def test_small_bf16_trajectory(family, tokens, n, m, r):
+    wl = wlm.Workload("small", 90, "bf16", tokens, [wlm.LayerShape("l", n, m, r)], steps=3, refresh_T=2,
+                      x_scale_inv_sqrt_n=True)
+    errs, epochs, dW = run_layer_trajectory(wl, 0, 3)
+    assert epochs == [0, 0, 1]
+    for k, v in errs.items():
+        assert v <= TOL["bf16"], (k, v)
+
+
+@pytest.mark.parametrize("tokens,n,m,r", [(96, 64, 40, 12), (257, 132, 260, 33)])
+def test_small_fp32_ragged(tokens, n, m, r):
+    wl = wlm.Workload("small32", 91, "f32", tokens, [wlm.LayerShape("l", n, m, r)], steps=2, refresh_T=1)
+    errs, epochs, _ = run_layer_trajectory(wl, 0, 2)
+    assert epochs == [0, 1]
+    for k, v in errs.items():
+        assert v <= TOL["f32"], (k, v)
+
+
+# ---- Z token indexing: bit-exact ----------------------------------------------------------
+def test_z_token_indexing_bit_exact(family):
+    n, m, r, tokens = 512, 256, 100, 640
+    lay = cb.CompactLinear(n, m, r, seed=4, layer_id=1)
+    Pb = lay.debug_projection()
+    rng = np.random.default_rng(0)
+    rows = rng.integers(0, n, size=tokens)
+    X = torch.zeros((tokens, n), dtype=torch.bfloat16)
+    X[torch.arange(tokens), torch.from_numpy(rows)] = 1.0
+    X[::7] = 0.0                                     # some all-zero tokens
+    W = wlm.draw_W(wlm.Workload("w", 92, "bf16", tokens, [wlm.LayerShape("l", n, m, r)]), 0).cuda()
+    _, Z, _ = lay.forward(X.cuda(), W)
+    want = Pb[torch.from_numpy(rows).cuda()].clone()
+    want[::7] = 0
+    assert torch.equal(Z[:, :r].view(torch.int16), want.view(torch.int16))
+    assert not Z[:, r:].any()
+    # permuting tokens permutes rows of Z bitwise
+    Xr = torch.randn((tokens, n), generator=torch.Generator().manual_seed(1)).to(torch.bfloat16).cuda()
+    perm = torch.randperm(tokens, generator=torch.Generator().manual_seed(2)).cuda()
+    _, Z1, _ = lay.forward(Xr, W)
+    _, Z2, _ = lay.forward(Xr[perm].contiguous(), W)
+    assert torch.equal(Z1[perm].view(torch.int16), Z2.view(torch.int16))
+
+
+# ---- determinism, accumulation, empty input, epoch guard -----------------------------------
+def test_run_twice_bitwise_and_accumulate(family):
+    wl = wlm.Workload("det", 93, "bf16", 1024, [wlm.LayerShape("l", 512, 768, 128)], x_scale_inv_sqrt_n=True)
+    gpu, ora, W0 = make_pair(wl, 0)
+    W = W0.cuda()
+    X, dY = wlm.draw_X(wl, 0, 0).cuda(), wlm.draw_dY(wl, 0, 0).cuda()
+    Y1, Z1, ep = gpu.forward(X, W)
+    Y2, Z2, _ = gpu.forward(X, W)
+    assert torch.equal(Y1.view(torch.int16), Y2.view(torch.int16)) and torch.equal(Z1.view(torch.int16), Z2.view(torch.int16))
+    dX1, G1 = gpu.backward(dY, Z1, W)
+    dX2, G2 = gpu.backward(dY, Z1, W)
+    assert torch.equal(G1, G2) and torch.equal(dX1.view(torch.int16), dX2.view(torch.int16))
+    # two half micro-batches accumulated == oracle on the full batch
+    h = 512
+    Ga = torch.empty_like(G1)
+    gpu.backward(dY[:h], Z1[:h], W, Gc=Ga, need_dX=False)
+    gpu.backward(dY[h:], Z1[h:], W, Gc=Ga, need_dX=False, accumulate=True)
+    _, Gco = ora.backward(to64(dY), to64(Z1[:, :128]))
+    assert co.rel_frobenius(to64(Ga), Gco) <= TOL["bf16"]
+    assert co.rel_frobenius(to64(G1), Gco) <= TOL["bf16"]
+
+
+def test_empty_batch_and_epoch_guard():
+    lay = cb.CompactLinear(128, 512, 16, refresh_T=1)
+    W = torch.zeros((128, 512), dtype=torch.bfloat16, device="cuda")
+    Y, Z, ep = lay.forward(torch.empty((0, 128), dtype=torch.bfloat16, device="cuda"), W)
+    assert Y.shape == (0, 512) and ep == 0
+    G = torch.full((16, 512), 7.0, device="cuda")
+    lay.backward(torch.empty((0, 512), dtype=torch.bfloat16, device="cuda"), Z, W, Gc=G, need_dX=False)
+    assert not G.any()
+    M, V = torch.zeros_like(G), torch.zeros_like(G)
+    with pytest.raises(cb.CompactError) as e:
+        lay.adam_update(W, G, M, V, epoch_of_Gc=1)
+    assert e.value.code == cb.ERR_EPOCH_MISMATCH
+    lay.adam_update(W, G, M, V, epoch_of_Gc=0)      # zero gradient: nothing changes
+    assert not W.any() and not M.any() and not V.any()
+    assert lay.status() == cb.OK
+
+
+def test_checkpoint_resume_bitwise():
+    wl = wlm.Workload("ckpt", 94, "bf16", 512, [wlm.LayerShape("l", 256, 384, 64)], refresh_T=2, x_scale_inv_sqrt_n=True)
+
+    def run(lay, W, M, V, s0, s1):
+        for s in range(s0, s1):
+            X, dY = wlm.draw_X(wl, 0, s).cuda(), wlm.draw_dY(wl, 0, s).cuda()
+            _, Z, ep = lay.forward(X, W)
+            _, Gc = lay.backward(dY, Z, W, need_dX=False)
+            lay.adam_update(W, Gc, M, V, ep)
+            lay.refresh_projection()
+
+    def fresh():
+        lay = cb.CompactLinear(256, 384, 64, refresh_T=2, seed=5, layer_id=1)
+        W = wlm.draw_W(wl, 0).cuda()
+        return lay, W, torch.zeros((64, 384), device="cuda"), torch.zeros((64, 384), device="cuda")
+
+    a, Wa, Ma, Va = fresh()
+    run(a, Wa, Ma, Va, 0, 5)
+    b, Wb, Mb, Vb = fresh()
+    run(b, Wb, Mb, Vb, 0, 2)
+    st = b.state()
+    c = cb.CompactLinear(256, 384, 64, refresh_T=2)
+    c.set_state(st.seed, st.layer_id, st.epoch, st.step)
+    Wc, Mc, Vc = Wb.clone(), Mb.clone(), Vb.clone()
+    run(c, Wc, Mc, Vc, 2, 5)
+    assert torch.equal(Wa.view(torch.int16), Wc.view(torch.int16)) and torch.equal(Ma, Mc) and torch.equal(Va, Vc)
+    assert a.epoch == c.epoch == 2
