@@ -207,7 +207,7 @@ compact_status_t compact_linear_fwd(compact_layer_t* L, int64_t tokens, const vo
     typedef __nv_bfloat16 T;
     if (g_family.load() == 0) {
       tc::LaunchInfo li{st, status_word(L), &g_launches};
-      s = tc::forward(li, make_pp(L, L->epoch), tokens, (const T*)X, ldx, (const T*)W, ldw, (T*)Y, ldy, (T*)Z, ldz,
+      s = tc::forward(li, make_pp(L, L->epoch), tokens, L->cfg.m, (const T*)X, ldx, (const T*)W, ldw, (T*)Y, ldy, (T*)Z, ldz,
                       (int)compact_z_ld(L));
       if (s != COMPACT_ERR_SHAPE) return s;   // SHAPE: the tensor-core kernel does not take it
     }
@@ -249,7 +249,7 @@ compact_status_t compact_linear_bwd(compact_layer_t* L, int64_t tokens, const vo
     typedef __nv_bfloat16 T;
     if (g_family.load() == 0) {
       tc::LaunchInfo li{st, status_word(L), &g_launches};
-      s = tc::backward(li, tokens, L->cfg.n, L->cfg.m, L->cfg.r, (const T*)dY, lddy, (const T*)Z, ldz, (const T*)W,
+      s = tc::backward(li, tokens, L->cfg.n, L->cfg.m, L->cfg.r, (int)compact_z_ld(L), (const T*)dY, lddy, (const T*)Z, ldz, (const T*)W,
                        ldw, (T*)dX, lddx, Gc, ldg, accumulate, workspace, workspace_bytes);
       if (s != COMPACT_ERR_SHAPE) return s;
     }

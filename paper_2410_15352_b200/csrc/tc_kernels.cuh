@@ -1,6 +1,15 @@
-// Tensor-core (tcgen05 / TMEM / TMA) kernels of the CompAct layer for sm_100a.
+// Tensor-core kernels of the CompAct layer for sm_100a: one persistent,
+// warp-specialised GEMM (TMA -> 128B-swizzled shared memory ring -> tcgen05.mma
+// with fp32 accumulators in TMEM -> tcgen05.ld epilogue) whose operands can come
+// from TMA in either major-ness or from the in-kernel Philox/Box-Muller generator
+// of P.  It serves
+//   forward  : [Y | Z] = X [W | P]        (Algorithm 1; P tiles generated as the B operand)
+//   backward : dX = dY W^T and Gc = Z^T dY (Algorithm 2; Gc split over tokens)
+//   update   : W <- W - eta alpha P N      (Algorithm 3 lines 6-9; P tiles generated as A)
 #pragma once
+#include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_runtime.h>
 #include <stdint.h>
 
 #include <atomic>
@@ -18,20 +27,647 @@ struct LaunchInfo {
   std::atomic<uint64_t>* launches;
 };
 
-inline size_t gc_workspace_bytes(int64_t, int, int) { return 0; }
+constexpr int BM = 128;              // rows of one accumulator (TMEM lanes)
+constexpr int BK = 64;               // K elements per pipeline stage (one 128-byte swizzle row)
+constexpr int BN_MAX = 256;          // widest accumulator (TMEM columns)
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;
+constexpr int B_BYTES = BN_MAX * BK * 2;
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int NUM_GEN_WARPS = 8;
+constexpr int THREADS_BASE = 192;    // producer warp, MMA warp, four epilogue warps
+constexpr int THREADS_GEN = THREADS_BASE + 32 * NUM_GEN_WARPS;
+constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + 256;
+constexpr int NUM_SMS = 148;
 
-inline compact_status_t forward(const LaunchInfo&, const ProjectionParams&, int64_t, const __nv_bfloat16*, int64_t,
-                                const __nv_bfloat16*, int64_t, __nv_bfloat16*, int64_t, __nv_bfloat16*, int64_t, int) {
-  return COMPACT_ERR_SHAPE;
+enum OperandMode { TMA_KMAJOR = 0, TMA_MNMAJOR = 1, GENERATED = 2 };
+enum EpiMode { EPI_BF16 = 0, EPI_F32 = 1, EPI_UPDATE_W = 2 };
+
+constexpr unsigned int STATUS_TIMEOUT = 1u;
+
+struct Problem {
+  int M, N, K;
+  int tiles_m, tiles_n, splits, ksteps_total, ksteps_per_split;
+  int bn;
+  int a_mode, b_mode, epi_mode;
+  int accumulate;
+  int tile_begin;
+  float scale;
+  void* out;
+  long long ld_out;
+  long long split_stride;
+};
+
+struct alignas(64) Params {
+  CUtensorMap tmA[2];
+  CUtensorMap tmB[2];
+  Problem prob[2];
+  int num_problems;
+  int total_tiles;
+  int has_generated;
+  ProjectionParams pp;
+  unsigned int* status;
+};
+
+// --------------------------------------------------------------------------------------
+// PTX wrappers
+// --------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
-inline compact_status_t backward(const LaunchInfo&, int64_t, int, int, int, const __nv_bfloat16*, int64_t,
-                                 const __nv_bfloat16*, int64_t, const __nv_bfloat16*, int64_t, __nv_bfloat16*, int64_t,
-                                 float*, int64_t, int, void*, size_t) {
-  return COMPACT_ERR_SHAPE;
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-inline compact_status_t update(const LaunchInfo&, const ProjectionParams&, const simt::AdamScalars&, int, int, int,
-                               __nv_bfloat16*, int64_t, const float*, int64_t, float*, float*, float, void*, size_t) {
-  return COMPACT_ERR_SHAPE;
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: gives up after about a second, records it, and lets the CTA drain.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned int* status) {
+  for (uint32_t it = 0; it < 8000000u; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (it > 128) {
+      __nanosleep(100);
+      if (*abort_flag) return false;
+    }
+  }
+  *abort_flag = 1;
+  atomicOr(status, STATUS_TIMEOUT);
+  return false;
+}
+
+__device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+      "l"(map), "r"(bar), "r"(x), "r"(y)
+      : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: 128-byte swizzle, 8-row groups 1024 bytes apart.
+// lbo_bytes: distance between 64-element blocks along M/N (MN-major operands only).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr >> 4) & 0x3FFF);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((1024u >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;   // descriptor version of sm_100
+  d |= (uint64_t)2 << 61;   // 128-byte swizzle
+  return d;
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+// Eight consecutive entries P[i, j0 .. j0+7] (j0 a multiple of 8) as packed bf16.
+__device__ __forceinline__ uint4 projection8_bf16(const ProjectionParams& pp, int i, int j0) {
+  const float4 a = projection4(pp, i, j0 >> 2);
+  const float4 b = projection4(pp, i, (j0 >> 2) + 1);
+  return make_uint4(pack_bf16x2(a.x, a.y), pack_bf16x2(a.z, a.w), pack_bf16x2(b.x, b.y), pack_bf16x2(b.z, b.w));
+}
+
+struct TileCoord {
+  int prob, m0, n0, k_begin, k_end, split;
+};
+
+__device__ __forceinline__ TileCoord decode_tile(const Params& prm, int tile) {
+  TileCoord t;
+  t.prob = (prm.num_problems > 1 && tile >= prm.prob[1].tile_begin) ? 1 : 0;
+  const Problem& p = prm.prob[t.prob];
+  int local = tile - p.tile_begin;
+  const int nb = local % p.tiles_n;
+  local /= p.tiles_n;
+  const int mb = local % p.tiles_m;
+  t.split = local / p.tiles_m;
+  t.m0 = mb * BM;
+  t.n0 = nb * p.bn;
+  t.k_begin = t.split * p.ksteps_per_split;
+  t.k_end = min(p.ksteps_total, t.k_begin + p.ksteps_per_split);
+  return t;
+}
+
+// --------------------------------------------------------------------------------------
+// The kernel
+// --------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __grid_constant__ Params prm) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));   // generic pointer to the aligned base
+  const uint32_t bars = smem_base + STAGES * STAGE_BYTES;
+  // barrier slots (8 bytes each): full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
+  auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };
+  auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };
+  uint8_t* tail = smem_gen + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 4);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 8);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 1 + (prm.has_generated ? NUM_GEN_WARPS : 0));
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);
+      mbar_init(tempty_bar(a), 4);
+    }
+    *abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async_smem();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32((const void*)tmem_slot), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < prm.total_tiles && ok; tile += gridDim.x) {
+        const TileCoord t = decode_tile(prm, tile);
+        const Problem& p = prm.prob[t.prob];
+        const CUtensorMap* mapA = &prm.tmA[t.prob];
+        const CUtensorMap* mapB = &prm.tmB[t.prob];
+        const uint32_t bytes = (p.a_mode != GENERATED ? A_BYTES : 0) + (p.b_mode != GENERATED ? p.bn * BK * 2 : 0);
+        for (int ks = t.k_begin; ks < t.k_end; ++ks) {
+          if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1, abort_flag, prm.status))) break;
+          const uint32_t sa = smem_base + stage * STAGE_BYTES, sb = sa + A_BYTES;
+          const uint32_t fb = full_bar(stage);
+          mbar_arrive_expect_tx(fb, bytes);
+          const int k0 = ks * BK;
+          if (p.a_mode == TMA_KMAJOR) {
+            tma_load_2d(sa, mapA, fb, k0, t.m0);
+          } else if (p.a_mode == TMA_MNMAJOR) {
+            tma_load_2d(sa, mapA, fb, t.m0, k0);
+            tma_load_2d(sa + 8192, mapA, fb, t.m0 + 64, k0);
+          }
+          if (p.b_mode == TMA_KMAJOR) {
+            tma_load_2d(sb, mapB, fb, k0, t.n0);
+          } else if (p.b_mode == TMA_MNMAJOR) {
+            for (int b = 0; b < p.bn / 64; ++b) tma_load_2d(sb + b * 8192, mapB, fb, t.n0 + 64 * b, k0);
+          }
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer ---------------------------------
+    if (lane == 0) {
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < prm.total_tiles && ok; tile += gridDim.x) {
+        const TileCoord t = decode_tile(prm, tile);
+        const Problem& p = prm.prob[t.prob];
+        const bool a_mn = p.a_mode == TMA_MNMAJOR;
+        const bool b_mn = p.b_mode != TMA_KMAJOR;          // generated B tiles are written MN-major
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+                               ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+        if (!(ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag, prm.status))) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BN_MAX;
+        for (int ks = t.k_begin; ks < t.k_end; ++ks) {
+          if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag, prm.status))) break;
+          tc_fence_after();
+          const uint32_t sa = smem_base + stage * STAGE_BYTES, sb = sa + A_BYTES;
+#pragma unroll
+          for (int k4 = 0; k4 < BK / 16; ++k4) {
+            const uint64_t adesc = a_mn ? smem_desc(sa + k4 * 2048, 8192) : smem_desc(sa + k4 * 32, 16);
+            const uint64_t bdesc = b_mn ? smem_desc(sb + k4 * 2048, 8192) : smem_desc(sb + k4 * 32, 16);
+            umma_bf16(d_tmem, adesc, bdesc, idesc, (ks > t.k_begin || k4 > 0) ? 1u : 0u);
+          }
+          umma_commit(empty_bar(stage));
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        umma_commit(tfull_bar(acc));
+        if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+      }
+    }
+  } else if (warp < 6) {
+    // ------------------------------ epilogue ------------------------------------
+    const int q = warp & 3;                 // TMEM lane quarter this warp may read
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < prm.total_tiles && ok; tile += gridDim.x) {
+      const TileCoord t = decode_tile(prm, tile);
+      const Problem& p = prm.prob[t.prob];
+      if (!(ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, prm.status))) break;
+      tc_fence_after();
+      const int row = t.m0 + q * 32 + lane;
+      const bool row_ok = row < p.M;
+      for (int c0 = 0; c0 < p.bn; c0 += 32) {
+        const int col = t.n0 + c0;
+        if (col >= p.N) break;
+        uint32_t v[32];
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN_MAX + c0, v);
+        tmem_ld_wait();
+        if (!row_ok) continue;
+        if (p.epi_mode == EPI_BF16) {
+          __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + (long long)row * p.ld_out + col;
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            if (col + g * 8 + 8 <= p.N) {
+              uint4 o;
+              o.x = pack_bf16x2(__uint_as_float(v[g * 8 + 0]), __uint_as_float(v[g * 8 + 1]));
+              o.y = pack_bf16x2(__uint_as_float(v[g * 8 + 2]), __uint_as_float(v[g * 8 + 3]));
+              o.z = pack_bf16x2(__uint_as_float(v[g * 8 + 4]), __uint_as_float(v[g * 8 + 5]));
+              o.w = pack_bf16x2(__uint_as_float(v[g * 8 + 6]), __uint_as_float(v[g * 8 + 7]));
+              *reinterpret_cast<uint4*>(dst + g * 8) = o;
+            }
+          }
+        } else if (p.epi_mode == EPI_F32) {
+          float* dst = reinterpret_cast<float*>(p.out) + (long long)t.split * p.split_stride + (long long)row * p.ld_out + col;
+#pragma unroll
+          for (int g = 0; g < 8; ++g) {
+            if (col + g * 4 + 4 <= p.N) {
+              float4 o = make_float4(__uint_as_float(v[g * 4 + 0]), __uint_as_float(v[g * 4 + 1]),
+                                     __uint_as_float(v[g * 4 + 2]), __uint_as_float(v[g * 4 + 3]));
+              if (p.accumulate) {
+                const float4 old = *reinterpret_cast<const float4*>(dst + g * 4);
+                o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+              }
+              *reinterpret_cast<float4*>(dst + g * 4) = o;
+            }
+          }
+        } else {
+          // Algorithm 3 line 9: W <- W - (eta alpha) (P N), one rounding of the result
+          __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + (long long)row * p.ld_out + col;
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            if (col + g * 8 + 8 <= p.N) {
+              uint4 w = *reinterpret_cast<const uint4*>(dst + g * 8);
+              const float s = -p.scale;
+              w.x = pack_bf16x2(fmaf(s, __uint_as_float(v[g * 8 + 0]), bf16lo(w.x)), fmaf(s, __uint_as_float(v[g * 8 + 1]), bf16hi(w.x)));
+              w.y = pack_bf16x2(fmaf(s, __uint_as_float(v[g * 8 + 2]), bf16lo(w.y)), fmaf(s, __uint_as_float(v[g * 8 + 3]), bf16hi(w.y)));
+              w.z = pack_bf16x2(fmaf(s, __uint_as_float(v[g * 8 + 4]), bf16lo(w.z)), fmaf(s, __uint_as_float(v[g * 8 + 5]), bf16hi(w.z)));
+              w.w = pack_bf16x2(fmaf(s, __uint_as_float(v[g * 8 + 6]), bf16lo(w.w)), fmaf(s, __uint_as_float(v[g * 8 + 7]), bf16hi(w.w)));
+              *reinterpret_cast<uint4*>(dst + g * 8) = w;
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+    }
+  } else {
+    // ------------------------------ P generators --------------------------------
+    // Write bf16 tiles of P straight into the swizzled operand layout the MMA reads.
+    const int gtid = threadIdx.x - THREADS_BASE;
+    int stage = 0;
+    uint32_t phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < prm.total_tiles && ok; tile += gridDim.x) {
+      const TileCoord t = decode_tile(prm, tile);
+      const Problem& p = prm.prob[t.prob];
+      for (int ks = t.k_begin; ks < t.k_end; ++ks) {
+        if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1, abort_flag, prm.status))) break;
+        uint8_t* sa = smem_gen + stage * STAGE_BYTES;
+        uint8_t* sb = sa + A_BYTES;
+        const int k0 = ks * BK;
+        if (p.b_mode == GENERATED) {
+          // B[k = row i of P][n = column j of P], MN-major: 64-column blocks of [64 k][128 B]
+          const int chunks = p.bn >> 3;
+          for (int id = gtid; id < BK * chunks; id += 32 * NUM_GEN_WARPS) {
+            const int c = id % chunks, kr = id / chunks;
+            const uint4 val = projection8_bf16(prm.pp, k0 + kr, t.n0 + c * 8);
+            *reinterpret_cast<uint4*>(sb + (c >> 3) * 8192 + kr * 128 + (((c & 7) ^ (kr & 7)) << 4)) = val;
+          }
+        }
+        if (p.a_mode == GENERATED) {
+          // A[m = row i of P][k = column j of P], K-major: [128 rows][128 B]
+          for (int id = gtid; id < BM * 8; id += 32 * NUM_GEN_WARPS) {
+            const int c = id & 7, rr = id >> 3;
+            const uint4 val = projection8_bf16(prm.pp, t.m0 + rr, k0 + c * 8);
+            *reinterpret_cast<uint4*>(sa + rr * 128 + ((c ^ (rr & 7)) << 4)) = val;
+          }
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(full_bar(stage));
+        if (++stage == STAGES) { stage = 0; phase ^= 1; }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// --------------------------------------------------------------------------------------
+// Element-wise kernels around the GEMMs
+// --------------------------------------------------------------------------------------
+// Algorithm 3 lines 1-5: moments in place, N rounded to bf16 into scratch (pitch m).
+__global__ void adam_moments_bf16_kernel(const float* __restrict__ Gc, long long ldg, float* __restrict__ Mo,
+                                         float* __restrict__ Vo, __nv_bfloat16* __restrict__ Nout, int r, int m,
+                                         simt::AdamScalars s) {
+  const int m4 = m >> 2;
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (long long)r * m4) return;
+  const int j = (int)(idx / m4), c = (int)(idx % m4) * 4;
+  const long long off = (long long)j * ldg + c;
+  const float4 g = *reinterpret_cast<const float4*>(Gc + off);
+  float4 mm = *reinterpret_cast<const float4*>(Mo + off);
+  float4 vv = *reinterpret_cast<const float4*>(Vo + off);
+  mm.x = fmaf(s.beta1, mm.x, s.one_minus_beta1 * g.x);
+  mm.y = fmaf(s.beta1, mm.y, s.one_minus_beta1 * g.y);
+  mm.z = fmaf(s.beta1, mm.z, s.one_minus_beta1 * g.z);
+  mm.w = fmaf(s.beta1, mm.w, s.one_minus_beta1 * g.w);
+  vv.x = fmaf(s.beta2, vv.x, s.one_minus_beta2 * g.x * g.x);
+  vv.y = fmaf(s.beta2, vv.y, s.one_minus_beta2 * g.y * g.y);
+  vv.z = fmaf(s.beta2, vv.z, s.one_minus_beta2 * g.z * g.z);
+  vv.w = fmaf(s.beta2, vv.w, s.one_minus_beta2 * g.w * g.w);
+  *reinterpret_cast<float4*>(Mo + off) = mm;
+  *reinterpret_cast<float4*>(Vo + off) = vv;
+  const float n0 = (mm.x * s.inv_bias1) / (sqrtf(vv.x * s.inv_bias2) + s.eps);
+  const float n1 = (mm.y * s.inv_bias1) / (sqrtf(vv.y * s.inv_bias2) + s.eps);
+  const float n2 = (mm.z * s.inv_bias1) / (sqrtf(vv.z * s.inv_bias2) + s.eps);
+  const float n3 = (mm.w * s.inv_bias1) / (sqrtf(vv.w * s.inv_bias2) + s.eps);
+  uint2 o = make_uint2(pack_bf16x2(n0, n1), pack_bf16x2(n2, n3));
+  *reinterpret_cast<uint2*>(Nout + (long long)j * m + c) = o;
+}
+
+// Deterministic reduction of the split-K partials of Gc, in split order.
+__global__ void reduce_partials_kernel(const float* __restrict__ part, long long split_stride, int splits,
+                                       float* __restrict__ Gc, long long ldg, int r, int m, int accumulate) {
+  const int m4 = m >> 2;
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (long long)r * m4) return;
+  const int j = (int)(idx / m4), c = (int)(idx % m4) * 4;
+  float4 acc = accumulate ? *reinterpret_cast<const float4*>(Gc + (long long)j * ldg + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s = 0; s < splits; ++s) {
+    const float4 p = *reinterpret_cast<const float4*>(part + s * split_stride + (long long)j * m + c);
+    acc.x += p.x; acc.y += p.y; acc.z += p.z; acc.w += p.w;
+  }
+  *reinterpret_cast<float4*>(Gc + (long long)j * ldg + c) = acc;
+}
+
+// --------------------------------------------------------------------------------------
+// Host side
+// --------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &p, 12000, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+    else
+      cudaGetLastError();
+  }
+  return fn;
+}
+
+// 2-D bf16 map over a row-major matrix: `inner` contiguous elements per row, `rows` rows, pitch in elements.
+inline bool make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t rows, int64_t pitch, int box_inner,
+                     int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)pitch * 2};
+  cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline int pick_bn(int N) { return N >= BN_MAX ? BN_MAX : (int)((N + 63) / 64 * 64); }
+
+inline void finish_problem(Problem& p, int splits_wanted) {
+  p.bn = pick_bn(p.N);
+  p.tiles_m = (p.M + BM - 1) / BM;
+  p.tiles_n = (p.N + p.bn - 1) / p.bn;
+  p.ksteps_total = (p.K + BK - 1) / BK;
+  int s = splits_wanted < 1 ? 1 : splits_wanted;
+  if (s > p.ksteps_total) s = p.ksteps_total;
+  p.ksteps_per_split = (p.ksteps_total + s - 1) / s;
+  p.splits = (p.ksteps_total + p.ksteps_per_split - 1) / p.ksteps_per_split;
+}
+
+// Number of token splits of Gc = Z^T dY: enough work items to occupy the SMs, at most 32.
+inline int plan_gc_splits(int64_t tokens, int r, int m) {
+  const int tiles = ((r + BM - 1) / BM) * ((m + pick_bn(m) - 1) / pick_bn(m));
+  const int ksteps = (int)((tokens + BK - 1) / BK);
+  if (ksteps < 1) return 1;
+  int s = NUM_SMS / tiles;
+  if (s < 1) s = 1;
+  if (s > 32) s = 32;
+  if (s > ksteps) s = ksteps;
+  const int per = (ksteps + s - 1) / s;
+  return (ksteps + per - 1) / per;
+}
+
+inline size_t gc_workspace_bytes(int64_t tokens, int r, int m) {
+  const int s = plan_gc_splits(tokens, r, m);
+  return s > 1 ? (size_t)s * r * m * sizeof(float) : 0;
+}
+
+inline compact_status_t launch(const LaunchInfo& li, Params& prm) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(compact_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
+      cudaGetLastError();
+      return COMPACT_ERR_CUDA;
+    }
+    attr_set = true;
+  }
+  int t = 0;
+  for (int i = 0; i < prm.num_problems; ++i) {
+    prm.prob[i].tile_begin = t;
+    t += prm.prob[i].tiles_m * prm.prob[i].tiles_n * prm.prob[i].splits;
+  }
+  prm.total_tiles = t;
+  prm.status = li.status;
+  const int grid = t < NUM_SMS ? t : NUM_SMS;
+  const int threads = prm.has_generated ? THREADS_GEN : THREADS_BASE;
+  compact_gemm_kernel<<<grid, threads, SMEM_BYTES, li.stream>>>(prm);
+  (*li.launches)++;
+  return cudaGetLastError() == cudaSuccess ? COMPACT_OK : COMPACT_ERR_CUDA;
+}
+
+inline bool tc_shape_ok(int64_t tokens, int n, int m) { return tokens >= 1 && n % 8 == 0 && m % 8 == 0; }
+
+// Algorithm 1: problem 0 = Z = X P (generated B operand; longest tiles go first), problem 1 = Y = X W.
+inline compact_status_t forward(const LaunchInfo& li, const ProjectionParams& pp, int64_t tokens, int m,
+                                const __nv_bfloat16* X, int64_t ldx, const __nv_bfloat16* W, int64_t ldw,
+                                __nv_bfloat16* Y, int64_t ldy, __nv_bfloat16* Z, int64_t ldz, int zcols) {
+  const int n = pp.n;
+  if (!tc_shape_ok(tokens, n, m)) return COMPACT_ERR_SHAPE;
+  if (!li.status) return COMPACT_ERR_CUDA;
+  Params prm;
+  memset(&prm, 0, sizeof(prm));
+  prm.pp = pp;
+  prm.num_problems = 2;
+  prm.has_generated = 1;
+  Problem& pz = prm.prob[0];
+  pz.M = (int)tokens; pz.N = zcols; pz.K = n;
+  pz.a_mode = TMA_KMAJOR; pz.b_mode = GENERATED; pz.epi_mode = EPI_BF16;
+  pz.out = Z; pz.ld_out = ldz;
+  finish_problem(pz, 1);
+  Problem& py = prm.prob[1];
+  py.M = (int)tokens; py.N = m; py.K = n;
+  py.a_mode = TMA_KMAJOR; py.b_mode = TMA_MNMAJOR; py.epi_mode = EPI_BF16;
+  py.out = Y; py.ld_out = ldy;
+  finish_problem(py, 1);
+  if (!make_map(&prm.tmA[0], X, n, tokens, ldx, BK, BM)) return COMPACT_ERR_CUDA;
+  prm.tmA[1] = prm.tmA[0];
+  if (!make_map(&prm.tmB[1], W, m, n, ldw, 64, BK)) return COMPACT_ERR_CUDA;
+  prm.tmB[0] = prm.tmB[1];   // unused by the generated operand
+  return launch(li, prm);
+}
+
+// Algorithm 2: problem 0 = Gc = Z^T dY (both operands MN-major, split over tokens), problem 1 = dX = dY W^T.
+inline compact_status_t backward(const LaunchInfo& li, int64_t tokens, int n, int m, int r, int zcols,
+                                 const __nv_bfloat16* dY, int64_t lddy, const __nv_bfloat16* Z, int64_t ldz,
+                                 const __nv_bfloat16* W, int64_t ldw, __nv_bfloat16* dX, int64_t lddx, float* Gc,
+                                 int64_t ldg, int accumulate, void* workspace, size_t workspace_bytes) {
+  if (!tc_shape_ok(tokens, n, m)) return COMPACT_ERR_SHAPE;
+  if (!li.status) return COMPACT_ERR_CUDA;
+  Params prm;
+  memset(&prm, 0, sizeof(prm));
+  prm.num_problems = dX ? 2 : 1;
+  prm.has_generated = 0;
+  const int splits = plan_gc_splits(tokens, r, m);
+  if (splits > 1 && workspace_bytes < (size_t)splits * r * m * sizeof(float)) return COMPACT_ERR_WORKSPACE;
+  Problem& pg = prm.prob[0];
+  pg.M = r; pg.N = m; pg.K = (int)tokens;
+  pg.a_mode = TMA_MNMAJOR; pg.b_mode = TMA_MNMAJOR; pg.epi_mode = EPI_F32;
+  finish_problem(pg, splits);
+  if (pg.splits > 1) {
+    pg.out = workspace; pg.ld_out = m; pg.split_stride = (long long)r * m; pg.accumulate = 0;
+  } else {
+    pg.out = Gc; pg.ld_out = ldg; pg.split_stride = 0; pg.accumulate = accumulate;
+  }
+  if (!make_map(&prm.tmA[0], Z, zcols, tokens, ldz, 64, BK)) return COMPACT_ERR_CUDA;
+  if (!make_map(&prm.tmB[0], dY, m, tokens, lddy, 64, BK)) return COMPACT_ERR_CUDA;
+  if (dX) {
+    Problem& px = prm.prob[1];
+    px.M = (int)tokens; px.N = n; px.K = m;
+    px.a_mode = TMA_KMAJOR; px.b_mode = TMA_KMAJOR; px.epi_mode = EPI_BF16;
+    px.out = dX; px.ld_out = lddx;
+    finish_problem(px, 1);
+    if (!make_map(&prm.tmA[1], dY, m, tokens, lddy, BK, BM)) return COMPACT_ERR_CUDA;
+    if (!make_map(&prm.tmB[1], W, m, n, ldw, BK, px.bn)) return COMPACT_ERR_CUDA;
+  }
+  compact_status_t s = launch(li, prm);
+  if (s != COMPACT_OK) return s;
+  if (pg.splits > 1) {
+    const long long cnt = (long long)r * (m / 4);
+    reduce_partials_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, li.stream>>>(
+        (const float*)workspace, (long long)r * m, pg.splits, Gc, ldg, r, m, accumulate);
+    (*li.launches)++;
+    if (cudaGetLastError() != cudaSuccess) return COMPACT_ERR_CUDA;
+  }
+  return COMPACT_OK;
+}
+
+// Algorithm 3: Adam moments -> N (bf16 scratch), then W <- W - scale * P N with P generated as the A operand.
+inline compact_status_t update(const LaunchInfo& li, const ProjectionParams& pp, const simt::AdamScalars& as, int n, int m,
+                               int r, __nv_bfloat16* W, int64_t ldw, const float* Gc, int64_t ldg, float* M, float* V,
+                               float scale, void* workspace, size_t workspace_bytes) {
+  if (!tc_shape_ok(1, n, m)) return COMPACT_ERR_SHAPE;
+  if (!li.status) return COMPACT_ERR_CUDA;
+  if (workspace_bytes < (size_t)r * m * 2) return COMPACT_ERR_WORKSPACE;
+  __nv_bfloat16* Nbuf = (__nv_bfloat16*)workspace;
+  const long long cnt = (long long)r * (m / 4);
+  adam_moments_bf16_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, li.stream>>>(Gc, ldg, M, V, Nbuf, r, m, as);
+  (*li.launches)++;
+  if (cudaGetLastError() != cudaSuccess) return COMPACT_ERR_CUDA;
+  Params prm;
+  memset(&prm, 0, sizeof(prm));
+  prm.pp = pp;
+  prm.num_problems = 1;
+  prm.has_generated = 1;
+  Problem& pu = prm.prob[0];
+  pu.M = n; pu.N = m; pu.K = r;
+  pu.a_mode = GENERATED; pu.b_mode = TMA_MNMAJOR; pu.epi_mode = EPI_UPDATE_W;
+  pu.out = W; pu.ld_out = ldw; pu.scale = scale;
+  finish_problem(pu, 1);
+  if (!make_map(&prm.tmB[0], Nbuf, m, r, m, 64, BK)) return COMPACT_ERR_CUDA;
+  prm.tmA[0] = prm.tmB[0];
+  return launch(li, prm);
 }
 
 }  // namespace tc
