@@ -6,7 +6,7 @@ import subprocess
 
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
-LIB_PATH = os.path.join(PKG_DIR, "libcompact.so")
+LIB_PATH = os.environ.get("COMPACT_LIB", os.path.join(PKG_DIR, "libcompact.so"))
 SOURCES = ["compact_api.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -66,6 +66,7 @@ ProjectionParams make_pp(const compact_layer_t* L, uint32_t epoch) {
   pp.n = L->cfg.n;
   pp.r = L->cfg.r;
   pp.inv_sqrt_r = (float)(1.0 / sqrt((double)L->cfg.r));
+  pp.neg2ln2_over_r = (float)(-2.0 * 0.6931471805599453 / (double)L->cfg.r);
   return pp;
 }
 
@@ -373,6 +374,17 @@ int compact_set_kernel_family(int family) {
 }
 
 uint64_t compact_kernel_launch_count(void) { return g_launches.load(); }
+
+#ifdef COMPACT_PROFILE
+// Profiling build only: cumulative clocks of the MMA-issuing threads
+// [wait accumulator, wait B, wait A, issue, total]; reading clears them.
+void compact_debug_profile(unsigned long long* out) {
+  cudaDeviceSynchronize();
+  cudaMemcpyFromSymbol(out, tc::g_prof, sizeof(unsigned long long) * 8);
+  unsigned long long z[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  cudaMemcpyToSymbol(tc::g_prof, z, sizeof(z));
+}
+#endif
 
 const char* compact_status_string(compact_status_t s) {
   switch (s) {

@@ -30,12 +30,12 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
                                                const PhiloxKey& key) {
 #pragma unroll
   for (int i = 0; i < 10; ++i) {
-    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
-    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
-    c0 = hi1 ^ c1 ^ key.k0[i];
-    c1 = lo1;
-    c2 = hi0 ^ c3 ^ key.k1[i];
-    c3 = lo0;
+    const uint64_t p0 = (uint64_t)0xD2511F53u * c0;   // one wide multiply each
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+    c0 = (uint32_t)(p1 >> 32) ^ c1 ^ key.k0[i];
+    c1 = (uint32_t)p1;
+    c2 = (uint32_t)(p0 >> 32) ^ c3 ^ key.k1[i];
+    c3 = (uint32_t)p0;
   }
   return make_uint4(c0, c1, c2, c3);
 }
@@ -55,6 +55,33 @@ __device__ __forceinline__ float4 gaussian4(uint4 x) {
   return make_float4(ra * ca, ra * sa, rb * cb, rb * sb);
 }
 
+// Same four values already scaled by 1/sqrt(r), built from the hardware
+// approximations (lg2/sqrt/sin/cos) and bit tricks instead of int->float
+// conversions.  Used where P is rounded to bf16 anyway.
+//   u1 = ((x>>9)+0.5) 2^-23 = float(1.m) - (1 - 2^-24)            (exact)
+//   2 pi u2 = pi*[x>>31] + pi * ((x>>8) & 0x7fffff) 2^-23: the top bit of u2
+//   adds pi to the angle, which flips the sign of both cos and sin.
+// neg2ln2_over_r = -2 ln(2) / r, so sqrt(lg2(u1) * neg2ln2_over_r) = sqrt(-2 ln u1) / sqrt(r).
+__device__ __forceinline__ float sqrt_approx(float x) {
+  float y;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ void box_muller_fast(uint32_t xa, uint32_t xb, float neg2ln2_over_r, float& c, float& s) {
+  const float u1 = __uint_as_float((xa >> 9) | 0x3F800000u) - 0.99999994f;
+  const float rad = sqrt_approx(fmaxf(__log2f(u1) * neg2ln2_over_r, 0.0f));
+  const float th = (__uint_as_float(((xb >> 8) & 0x007FFFFFu) | 0x3F800000u) - 1.0f) * 3.14159265358979f;
+  const float rs = __uint_as_float(__float_as_uint(rad) ^ (xb & 0x80000000u));
+  c = rs * __cosf(th);
+  s = rs * __sinf(th);
+}
+__device__ __forceinline__ float4 gaussian4_fast_scaled(uint4 x, float neg2ln2_over_r) {
+  float4 g;
+  box_muller_fast(x.x, x.y, neg2ln2_over_r, g.x, g.y);
+  box_muller_fast(x.z, x.w, neg2ln2_over_r, g.z, g.w);
+  return g;
+}
+
 struct ProjectionParams {
   PhiloxKey key;
   uint32_t layer_id;
@@ -62,21 +89,33 @@ struct ProjectionParams {
   int32_t n;
   int32_t r;
   float inv_sqrt_r;
+  float neg2ln2_over_r;
 };
 
 // P[i, 4q .. 4q+3] in fp32; columns >= r are zero, rows >= n are zero.
+// kFast selects the approximate Box-Muller (bf16 layers); fp32 layers use the accurate one.
+template <bool kFast>
 __device__ __forceinline__ float4 projection4(const ProjectionParams& pp, int i, int q) {
   if (i >= pp.n || 4 * q >= pp.r) return make_float4(0.f, 0.f, 0.f, 0.f);
-  float4 g = gaussian4(philox4x32_10((uint32_t)q, (uint32_t)i, pp.layer_id, pp.epoch, pp.key));
-  g.x *= pp.inv_sqrt_r;
-  g.y = (4 * q + 1 < pp.r) ? g.y * pp.inv_sqrt_r : 0.f;
-  g.z = (4 * q + 2 < pp.r) ? g.z * pp.inv_sqrt_r : 0.f;
-  g.w = (4 * q + 3 < pp.r) ? g.w * pp.inv_sqrt_r : 0.f;
+  const uint4 x = philox4x32_10((uint32_t)q, (uint32_t)i, pp.layer_id, pp.epoch, pp.key);
+  float4 g;
+  if (kFast) {
+    g = gaussian4_fast_scaled(x, pp.neg2ln2_over_r);
+  } else {
+    g = gaussian4(x);
+    g.x *= pp.inv_sqrt_r; g.y *= pp.inv_sqrt_r; g.z *= pp.inv_sqrt_r; g.w *= pp.inv_sqrt_r;
+  }
+  if (4 * q + 4 > pp.r) {
+    if (4 * q + 1 >= pp.r) g.y = 0.f;
+    if (4 * q + 2 >= pp.r) g.z = 0.f;
+    if (4 * q + 3 >= pp.r) g.w = 0.f;
+  }
   return g;
 }
 
+template <bool kFast>
 __device__ __forceinline__ float projection1(const ProjectionParams& pp, int i, int j) {
-  const float4 g = projection4(pp, i, j >> 2);
+  const float4 g = projection4<kFast>(pp, i, j >> 2);
   const int l = j & 3;
   return l == 0 ? g.x : (l == 1 ? g.y : (l == 2 ? g.z : g.w));
 }

@@ -35,7 +35,7 @@ template <bool kRoundBf16, bool kAsB> struct GeneratedP {
   ProjectionParams pp;
   __device__ __forceinline__ float operator()(int a, int b) const {
     const int i = kAsB ? b : a, j = kAsB ? a : b;
-    float v = projection1(pp, i, j);
+    float v = projection1<kRoundBf16>(pp, i, j);
     if (kRoundBf16) v = __bfloat162float(__float2bfloat16_rn(v));
     return v;
   }
@@ -157,7 +157,7 @@ __global__ void debug_projection_kernel(ProjectionParams pp, T* P) {
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (int64_t)pp.n * groups) return;
   const int i = (int)(idx / groups), q = (int)(idx % groups);
-  const float4 g = projection4(pp, i, q);
+  const float4 g = projection4<sizeof(T) == 2>(pp, i, q);
   const float v[4] = {g.x, g.y, g.z, g.w};
   for (int l = 0; l < 4; ++l)
     if (4 * q + l < pp.r) P[(int64_t)i * pp.r + 4 * q + l] = simt::from_f32<T>(v[l]);

@@ -29,26 +29,46 @@ struct LaunchInfo {
 
 constexpr int BM = 128;              // rows of one accumulator (TMEM lanes)
 constexpr int BK = 64;               // K elements per pipeline stage (one 128-byte swizzle row)
-constexpr int BN_MAX = 256;          // widest accumulator (TMEM columns)
-constexpr int STAGES = 4;
+constexpr int BN_MAX = 256;          // columns of one accumulator slot (TMEM has two slots)
+#ifndef CFG_STAGES_A
+#define CFG_STAGES_A 6
+#endif
+#ifndef CFG_STAGES_B
+#define CFG_STAGES_B 4
+#endif
+constexpr int STAGES_A = CFG_STAGES_A;          // ring of A tiles (128 x 64 bf16)
+constexpr int STAGES_B = CFG_STAGES_B;          // ring of B tiles (up to 256 x 64 bf16)
 constexpr int A_BYTES = BM * BK * 2;
 constexpr int B_BYTES = BN_MAX * BK * 2;
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int NUM_GEN_WARPS = 8;
+constexpr int RING_BYTES = STAGES_A * A_BYTES + STAGES_B * B_BYTES;
+constexpr int NUM_GEN_WARPS = 16;
 constexpr int THREADS_BASE = 192;    // producer warp, MMA warp, four epilogue warps
 constexpr int THREADS_GEN = THREADS_BASE + 32 * NUM_GEN_WARPS;
-constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + 256;
+constexpr int SMEM_BYTES = 1024 + RING_BYTES + 256;
 constexpr int NUM_SMS = 148;
+constexpr int MAX_SUB = 4;           // row blocks of 128 that share one generated B tile
 
 enum OperandMode { TMA_KMAJOR = 0, TMA_MNMAJOR = 1, GENERATED = 2 };
 enum EpiMode { EPI_BF16 = 0, EPI_F32 = 1, EPI_UPDATE_W = 2 };
+enum GenRing { GEN_NONE = 0, GEN_A = 1, GEN_B = 2 };
 
 constexpr unsigned int STATUS_TIMEOUT = 1u;
+#ifdef COMPACT_PROFILE
+__device__ unsigned long long g_prof[8];
+#define PROF_T() clock64()
+#define PROF_ADD(i, t0) prof[i] += clock64() - (t0)
+#else
+#define PROF_T() 0
+#define PROF_ADD(i, t0)
+#endif
 
+// One GEMM inside a launch.  An item is nsub row blocks of 128 rows by bn columns;
+// its nsub accumulators sit side by side in TMEM (nsub * bn <= 512 columns).
 struct Problem {
   int M, N, K;
   int tiles_m, tiles_n, splits, ksteps_total, ksteps_per_split;
   int bn;
+  int nsub;
   int a_mode, b_mode, epi_mode;
   int accumulate;
   int tile_begin;
@@ -64,7 +84,7 @@ struct alignas(64) Params {
   Problem prob[2];
   int num_problems;
   int total_tiles;
-  int has_generated;
+  int gen_ring;
   ProjectionParams pp;
   unsigned int* status;
 };
@@ -96,6 +116,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait: gives up after about a second, records it, and lets the CTA drain.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned int* status) {
+  if (mbar_try_wait(bar, parity)) return true;
   for (uint32_t it = 0; it < 8000000u; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if (it > 128) {
@@ -130,12 +151,16 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+// Descriptors travel as (lo, hi) 32-bit halves so that stepping along K is one 32-bit add.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                          uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %2};\n\t"
+      "mov.b64 db, {%3, %4};\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
@@ -156,16 +181,14 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-// Shared-memory matrix descriptor: 128-byte swizzle, 8-row groups 1024 bytes apart.
-// lbo_bytes: distance between 64-element blocks along M/N (MN-major operands only).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes) {
-  uint64_t d = 0;
-  d |= (uint64_t)((addr >> 4) & 0x3FFF);
-  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
-  d |= (uint64_t)((1024u >> 4) & 0x3FFF) << 32;
-  d |= (uint64_t)1 << 46;   // descriptor version of sm_100
-  d |= (uint64_t)2 << 61;   // 128-byte swizzle
-  return d;
+// Shared-memory matrix descriptor (64 bits), 128-byte swizzle, 8-row groups 1024 bytes apart:
+//   lo: start address >> 4 in bits [0,14), leading byte offset >> 4 in bits [16,30)
+//   hi: stride byte offset >> 4 in bits [0,14), descriptor version 1 in bit 14, swizzle mode 2 in bits [29,32)
+// The leading byte offset is the distance between 64-element blocks along M/N of an
+// MN-major operand (8192 here); K-major operands do not use it.
+constexpr uint32_t DESC_HI = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr, bool mn_major) {
+  return ((addr >> 4) & 0x3FFFu) | ((mn_major ? (8192u >> 4) : 1u) << 16);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -177,13 +200,13 @@ __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w &
 
 // Eight consecutive entries P[i, j0 .. j0+7] (j0 a multiple of 8) as packed bf16.
 __device__ __forceinline__ uint4 projection8_bf16(const ProjectionParams& pp, int i, int j0) {
-  const float4 a = projection4(pp, i, j0 >> 2);
-  const float4 b = projection4(pp, i, (j0 >> 2) + 1);
+  const float4 a = projection4<true>(pp, i, j0 >> 2);
+  const float4 b = projection4<true>(pp, i, (j0 >> 2) + 1);
   return make_uint4(pack_bf16x2(a.x, a.y), pack_bf16x2(a.z, a.w), pack_bf16x2(b.x, b.y), pack_bf16x2(b.z, b.w));
 }
 
 struct TileCoord {
-  int prob, m0, n0, k_begin, k_end, split;
+  int prob, m0, n0, k_begin, k_end, split, nsub;
 };
 
 __device__ __forceinline__ TileCoord decode_tile(const Params& prm, int tile) {
@@ -195,10 +218,11 @@ __device__ __forceinline__ TileCoord decode_tile(const Params& prm, int tile) {
   local /= p.tiles_n;
   const int mb = local % p.tiles_m;
   t.split = local / p.tiles_m;
-  t.m0 = mb * BM;
+  t.m0 = mb * BM * p.nsub;
   t.n0 = nb * p.bn;
   t.k_begin = t.split * p.ksteps_per_split;
   t.k_end = min(p.ksteps_total, t.k_begin + p.ksteps_per_split);
+  t.nsub = min(p.nsub, (p.M - t.m0 + BM - 1) / BM);   // row blocks that hold at least one valid row
   return t;
 }
 
@@ -209,13 +233,16 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));   // generic pointer to the aligned base
-  const uint32_t bars = smem_base + STAGES * STAGE_BYTES;
-  // barrier slots (8 bytes each): full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2]
-  auto full_bar = [&](int s) { return bars + 8u * s; };
-  auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };
-  auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };
-  auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };
-  uint8_t* tail = smem_gen + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 4);
+  const uint32_t ringA = smem_base, ringB = smem_base + STAGES_A * A_BYTES;
+  const uint32_t bars = smem_base + RING_BYTES;
+  // barrier slots (8 bytes each)
+  auto fullA = [&](int s) { return bars + 8u * s; };
+  auto emptyA = [&](int s) { return bars + 8u * (STAGES_A + s); };
+  auto fullB = [&](int s) { return bars + 8u * (2 * STAGES_A + s); };
+  auto emptyB = [&](int s) { return bars + 8u * (2 * STAGES_A + STAGES_B + s); };
+  auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES_A + 2 * STAGES_B + a); };
+  auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES_A + 2 * STAGES_B + 2 + a); };
+  uint8_t* tail = smem_gen + RING_BYTES + 8 * (2 * STAGES_A + 2 * STAGES_B + 4);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 8);
 
@@ -223,9 +250,13 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
   const int lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) {
-      mbar_init(full_bar(s), 1 + (prm.has_generated ? NUM_GEN_WARPS : 0));
-      mbar_init(empty_bar(s), 1);
+    for (int s = 0; s < STAGES_A; ++s) {
+      mbar_init(fullA(s), 1 + (prm.gen_ring == GEN_A ? NUM_GEN_WARPS : 0));
+      mbar_init(emptyA(s), 1);
+    }
+    for (int s = 0; s < STAGES_B; ++s) {
+      mbar_init(fullB(s), 1 + (prm.gen_ring == GEN_B ? NUM_GEN_WARPS : 0));
+      mbar_init(emptyB(s), 1);
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);
@@ -247,42 +278,64 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
+      int sa = 0, sb = 0;
+      uint32_t pha = 0, phb = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < prm.total_tiles && ok; tile += gridDim.x) {
         const TileCoord t = decode_tile(prm, tile);
         const Problem& p = prm.prob[t.prob];
         const CUtensorMap* mapA = &prm.tmA[t.prob];
         const CUtensorMap* mapB = &prm.tmB[t.prob];
-        const uint32_t bytes = (p.a_mode != GENERATED ? A_BYTES : 0) + (p.b_mode != GENERATED ? p.bn * BK * 2 : 0);
-        for (int ks = t.k_begin; ks < t.k_end; ++ks) {
-          if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1, abort_flag, prm.status))) break;
-          const uint32_t sa = smem_base + stage * STAGE_BYTES, sb = sa + A_BYTES;
-          const uint32_t fb = full_bar(stage);
-          mbar_arrive_expect_tx(fb, bytes);
+        for (int ks = t.k_begin; ks < t.k_end && ok; ++ks) {
           const int k0 = ks * BK;
-          if (p.a_mode == TMA_KMAJOR) {
-            tma_load_2d(sa, mapA, fb, k0, t.m0);
-          } else if (p.a_mode == TMA_MNMAJOR) {
-            tma_load_2d(sa, mapA, fb, t.m0, k0);
-            tma_load_2d(sa + 8192, mapA, fb, t.m0 + 64, k0);
+          // B tile of this k-step (shared by all row blocks of the item)
+          if (!(ok = mbar_wait(emptyB(sb), phb ^ 1, abort_flag, prm.status))) break;
+          {
+            const uint32_t dst = ringB + sb * B_BYTES, fb = fullB(sb);
+            if (p.b_mode == GENERATED) {
+              mbar_arrive(fb);
+            } else {
+              mbar_arrive_expect_tx(fb, p.bn * BK * 2);
+              if (p.b_mode == TMA_KMAJOR) {
+                tma_load_2d(dst, mapB, fb, k0, t.n0);
+              } else {
+                for (int b = 0; b < p.bn / 64; ++b) tma_load_2d(dst + b * 8192, mapB, fb, t.n0 + 64 * b, k0);
+              }
+            }
+            if (++sb == STAGES_B) { sb = 0; phb ^= 1; }
           }
-          if (p.b_mode == TMA_KMAJOR) {
-            tma_load_2d(sb, mapB, fb, k0, t.n0);
-          } else if (p.b_mode == TMA_MNMAJOR) {
-            for (int b = 0; b < p.bn / 64; ++b) tma_load_2d(sb + b * 8192, mapB, fb, t.n0 + 64 * b, k0);
+          for (int mi = 0; mi < t.nsub; ++mi) {
+            if (!(ok = mbar_wait(emptyA(sa), pha ^ 1, abort_flag, prm.status))) break;
+            const uint32_t dst = ringA + sa * A_BYTES, fa = fullA(sa);
+            const int m0 = t.m0 + mi * BM;
+            if (p.a_mode == GENERATED) {
+              mbar_arrive(fa);
+            } else {
+              mbar_arrive_expect_tx(fa, A_BYTES);
+              if (p.a_mode == TMA_KMAJOR) {
+                tma_load_2d(dst, mapA, fa, k0, m0);
+              } else {
+                tma_load_2d(dst, mapA, fa, m0, k0);
+                tma_load_2d(dst + 8192, mapA, fa, m0 + 64, k0);
+              }
+            }
+            if (++sa == STAGES_A) { sa = 0; pha ^= 1; }
           }
-          if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
       }
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ---------------------------------
     if (lane == 0) {
-      int stage = 0, acc = 0;
-      uint32_t phase = 0, acc_phase = 0;
+      int sa = 0, sb = 0, acc = 0;
+      uint32_t pha = 0, phb = 0, acc_phase = 0;
       bool ok = true;
+#ifdef COMPACT_PROFILE
+      unsigned long long prof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+      const long long t_start = clock64();
+      unsigned long long ns0;
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(ns0));
+#endif
       for (int tile = blockIdx.x; tile < prm.total_tiles && ok; tile += gridDim.x) {
         const TileCoord t = decode_tile(prm, tile);
         const Problem& p = prm.prob[t.prob];
@@ -290,26 +343,56 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const bool b_mn = p.b_mode != TMA_KMAJOR;          // generated B tiles are written MN-major
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
                                ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-        if (!(ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag, prm.status))) break;
+        const int slots = (p.nsub * p.bn + BN_MAX - 1) / BN_MAX;   // accumulator slots this item occupies
+        const int acc0 = acc;
+        const long long tp0 = PROF_T();
+        for (int sl = 0; sl < slots && ok; ++sl) {
+          ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag, prm.status);
+          if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+        }
+        PROF_ADD(0, tp0);
+        if (!ok) break;
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * BN_MAX;
-        for (int ks = t.k_begin; ks < t.k_end; ++ks) {
-          if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag, prm.status))) break;
-          tc_fence_after();
-          const uint32_t sa = smem_base + stage * STAGE_BYTES, sb = sa + A_BYTES;
-#pragma unroll
-          for (int k4 = 0; k4 < BK / 16; ++k4) {
-            const uint64_t adesc = a_mn ? smem_desc(sa + k4 * 2048, 8192) : smem_desc(sa + k4 * 32, 16);
-            const uint64_t bdesc = b_mn ? smem_desc(sb + k4 * 2048, 8192) : smem_desc(sb + k4 * 32, 16);
-            umma_bf16(d_tmem, adesc, bdesc, idesc, (ks > t.k_begin || k4 > 0) ? 1u : 0u);
+        const uint32_t d_base = tmem_base + acc0 * BN_MAX;
+        // one UMMA consumes K = 16: 32 bytes along a K-major row, or two 8-row groups (2048 bytes) MN-major
+        const uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4), b_step = b_mn ? (2048u >> 4) : (32u >> 4);
+        const int nsub = t.nsub, bn = p.bn;
+        for (int ks = t.k_begin; ks < t.k_end && ok; ++ks) {
+          const long long tp1 = PROF_T();
+          if (!(ok = mbar_wait(fullB(sb), phb, abort_flag, prm.status))) break;
+          PROF_ADD(1, tp1);
+          const uint32_t b_lo = desc_lo(ringB + sb * B_BYTES, b_mn);
+          const uint32_t first = ks > t.k_begin ? 1u : 0u;
+          for (int mi = 0; mi < nsub; ++mi) {
+            const long long tp2 = PROF_T();
+            if (!(ok = mbar_wait(fullA(sa), pha, abort_flag, prm.status))) break;
+            PROF_ADD(2, tp2);
+            const long long tp3 = PROF_T();
+            tc_fence_after();
+            const uint32_t a_lo = desc_lo(ringA + sa * A_BYTES, a_mn);
+            const uint32_t d = d_base + mi * bn;
+            umma_bf16(d, a_lo, DESC_HI, b_lo, DESC_HI, idesc, first);
+            umma_bf16(d, a_lo + a_step, DESC_HI, b_lo + b_step, DESC_HI, idesc, 1u);
+            umma_bf16(d, a_lo + 2 * a_step, DESC_HI, b_lo + 2 * b_step, DESC_HI, idesc, 1u);
+            umma_bf16(d, a_lo + 3 * a_step, DESC_HI, b_lo + 3 * b_step, DESC_HI, idesc, 1u);
+            umma_commit(emptyA(sa));
+            PROF_ADD(3, tp3);
+            if (++sa == STAGES_A) { sa = 0; pha ^= 1; }
           }
-          umma_commit(empty_bar(stage));
-          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+          if (!ok) break;
+          umma_commit(emptyB(sb));
+          if (++sb == STAGES_B) { sb = 0; phb ^= 1; }
         }
         if (!ok) break;
-        umma_commit(tfull_bar(acc));
-        if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+        for (int sl = 0; sl < slots; ++sl) umma_commit(tfull_bar((acc0 + sl) & 1));
       }
+#ifdef COMPACT_PROFILE
+      prof[4] = clock64() - t_start;
+      unsigned long long ns1;
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(ns1));
+      prof[5] = ns1 - ns0;
+      for (int i = 0; i < 6; ++i) atomicAdd(&g_prof[i], prof[i]);
+#endif
     }
   } else if (warp < 6) {
     // ------------------------------ epilogue ------------------------------------
@@ -320,102 +403,127 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
     for (int tile = blockIdx.x; tile < prm.total_tiles && ok; tile += gridDim.x) {
       const TileCoord t = decode_tile(prm, tile);
       const Problem& p = prm.prob[t.prob];
-      if (!(ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, prm.status))) break;
-      tc_fence_after();
-      const int row = t.m0 + q * 32 + lane;
-      const bool row_ok = row < p.M;
-      for (int c0 = 0; c0 < p.bn; c0 += 32) {
-        const int col = t.n0 + c0;
-        if (col >= p.N) break;
-        uint32_t v[32];
-        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN_MAX + c0, v);
-        tmem_ld_wait();
-        if (!row_ok) continue;
-        if (p.epi_mode == EPI_BF16) {
-          __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + (long long)row * p.ld_out + col;
+      const int slots = (p.nsub * p.bn + BN_MAX - 1) / BN_MAX;
+      const int sub_per_slot = BN_MAX / p.bn > p.nsub ? p.nsub : BN_MAX / p.bn;
+      for (int sl = 0; sl < slots && ok; ++sl) {
+        if (!(ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, prm.status))) break;
+        tc_fence_after();
+        for (int su = 0; su < sub_per_slot; ++su) {
+          const int mi = sl * sub_per_slot + su;
+          if (mi >= t.nsub) break;
+          const int row = t.m0 + mi * BM + q * 32 + lane;
+          const bool row_ok = row < p.M;
+          for (int c0 = 0; c0 < p.bn; c0 += 32) {
+            const int col = t.n0 + c0;
+            if (col >= p.N) break;
+            uint32_t v[32];
+            tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN_MAX + su * p.bn + c0, v);
+            tmem_ld_wait();
+            if (!row_ok) continue;
+            if (p.epi_mode == EPI_BF16) {
+              __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + (long long)row * p.ld_out + col;
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            if (col + g * 8 + 8 <= p.N) {
-              uint4 o;
-              o.x = pack_bf16x2(__uint_as_float(v[g * 8 + 0]), __uint_as_float(v[g * 8 + 1]));
-              o.y = pack_bf16x2(__uint_as_float(v[g * 8 + 2]), __uint_as_float(v[g * 8 + 3]));
-              o.z = pack_bf16x2(__uint_as_float(v[g * 8 + 4]), __uint_as_float(v[g * 8 + 5]));
-              o.w = pack_bf16x2(__uint_as_float(v[g * 8 + 6]), __uint_as_float(v[g * 8 + 7]));
-              *reinterpret_cast<uint4*>(dst + g * 8) = o;
-            }
-          }
-        } else if (p.epi_mode == EPI_F32) {
-          float* dst = reinterpret_cast<float*>(p.out) + (long long)t.split * p.split_stride + (long long)row * p.ld_out + col;
-#pragma unroll
-          for (int g = 0; g < 8; ++g) {
-            if (col + g * 4 + 4 <= p.N) {
-              float4 o = make_float4(__uint_as_float(v[g * 4 + 0]), __uint_as_float(v[g * 4 + 1]),
-                                     __uint_as_float(v[g * 4 + 2]), __uint_as_float(v[g * 4 + 3]));
-              if (p.accumulate) {
-                const float4 old = *reinterpret_cast<const float4*>(dst + g * 4);
-                o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+              for (int g = 0; g < 4; ++g) {
+                if (col + g * 8 + 8 <= p.N) {
+                  uint4 o;
+                  o.x = pack_bf16x2(__uint_as_float(v[g * 8 + 0]), __uint_as_float(v[g * 8 + 1]));
+                  o.y = pack_bf16x2(__uint_as_float(v[g * 8 + 2]), __uint_as_float(v[g * 8 + 3]));
+                  o.z = pack_bf16x2(__uint_as_float(v[g * 8 + 4]), __uint_as_float(v[g * 8 + 5]));
+                  o.w = pack_bf16x2(__uint_as_float(v[g * 8 + 6]), __uint_as_float(v[g * 8 + 7]));
+                  *reinterpret_cast<uint4*>(dst + g * 8) = o;
+                }
               }
-              *reinterpret_cast<float4*>(dst + g * 4) = o;
-            }
-          }
-        } else {
-          // Algorithm 3 line 9: W <- W - (eta alpha) (P N), one rounding of the result
-          __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + (long long)row * p.ld_out + col;
+            } else if (p.epi_mode == EPI_F32) {
+              float* dst = reinterpret_cast<float*>(p.out) + (long long)t.split * p.split_stride + (long long)row * p.ld_out + col;
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            if (col + g * 8 + 8 <= p.N) {
-              uint4 w = *reinterpret_cast<const uint4*>(dst + g * 8);
-              const float s = -p.scale;
-              w.x = pack_bf16x2(fmaf(s, __uint_as_float(v[g * 8 + 0]), bf16lo(w.x)), fmaf(s, __uint_as_float(v[g * 8 + 1]), bf16hi(w.x)));
-              w.y = pack_bf16x2(fmaf(s, __uint_as_float(v[g * 8 + 2]), bf16lo(w.y)), fmaf(s, __uint_as_float(v[g * 8 + 3]), bf16hi(w.y)));
-              w.z = pack_bf16x2(fmaf(s, __uint_as_float(v[g * 8 + 4]), bf16lo(w.z)), fmaf(s, __uint_as_float(v[g * 8 + 5]), bf16hi(w.z)));
-              w.w = pack_bf16x2(fmaf(s, __uint_as_float(v[g * 8 + 6]), bf16lo(w.w)), fmaf(s, __uint_as_float(v[g * 8 + 7]), bf16hi(w.w)));
-              *reinterpret_cast<uint4*>(dst + g * 8) = w;
+              for (int g = 0; g < 8; ++g) {
+                if (col + g * 4 + 4 <= p.N) {
+                  float4 o = make_float4(__uint_as_float(v[g * 4 + 0]), __uint_as_float(v[g * 4 + 1]),
+                                         __uint_as_float(v[g * 4 + 2]), __uint_as_float(v[g * 4 + 3]));
+                  if (p.accumulate) {
+                    const float4 old = *reinterpret_cast<const float4*>(dst + g * 4);
+                    o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                  }
+                  *reinterpret_cast<float4*>(dst + g * 4) = o;
+                }
+              }
+            } else {
+              // Algorithm 3 line 9: W <- W - (eta alpha) (P N), one rounding of the result
+              __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + (long long)row * p.ld_out + col;
+#pragma unroll
+              for (int g = 0; g < 4; ++g) {
+                if (col + g * 8 + 8 <= p.N) {
+                  uint4 w = *reinterpret_cast<const uint4*>(dst + g * 8);
+                  const float s = -p.scale;
+                  w.x = pack_bf16x2(fmaf(s, __uint_as_float(v[g * 8 + 0]), bf16lo(w.x)), fmaf(s, __uint_as_float(v[g * 8 + 1]), bf16hi(w.x)));
+                  w.y = pack_bf16x2(fmaf(s, __uint_as_float(v[g * 8 + 2]), bf16lo(w.y)), fmaf(s, __uint_as_float(v[g * 8 + 3]), bf16hi(w.y)));
+                  w.z = pack_bf16x2(fmaf(s, __uint_as_float(v[g * 8 + 4]), bf16lo(w.z)), fmaf(s, __uint_as_float(v[g * 8 + 5]), bf16hi(w.z)));
+                  w.w = pack_bf16x2(fmaf(s, __uint_as_float(v[g * 8 + 6]), bf16lo(w.w)), fmaf(s, __uint_as_float(v[g * 8 + 7]), bf16hi(w.w)));
+                  *reinterpret_cast<uint4*>(dst + g * 8) = w;
+                }
+              }
             }
           }
         }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar(acc));
+        if (++acc == 2) { acc = 0; acc_phase ^= 1; }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(acc));
-      if (++acc == 2) { acc = 0; acc_phase ^= 1; }
     }
   } else {
     // ------------------------------ P generators --------------------------------
     // Write bf16 tiles of P straight into the swizzled operand layout the MMA reads.
     const int gtid = threadIdx.x - THREADS_BASE;
-    int stage = 0;
-    uint32_t phase = 0;
+    int st = 0;
+    uint32_t ph = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < prm.total_tiles && ok; tile += gridDim.x) {
-      const TileCoord t = decode_tile(prm, tile);
-      const Problem& p = prm.prob[t.prob];
-      for (int ks = t.k_begin; ks < t.k_end; ++ks) {
-        if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1, abort_flag, prm.status))) break;
-        uint8_t* sa = smem_gen + stage * STAGE_BYTES;
-        uint8_t* sb = sa + A_BYTES;
-        const int k0 = ks * BK;
-        if (p.b_mode == GENERATED) {
-          // B[k = row i of P][n = column j of P], MN-major: 64-column blocks of [64 k][128 B]
-          const int chunks = p.bn >> 3;
-          for (int id = gtid; id < BK * chunks; id += 32 * NUM_GEN_WARPS) {
-            const int c = id % chunks, kr = id / chunks;
-            const uint4 val = projection8_bf16(prm.pp, k0 + kr, t.n0 + c * 8);
-            *reinterpret_cast<uint4*>(sb + (c >> 3) * 8192 + kr * 128 + (((c & 7) ^ (kr & 7)) << 4)) = val;
+    if (prm.gen_ring == GEN_B) {
+      for (int tile = blockIdx.x; tile < prm.total_tiles && ok; tile += gridDim.x) {
+        const TileCoord t = decode_tile(prm, tile);
+        const Problem& p = prm.prob[t.prob];
+        const int chunks = p.bn >> 3;
+        for (int ks = t.k_begin; ks < t.k_end; ++ks) {
+          if (!(ok = mbar_wait(emptyB(st), ph ^ 1, abort_flag, prm.status))) break;
+          if (p.b_mode == GENERATED) {
+            // B[k = row i of P][n = column j of P], MN-major: 64-column blocks of [64 k][128 B]
+            uint8_t* sbp = smem_gen + STAGES_A * A_BYTES + st * B_BYTES;
+            const int k0 = ks * BK;
+            for (int id = gtid; id < BK * chunks; id += 32 * NUM_GEN_WARPS) {
+              const int c = id % chunks, kr = id / chunks;
+              const uint4 val = projection8_bf16(prm.pp, k0 + kr, t.n0 + c * 8);
+              *reinterpret_cast<uint4*>(sbp + (c >> 3) * 8192 + kr * 128 + (((c & 7) ^ (kr & 7)) << 4)) = val;
+            }
+            fence_proxy_async_smem();
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(fullB(st));
+          if (++st == STAGES_B) { st = 0; ph ^= 1; }
+        }
+      }
+    } else if (prm.gen_ring == GEN_A) {
+      for (int tile = blockIdx.x; tile < prm.total_tiles && ok; tile += gridDim.x) {
+        const TileCoord t = decode_tile(prm, tile);
+        const Problem& p = prm.prob[t.prob];
+        for (int ks = t.k_begin; ks < t.k_end && ok; ++ks) {
+          for (int mi = 0; mi < t.nsub; ++mi) {
+            if (!(ok = mbar_wait(emptyA(st), ph ^ 1, abort_flag, prm.status))) break;
+            if (p.a_mode == GENERATED) {
+              // A[m = row i of P][k = column j of P], K-major: [128 rows][128 B]
+              uint8_t* sap = smem_gen + st * A_BYTES;
+              const int k0 = ks * BK, m0 = t.m0 + mi * BM;
+              for (int id = gtid; id < BM * 8; id += 32 * NUM_GEN_WARPS) {
+                const int c = id & 7, rr = id >> 3;
+                const uint4 val = projection8_bf16(prm.pp, m0 + rr, k0 + c * 8);
+                *reinterpret_cast<uint4*>(sap + rr * 128 + ((c ^ (rr & 7)) << 4)) = val;
+              }
+              fence_proxy_async_smem();
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(fullA(st));
+            if (++st == STAGES_A) { st = 0; ph ^= 1; }
           }
         }
-        if (p.a_mode == GENERATED) {
-          // A[m = row i of P][k = column j of P], K-major: [128 rows][128 B]
-          for (int id = gtid; id < BM * 8; id += 32 * NUM_GEN_WARPS) {
-            const int c = id & 7, rr = id >> 3;
-            const uint4 val = projection8_bf16(prm.pp, t.m0 + rr, k0 + c * 8);
-            *reinterpret_cast<uint4*>(sa + rr * 128 + ((c ^ (rr & 7)) << 4)) = val;
-          }
-        }
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(full_bar(stage));
-        if (++stage == STAGES) { stage = 0; phase ^= 1; }
       }
     }
   }
@@ -516,8 +624,13 @@ inline bool make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t 
 inline int pick_bn(int N) { return N >= BN_MAX ? BN_MAX : (int)((N + 63) / 64 * 64); }
 
 inline void finish_problem(Problem& p, int splits_wanted) {
-  p.bn = pick_bn(p.N);
-  p.tiles_m = (p.M + BM - 1) / BM;
+  if (p.bn == 0) p.bn = pick_bn(p.N);
+  // two row blocks share each B tile: 256 x 256 items halve the L2 -> shared-memory traffic per flop
+#ifndef CFG_NSUB
+#define CFG_NSUB 2
+#endif
+  if (p.nsub == 0) p.nsub = p.M > BM ? CFG_NSUB : 1;
+  p.tiles_m = (p.M + BM * p.nsub - 1) / (BM * p.nsub);
   p.tiles_n = (p.N + p.bn - 1) / p.bn;
   p.ksteps_total = (p.K + BK - 1) / BK;
   int s = splits_wanted < 1 ? 1 : splits_wanted;
@@ -561,7 +674,7 @@ inline compact_status_t launch(const LaunchInfo& li, Params& prm) {
   prm.total_tiles = t;
   prm.status = li.status;
   const int grid = t < NUM_SMS ? t : NUM_SMS;
-  const int threads = prm.has_generated ? THREADS_GEN : THREADS_BASE;
+  const int threads = prm.gen_ring != GEN_NONE ? THREADS_GEN : THREADS_BASE;
   compact_gemm_kernel<<<grid, threads, SMEM_BYTES, li.stream>>>(prm);
   (*li.launches)++;
   return cudaGetLastError() == cudaSuccess ? COMPACT_OK : COMPACT_ERR_CUDA;
@@ -580,9 +693,12 @@ inline compact_status_t forward(const LaunchInfo& li, const ProjectionParams& pp
   memset(&prm, 0, sizeof(prm));
   prm.pp = pp;
   prm.num_problems = 2;
-  prm.has_generated = 1;
+  prm.gen_ring = GEN_B;
   Problem& pz = prm.prob[0];
   pz.M = (int)tokens; pz.N = zcols; pz.K = n;
+  // one generated 64 x 128 tile of P feeds up to four row blocks of X (512 tokens)
+  pz.bn = zcols >= 128 ? 128 : (int)((zcols + 63) / 64 * 64);
+  pz.nsub = (int)((tokens + BM - 1) / BM) < MAX_SUB ? (int)((tokens + BM - 1) / BM) : MAX_SUB;
   pz.a_mode = TMA_KMAJOR; pz.b_mode = GENERATED; pz.epi_mode = EPI_BF16;
   pz.out = Z; pz.ld_out = ldz;
   finish_problem(pz, 1);
@@ -608,7 +724,7 @@ inline compact_status_t backward(const LaunchInfo& li, int64_t tokens, int n, in
   Params prm;
   memset(&prm, 0, sizeof(prm));
   prm.num_problems = dX ? 2 : 1;
-  prm.has_generated = 0;
+  prm.gen_ring = GEN_NONE;
   const int splits = plan_gc_splits(tokens, r, m);
   if (splits > 1 && workspace_bytes < (size_t)splits * r * m * sizeof(float)) return COMPACT_ERR_WORKSPACE;
   Problem& pg = prm.prob[0];
@@ -659,7 +775,7 @@ inline compact_status_t update(const LaunchInfo& li, const ProjectionParams& pp,
   memset(&prm, 0, sizeof(prm));
   prm.pp = pp;
   prm.num_problems = 1;
-  prm.has_generated = 1;
+  prm.gen_ring = GEN_A;
   Problem& pu = prm.prob[0];
   pu.M = n; pu.N = m; pu.K = r;
   pu.a_mode = GENERATED; pu.b_mode = TMA_MNMAJOR; pu.epi_mode = EPI_UPDATE_W;
