@@ -32,6 +32,9 @@ std::atomic<int> g_next_slot{0};
 
 constexpr int kStatusSlots = 256;
 __device__ unsigned int g_status_words[kStatusSlots];
+// Two words per layer slot for the dynamic item scheduler of the tensor-core kernel
+// (next item, finished CTAs).  Zero at load; each launch leaves them zero again.
+__device__ unsigned int g_sched_words[kStatusSlots][2];
 
 inline size_t elem_size(int dtype) { return dtype == COMPACT_BF16 ? 2 : 4; }
 inline int64_t round_up(int64_t a, int64_t b) { return (a + b - 1) / b * b; }
@@ -56,6 +59,12 @@ unsigned int* status_word(const compact_layer_t* L) {
   unsigned int* base = nullptr;
   if (cudaGetSymbolAddress((void**)&base, g_status_words) != cudaSuccess) { cudaGetLastError(); return nullptr; }
   return base + L->status_slot;
+}
+
+unsigned int* sched_words(const compact_layer_t* L) {
+  unsigned int* base = nullptr;
+  if (cudaGetSymbolAddress((void**)&base, g_sched_words) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+  return base + 2 * L->status_slot;
 }
 
 ProjectionParams make_pp(const compact_layer_t* L, uint32_t epoch) {
@@ -207,7 +216,7 @@ compact_status_t compact_linear_fwd(compact_layer_t* L, int64_t tokens, const vo
   if (L->cfg.dtype == COMPACT_BF16) {
     typedef __nv_bfloat16 T;
     if (g_family.load() == 0) {
-      tc::LaunchInfo li{st, status_word(L), &g_launches};
+      tc::LaunchInfo li{st, status_word(L), sched_words(L), &g_launches};
       s = tc::forward(li, make_pp(L, L->epoch), tokens, L->cfg.m, (const T*)X, ldx, (const T*)W, ldw, (T*)Y, ldy, (T*)Z, ldz,
                       (int)compact_z_ld(L));
       if (s != COMPACT_ERR_SHAPE) return s;   // SHAPE: the tensor-core kernel does not take it
@@ -249,7 +258,7 @@ compact_status_t compact_linear_bwd(compact_layer_t* L, int64_t tokens, const vo
   if (L->cfg.dtype == COMPACT_BF16) {
     typedef __nv_bfloat16 T;
     if (g_family.load() == 0) {
-      tc::LaunchInfo li{st, status_word(L), &g_launches};
+      tc::LaunchInfo li{st, status_word(L), sched_words(L), &g_launches};
       s = tc::backward(li, tokens, L->cfg.n, L->cfg.m, L->cfg.r, (int)compact_z_ld(L), (const T*)dY, lddy, (const T*)Z, ldz, (const T*)W,
                        ldw, (T*)dX, lddx, Gc, ldg, accumulate, workspace, workspace_bytes);
       if (s != COMPACT_ERR_SHAPE) return s;
@@ -279,7 +288,7 @@ compact_status_t compact_adam_update(compact_layer_t* L, void* W, int64_t ldw, c
     typedef __nv_bfloat16 T;
     s = COMPACT_ERR_SHAPE;
     if (g_family.load() == 0) {
-      tc::LaunchInfo li{st, status_word(L), &g_launches};
+      tc::LaunchInfo li{st, status_word(L), sched_words(L), &g_launches};
       s = tc::update(li, make_pp(L, L->epoch), adam_scalars(L, L->step + 1), L->cfg.n, L->cfg.m, L->cfg.r, (T*)W, ldw,
                      Gc, ldg, M, V, lr * L->cfg.alpha, workspace, workspace_bytes);
     }

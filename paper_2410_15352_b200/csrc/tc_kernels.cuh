@@ -1,11 +1,12 @@
 // Tensor-core kernels of the CompAct layer for sm_100a: one persistent,
-// warp-specialised GEMM (TMA -> 128B-swizzled shared memory ring -> tcgen05.mma
-// with fp32 accumulators in TMEM -> tcgen05.ld epilogue) whose operands can come
-// from TMA in either major-ness or from the in-kernel Philox/Box-Muller generator
-// of P.  It serves
+// warp-specialised GEMM (TMA -> 128B-swizzled shared memory rings -> tcgen05.mma
+// with fp32 accumulators in TMEM -> tcgen05.ld -> swizzled staging -> TMA store)
+// whose operands come from TMA in either major-ness or from the in-kernel
+// Philox/Box-Muller generator of P.  It serves
 //   forward  : [Y | Z] = X [W | P]        (Algorithm 1; P tiles generated as the B operand)
 //   backward : dX = dY W^T and Gc = Z^T dY (Algorithm 2; Gc split over tokens)
 //   update   : W <- W - eta alpha P N      (Algorithm 3 lines 6-9; P tiles generated as A)
+// Work items are handed out dynamically (one atomic counter per launch), longest first.
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -23,7 +24,8 @@ namespace tc {
 
 struct LaunchInfo {
   cudaStream_t stream;
-  unsigned int* status;
+  unsigned int* status;   // device word: kernels OR error bits into it
+  unsigned int* sched;    // two device words, zero between launches: next item, finished CTAs
   std::atomic<uint64_t>* launches;
 };
 
@@ -31,22 +33,28 @@ constexpr int BM = 128;              // rows of one accumulator (TMEM lanes)
 constexpr int BK = 64;               // K elements per pipeline stage (one 128-byte swizzle row)
 constexpr int BN_MAX = 256;          // columns of one accumulator slot (TMEM has two slots)
 #ifndef CFG_STAGES_A
-#define CFG_STAGES_A 6
+#define CFG_STAGES_A 5
 #endif
 #ifndef CFG_STAGES_B
 #define CFG_STAGES_B 4
 #endif
-constexpr int STAGES_A = CFG_STAGES_A;          // ring of A tiles (128 x 64 bf16)
-constexpr int STAGES_B = CFG_STAGES_B;          // ring of B tiles (up to 256 x 64 bf16)
+constexpr int STAGES_A = CFG_STAGES_A;   // ring of A tiles (128 x 64 bf16)
+constexpr int STAGES_B = CFG_STAGES_B;   // ring of B tiles (up to 256 x 64 bf16)
 constexpr int A_BYTES = BM * BK * 2;
 constexpr int B_BYTES = BN_MAX * BK * 2;
 constexpr int RING_BYTES = STAGES_A * A_BYTES + STAGES_B * B_BYTES;
+constexpr int STAGING_BYTES = 4096;      // per epilogue warp: 32 rows x 128 bytes
+constexpr int QDEPTH = 4;                // work items the scheduler may run ahead
+constexpr int NUM_EPI_WARPS = 4;
 constexpr int NUM_GEN_WARPS = 16;
-constexpr int THREADS_BASE = 192;    // producer warp, MMA warp, four epilogue warps
+constexpr int THREADS_BASE = 64 + 32 * NUM_EPI_WARPS;   // producer warp, MMA warp, epilogue warps
 constexpr int THREADS_GEN = THREADS_BASE + 32 * NUM_GEN_WARPS;
-constexpr int SMEM_BYTES = 1024 + RING_BYTES + 256;
+constexpr int NUM_BARRIERS = 2 * STAGES_A + 2 * STAGES_B + 4 + 2 * QDEPTH + NUM_EPI_WARPS;
+constexpr int TAIL_BYTES = 8 * NUM_BARRIERS + 4 * QDEPTH + 16;
+constexpr int SMEM_BYTES = 1024 + RING_BYTES + NUM_EPI_WARPS * STAGING_BYTES + ((TAIL_BYTES + 127) / 128) * 128;
 constexpr int NUM_SMS = 148;
-constexpr int MAX_SUB = 4;           // row blocks of 128 that share one generated B tile
+constexpr int MAX_SUB = 4;           // row blocks of 128 that share one B tile
+static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 
 enum OperandMode { TMA_KMAJOR = 0, TMA_MNMAJOR = 1, GENERATED = 2 };
 enum EpiMode { EPI_BF16 = 0, EPI_F32 = 1, EPI_UPDATE_W = 2 };
@@ -59,7 +67,7 @@ __device__ unsigned long long g_prof[8];
 #define PROF_ADD(i, t0) prof[i] += clock64() - (t0)
 #else
 #define PROF_T() 0
-#define PROF_ADD(i, t0)
+#define PROF_ADD(i, t0) ((void)(t0))
 #endif
 
 // One GEMM inside a launch.  An item is nsub row blocks of 128 rows by bn columns;
@@ -70,23 +78,21 @@ struct Problem {
   int bn;
   int nsub;
   int a_mode, b_mode, epi_mode;
-  int accumulate;
   int tile_begin;
   float scale;
-  void* out;
-  long long ld_out;
-  long long split_stride;
 };
 
 struct alignas(64) Params {
   CUtensorMap tmA[2];
   CUtensorMap tmB[2];
+  CUtensorMap tmC[2];     // output (and, for the update, input) tiles of the epilogue
   Problem prob[2];
   int num_problems;
   int total_tiles;
   int gen_ring;
   ProjectionParams pp;
   unsigned int* status;
+  unsigned int* sched;
 };
 
 // --------------------------------------------------------------------------------------
@@ -138,6 +144,19 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "l"(map), "r"(bar), "r"(x), "r"(y)
       : "memory");
 }
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src), "r"(x),
+               "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(map), "r"(src),
+               "r"(x), "r"(y), "r"(z)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
@@ -234,20 +253,27 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));   // generic pointer to the aligned base
   const uint32_t ringA = smem_base, ringB = smem_base + STAGES_A * A_BYTES;
-  const uint32_t bars = smem_base + RING_BYTES;
+  const uint32_t staging = smem_base + RING_BYTES;
+  const uint32_t bars = staging + NUM_EPI_WARPS * STAGING_BYTES;
   // barrier slots (8 bytes each)
   auto fullA = [&](int s) { return bars + 8u * s; };
   auto emptyA = [&](int s) { return bars + 8u * (STAGES_A + s); };
   auto fullB = [&](int s) { return bars + 8u * (2 * STAGES_A + s); };
   auto emptyB = [&](int s) { return bars + 8u * (2 * STAGES_A + STAGES_B + s); };
-  auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES_A + 2 * STAGES_B + a); };
-  auto tempty_bar = [&](int a) { return bars + 8u * (2 * STAGES_A + 2 * STAGES_B + 2 + a); };
-  uint8_t* tail = smem_gen + RING_BYTES + 8 * (2 * STAGES_A + 2 * STAGES_B + 4);
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 8);
+  constexpr int kT = 2 * STAGES_A + 2 * STAGES_B;
+  auto tfull_bar = [&](int a) { return bars + 8u * (kT + a); };
+  auto tempty_bar = [&](int a) { return bars + 8u * (kT + 2 + a); };
+  auto qfull = [&](int s) { return bars + 8u * (kT + 4 + s); };
+  auto qempty = [&](int s) { return bars + 8u * (kT + 4 + QDEPTH + s); };
+  auto wbar = [&](int w) { return bars + 8u * (kT + 4 + 2 * QDEPTH + w); };
+  uint8_t* tail = smem_gen + RING_BYTES + NUM_EPI_WARPS * STAGING_BYTES + 8 * NUM_BARRIERS;
+  volatile int* tile_q = reinterpret_cast<volatile int*>(tail);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail + 4 * QDEPTH);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 4 * QDEPTH + 8);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const bool has_gen = prm.gen_ring != GEN_NONE;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES_A; ++s) {
@@ -260,8 +286,13 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);
-      mbar_init(tempty_bar(a), 4);
+      mbar_init(tempty_bar(a), NUM_EPI_WARPS);
     }
+    for (int s = 0; s < QDEPTH; ++s) {
+      mbar_init(qfull(s), 1);
+      mbar_init(qempty(s), 1 + NUM_EPI_WARPS + (has_gen ? NUM_GEN_WARPS : 0));   // MMA thread, epilogue warps, generator warps
+    }
+    for (int w = 0; w < NUM_EPI_WARPS; ++w) mbar_init(wbar(w), 1);
     *abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async_smem();
@@ -275,13 +306,32 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  // Every consumer role reads the next item from the queue the producer fills.
+  int qs = 0;
+  uint32_t qph = 0;
+  auto next_tile = [&](bool whole_warp, bool elected) -> int {
+    if (!mbar_wait(qfull(qs), qph, abort_flag, prm.status)) return -1;
+    const int tile = tile_q[qs];
+    if (whole_warp) __syncwarp();           // every lane has read the slot before it is handed back
+    if (elected) mbar_arrive(qempty(qs));
+    if (++qs == QDEPTH) { qs = 0; qph ^= 1; }
+    return tile;
+  };
+
   if (warp == 0) {
-    // ------------------------------ TMA producer ------------------------------
+    // ------------------------- scheduler + TMA producer -------------------------
     if (lane == 0) {
       int sa = 0, sb = 0;
       uint32_t pha = 0, phb = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < prm.total_tiles && ok; tile += gridDim.x) {
+      while (ok) {
+        if (!(ok = mbar_wait(qempty(qs), qph ^ 1, abort_flag, prm.status))) break;
+        int tile = (int)atomicAdd(prm.sched, 1u);
+        if (tile >= prm.total_tiles) tile = -1;
+        tile_q[qs] = tile;
+        mbar_arrive(qfull(qs));
+        if (++qs == QDEPTH) { qs = 0; qph ^= 1; }
+        if (tile < 0) break;
         const TileCoord t = decode_tile(prm, tile);
         const Problem& p = prm.prob[t.prob];
         const CUtensorMap* mapA = &prm.tmA[t.prob];
@@ -336,7 +386,9 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       unsigned long long ns0;
       asm volatile("mov.u64 %0, %globaltimer;" : "=l"(ns0));
 #endif
-      for (int tile = blockIdx.x; tile < prm.total_tiles && ok; tile += gridDim.x) {
+      while (ok) {
+        const int tile = next_tile(false, true);
+        if (tile < 0) break;
         const TileCoord t = decode_tile(prm, tile);
         const Problem& p = prm.prob[t.prob];
         const bool a_mn = p.a_mode == TMA_MNMAJOR;
@@ -344,8 +396,15 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
                                ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
         const int slots = (p.nsub * p.bn + BN_MAX - 1) / BN_MAX;   // accumulator slots this item occupies
-        const int acc0 = acc;
         const long long tp0 = PROF_T();
+        if (slots == 2 && acc == 1) {
+          // a two-slot item starts at slot 0: pass slot 1 through unused
+          if (!(ok = mbar_wait(tempty_bar(1), acc_phase ^ 1, abort_flag, prm.status))) break;
+          umma_commit(tfull_bar(1));
+          acc = 0;
+          acc_phase ^= 1;
+        }
+        const int acc0 = acc;
         for (int sl = 0; sl < slots && ok; ++sl) {
           ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag, prm.status);
           if (++acc == 2) { acc = 0; acc_phase ^= 1; }
@@ -394,83 +453,128 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       for (int i = 0; i < 6; ++i) atomicAdd(&g_prof[i], prof[i]);
 #endif
     }
-  } else if (warp < 6) {
+  } else if (warp < 2 + NUM_EPI_WARPS) {
     // ------------------------------ epilogue ------------------------------------
+    // TMEM -> registers -> 128B-swizzled staging tile (32 rows x 128 bytes per warp) -> TMA store.
     const int q = warp & 3;                 // TMEM lane quarter this warp may read
+    const uint32_t stg = staging + (warp - 2) * STAGING_BYTES;
+    uint8_t* stg_gen = smem_gen + RING_BYTES + (warp - 2) * STAGING_BYTES;
+    const uint32_t my_wbar = wbar(warp - 2);
+    uint32_t wph = 0;
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < prm.total_tiles && ok; tile += gridDim.x) {
+    const int sw = lane & 7;
+    while (ok) {
+      const int tile = next_tile(true, lane == 0);
+      if (tile < 0) break;
       const TileCoord t = decode_tile(prm, tile);
       const Problem& p = prm.prob[t.prob];
+      const CUtensorMap* mapC = &prm.tmC[t.prob];
       const int slots = (p.nsub * p.bn + BN_MAX - 1) / BN_MAX;
       const int sub_per_slot = BN_MAX / p.bn > p.nsub ? p.nsub : BN_MAX / p.bn;
+      if (slots == 2 && acc == 1) {
+        if (!(ok = mbar_wait(tfull_bar(1), acc_phase, abort_flag, prm.status))) break;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar(1));
+        acc = 0;
+        acc_phase ^= 1;
+      }
       for (int sl = 0; sl < slots && ok; ++sl) {
         if (!(ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, prm.status))) break;
         tc_fence_after();
-        for (int su = 0; su < sub_per_slot; ++su) {
+        for (int su = 0; su < sub_per_slot && ok; ++su) {
           const int mi = sl * sub_per_slot + su;
           if (mi >= t.nsub) break;
-          const int row = t.m0 + mi * BM + q * 32 + lane;
-          const bool row_ok = row < p.M;
-          for (int c0 = 0; c0 < p.bn; c0 += 32) {
-            const int col = t.n0 + c0;
-            if (col >= p.N) break;
-            uint32_t v[32];
-            tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN_MAX + su * p.bn + c0, v);
-            tmem_ld_wait();
-            if (!row_ok) continue;
-            if (p.epi_mode == EPI_BF16) {
-              __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + (long long)row * p.ld_out + col;
+          const int row0 = t.m0 + mi * BM + q * 32;
+          if (row0 >= p.M) continue;          // this warp's 32 rows are all padding
+          const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN_MAX + su * p.bn;
+          if (p.epi_mode == EPI_F32) {
+            // fp32 output: 32 columns (128 bytes) per staged tile
+            for (int c0 = 0; c0 < p.bn; c0 += 32) {
+              const int col = t.n0 + c0;
+              if (col >= p.N) break;
+              uint32_t v[32];
+              tmem_ld32(tcol + c0, v);
+              if (lane == 0) tma_store_wait_read();
+              __syncwarp();
+              tmem_ld_wait();
 #pragma unroll
-              for (int g = 0; g < 4; ++g) {
-                if (col + g * 8 + 8 <= p.N) {
-                  uint4 o;
-                  o.x = pack_bf16x2(__uint_as_float(v[g * 8 + 0]), __uint_as_float(v[g * 8 + 1]));
-                  o.y = pack_bf16x2(__uint_as_float(v[g * 8 + 2]), __uint_as_float(v[g * 8 + 3]));
-                  o.z = pack_bf16x2(__uint_as_float(v[g * 8 + 4]), __uint_as_float(v[g * 8 + 5]));
-                  o.w = pack_bf16x2(__uint_as_float(v[g * 8 + 6]), __uint_as_float(v[g * 8 + 7]));
-                  *reinterpret_cast<uint4*>(dst + g * 8) = o;
+              for (int j = 0; j < 8; ++j)
+                *reinterpret_cast<uint4*>(stg_gen + lane * 128 + ((j ^ sw) << 4)) =
+                    make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+              fence_proxy_async_smem();
+              __syncwarp();
+              if (lane == 0) {
+                tma_store_3d(mapC, stg, col, row0, t.split);
+                tma_store_commit();
+              }
+            }
+          } else {
+            // bf16 output: 64 columns (128 bytes) per staged tile
+            for (int c0 = 0; c0 < p.bn; c0 += 64) {
+              const int col = t.n0 + c0;
+              if (col >= p.N) break;
+              if (lane == 0) tma_store_wait_read();
+              __syncwarp();
+              if (p.epi_mode == EPI_UPDATE_W) {
+                // bring the W tile in first: W <- W - (eta alpha) (P N), one rounding (Algorithm 3 line 9)
+                if (lane == 0) {
+                  mbar_arrive_expect_tx(my_wbar, STAGING_BYTES);
+                  tma_load_2d(stg, mapC, my_wbar, col, row0);
                 }
               }
-            } else if (p.epi_mode == EPI_F32) {
-              float* dst = reinterpret_cast<float*>(p.out) + (long long)t.split * p.split_stride + (long long)row * p.ld_out + col;
 #pragma unroll
-              for (int g = 0; g < 8; ++g) {
-                if (col + g * 4 + 4 <= p.N) {
-                  float4 o = make_float4(__uint_as_float(v[g * 4 + 0]), __uint_as_float(v[g * 4 + 1]),
-                                         __uint_as_float(v[g * 4 + 2]), __uint_as_float(v[g * 4 + 3]));
-                  if (p.accumulate) {
-                    const float4 old = *reinterpret_cast<const float4*>(dst + g * 4);
-                    o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+              for (int h = 0; h < 2; ++h) {
+                uint32_t v[32];
+                tmem_ld32(tcol + c0 + 32 * h, v);
+                tmem_ld_wait();
+                if (p.epi_mode == EPI_UPDATE_W) {
+                  if (h == 0) {
+                    if (!(ok = mbar_wait(my_wbar, wph, abort_flag, prm.status))) break;
+                    wph ^= 1;
                   }
-                  *reinterpret_cast<float4*>(dst + g * 4) = o;
+                  const float s = -p.scale;
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) {
+                    uint4* cell = reinterpret_cast<uint4*>(stg_gen + lane * 128 + (((4 * h + j) ^ sw) << 4));
+                    uint4 w = *cell;
+                    w.x = pack_bf16x2(fmaf(s, __uint_as_float(v[8 * j + 0]), bf16lo(w.x)), fmaf(s, __uint_as_float(v[8 * j + 1]), bf16hi(w.x)));
+                    w.y = pack_bf16x2(fmaf(s, __uint_as_float(v[8 * j + 2]), bf16lo(w.y)), fmaf(s, __uint_as_float(v[8 * j + 3]), bf16hi(w.y)));
+                    w.z = pack_bf16x2(fmaf(s, __uint_as_float(v[8 * j + 4]), bf16lo(w.z)), fmaf(s, __uint_as_float(v[8 * j + 5]), bf16hi(w.z)));
+                    w.w = pack_bf16x2(fmaf(s, __uint_as_float(v[8 * j + 6]), bf16lo(w.w)), fmaf(s, __uint_as_float(v[8 * j + 7]), bf16hi(w.w)));
+                    *cell = w;
+                  }
+                } else {
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) {
+                    uint4 o;
+                    o.x = pack_bf16x2(__uint_as_float(v[8 * j + 0]), __uint_as_float(v[8 * j + 1]));
+                    o.y = pack_bf16x2(__uint_as_float(v[8 * j + 2]), __uint_as_float(v[8 * j + 3]));
+                    o.z = pack_bf16x2(__uint_as_float(v[8 * j + 4]), __uint_as_float(v[8 * j + 5]));
+                    o.w = pack_bf16x2(__uint_as_float(v[8 * j + 6]), __uint_as_float(v[8 * j + 7]));
+                    *reinterpret_cast<uint4*>(stg_gen + lane * 128 + (((4 * h + j) ^ sw) << 4)) = o;
+                  }
                 }
               }
-            } else {
-              // Algorithm 3 line 9: W <- W - (eta alpha) (P N), one rounding of the result
-              __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.out) + (long long)row * p.ld_out + col;
-#pragma unroll
-              for (int g = 0; g < 4; ++g) {
-                if (col + g * 8 + 8 <= p.N) {
-                  uint4 w = *reinterpret_cast<const uint4*>(dst + g * 8);
-                  const float s = -p.scale;
-                  w.x = pack_bf16x2(fmaf(s, __uint_as_float(v[g * 8 + 0]), bf16lo(w.x)), fmaf(s, __uint_as_float(v[g * 8 + 1]), bf16hi(w.x)));
-                  w.y = pack_bf16x2(fmaf(s, __uint_as_float(v[g * 8 + 2]), bf16lo(w.y)), fmaf(s, __uint_as_float(v[g * 8 + 3]), bf16hi(w.y)));
-                  w.z = pack_bf16x2(fmaf(s, __uint_as_float(v[g * 8 + 4]), bf16lo(w.z)), fmaf(s, __uint_as_float(v[g * 8 + 5]), bf16hi(w.z)));
-                  w.w = pack_bf16x2(fmaf(s, __uint_as_float(v[g * 8 + 6]), bf16lo(w.w)), fmaf(s, __uint_as_float(v[g * 8 + 7]), bf16hi(w.w)));
-                  *reinterpret_cast<uint4*>(dst + g * 8) = w;
-                }
+              if (!ok) break;
+              fence_proxy_async_smem();
+              __syncwarp();
+              if (lane == 0) {
+                tma_store_2d(mapC, stg, col, row0);
+                tma_store_commit();
               }
             }
           }
         }
+        if (!ok) break;
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(tempty_bar(acc));
         if (++acc == 2) { acc = 0; acc_phase ^= 1; }
       }
     }
+    if (lane == 0) tma_store_wait_all();
   } else {
     // ------------------------------ P generators --------------------------------
     // Write bf16 tiles of P straight into the swizzled operand layout the MMA reads.
@@ -478,10 +582,12 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
     int st = 0;
     uint32_t ph = 0;
     bool ok = true;
-    if (prm.gen_ring == GEN_B) {
-      for (int tile = blockIdx.x; tile < prm.total_tiles && ok; tile += gridDim.x) {
-        const TileCoord t = decode_tile(prm, tile);
-        const Problem& p = prm.prob[t.prob];
+    while (ok) {
+      const int tile = next_tile(true, lane == 0);
+      if (tile < 0) break;
+      const TileCoord t = decode_tile(prm, tile);
+      const Problem& p = prm.prob[t.prob];
+      if (prm.gen_ring == GEN_B) {
         const int chunks = p.bn >> 3;
         for (int ks = t.k_begin; ks < t.k_end; ++ks) {
           if (!(ok = mbar_wait(emptyB(st), ph ^ 1, abort_flag, prm.status))) break;
@@ -500,11 +606,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
           if (lane == 0) mbar_arrive(fullB(st));
           if (++st == STAGES_B) { st = 0; ph ^= 1; }
         }
-      }
-    } else if (prm.gen_ring == GEN_A) {
-      for (int tile = blockIdx.x; tile < prm.total_tiles && ok; tile += gridDim.x) {
-        const TileCoord t = decode_tile(prm, tile);
-        const Problem& p = prm.prob[t.prob];
+      } else {
         for (int ks = t.k_begin; ks < t.k_end && ok; ++ks) {
           for (int mi = 0; mi < t.nsub; ++mi) {
             if (!(ok = mbar_wait(emptyA(st), ph ^ 1, abort_flag, prm.status))) break;
@@ -533,6 +635,15 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
+  }
+  // the last CTA to finish re-arms the scheduler words for the next launch
+  if (threadIdx.x == 0) {
+    __threadfence();
+    if (atomicAdd(prm.sched + 1, 1u) == gridDim.x - 1) {
+      prm.sched[0] = 0u;
+      prm.sched[1] = 0u;
+      __threadfence();
+    }
   }
 }
 
@@ -621,14 +732,30 @@ inline bool make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 3-D fp32 map over `planes` row-major matrices of rows x inner (pitch and plane stride in elements);
+// boxes are 32 columns x 32 rows of one plane.
+inline bool make_map_f32_3d(CUtensorMap* map, const void* base, int64_t inner, int64_t rows, int64_t planes, int64_t pitch,
+                            int64_t plane_stride) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)rows, (cuuint64_t)planes};
+  cuuint64_t strides[2] = {(cuuint64_t)pitch * 4, (cuuint64_t)plane_stride * 4};
+  cuuint32_t box[3] = {32, 32, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 inline int pick_bn(int N) { return N >= BN_MAX ? BN_MAX : (int)((N + 63) / 64 * 64); }
+
+#ifndef CFG_NSUB
+#define CFG_NSUB 2
+#endif
 
 inline void finish_problem(Problem& p, int splits_wanted) {
   if (p.bn == 0) p.bn = pick_bn(p.N);
   // two row blocks share each B tile: 256 x 256 items halve the L2 -> shared-memory traffic per flop
-#ifndef CFG_NSUB
-#define CFG_NSUB 2
-#endif
   if (p.nsub == 0) p.nsub = p.M > BM ? CFG_NSUB : 1;
   p.tiles_m = (p.M + BM * p.nsub - 1) / (BM * p.nsub);
   p.tiles_n = (p.N + p.bn - 1) / p.bn;
@@ -639,12 +766,18 @@ inline void finish_problem(Problem& p, int splits_wanted) {
   p.splits = (p.ksteps_total + p.ksteps_per_split - 1) / p.ksteps_per_split;
 }
 
-// Number of token splits of Gc = Z^T dY: enough work items to occupy the SMs, at most 32.
+// Number of token splits of Gc = Z^T dY.  A split should be about as long as one dX item
+// (m / 64 k-steps) so that the dynamic scheduler balances well, and there should be enough
+// items to occupy the SMs; at most 32.
 inline int plan_gc_splits(int64_t tokens, int r, int m) {
-  const int tiles = ((r + BM - 1) / BM) * ((m + pick_bn(m) - 1) / pick_bn(m));
+  const int nsub = r > BM ? CFG_NSUB : 1;
+  const int items = ((r + BM * nsub - 1) / (BM * nsub)) * ((m + pick_bn(m) - 1) / pick_bn(m));
   const int ksteps = (int)((tokens + BK - 1) / BK);
   if (ksteps < 1) return 1;
-  int s = NUM_SMS / tiles;
+  const int dx_ksteps = (m + BK - 1) / BK;
+  const int by_len = (ksteps + dx_ksteps - 1) / dx_ksteps;
+  const int by_fill = (NUM_SMS + items - 1) / items;
+  int s = by_len > by_fill ? by_len : by_fill;
   if (s < 1) s = 1;
   if (s > 32) s = 32;
   if (s > ksteps) s = ksteps;
@@ -652,9 +785,10 @@ inline int plan_gc_splits(int64_t tokens, int r, int m) {
   return (ksteps + per - 1) / per;
 }
 
+// Partials are staged in the workspace when there is more than one split or when the call
+// accumulates into Gc; the size covers both.
 inline size_t gc_workspace_bytes(int64_t tokens, int r, int m) {
-  const int s = plan_gc_splits(tokens, r, m);
-  return s > 1 ? (size_t)s * r * m * sizeof(float) : 0;
+  return (size_t)plan_gc_splits(tokens, r, m) * r * m * sizeof(float);
 }
 
 inline compact_status_t launch(const LaunchInfo& li, Params& prm) {
@@ -673,6 +807,7 @@ inline compact_status_t launch(const LaunchInfo& li, Params& prm) {
   }
   prm.total_tiles = t;
   prm.status = li.status;
+  prm.sched = li.sched;
   const int grid = t < NUM_SMS ? t : NUM_SMS;
   const int threads = prm.gen_ring != GEN_NONE ? THREADS_GEN : THREADS_BASE;
   compact_gemm_kernel<<<grid, threads, SMEM_BYTES, li.stream>>>(prm);
@@ -682,13 +817,13 @@ inline compact_status_t launch(const LaunchInfo& li, Params& prm) {
 
 inline bool tc_shape_ok(int64_t tokens, int n, int m) { return tokens >= 1 && n % 8 == 0 && m % 8 == 0; }
 
-// Algorithm 1: problem 0 = Z = X P (generated B operand; longest tiles go first), problem 1 = Y = X W.
+// Algorithm 1: problem 0 = Z = X P (generated B operand; longest items go first), problem 1 = Y = X W.
 inline compact_status_t forward(const LaunchInfo& li, const ProjectionParams& pp, int64_t tokens, int m,
                                 const __nv_bfloat16* X, int64_t ldx, const __nv_bfloat16* W, int64_t ldw,
                                 __nv_bfloat16* Y, int64_t ldy, __nv_bfloat16* Z, int64_t ldz, int zcols) {
   const int n = pp.n;
   if (!tc_shape_ok(tokens, n, m)) return COMPACT_ERR_SHAPE;
-  if (!li.status) return COMPACT_ERR_CUDA;
+  if (!li.status || !li.sched) return COMPACT_ERR_CUDA;
   Params prm;
   memset(&prm, 0, sizeof(prm));
   prm.pp = pp;
@@ -700,17 +835,17 @@ inline compact_status_t forward(const LaunchInfo& li, const ProjectionParams& pp
   pz.bn = zcols >= 128 ? 128 : (int)((zcols + 63) / 64 * 64);
   pz.nsub = (int)((tokens + BM - 1) / BM) < MAX_SUB ? (int)((tokens + BM - 1) / BM) : MAX_SUB;
   pz.a_mode = TMA_KMAJOR; pz.b_mode = GENERATED; pz.epi_mode = EPI_BF16;
-  pz.out = Z; pz.ld_out = ldz;
   finish_problem(pz, 1);
   Problem& py = prm.prob[1];
   py.M = (int)tokens; py.N = m; py.K = n;
   py.a_mode = TMA_KMAJOR; py.b_mode = TMA_MNMAJOR; py.epi_mode = EPI_BF16;
-  py.out = Y; py.ld_out = ldy;
   finish_problem(py, 1);
   if (!make_map(&prm.tmA[0], X, n, tokens, ldx, BK, BM)) return COMPACT_ERR_CUDA;
   prm.tmA[1] = prm.tmA[0];
   if (!make_map(&prm.tmB[1], W, m, n, ldw, 64, BK)) return COMPACT_ERR_CUDA;
   prm.tmB[0] = prm.tmB[1];   // unused by the generated operand
+  if (!make_map(&prm.tmC[0], Z, zcols, tokens, ldz, 64, 32)) return COMPACT_ERR_CUDA;
+  if (!make_map(&prm.tmC[1], Y, m, tokens, ldy, 64, 32)) return COMPACT_ERR_CUDA;
   return launch(li, prm);
 }
 
@@ -720,21 +855,22 @@ inline compact_status_t backward(const LaunchInfo& li, int64_t tokens, int n, in
                                  const __nv_bfloat16* W, int64_t ldw, __nv_bfloat16* dX, int64_t lddx, float* Gc,
                                  int64_t ldg, int accumulate, void* workspace, size_t workspace_bytes) {
   if (!tc_shape_ok(tokens, n, m)) return COMPACT_ERR_SHAPE;
-  if (!li.status) return COMPACT_ERR_CUDA;
+  if (!li.status || !li.sched) return COMPACT_ERR_CUDA;
   Params prm;
   memset(&prm, 0, sizeof(prm));
   prm.num_problems = dX ? 2 : 1;
   prm.gen_ring = GEN_NONE;
   const int splits = plan_gc_splits(tokens, r, m);
-  if (splits > 1 && workspace_bytes < (size_t)splits * r * m * sizeof(float)) return COMPACT_ERR_WORKSPACE;
+  const bool staged = splits > 1 || accumulate;
+  if (staged && workspace_bytes < (size_t)splits * r * m * sizeof(float)) return COMPACT_ERR_WORKSPACE;
   Problem& pg = prm.prob[0];
   pg.M = r; pg.N = m; pg.K = (int)tokens;
   pg.a_mode = TMA_MNMAJOR; pg.b_mode = TMA_MNMAJOR; pg.epi_mode = EPI_F32;
   finish_problem(pg, splits);
-  if (pg.splits > 1) {
-    pg.out = workspace; pg.ld_out = m; pg.split_stride = (long long)r * m; pg.accumulate = 0;
+  if (staged) {
+    if (!make_map_f32_3d(&prm.tmC[0], workspace, m, r, pg.splits, m, (int64_t)r * m)) return COMPACT_ERR_CUDA;
   } else {
-    pg.out = Gc; pg.ld_out = ldg; pg.split_stride = 0; pg.accumulate = accumulate;
+    if (!make_map_f32_3d(&prm.tmC[0], Gc, m, r, 1, ldg, (int64_t)r * ldg)) return COMPACT_ERR_CUDA;
   }
   if (!make_map(&prm.tmA[0], Z, zcols, tokens, ldz, 64, BK)) return COMPACT_ERR_CUDA;
   if (!make_map(&prm.tmB[0], dY, m, tokens, lddy, 64, BK)) return COMPACT_ERR_CUDA;
@@ -742,14 +878,14 @@ inline compact_status_t backward(const LaunchInfo& li, int64_t tokens, int n, in
     Problem& px = prm.prob[1];
     px.M = (int)tokens; px.N = n; px.K = m;
     px.a_mode = TMA_KMAJOR; px.b_mode = TMA_KMAJOR; px.epi_mode = EPI_BF16;
-    px.out = dX; px.ld_out = lddx;
     finish_problem(px, 1);
     if (!make_map(&prm.tmA[1], dY, m, tokens, lddy, BK, BM)) return COMPACT_ERR_CUDA;
     if (!make_map(&prm.tmB[1], W, m, n, ldw, BK, px.bn)) return COMPACT_ERR_CUDA;
+    if (!make_map(&prm.tmC[1], dX, n, tokens, lddx, 64, 32)) return COMPACT_ERR_CUDA;
   }
   compact_status_t s = launch(li, prm);
   if (s != COMPACT_OK) return s;
-  if (pg.splits > 1) {
+  if (staged) {
     const long long cnt = (long long)r * (m / 4);
     reduce_partials_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, li.stream>>>(
         (const float*)workspace, (long long)r * m, pg.splits, Gc, ldg, r, m, accumulate);
@@ -764,7 +900,7 @@ inline compact_status_t update(const LaunchInfo& li, const ProjectionParams& pp,
                                int r, __nv_bfloat16* W, int64_t ldw, const float* Gc, int64_t ldg, float* M, float* V,
                                float scale, void* workspace, size_t workspace_bytes) {
   if (!tc_shape_ok(1, n, m)) return COMPACT_ERR_SHAPE;
-  if (!li.status) return COMPACT_ERR_CUDA;
+  if (!li.status || !li.sched) return COMPACT_ERR_CUDA;
   if (workspace_bytes < (size_t)r * m * 2) return COMPACT_ERR_WORKSPACE;
   __nv_bfloat16* Nbuf = (__nv_bfloat16*)workspace;
   const long long cnt = (long long)r * (m / 4);
@@ -778,11 +914,13 @@ inline compact_status_t update(const LaunchInfo& li, const ProjectionParams& pp,
   prm.gen_ring = GEN_A;
   Problem& pu = prm.prob[0];
   pu.M = n; pu.N = m; pu.K = r;
+  pu.nsub = 1;     // one accumulator slot per item keeps the W read-modify-write overlapped with the next item
   pu.a_mode = GENERATED; pu.b_mode = TMA_MNMAJOR; pu.epi_mode = EPI_UPDATE_W;
-  pu.out = W; pu.ld_out = ldw; pu.scale = scale;
+  pu.scale = scale;
   finish_problem(pu, 1);
   if (!make_map(&prm.tmB[0], Nbuf, m, r, m, 64, BK)) return COMPACT_ERR_CUDA;
   prm.tmA[0] = prm.tmB[0];
+  if (!make_map(&prm.tmC[0], W, m, n, ldw, 64, 32)) return COMPACT_ERR_CUDA;
   return launch(li, prm);
 }
 
