@@ -201,6 +201,7 @@ class LayerBuffers:
 def run_ours(args):
     import torch.distributed as dist
     from paper_2410_15352_b200 import binding as cb
+    from paper_2410_15352_b200 import dp
     from paper_2410_15352_b200.build import build_library
 
     rank = int(os.environ.get("RANK", "0"))
@@ -238,7 +239,7 @@ def run_ours(args):
             lb.lay.backward(lb.dY, lb.Z, lb.W, lb.Gc, lb.dX)
             if ev: ev[2].record(stream)
             if world > 1:                  # data parallel: the only exchange is the r x m compressed gradient
-                dist.all_reduce(lb.Gc)
+                dp.allreduce_compressed_grad(lb.Gc)
             lb.lay.adam_update(lb.W, lb.Gc, lb.M, lb.V, ep)
             if ev: ev[3].record(stream)
             lb.lay.refresh_projection()
@@ -319,7 +320,7 @@ def run_ours(args):
                 _, _, ep = lb.lay.forward(lb.X, lb.W, lb.Y, lb.Z)
                 lb.lay.backward(lb.dY, lb.Z, lb.W, lb.Gc, lb.dX)
                 if world > 1:
-                    dist.all_reduce(lb.Gc)
+                    dp.allreduce_compressed_grad(lb.Gc)
                 lb.lay.adam_update(lb.W, lb.Gc, lb.M, lb.V, ep)
                 lb.lay.refresh_projection()
                 g.copy_(lb.Gc, non_blocking=True)

@@ -53,7 +53,10 @@ constexpr int NUM_BARRIERS = 2 * STAGES_A + 2 * STAGES_B + 4 + 2 * QDEPTH + NUM_
 constexpr int TAIL_BYTES = 8 * NUM_BARRIERS + 4 * QDEPTH + 16;
 constexpr int SMEM_BYTES = 1024 + RING_BYTES + NUM_EPI_WARPS * STAGING_BYTES + ((TAIL_BYTES + 127) / 128) * 128;
 constexpr int NUM_SMS = 148;
-constexpr int MAX_SUB = 4;           // row blocks of 128 that share one B tile
+#ifndef CFG_ZSUB
+#define CFG_ZSUB 4
+#endif
+constexpr int MAX_SUB = CFG_ZSUB;    // row blocks of 128 that share one generated B tile
 static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 
 enum OperandMode { TMA_KMAJOR = 0, TMA_MNMAJOR = 1, GENERATED = 2 };
@@ -832,7 +835,7 @@ inline compact_status_t forward(const LaunchInfo& li, const ProjectionParams& pp
   Problem& pz = prm.prob[0];
   pz.M = (int)tokens; pz.N = zcols; pz.K = n;
   // one generated 64 x 128 tile of P feeds up to four row blocks of X (512 tokens)
-  pz.bn = zcols >= 128 ? 128 : (int)((zcols + 63) / 64 * 64);
+  pz.bn = zcols >= 512 / MAX_SUB ? 512 / MAX_SUB : (int)((zcols + 63) / 64 * 64);
   pz.nsub = (int)((tokens + BM - 1) / BM) < MAX_SUB ? (int)((tokens + BM - 1) / BM) : MAX_SUB;
   pz.a_mode = TMA_KMAJOR; pz.b_mode = GENERATED; pz.epi_mode = EPI_BF16;
   finish_problem(pz, 1);

@@ -1,0 +1,110 @@
+"""Parity at the benchmark configurations' full sizes, through the C ABI, in the
+launch configuration bench.py times.  Small configurations run whole
+trajectories against the oracle; at the large shapes the oracle checks sampled
+rows of Y, Z, dX, sampled rows of Gc (reduced over all tokens) and sampled rows
+of the updated W (which needs the full Gc), all on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import compact_oracle as co
+from paper_2410_15352_b200 import binding as cb
+from paper_2410_15352_b200 import workloads as wlm
+from paper_2410_15352_b200.build import build_library
+from tests._harness import TOL, f32, make_pair, run_layer_trajectory, to64
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build_library()
+    cb.set_kernel_family(0)
+
+
+# ---- config 2: whole trajectories with refresh, one layer of each distinct shape ----------
+@pytest.mark.parametrize("li", [0, 4, 6])
+def test_config2_trajectory(li):
+    wl = wlm.config2()
+    errs, epochs, dW = run_layer_trajectory(wl, li, steps=wl.steps, check_every_step=True)
+    assert epochs == [0] * 10 + [1] * 10
+    for k, v in errs.items():
+        assert v <= TOL["bf16"], (k, v)
+    assert dW <= 0.1     # accumulated update, relative to itself (sign flips of tiny Gc entries)
+
+
+def _sampled_step(wl, li, tokens, rng, n_rows=48, n_gc=32, n_w=32):
+    """One fwd+bwd+update on both sides at full size; returns relative errors on samples."""
+    L = wl.layers[li]
+    gpu, ora, W0 = make_pair(wl, li)
+    X, dY = wlm.draw_X(wl, li, 0, tokens), wlm.draw_dY(wl, li, 0, tokens)
+    W = W0.cuda()
+    M = torch.zeros((L.r, L.m), dtype=torch.float32, device="cuda")
+    V = torch.zeros_like(M)
+    Y, Z, ep = gpu.forward(X.cuda(), W)
+    dX, Gc = gpu.backward(dY.cuda(), Z, W)
+    gpu.adam_update(W, Gc, M, V, ep)
+    assert gpu.status() == cb.OK
+    assert not Z[:, L.r:].any()
+
+    X64, dY64, W64 = to64(X), to64(dY), to64(W0)
+    P = ora.P()
+    rows = np.sort(rng.choice(tokens, size=min(n_rows, tokens), replace=False))
+    rows[0], rows[-1] = 0, tokens - 1
+    Yo, Zo = co.linear_fwd(X64[rows], W64, P, "bf16")
+    dXo = co.round_bf16(dY64[rows] @ W64.T)
+    out = {"Y": co.rel_frobenius(to64(Y)[rows], Yo), "Z": co.rel_frobenius(to64(Z)[rows, :L.r], Zo),
+           "dX": co.rel_frobenius(to64(dX)[rows], dXo)}
+    # full Z and Gc on the oracle side (the update needs every entry of Gc)
+    Zfull = co.round_bf16(X64 @ P)
+    Gco = Zfull.T @ dY64
+    jr = np.sort(rng.choice(L.r, size=min(n_gc, L.r), replace=False))
+    jr[0], jr[-1] = 0, L.r - 1
+    out["Gc"] = co.rel_frobenius(to64(Gc)[jr], Gco[jr])
+    out["Gc_full"] = co.rel_frobenius(to64(Gc), Gco)
+    Wn, Mn, Vn = co.adam_update(W64, Gco, np.zeros_like(Gco), np.zeros_like(Gco), 1, P, f32(wl.lr), f32(wl.beta1),
+                                f32(wl.beta2), f32(wl.eps), f32(wl.alpha), "bf16")
+    ir = np.sort(rng.choice(L.n, size=min(n_w, L.n), replace=False))
+    ir[0], ir[-1] = 0, L.n - 1
+    out["W"] = co.rel_frobenius(to64(W)[ir], Wn[ir])
+    out["M"] = co.rel_frobenius(to64(M), Mn)
+    out["V"] = co.rel_frobenius(to64(V), Vn)
+    return out
+
+
+FULL_SIZE = [
+    ("c5", 0), ("c5", 4), ("c5", 6),          # LLaMA-7B shapes: 4096x4096 r512, 4096x11008 r512, 11008x4096 r1376
+    ("c3r8", 6), ("c3r4", 6), ("c3r8", 4),    # ragged ranks 342 and 684, ragged m 2736, outlier channels
+    ("c4", 5), ("c4", 4),                      # r = n/2 = 1536 with GELU inputs; 768 -> 3072
+]
+
+
+@pytest.mark.parametrize("cfg,li", FULL_SIZE)
+def test_full_size_sampled(cfg, li):
+    wl = {"c5": wlm.config5, "c4": wlm.config4, "c3r8": lambda: wlm.config3(8), "c3r4": lambda: wlm.config3(4)}[cfg]()
+    rng = np.random.default_rng(li)
+    errs = _sampled_step(wl, li, wl.tokens, rng)
+    for k, v in errs.items():
+        assert v <= TOL["bf16"], (cfg, li, k, v)
+
+
+def test_config5_reduced_tokens_trajectory():
+    # whole-tensor parity over 3 steps at the 7B layer shape with fewer tokens
+    wl = wlm.config5().with_tokens(2048)
+    errs, epochs, _ = run_layer_trajectory(wl, 0, steps=3)
+    assert epochs == [0, 0, 0]
+    for k, v in errs.items():
+        assert v <= TOL["bf16"], (k, v)
+
+
+def test_forced_refresh_changes_projection():
+    wl = wlm.config5().with_tokens(512)
+    gpu, ora, W0 = make_pair(wl, 0)
+    X = wlm.draw_X(wl, 0, 0, 512).cuda()
+    W = W0.cuda()
+    _, Z0, ep0 = gpu.forward(X, W)
+    assert gpu.refresh_projection(force=True) == ep0 + 1
+    _, Z1, ep1 = gpu.forward(X, W)
+    assert ep1 == ep0 + 1 and not torch.equal(Z0, Z1)
+    Zo = co.round_bf16(to64(X) @ co.projection(wl.seed, 0, 1, 4096, 512, "bf16"))
+    assert co.rel_frobenius(to64(Z1), Zo) <= TOL["bf16"]
