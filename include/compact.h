@@ -48,7 +48,8 @@ typedef enum {
   COMPACT_ERR_WORKSPACE = 6,
   COMPACT_ERR_UNSUPPORTED_ARCH = 7,
   COMPACT_ERR_CUDA = 8,
-  COMPACT_ERR_DEVICE_TIMEOUT = 9
+  COMPACT_ERR_DEVICE_TIMEOUT = 9,
+  COMPACT_ERR_SCRATCH_LIMIT = 10
 } compact_status_t;
 
 typedef enum { COMPACT_F32 = 0, COMPACT_BF16 = 1 } compact_dtype_t;
@@ -121,6 +122,36 @@ compact_status_t compact_adam_update(compact_layer_t* layer,
                                      float* M, float* V,
                                      uint32_t epoch_of_Gc, float lr,
                                      void* workspace, size_t workspace_bytes, void* stream);
+
+/* Allocation-free variant of compact_adam_update (the paper has no counterpart: this is
+ * a deployment convenience, not part of the method).
+ *
+ * Who needs it: a caller that is not allowed to obtain device memory at the moment it
+ * wants to step the optimizer -- a serving or training process whose framework has
+ * already claimed all of HBM for its own pool, a plugin running inside another runtime's
+ * callback where cudaMalloc would serialise the whole device, or code whose memory budget
+ * was fixed at start-up.  Such a caller cannot provide the workspace compact_adam_update
+ * asks for.  Here the scratch (the normalised step N of Algorithm 3 line 5) lives in an
+ * array that is part of the library image: COMPACT_NOALLOC_SCRATCH_BYTES of device memory
+ * on every GPU that loads the library, held until the process exits.
+ *
+ * Same arguments, results and step/epoch bookkeeping as compact_adam_update, without the
+ * workspace pair.  The call itself performs no cudaMalloc/cudaFree and calls nothing
+ * that allocates.  Layers with r * m * 4 bytes > COMPACT_NOALLOC_SCRATCH_BYTES are
+ * rejected with COMPACT_ERR_SCRATCH_LIMIT before anything is launched.
+ *
+ * The first call on each device looks up the array's device address (one runtime query,
+ * no allocation); make that first call outside any stream capture.  All calls on a device
+ * share the one array, and it keeps whatever the previous call left in it (each call
+ * overwrites the r x m entries it reads, so nothing needs clearing).  Two calls whose
+ * kernels can overlap on the GPU -- different streams, different layers -- race on it:
+ * keep them ordered on one stream or synchronise between them. */
+#define COMPACT_NOALLOC_SCRATCH_BYTES (32u << 20)
+compact_status_t compact_adam_update_noalloc(compact_layer_t* layer,
+                                             void* W, int64_t ldw,
+                                             const float* Gc, int64_t ldg,
+                                             float* M, float* V,
+                                             uint32_t epoch_of_Gc, float lr, void* stream);
 
 /* Algorithm 3 lines 11-13 and Section 3.3: changing the projection only
  * replaces the seed.  If force != 0, or refresh_T > 0 and the step count is a

@@ -19,11 +19,13 @@ from .build import LIB_PATH
 OK = 0
 ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGNMENT, ERR_DTYPE, ERR_EPOCH_MISMATCH, ERR_WORKSPACE, \
     ERR_UNSUPPORTED_ARCH, ERR_CUDA, ERR_DEVICE_TIMEOUT = range(1, 10)
+ERR_SCRATCH_LIMIT = 10
+NOALLOC_SCRATCH_BYTES = 32 << 20
 F32, BF16 = 0, 1
 
 EXPORTS = [
     "compact_layer_create", "compact_layer_destroy", "compact_z_ld", "compact_workspace_bytes",
-    "compact_saved_bytes", "compact_linear_fwd", "compact_linear_bwd", "compact_adam_update",
+    "compact_saved_bytes", "compact_linear_fwd", "compact_linear_bwd", "compact_adam_update", "compact_adam_update_noalloc",
     "compact_refresh_projection", "compact_layer_get_state", "compact_layer_set_state",
     "compact_layer_status", "compact_debug_philox_u32", "compact_debug_projection",
     "compact_set_kernel_family", "compact_kernel_launch_count", "compact_status_string",
@@ -66,6 +68,7 @@ def lib() -> C.CDLL:
     L.compact_linear_bwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, i64, vp, i64, C.c_int, vp,
                                      C.c_size_t, vp]
     L.compact_adam_update.argtypes = [vp, vp, i64, vp, i64, vp, vp, C.c_uint32, C.c_float, vp, C.c_size_t, vp]
+    L.compact_adam_update_noalloc.argtypes = [vp, vp, i64, vp, i64, vp, vp, C.c_uint32, C.c_float, vp]
     L.compact_refresh_projection.argtypes = [vp, C.c_int, u32p]
     L.compact_layer_get_state.argtypes = [vp, C.POINTER(LayerState)]
     L.compact_layer_set_state.argtypes = [vp, C.POINTER(LayerState)]
@@ -212,6 +215,16 @@ class CompactLinear:
         _check(lib().compact_adam_update(self._h, _ptr(W), W.stride(0), _ptr(Gc), Gc.stride(0), _ptr(M), _ptr(V),
                                          epoch_of_Gc, lr, _ptr(ws), ws.numel(), _stream(stream)),
                "compact_adam_update")
+
+    def adam_update_noalloc(self, W: torch.Tensor, Gc: torch.Tensor, M: torch.Tensor, V: torch.Tensor,
+                            epoch_of_Gc: int, lr: float = math.nan, stream=None) -> None:
+        """Same update, for callers that cannot provide device memory: the scratch is a
+        fixed array inside the library (NOALLOC_SCRATCH_BYTES per GPU).  Nothing is
+        allocated here either: no workspace tensor is created.  Calls that may overlap
+        on the GPU share that array and race; keep them on one stream."""
+        _check(lib().compact_adam_update_noalloc(self._h, _ptr(W), W.stride(0), _ptr(Gc), Gc.stride(0), _ptr(M),
+                                                 _ptr(V), epoch_of_Gc, lr, _stream(stream)),
+               "compact_adam_update_noalloc")
 
     def refresh_projection(self, force: bool = False) -> int:
         ep = C.c_uint32()

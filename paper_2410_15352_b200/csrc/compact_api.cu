@@ -300,6 +300,45 @@ compact_status_t compact_adam_update(compact_layer_t* L, void* W, int64_t ldw, c
   return s;
 }
 
+// ---- allocation-free update -------------------------------------------------------------
+// Scratch for callers that cannot hand over device memory: part of the library image, so
+// every GPU that loads the library carries it until the process ends.  In host code the
+// array's name is only a handle; the device address comes from cudaGetSymbolAddress, asked
+// once per device with that device current.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[COMPACT_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::atomic<void*> g_noalloc_ptr[kMaxDevices];
+
+// Device address of the scratch array on the current device (looked up on first use).
+compact_status_t noalloc_scratch(void** out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return COMPACT_ERR_CUDA; }
+  if (dev < 0 || dev >= kMaxDevices) return COMPACT_ERR_INVALID_ARG;
+  void* p = g_noalloc_ptr[dev].load(std::memory_order_acquire);
+  if (!p) {
+    if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) { cudaGetLastError(); return COMPACT_ERR_CUDA; }
+    g_noalloc_ptr[dev].store(p, std::memory_order_release);
+  }
+  *out = p;
+  return COMPACT_OK;
+}
+}  // namespace
+
+compact_status_t compact_adam_update_noalloc(compact_layer_t* L, void* W, int64_t ldw, const float* Gc, int64_t ldg,
+                                             float* M, float* V, uint32_t epoch_of_Gc, float lr, void* stream) {
+  if (!L) return COMPACT_ERR_INVALID_ARG;
+  // the update needs r x m scratch entries (fp32 in the plain kernels, bf16 in the tensor-core ones)
+  if (compact_workspace_bytes(L, 0) > (size_t)COMPACT_NOALLOC_SCRATCH_BYTES) return COMPACT_ERR_SCRATCH_LIMIT;
+  compact_status_t s = check_device(L);
+  if (s != COMPACT_OK) return s;
+  void* scratch = nullptr;
+  s = noalloc_scratch(&scratch);
+  if (s != COMPACT_OK) return s;
+  return compact_adam_update(L, W, ldw, Gc, ldg, M, V, epoch_of_Gc, lr, scratch, (size_t)COMPACT_NOALLOC_SCRATCH_BYTES, stream);
+}
+
 compact_status_t compact_refresh_projection(compact_layer_t* L, int force, uint32_t* new_epoch) {
   if (!L) return COMPACT_ERR_INVALID_ARG;
   const uint32_t T = L->cfg.refresh_T;
@@ -407,6 +446,7 @@ const char* compact_status_string(compact_status_t s) {
     case COMPACT_ERR_UNSUPPORTED_ARCH: return "device is not compute capability 10.x";
     case COMPACT_ERR_CUDA: return "CUDA runtime error";
     case COMPACT_ERR_DEVICE_TIMEOUT: return "a kernel gave up on a bounded wait";
+    case COMPACT_ERR_SCRATCH_LIMIT: return "layer needs more scratch than the allocation-free entry point carries (r*m*4 > 32 MiB)";
   }
   return "unknown status";
 }
