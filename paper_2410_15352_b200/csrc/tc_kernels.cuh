@@ -12,6 +12,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdlib.h>
 
 #include <atomic>
 
@@ -32,32 +33,34 @@ struct LaunchInfo {
 constexpr int BM = 128;              // rows of one accumulator (TMEM lanes)
 constexpr int BK = 64;               // K elements per pipeline stage (one 128-byte swizzle row)
 constexpr int BN_MAX = 256;          // columns of one accumulator slot (TMEM has two slots)
-#ifndef CFG_STAGES_A
-#define CFG_STAGES_A 5
-#endif
-#ifndef CFG_STAGES_B
-#define CFG_STAGES_B 4
-#endif
-constexpr int STAGES_A = CFG_STAGES_A;   // ring of A tiles (128 x 64 bf16)
-constexpr int STAGES_B = CFG_STAGES_B;   // ring of B tiles (up to 256 x 64 bf16)
 constexpr int A_BYTES = BM * BK * 2;
-constexpr int B_BYTES = BN_MAX * BK * 2;
-constexpr int RING_BYTES = STAGES_A * A_BYTES + STAGES_B * B_BYTES;
 constexpr int STAGING_BYTES = 4096;      // per epilogue warp: 32 rows x 128 bytes
 constexpr int QDEPTH = 4;                // work items the scheduler may run ahead
 constexpr int NUM_EPI_WARPS = 4;
 constexpr int NUM_GEN_WARPS = 16;
-constexpr int THREADS_BASE = 64 + 32 * NUM_EPI_WARPS;   // producer warp, MMA warp, epilogue warps
+constexpr int NUM_PROD = 2;              // producer threads per operand ring (each in its own warp)
+constexpr int THREADS_BASE = 64 + 32 * NUM_EPI_WARPS + 32 * (2 * NUM_PROD - 1);   // scheduler + B producer, MMA, epilogue, other producers
 constexpr int THREADS_GEN = THREADS_BASE + 32 * NUM_GEN_WARPS;
-constexpr int NUM_BARRIERS = 2 * STAGES_A + 2 * STAGES_B + 4 + 2 * QDEPTH + NUM_EPI_WARPS;
-constexpr int TAIL_BYTES = 8 * NUM_BARRIERS + 4 * QDEPTH + 16;
-constexpr int SMEM_BYTES = 1024 + RING_BYTES + NUM_EPI_WARPS * STAGING_BYTES + ((TAIL_BYTES + 127) / 128) * 128;
 constexpr int NUM_SMS = 148;
 #ifndef CFG_ZSUB
 #define CFG_ZSUB 4
 #endif
-constexpr int MAX_SUB = CFG_ZSUB;    // row blocks of 128 that share one generated B tile
-static_assert(SMEM_BYTES <= 232448, "shared memory budget");
+constexpr int MAX_SUB = CFG_ZSUB;    // row blocks that share one generated B tile
+
+// Shared-memory plan.  kPair = false: one CTA per item, B tiles up to 256 columns (32 KB).
+// kPair = true: two CTAs (one cluster) per item, tcgen05 cta_group::2; each CTA holds its own
+// 128 rows of A and its half of the B tile (16 KB), so the rings are deeper.
+template <bool kPair> struct Plan {
+  static constexpr int STAGES_A = kPair ? 7 : 5;
+  static constexpr int STAGES_B = kPair ? 6 : 4;
+  static constexpr int B_BYTES = (kPair ? BN_MAX / 2 : BN_MAX) * BK * 2;
+  static constexpr int RING_BYTES = STAGES_A * A_BYTES + STAGES_B * B_BYTES;
+  static constexpr int NUM_BARRIERS = 2 * STAGES_A + 2 * STAGES_B + 4 + 2 * QDEPTH + NUM_EPI_WARPS;
+  static constexpr int TAIL_BYTES = 8 * NUM_BARRIERS + 4 * QDEPTH + 16;
+  static constexpr int SMEM_BYTES = 1024 + RING_BYTES + NUM_EPI_WARPS * STAGING_BYTES + ((TAIL_BYTES + 127) / 128) * 128;
+  static constexpr int CTAS = kPair ? 2 : 1;
+};
+static_assert(Plan<false>::SMEM_BYTES <= 232448 && Plan<true>::SMEM_BYTES <= 232448, "shared memory budget");
 
 enum OperandMode { TMA_KMAJOR = 0, TMA_MNMAJOR = 1, GENERATED = 2 };
 enum EpiMode { EPI_BF16 = 0, EPI_F32 = 1, EPI_UPDATE_W = 2 };
@@ -77,6 +80,7 @@ __device__ unsigned long long g_prof[8];
 // its nsub accumulators sit side by side in TMEM (nsub * bn <= 512 columns).
 struct Problem {
   int M, N, K;
+  int rows_per_block;   // 128, or 256 when a CTA pair shares the item
   int tiles_m, tiles_n, splits, ksteps_total, ksteps_per_split;
   int bn;
   int nsub;
@@ -93,6 +97,7 @@ struct alignas(64) Params {
   int num_problems;
   int total_tiles;
   int gen_ring;
+  int debug_flags;        // profiling builds only: bit 0 = issue no MMAs (measures the load path alone)
   ProjectionParams pp;
   unsigned int* status;
   unsigned int* sched;
@@ -108,6 +113,27 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_n(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// the generator warps meet on hardware barrier 1 (barrier 0 is __syncthreads)
+// and agree on one answer (true only if every thread's `ok` is true), so that a thread whose
+// bounded wait expired takes the whole group out with it instead of leaving the rest at the barrier
+__device__ __forceinline__ bool gen_group_all(bool ok) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.and.pred p, 1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r)
+      : "r"((uint32_t)ok), "r"(32 * 16)
+      : "memory");
+  return r != 0;
 }
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -128,6 +154,80 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   if (mbar_try_wait(bar, parity)) return true;
   for (uint32_t it = 0; it < 8000000u; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
+    if (it > 128) {
+      __nanosleep(100);
+      if (*abort_flag) return false;
+    }
+  }
+  *abort_flag = 1;
+  atomicOr(status, STATUS_TIMEOUT);
+  return false;
+}
+
+// ---- cluster (CTA pair) helpers ----
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
+  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// TMA load issued by either CTA of a pair; completes on the barrier `bar_cluster` (a shared::cluster
+// address, normally the leader's) and writes this CTA's own shared memory.  No multicast.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+      "l"(map), "r"(bar_cluster), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                               uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %2};\n\t"
+      "mov.b64 db, {%3, %4};\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Completion of all earlier MMAs of this thread arrives on the barrier at this offset in both CTAs of the pair.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+               "h"((uint16_t)3)
+               : "memory");
+}
+
+template <bool kCluster>
+__device__ __forceinline__ bool mbar_wait_t(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned int* status) {
+  if (!kCluster) return mbar_wait(bar, parity, abort_flag, status);
+  if (mbar_try_wait_cluster(bar, parity)) return true;
+  for (uint32_t it = 0; it < 8000000u; ++it) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
     if (it > 128) {
       __nanosleep(100);
       if (*abort_flag) return false;
@@ -240,18 +340,29 @@ __device__ __forceinline__ TileCoord decode_tile(const Params& prm, int tile) {
   local /= p.tiles_n;
   const int mb = local % p.tiles_m;
   t.split = local / p.tiles_m;
-  t.m0 = mb * BM * p.nsub;
+  t.m0 = mb * p.rows_per_block * p.nsub;
   t.n0 = nb * p.bn;
   t.k_begin = t.split * p.ksteps_per_split;
   t.k_end = min(p.ksteps_total, t.k_begin + p.ksteps_per_split);
-  t.nsub = min(p.nsub, (p.M - t.m0 + BM - 1) / BM);   // row blocks that hold at least one valid row
+  t.nsub = min(p.nsub, (p.M - t.m0 + p.rows_per_block - 1) / p.rows_per_block);   // row blocks with a valid row
   return t;
 }
 
 // --------------------------------------------------------------------------------------
-// The kernel
+// The kernel.  kPair = true runs two CTAs (a cluster of 2) per item with tcgen05 cta_group::2:
+// the leader CTA (cluster rank 0) issues the MMAs over 256 rows; each CTA loads or generates its
+// own 128 rows of A and its own half of the B columns into its own shared memory and drains its
+// own half of the accumulator.  Full barriers and the item queue's hand-back barrier live in the
+// leader; empty and accumulator-full barriers are signalled in both CTAs by multicast commits.
 // --------------------------------------------------------------------------------------
+template <bool kPair>
 __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __grid_constant__ Params prm) {
+  using PL = Plan<kPair>;
+  constexpr int STAGES_A = PL::STAGES_A, STAGES_B = PL::STAGES_B, B_BYTES = PL::B_BYTES, RING_BYTES = PL::RING_BYTES;
+  constexpr int NCTA = PL::CTAS;
+  // generator arrivals on a barrier of the leader: one per local warp, plus one for the whole group of the
+  // second CTA (arrivals across the cluster are slow, so that group meets on a hardware barrier first)
+  constexpr int GEN_ARRIVALS = NUM_GEN_WARPS + (kPair ? 1 : 0);
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));   // generic pointer to the aligned base
@@ -269,7 +380,8 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
   auto qfull = [&](int s) { return bars + 8u * (kT + 4 + s); };
   auto qempty = [&](int s) { return bars + 8u * (kT + 4 + QDEPTH + s); };
   auto wbar = [&](int w) { return bars + 8u * (kT + 4 + 2 * QDEPTH + w); };
-  uint8_t* tail = smem_gen + RING_BYTES + NUM_EPI_WARPS * STAGING_BYTES + 8 * NUM_BARRIERS;
+  const uint32_t tail_u32 = bars + 8 * PL::NUM_BARRIERS;
+  uint8_t* tail = smem_gen + RING_BYTES + NUM_EPI_WARPS * STAGING_BYTES + 8 * PL::NUM_BARRIERS;
   volatile int* tile_q = reinterpret_cast<volatile int*>(tail);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail + 4 * QDEPTH);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 4 * QDEPTH + 8);
@@ -277,23 +389,36 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const bool has_gen = prm.gen_ring != GEN_NONE;
+  const uint32_t rank = kPair ? cluster_ctarank() : 0u;        // 0 = leader
+  const bool leader = rank == 0;
+  // arrive on a barrier that lives in the leader CTA
+  auto arrive_leader = [&](uint32_t bar) {
+    if (!kPair || leader) mbar_arrive(bar);
+    else mbar_arrive_cluster(map_to_cta(bar, 0));
+  };
+  auto commit = [&](uint32_t bar) {
+    if (kPair) umma_commit_pair(bar); else umma_commit(bar);
+  };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES_A; ++s) {
-      mbar_init(fullA(s), 1 + (prm.gen_ring == GEN_A ? NUM_GEN_WARPS : 0));
+      mbar_init(fullA(s), 1 + (prm.gen_ring == GEN_A ? GEN_ARRIVALS : 0));
       mbar_init(emptyA(s), 1);
     }
     for (int s = 0; s < STAGES_B; ++s) {
-      mbar_init(fullB(s), 1 + (prm.gen_ring == GEN_B ? NUM_GEN_WARPS : 0));
+      mbar_init(fullB(s), 1 + (prm.gen_ring == GEN_B ? GEN_ARRIVALS : 0));
       mbar_init(emptyB(s), 1);
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);
-      mbar_init(tempty_bar(a), NUM_EPI_WARPS);
+      mbar_init(tempty_bar(a), NCTA * NUM_EPI_WARPS);
     }
+    // consumers of the item queue: the MMA thread (leader); the producers other than the scheduler,
+    // the epilogue warps and the generator group (one arrival) of each CTA; the second CTA's first B producer
+    const int consumers = 1 + NCTA * (2 * NUM_PROD - 1 + NUM_EPI_WARPS) + (has_gen ? GEN_ARRIVALS : 0) + (kPair ? 1 : 0);
     for (int s = 0; s < QDEPTH; ++s) {
       mbar_init(qfull(s), 1);
-      mbar_init(qempty(s), 1 + NUM_EPI_WARPS + (has_gen ? NUM_GEN_WARPS : 0));   // MMA thread, epilogue warps, generator warps
+      mbar_init(qempty(s), consumers);
     }
     for (int w = 0; w < NUM_EPI_WARPS; ++w) mbar_init(wbar(w), 1);
     *abort_flag = 0;
@@ -306,80 +431,96 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
   }
   tc_fence_before();
   __syncthreads();
+  if (kPair) cluster_sync_all();          // both CTAs' barriers exist before anyone signals across
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  // Every consumer role reads the next item from the queue the producer fills.
+  // Every consumer role reads the next item from the queue the (leader's) producer fills.
   int qs = 0;
   uint32_t qph = 0;
   auto next_tile = [&](bool whole_warp, bool elected) -> int {
-    if (!mbar_wait(qfull(qs), qph, abort_flag, prm.status)) return -1;
+    // the second CTA's slot is written by the leader from across the cluster: acquire at cluster scope there
+    const bool got = (kPair && !leader) ? mbar_wait_t<true>(qfull(qs), qph, abort_flag, prm.status)
+                                        : mbar_wait(qfull(qs), qph, abort_flag, prm.status);
+    if (!got) return -1;
     const int tile = tile_q[qs];
     if (whole_warp) __syncwarp();           // every lane has read the slot before it is handed back
-    if (elected) mbar_arrive(qempty(qs));
+    if (elected) arrive_leader(qempty(qs));
     if (++qs == QDEPTH) { qs = 0; qph ^= 1; }
     return tile;
   };
 
-  if (warp == 0) {
-    // ------------------------- scheduler + TMA producer -------------------------
+  // Producer threads: NUM_PROD per operand ring, each lane 0 of its own warp.  Thread j of a ring
+  // loads the tiles whose running index is j modulo NUM_PROD: every barrier wait / expect / TMA issue
+  // is a dependent long-latency step, and several threads overlap them.
+  const int prodB = warp == 0 ? 0 : ((warp >= 2 + NUM_EPI_WARPS && warp < 2 + NUM_EPI_WARPS + 2 * NUM_PROD - 1 && ((warp - 2 - NUM_EPI_WARPS) & 1)) ? (warp - 2 - NUM_EPI_WARPS + 1) / 2 : -1);
+  const int prodA = (warp >= 2 + NUM_EPI_WARPS && warp < 2 + NUM_EPI_WARPS + 2 * NUM_PROD - 1 && !((warp - 2 - NUM_EPI_WARPS) & 1)) ? (warp - 2 - NUM_EPI_WARPS) / 2 : -1;
+  if (prodB >= 0) {
+    // ------------------------- producers of B tiles (thread 0 is also the scheduler) ----------
     if (lane == 0) {
-      int sa = 0, sb = 0;
-      uint32_t pha = 0, phb = 0;
+      uint32_t ib = 0;                     // running index of B tiles in this CTA
       bool ok = true;
       while (ok) {
-        if (!(ok = mbar_wait(qempty(qs), qph ^ 1, abort_flag, prm.status))) break;
-        int tile = (int)atomicAdd(prm.sched, 1u);
-        if (tile >= prm.total_tiles) tile = -1;
-        tile_q[qs] = tile;
-        mbar_arrive(qfull(qs));
-        if (++qs == QDEPTH) { qs = 0; qph ^= 1; }
+        int tile;
+        if (prodB == 0 && leader) {
+          if (!(ok = mbar_wait(qempty(qs), qph ^ 1, abort_flag, prm.status))) break;
+          tile = (int)atomicAdd(prm.sched, 1u);
+          if (tile >= prm.total_tiles) tile = -1;
+          tile_q[qs] = tile;
+          mbar_arrive(qfull(qs));
+          if (kPair) {
+            st_cluster_u32(map_to_cta(tail_u32 + 4u * qs, 1), (uint32_t)tile);
+            mbar_arrive_cluster(map_to_cta(qfull(qs), 1));
+          }
+          if (++qs == QDEPTH) { qs = 0; qph ^= 1; }
+        } else {
+          tile = next_tile(false, true);
+        }
         if (tile < 0) break;
         const TileCoord t = decode_tile(prm, tile);
         const Problem& p = prm.prob[t.prob];
-        const CUtensorMap* mapA = &prm.tmA[t.prob];
         const CUtensorMap* mapB = &prm.tmB[t.prob];
-        for (int ks = t.k_begin; ks < t.k_end && ok; ++ks) {
+        const int bn_cta = p.bn / NCTA;                 // B columns this CTA holds
+        const int n0 = t.n0 + (int)rank * bn_cta;
+        for (int ks = t.k_begin; ks < t.k_end && ok; ++ks, ++ib) {
+          if ((int)(ib % NUM_PROD) != prodB) continue;
+          const int sb = (int)(ib % STAGES_B);
+          const uint32_t phb = (ib / STAGES_B) & 1u;
           const int k0 = ks * BK;
           // B tile of this k-step (shared by all row blocks of the item)
           if (!(ok = mbar_wait(emptyB(sb), phb ^ 1, abort_flag, prm.status))) break;
-          {
-            const uint32_t dst = ringB + sb * B_BYTES, fb = fullB(sb);
-            if (p.b_mode == GENERATED) {
-              mbar_arrive(fb);
-            } else {
-              mbar_arrive_expect_tx(fb, p.bn * BK * 2);
+          const uint32_t dst = ringB + sb * B_BYTES, fb = fullB(sb);
+          if (p.b_mode == GENERATED) {
+            if (leader) mbar_arrive(fb);                                 // the generator groups arrive for the data
+          } else {
+            if (leader) {
+              // both CTAs' halves land on this barrier; the generators sit this item out, so arrive for them too
+              mbar_expect_tx(fb, p.bn * BK * 2);
+              mbar_arrive_n(fb, 1 + (prm.gen_ring == GEN_B ? GEN_ARRIVALS : 0));
+            }
+            if (!kPair || leader) {
+              // ordinary loads onto this CTA's own barrier
               if (p.b_mode == TMA_KMAJOR) {
-                tma_load_2d(dst, mapB, fb, k0, t.n0);
+                tma_load_2d(dst, mapB, fb, k0, n0);
               } else {
-                for (int b = 0; b < p.bn / 64; ++b) tma_load_2d(dst + b * 8192, mapB, fb, t.n0 + 64 * b, k0);
+                for (int b = 0; b < bn_cta / 64; ++b) tma_load_2d(dst + b * 8192, mapB, fb, n0 + 64 * b, k0);
               }
-            }
-            if (++sb == STAGES_B) { sb = 0; phb ^= 1; }
-          }
-          for (int mi = 0; mi < t.nsub; ++mi) {
-            if (!(ok = mbar_wait(emptyA(sa), pha ^ 1, abort_flag, prm.status))) break;
-            const uint32_t dst = ringA + sa * A_BYTES, fa = fullA(sa);
-            const int m0 = t.m0 + mi * BM;
-            if (p.a_mode == GENERATED) {
-              mbar_arrive(fa);
             } else {
-              mbar_arrive_expect_tx(fa, A_BYTES);
-              if (p.a_mode == TMA_KMAJOR) {
-                tma_load_2d(dst, mapA, fa, k0, m0);
+              // second CTA: data into its own shared memory, completion onto the leader's barrier
+              const uint32_t fb_sig = map_to_cta(fb, 0);
+              if (p.b_mode == TMA_KMAJOR) {
+                tma_load_2d_pair(dst, mapB, fb_sig, k0, n0);
               } else {
-                tma_load_2d(dst, mapA, fa, m0, k0);
-                tma_load_2d(dst + 8192, mapA, fa, m0 + 64, k0);
+                for (int b = 0; b < bn_cta / 64; ++b) tma_load_2d_pair(dst + b * 8192, mapB, fb_sig, n0 + 64 * b, k0);
               }
             }
-            if (++sa == STAGES_A) { sa = 0; pha ^= 1; }
           }
         }
       }
     }
   } else if (warp == 1) {
-    // ------------------------------ MMA issuer ---------------------------------
-    if (lane == 0) {
+    // ------------------------------ MMA issuer (leader CTA only) ----------------
+    if (lane == 0 && leader) {
       int sa = 0, sb = 0, acc = 0;
       uint32_t pha = 0, phb = 0, acc_phase = 0;
       bool ok = true;
@@ -397,13 +538,13 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const bool a_mn = p.a_mode == TMA_MNMAJOR;
         const bool b_mn = p.b_mode != TMA_KMAJOR;          // generated B tiles are written MN-major
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
-                               ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+                               ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)((NCTA * BM) >> 4) << 24);
         const int slots = (p.nsub * p.bn + BN_MAX - 1) / BN_MAX;   // accumulator slots this item occupies
         const long long tp0 = PROF_T();
         if (slots == 2 && acc == 1) {
           // a two-slot item starts at slot 0: pass slot 1 through unused
           if (!(ok = mbar_wait(tempty_bar(1), acc_phase ^ 1, abort_flag, prm.status))) break;
-          umma_commit(tfull_bar(1));
+          commit(tfull_bar(1));
           acc = 0;
           acc_phase ^= 1;
         }
@@ -429,31 +570,46 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             const long long tp2 = PROF_T();
             if (!(ok = mbar_wait(fullA(sa), pha, abort_flag, prm.status))) break;
             PROF_ADD(2, tp2);
-            const long long tp3 = PROF_T();
+            const long long tp7 = PROF_T();
             tc_fence_after();
+            PROF_ADD(7, tp7);
+            const long long tp3 = PROF_T();
             const uint32_t a_lo = desc_lo(ringA + sa * A_BYTES, a_mn);
             const uint32_t d = d_base + mi * bn;
-            umma_bf16(d, a_lo, DESC_HI, b_lo, DESC_HI, idesc, first);
-            umma_bf16(d, a_lo + a_step, DESC_HI, b_lo + b_step, DESC_HI, idesc, 1u);
-            umma_bf16(d, a_lo + 2 * a_step, DESC_HI, b_lo + 2 * b_step, DESC_HI, idesc, 1u);
-            umma_bf16(d, a_lo + 3 * a_step, DESC_HI, b_lo + 3 * b_step, DESC_HI, idesc, 1u);
-            umma_commit(emptyA(sa));
+#ifdef COMPACT_PROFILE
+            if (prm.debug_flags & 1) {
+            } else
+#endif
+            if (kPair) {
+              umma_bf16_pair(d, a_lo, DESC_HI, b_lo, DESC_HI, idesc, first);
+              umma_bf16_pair(d, a_lo + a_step, DESC_HI, b_lo + b_step, DESC_HI, idesc, 1u);
+              umma_bf16_pair(d, a_lo + 2 * a_step, DESC_HI, b_lo + 2 * b_step, DESC_HI, idesc, 1u);
+              umma_bf16_pair(d, a_lo + 3 * a_step, DESC_HI, b_lo + 3 * b_step, DESC_HI, idesc, 1u);
+            } else {
+              umma_bf16(d, a_lo, DESC_HI, b_lo, DESC_HI, idesc, first);
+              umma_bf16(d, a_lo + a_step, DESC_HI, b_lo + b_step, DESC_HI, idesc, 1u);
+              umma_bf16(d, a_lo + 2 * a_step, DESC_HI, b_lo + 2 * b_step, DESC_HI, idesc, 1u);
+              umma_bf16(d, a_lo + 3 * a_step, DESC_HI, b_lo + 3 * b_step, DESC_HI, idesc, 1u);
+            }
+            commit(emptyA(sa));
             PROF_ADD(3, tp3);
             if (++sa == STAGES_A) { sa = 0; pha ^= 1; }
           }
           if (!ok) break;
-          umma_commit(emptyB(sb));
+          const long long tp6 = PROF_T();
+          commit(emptyB(sb));
+          PROF_ADD(6, tp6);
           if (++sb == STAGES_B) { sb = 0; phb ^= 1; }
         }
         if (!ok) break;
-        for (int sl = 0; sl < slots; ++sl) umma_commit(tfull_bar((acc0 + sl) & 1));
+        for (int sl = 0; sl < slots; ++sl) commit(tfull_bar((acc0 + sl) & 1));
       }
 #ifdef COMPACT_PROFILE
       prof[4] = clock64() - t_start;
       unsigned long long ns1;
       asm volatile("mov.u64 %0, %globaltimer;" : "=l"(ns1));
       prof[5] = ns1 - ns0;
-      for (int i = 0; i < 6; ++i) atomicAdd(&g_prof[i], prof[i]);
+      for (int i = 0; i < 8; ++i) atomicAdd(&g_prof[i], prof[i]);
 #endif
     }
   } else if (warp < 2 + NUM_EPI_WARPS) {
@@ -479,7 +635,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       if (slots == 2 && acc == 1) {
         if (!(ok = mbar_wait(tfull_bar(1), acc_phase, abort_flag, prm.status))) break;
         __syncwarp();
-        if (lane == 0) mbar_arrive(tempty_bar(1));
+        if (lane == 0) arrive_leader(tempty_bar(1));
         acc = 0;
         acc_phase ^= 1;
       }
@@ -489,7 +645,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         for (int su = 0; su < sub_per_slot && ok; ++su) {
           const int mi = sl * sub_per_slot + su;
           if (mi >= t.nsub) break;
-          const int row0 = t.m0 + mi * BM + q * 32;
+          const int row0 = t.m0 + mi * p.rows_per_block + (int)rank * BM + q * 32;
           if (row0 >= p.M) continue;          // this warp's 32 rows are all padding
           const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN_MAX + su * p.bn;
           if (p.epi_mode == EPI_F32) {
@@ -573,50 +729,119 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         if (!ok) break;
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(tempty_bar(acc));
+        if (lane == 0) arrive_leader(tempty_bar(acc));
         if (++acc == 2) { acc = 0; acc_phase ^= 1; }
       }
     }
     if (lane == 0) tma_store_wait_all();
+  } else if (prodA >= 0) {
+    // ------------------------------ producers of A tiles ------------------------
+    if (lane == 0) {
+      uint32_t ia = 0;                     // running index of A tiles in this CTA
+      bool ok = true;
+      while (ok) {
+        const int tile = next_tile(false, true);
+        if (tile < 0) break;
+        const TileCoord t = decode_tile(prm, tile);
+        const Problem& p = prm.prob[t.prob];
+        const CUtensorMap* mapA = &prm.tmA[t.prob];
+        for (int ks = t.k_begin; ks < t.k_end && ok; ++ks) {
+          const int k0 = ks * BK;
+          for (int mi = 0; mi < t.nsub; ++mi, ++ia) {
+            if ((int)(ia % NUM_PROD) != prodA) continue;
+            const int sa = (int)(ia % STAGES_A);
+            const uint32_t pha = (ia / STAGES_A) & 1u;
+            if (!(ok = mbar_wait(emptyA(sa), pha ^ 1, abort_flag, prm.status))) break;
+            const uint32_t dst = ringA + sa * A_BYTES, fa = fullA(sa);
+            const int m0 = t.m0 + mi * p.rows_per_block + (int)rank * BM;
+            if (p.a_mode == GENERATED) {
+              if (leader) mbar_arrive(fa);
+            } else {
+              if (leader) {
+                mbar_expect_tx(fa, NCTA * A_BYTES);
+                mbar_arrive_n(fa, 1 + (prm.gen_ring == GEN_A ? GEN_ARRIVALS : 0));
+              }
+              if (!kPair || leader) {
+                if (p.a_mode == TMA_KMAJOR) {
+                  tma_load_2d(dst, mapA, fa, k0, m0);
+                } else {
+                  tma_load_2d(dst, mapA, fa, m0, k0);
+                  tma_load_2d(dst + 8192, mapA, fa, m0 + 64, k0);
+                }
+              } else {
+                const uint32_t fa_sig = map_to_cta(fa, 0);
+                if (p.a_mode == TMA_KMAJOR) {
+                  tma_load_2d_pair(dst, mapA, fa_sig, k0, m0);
+                } else {
+                  tma_load_2d_pair(dst, mapA, fa_sig, m0, k0);
+                  tma_load_2d_pair(dst + 8192, mapA, fa_sig, m0 + 64, k0);
+                }
+              }
+            }
+          }
+        }
+      }
+    }
   } else {
     // ------------------------------ P generators --------------------------------
-    // Write bf16 tiles of P straight into the swizzled operand layout the MMA reads.
+    // Write bf16 tiles of P straight into the swizzled operand layout the MMA reads.  The group
+    // meets on a hardware barrier and signals each tile (and each item hand-back) once.
     const int gtid = threadIdx.x - THREADS_BASE;
-    int st = 0;
-    uint32_t ph = 0;
+    uint32_t it = 0;                       // running index of tiles in the ring this launch generates into
     bool ok = true;
+    // Signal `bar` of the leader once this thread's warp (leader CTA) or the whole group (second CTA)
+    // is done; returns false if some participant's wait had expired.
+    auto signal = [&](uint32_t bar, bool w) -> bool {
+      if (!kPair || leader) {
+        const bool all = __all_sync(0xffffffffu, w);
+        if (all && lane == 0) mbar_arrive(bar);
+        return all;
+      }
+      const bool all = gen_group_all(w);
+      if (all && gtid == 0) mbar_arrive_cluster(map_to_cta(bar, 0));
+      return all;
+    };
     while (ok) {
-      const int tile = next_tile(true, lane == 0);
+      const bool got = (kPair && !leader) ? mbar_wait_t<true>(qfull(qs), qph, abort_flag, prm.status)
+                                          : mbar_wait(qfull(qs), qph, abort_flag, prm.status);
+      const int tile = got ? tile_q[qs] : -1;
+      if (!(ok = signal(qempty(qs), got))) break;     // every participating thread has read the slot
+      if (++qs == QDEPTH) { qs = 0; qph ^= 1; }
       if (tile < 0) break;
       const TileCoord t = decode_tile(prm, tile);
       const Problem& p = prm.prob[t.prob];
+      const int klen = t.k_end - t.k_begin;
       if (prm.gen_ring == GEN_B) {
-        const int chunks = p.bn >> 3;
-        for (int ks = t.k_begin; ks < t.k_end; ++ks) {
-          if (!(ok = mbar_wait(emptyB(st), ph ^ 1, abort_flag, prm.status))) break;
-          if (p.b_mode == GENERATED) {
+        if (p.b_mode != GENERATED) { it += klen; continue; }      // the producer arrives for this item
+        const int bn_cta = p.bn / NCTA;
+        const int n0 = t.n0 + (int)rank * bn_cta;
+        const int chunks = bn_cta >> 3;
+        for (int ks = t.k_begin; ks < t.k_end; ++ks, ++it) {
+          const int st = (int)(it % STAGES_B);
+          const bool w = mbar_wait(emptyB(st), ((it / STAGES_B) & 1u) ^ 1, abort_flag, prm.status);
+          if (w) {
             // B[k = row i of P][n = column j of P], MN-major: 64-column blocks of [64 k][128 B]
             uint8_t* sbp = smem_gen + STAGES_A * A_BYTES + st * B_BYTES;
             const int k0 = ks * BK;
             for (int id = gtid; id < BK * chunks; id += 32 * NUM_GEN_WARPS) {
               const int c = id % chunks, kr = id / chunks;
-              const uint4 val = projection8_bf16(prm.pp, k0 + kr, t.n0 + c * 8);
+              const uint4 val = projection8_bf16(prm.pp, k0 + kr, n0 + c * 8);
               *reinterpret_cast<uint4*>(sbp + (c >> 3) * 8192 + kr * 128 + (((c & 7) ^ (kr & 7)) << 4)) = val;
             }
             fence_proxy_async_smem();
           }
-          __syncwarp();
-          if (lane == 0) mbar_arrive(fullB(st));
-          if (++st == STAGES_B) { st = 0; ph ^= 1; }
+          if (!(ok = signal(fullB(st), w))) break;
         }
       } else {
+        if (p.a_mode != GENERATED) { it += klen * t.nsub; continue; }
         for (int ks = t.k_begin; ks < t.k_end && ok; ++ks) {
-          for (int mi = 0; mi < t.nsub; ++mi) {
-            if (!(ok = mbar_wait(emptyA(st), ph ^ 1, abort_flag, prm.status))) break;
-            if (p.a_mode == GENERATED) {
+          for (int mi = 0; mi < t.nsub; ++mi, ++it) {
+            const int st = (int)(it % STAGES_A);
+            const bool w = mbar_wait(emptyA(st), ((it / STAGES_A) & 1u) ^ 1, abort_flag, prm.status);
+            if (w) {
               // A[m = row i of P][k = column j of P], K-major: [128 rows][128 B]
               uint8_t* sap = smem_gen + st * A_BYTES;
-              const int k0 = ks * BK, m0 = t.m0 + mi * BM;
+              const int k0 = ks * BK, m0 = t.m0 + mi * p.rows_per_block + (int)rank * BM;
               for (int id = gtid; id < BM * 8; id += 32 * NUM_GEN_WARPS) {
                 const int c = id & 7, rr = id >> 3;
                 const uint4 val = projection8_bf16(prm.pp, m0 + rr, k0 + c * 8);
@@ -624,9 +849,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
               }
               fence_proxy_async_smem();
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(fullA(st));
-            if (++st == STAGES_A) { st = 0; ph ^= 1; }
+            if (!(ok = signal(fullA(st), w))) break;
           }
         }
       }
@@ -635,6 +858,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
 
   tc_fence_before();
   __syncthreads();
+  if (kPair) cluster_sync_all();          // the partner may still signal into this CTA until it is done too
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
@@ -750,17 +974,24 @@ inline bool make_map_f32_3d(CUtensorMap* map, const void* base, int64_t inner, i
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-inline int pick_bn(int N) { return N >= BN_MAX ? BN_MAX : (int)((N + 63) / 64 * 64); }
+// Tile width: up to 256 columns; a CTA pair splits it in two halves of whole 64-column blocks.
+inline int pick_bn(int N, bool pair) {
+  if (N >= BN_MAX) return BN_MAX;
+  const int g = pair ? 128 : 64;
+  return (int)((N + g - 1) / g * g);
+}
 
 #ifndef CFG_NSUB
 #define CFG_NSUB 2
 #endif
 
-inline void finish_problem(Problem& p, int splits_wanted) {
-  if (p.bn == 0) p.bn = pick_bn(p.N);
-  // two row blocks share each B tile: 256 x 256 items halve the L2 -> shared-memory traffic per flop
-  if (p.nsub == 0) p.nsub = p.M > BM ? CFG_NSUB : 1;
-  p.tiles_m = (p.M + BM * p.nsub - 1) / (BM * p.nsub);
+inline void finish_problem(Problem& p, int splits_wanted, bool pair) {
+  p.rows_per_block = pair ? 2 * BM : BM;
+  if (p.bn == 0) p.bn = pick_bn(p.N, pair);
+  // single CTA: two row blocks share each B tile (256 x 256 items halve the shared-memory refill per flop);
+  // CTA pair: one 256-row block per item, accumulators double-buffered
+  if (p.nsub == 0) p.nsub = pair ? 1 : (p.M > BM ? CFG_NSUB : 1);
+  p.tiles_m = (p.M + p.rows_per_block * p.nsub - 1) / (p.rows_per_block * p.nsub);
   p.tiles_n = (p.N + p.bn - 1) / p.bn;
   p.ksteps_total = (p.K + BK - 1) / BK;
   int s = splits_wanted < 1 ? 1 : splits_wanted;
@@ -773,8 +1004,7 @@ inline void finish_problem(Problem& p, int splits_wanted) {
 // (m / 64 k-steps) so that the dynamic scheduler balances well, and there should be enough
 // items to occupy the SMs; at most 32.
 inline int plan_gc_splits(int64_t tokens, int r, int m) {
-  const int nsub = r > BM ? CFG_NSUB : 1;
-  const int items = ((r + BM * nsub - 1) / (BM * nsub)) * ((m + pick_bn(m) - 1) / pick_bn(m));
+  const int items = ((r + 2 * BM - 1) / (2 * BM)) * ((m + pick_bn(m, false) - 1) / pick_bn(m, false));
   const int ksteps = (int)((tokens + BK - 1) / BK);
   if (ksteps < 1) return 1;
   const int dx_ksteps = (m + BK - 1) / BK;
@@ -794,10 +1024,12 @@ inline size_t gc_workspace_bytes(int64_t tokens, int r, int m) {
   return (size_t)plan_gc_splits(tokens, r, m) * r * m * sizeof(float);
 }
 
-inline compact_status_t launch(const LaunchInfo& li, Params& prm) {
+template <bool kPair>
+inline compact_status_t launch_t(const LaunchInfo& li, Params& prm) {
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(compact_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
+    if (cudaFuncSetAttribute(compact_gemm_kernel<kPair>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             Plan<kPair>::SMEM_BYTES) != cudaSuccess) {
       cudaGetLastError();
       return COMPACT_ERR_CUDA;
     }
@@ -811,17 +1043,42 @@ inline compact_status_t launch(const LaunchInfo& li, Params& prm) {
   prm.total_tiles = t;
   prm.status = li.status;
   prm.sched = li.sched;
-  const int grid = t < NUM_SMS ? t : NUM_SMS;
+#ifdef COMPACT_PROFILE
+  prm.debug_flags = getenv("COMPACT_SKIP_MMA") ? 1 : 0;
+#endif
   const int threads = prm.gen_ring != GEN_NONE ? THREADS_GEN : THREADS_BASE;
-  compact_gemm_kernel<<<grid, threads, SMEM_BYTES, li.stream>>>(prm);
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.blockDim = dim3(threads, 1, 1);
+  cfg.dynamicSmemBytes = Plan<kPair>::SMEM_BYTES;
+  cfg.stream = li.stream;
+  cudaLaunchAttribute attr[1];
+  if (kPair) {
+    int pairs = t < NUM_SMS / 2 ? t : NUM_SMS / 2;
+    cfg.gridDim = dim3(2 * pairs, 1, 1);
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+  } else {
+    cfg.gridDim = dim3(t < NUM_SMS ? t : NUM_SMS, 1, 1);
+  }
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, compact_gemm_kernel<kPair>, prm);
   (*li.launches)++;
+  if (e != cudaSuccess) { cudaGetLastError(); return COMPACT_ERR_CUDA; }
   return cudaGetLastError() == cudaSuccess ? COMPACT_OK : COMPACT_ERR_CUDA;
+}
+
+inline compact_status_t launch(const LaunchInfo& li, Params& prm, bool pair) {
+  return pair ? launch_t<true>(li, prm) : launch_t<false>(li, prm);
 }
 
 inline bool tc_shape_ok(int64_t tokens, int n, int m) { return tokens >= 1 && n % 8 == 0 && m % 8 == 0; }
 
 // Algorithm 1: problem 0 = Z = X P (generated B operand; longest items go first), problem 1 = Y = X W.
-inline compact_status_t forward(const LaunchInfo& li, const ProjectionParams& pp, int64_t tokens, int m,
+inline compact_status_t forward(const LaunchInfo& li, bool pair, const ProjectionParams& pp, int64_t tokens, int m,
                                 const __nv_bfloat16* X, int64_t ldx, const __nv_bfloat16* W, int64_t ldw,
                                 __nv_bfloat16* Y, int64_t ldy, __nv_bfloat16* Z, int64_t ldz, int zcols) {
   const int n = pp.n;
@@ -834,26 +1091,28 @@ inline compact_status_t forward(const LaunchInfo& li, const ProjectionParams& pp
   prm.gen_ring = GEN_B;
   Problem& pz = prm.prob[0];
   pz.M = (int)tokens; pz.N = zcols; pz.K = n;
-  // one generated 64 x 128 tile of P feeds up to four row blocks of X (512 tokens)
-  pz.bn = zcols >= 512 / MAX_SUB ? 512 / MAX_SUB : (int)((zcols + 63) / 64 * 64);
-  pz.nsub = (int)((tokens + BM - 1) / BM) < MAX_SUB ? (int)((tokens + BM - 1) / BM) : MAX_SUB;
+  // one generated 64 x 128 tile of P feeds up to four row blocks of X: 512 tokens per CTA,
+  // 1024 per CTA pair (each CTA of a pair generates 64 of the 128 columns)
+  const int rows_pb = pair ? 2 * BM : BM;
+  pz.bn = (zcols >= 512 / MAX_SUB || pair) ? 512 / MAX_SUB : (int)((zcols + 63) / 64 * 64);
+  pz.nsub = (int)((tokens + rows_pb - 1) / rows_pb) < MAX_SUB ? (int)((tokens + rows_pb - 1) / rows_pb) : MAX_SUB;
   pz.a_mode = TMA_KMAJOR; pz.b_mode = GENERATED; pz.epi_mode = EPI_BF16;
-  finish_problem(pz, 1);
+  finish_problem(pz, 1, pair);
   Problem& py = prm.prob[1];
   py.M = (int)tokens; py.N = m; py.K = n;
   py.a_mode = TMA_KMAJOR; py.b_mode = TMA_MNMAJOR; py.epi_mode = EPI_BF16;
-  finish_problem(py, 1);
+  finish_problem(py, 1, pair);
   if (!make_map(&prm.tmA[0], X, n, tokens, ldx, BK, BM)) return COMPACT_ERR_CUDA;
   prm.tmA[1] = prm.tmA[0];
   if (!make_map(&prm.tmB[1], W, m, n, ldw, 64, BK)) return COMPACT_ERR_CUDA;
   prm.tmB[0] = prm.tmB[1];   // unused by the generated operand
   if (!make_map(&prm.tmC[0], Z, zcols, tokens, ldz, 64, 32)) return COMPACT_ERR_CUDA;
   if (!make_map(&prm.tmC[1], Y, m, tokens, ldy, 64, 32)) return COMPACT_ERR_CUDA;
-  return launch(li, prm);
+  return launch(li, prm, pair);
 }
 
 // Algorithm 2: problem 0 = Gc = Z^T dY (both operands MN-major, split over tokens), problem 1 = dX = dY W^T.
-inline compact_status_t backward(const LaunchInfo& li, int64_t tokens, int n, int m, int r, int zcols,
+inline compact_status_t backward(const LaunchInfo& li, bool pair, int64_t tokens, int n, int m, int r, int zcols,
                                  const __nv_bfloat16* dY, int64_t lddy, const __nv_bfloat16* Z, int64_t ldz,
                                  const __nv_bfloat16* W, int64_t ldw, __nv_bfloat16* dX, int64_t lddx, float* Gc,
                                  int64_t ldg, int accumulate, void* workspace, size_t workspace_bytes) {
@@ -869,7 +1128,7 @@ inline compact_status_t backward(const LaunchInfo& li, int64_t tokens, int n, in
   Problem& pg = prm.prob[0];
   pg.M = r; pg.N = m; pg.K = (int)tokens;
   pg.a_mode = TMA_MNMAJOR; pg.b_mode = TMA_MNMAJOR; pg.epi_mode = EPI_F32;
-  finish_problem(pg, splits);
+  finish_problem(pg, splits, pair);
   if (staged) {
     if (!make_map_f32_3d(&prm.tmC[0], workspace, m, r, pg.splits, m, (int64_t)r * m)) return COMPACT_ERR_CUDA;
   } else {
@@ -881,12 +1140,12 @@ inline compact_status_t backward(const LaunchInfo& li, int64_t tokens, int n, in
     Problem& px = prm.prob[1];
     px.M = (int)tokens; px.N = n; px.K = m;
     px.a_mode = TMA_KMAJOR; px.b_mode = TMA_KMAJOR; px.epi_mode = EPI_BF16;
-    finish_problem(px, 1);
+    finish_problem(px, 1, pair);
     if (!make_map(&prm.tmA[1], dY, m, tokens, lddy, BK, BM)) return COMPACT_ERR_CUDA;
-    if (!make_map(&prm.tmB[1], W, m, n, ldw, BK, px.bn)) return COMPACT_ERR_CUDA;
+    if (!make_map(&prm.tmB[1], W, m, n, ldw, BK, pair ? px.bn / 2 : px.bn)) return COMPACT_ERR_CUDA;
     if (!make_map(&prm.tmC[1], dX, n, tokens, lddx, 64, 32)) return COMPACT_ERR_CUDA;
   }
-  compact_status_t s = launch(li, prm);
+  compact_status_t s = launch(li, prm, pair);
   if (s != COMPACT_OK) return s;
   if (staged) {
     const long long cnt = (long long)r * (m / 4);
@@ -920,11 +1179,11 @@ inline compact_status_t update(const LaunchInfo& li, const ProjectionParams& pp,
   pu.nsub = 1;     // one accumulator slot per item keeps the W read-modify-write overlapped with the next item
   pu.a_mode = GENERATED; pu.b_mode = TMA_MNMAJOR; pu.epi_mode = EPI_UPDATE_W;
   pu.scale = scale;
-  finish_problem(pu, 1);
+  finish_problem(pu, 1, false);
   if (!make_map(&prm.tmB[0], Nbuf, m, r, m, 64, BK)) return COMPACT_ERR_CUDA;
   prm.tmA[0] = prm.tmB[0];
   if (!make_map(&prm.tmC[0], W, m, n, ldw, 64, 32)) return COMPACT_ERR_CUDA;
-  return launch(li, prm);
+  return launch(li, prm, false);
 }
 
 }  // namespace tc
