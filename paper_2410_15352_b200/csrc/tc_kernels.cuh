@@ -34,7 +34,8 @@ constexpr int BM = 128;              // rows of one accumulator (TMEM lanes)
 constexpr int BK = 64;               // K elements per pipeline stage (one 128-byte swizzle row)
 constexpr int BN_MAX = 256;          // columns of one accumulator slot (TMEM has two slots)
 constexpr int A_BYTES = BM * BK * 2;
-constexpr int STAGING_BYTES = 4096;      // per epilogue warp: 32 rows x 128 bytes
+constexpr int STAGING_BYTES = 4096;      // one staged tile: 32 rows x 128 bytes
+constexpr int STAGING_BUFS = 2;          // staged tiles per epilogue warp
 constexpr int QDEPTH = 4;                // work items the scheduler may run ahead
 constexpr int NUM_EPI_WARPS = 4;
 constexpr int NUM_GEN_WARPS = 16;
@@ -51,13 +52,19 @@ constexpr int MAX_SUB = CFG_ZSUB;    // row blocks that share one generated B ti
 // kPair = true: two CTAs (one cluster) per item, tcgen05 cta_group::2; each CTA holds its own
 // 128 rows of A and its half of the B tile (16 KB), so the rings are deeper.
 template <bool kPair> struct Plan {
-  static constexpr int STAGES_A = kPair ? 7 : 5;
-  static constexpr int STAGES_B = kPair ? 6 : 4;
+#ifndef CFG_SA
+#define CFG_SA 4
+#endif
+#ifndef CFG_SB
+#define CFG_SB 4
+#endif
+  static constexpr int STAGES_A = kPair ? 6 : CFG_SA;
+  static constexpr int STAGES_B = kPair ? 6 : CFG_SB;
   static constexpr int B_BYTES = (kPair ? BN_MAX / 2 : BN_MAX) * BK * 2;
   static constexpr int RING_BYTES = STAGES_A * A_BYTES + STAGES_B * B_BYTES;
-  static constexpr int NUM_BARRIERS = 2 * STAGES_A + 2 * STAGES_B + 4 + 2 * QDEPTH + NUM_EPI_WARPS;
+  static constexpr int NUM_BARRIERS = 2 * STAGES_A + 2 * STAGES_B + 4 + 2 * QDEPTH + NUM_EPI_WARPS * STAGING_BUFS;
   static constexpr int TAIL_BYTES = 8 * NUM_BARRIERS + 4 * QDEPTH + 16;
-  static constexpr int SMEM_BYTES = 1024 + RING_BYTES + NUM_EPI_WARPS * STAGING_BYTES + ((TAIL_BYTES + 127) / 128) * 128;
+  static constexpr int SMEM_BYTES = 1024 + RING_BYTES + NUM_EPI_WARPS * STAGING_BUFS * STAGING_BYTES + ((TAIL_BYTES + 127) / 128) * 128;
   static constexpr int CTAS = kPair ? 2 : 1;
 };
 static_assert(Plan<false>::SMEM_BYTES <= 232448 && Plan<true>::SMEM_BYTES <= 232448, "shared memory budget");
@@ -76,14 +83,16 @@ __device__ unsigned long long g_prof[8];
 #define PROF_ADD(i, t0) ((void)(t0))
 #endif
 
-// One GEMM inside a launch.  An item is nsub row blocks of 128 rows by bn columns;
-// its nsub accumulators sit side by side in TMEM (nsub * bn <= 512 columns).
+// One GEMM inside a launch.  An item is nsub row blocks (sharing each B tile) by ncol column
+// blocks of bn columns (sharing each A tile; ncol > 1 only with nsub == 1); its accumulators sit
+// side by side in TMEM (nsub * ncol * bn <= 512 columns).
 struct Problem {
   int M, N, K;
   int rows_per_block;   // 128, or 256 when a CTA pair shares the item
   int tiles_m, tiles_n, splits, ksteps_total, ksteps_per_split;
   int bn;
   int nsub;
+  int ncol;
   int a_mode, b_mode, epi_mode;
   int tile_begin;
   float scale;
@@ -259,6 +268,7 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t sr
 }
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
@@ -328,7 +338,7 @@ __device__ __forceinline__ uint4 projection8_bf16(const ProjectionParams& pp, in
 }
 
 struct TileCoord {
-  int prob, m0, n0, k_begin, k_end, split, nsub;
+  int prob, m0, n0, k_begin, k_end, split, nsub, ncol;
 };
 
 __device__ __forceinline__ TileCoord decode_tile(const Params& prm, int tile) {
@@ -341,10 +351,11 @@ __device__ __forceinline__ TileCoord decode_tile(const Params& prm, int tile) {
   const int mb = local % p.tiles_m;
   t.split = local / p.tiles_m;
   t.m0 = mb * p.rows_per_block * p.nsub;
-  t.n0 = nb * p.bn;
+  t.n0 = nb * p.bn * p.ncol;
   t.k_begin = t.split * p.ksteps_per_split;
   t.k_end = min(p.ksteps_total, t.k_begin + p.ksteps_per_split);
   t.nsub = min(p.nsub, (p.M - t.m0 + p.rows_per_block - 1) / p.rows_per_block);   // row blocks with a valid row
+  t.ncol = min(p.ncol, (p.N - t.n0 + p.bn - 1) / p.bn);                            // column blocks with a valid column
   return t;
 }
 
@@ -368,7 +379,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));   // generic pointer to the aligned base
   const uint32_t ringA = smem_base, ringB = smem_base + STAGES_A * A_BYTES;
   const uint32_t staging = smem_base + RING_BYTES;
-  const uint32_t bars = staging + NUM_EPI_WARPS * STAGING_BYTES;
+  const uint32_t bars = staging + NUM_EPI_WARPS * STAGING_BUFS * STAGING_BYTES;
   // barrier slots (8 bytes each)
   auto fullA = [&](int s) { return bars + 8u * s; };
   auto emptyA = [&](int s) { return bars + 8u * (STAGES_A + s); };
@@ -381,7 +392,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
   auto qempty = [&](int s) { return bars + 8u * (kT + 4 + QDEPTH + s); };
   auto wbar = [&](int w) { return bars + 8u * (kT + 4 + 2 * QDEPTH + w); };
   const uint32_t tail_u32 = bars + 8 * PL::NUM_BARRIERS;
-  uint8_t* tail = smem_gen + RING_BYTES + NUM_EPI_WARPS * STAGING_BYTES + 8 * PL::NUM_BARRIERS;
+  uint8_t* tail = smem_gen + RING_BYTES + NUM_EPI_WARPS * STAGING_BUFS * STAGING_BYTES + 8 * PL::NUM_BARRIERS;
   volatile int* tile_q = reinterpret_cast<volatile int*>(tail);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail + 4 * QDEPTH);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 4 * QDEPTH + 8);
@@ -420,7 +431,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       mbar_init(qfull(s), 1);
       mbar_init(qempty(s), consumers);
     }
-    for (int w = 0; w < NUM_EPI_WARPS; ++w) mbar_init(wbar(w), 1);
+    for (int w = 0; w < NUM_EPI_WARPS * STAGING_BUFS; ++w) mbar_init(wbar(w), 1);
     *abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async_smem();
@@ -481,15 +492,22 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const Problem& p = prm.prob[t.prob];
         const CUtensorMap* mapB = &prm.tmB[t.prob];
         const int bn_cta = p.bn / NCTA;                 // B columns this CTA holds
-        const int n0 = t.n0 + (int)rank * bn_cta;
-        for (int ks = t.k_begin; ks < t.k_end && ok; ++ks, ++ib) {
+        const int n_first = t.n0 + (int)rank * bn_cta;
+        for (int kc = 0; kc < (t.k_end - t.k_begin) * t.ncol && ok; ++kc, ++ib) {
           if ((int)(ib % NUM_PROD) != prodB) continue;
           const int sb = (int)(ib % STAGES_B);
           const uint32_t phb = (ib / STAGES_B) & 1u;
-          const int k0 = ks * BK;
+          const int k0 = (t.k_begin + kc / t.ncol) * BK;
+          const int n0 = n_first + (kc % t.ncol) * p.bn;
           // B tile of this k-step (shared by all row blocks of the item)
           if (!(ok = mbar_wait(emptyB(sb), phb ^ 1, abort_flag, prm.status))) break;
           const uint32_t dst = ringB + sb * B_BYTES, fb = fullB(sb);
+#if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
+          if ((prm.debug_flags & 2) && p.b_mode != GENERATED) {          // no loads: MMAs run on whatever is in the ring
+            if (leader) mbar_arrive_n(fb, 1 + (prm.gen_ring == GEN_B ? GEN_ARRIVALS : 0));
+            continue;
+          }
+#endif
           if (p.b_mode == GENERATED) {
             if (leader) mbar_arrive(fb);                                 // the generator groups arrive for the data
           } else {
@@ -539,7 +557,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const bool b_mn = p.b_mode != TMA_KMAJOR;          // generated B tiles are written MN-major
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
                                ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)((NCTA * BM) >> 4) << 24);
-        const int slots = (p.nsub * p.bn + BN_MAX - 1) / BN_MAX;   // accumulator slots this item occupies
+        const int slots = (p.nsub * p.ncol * p.bn + BN_MAX - 1) / BN_MAX;   // accumulator slots this item occupies
         const long long tp0 = PROF_T();
         if (slots == 2 && acc == 1) {
           // a two-slot item starts at slot 0: pass slot 1 through unused
@@ -559,13 +577,45 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const uint32_t d_base = tmem_base + acc0 * BN_MAX;
         // one UMMA consumes K = 16: 32 bytes along a K-major row, or two 8-row groups (2048 bytes) MN-major
         const uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4), b_step = b_mn ? (2048u >> 4) : (32u >> 4);
-        const int nsub = t.nsub, bn = p.bn;
+        const int nsub = t.nsub, ncol = t.ncol, bn = p.bn;
+        auto issue4 = [&](uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t first) {
+#if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
+          if (prm.debug_flags & 1) return;
+#endif
+          if (kPair) {
+            umma_bf16_pair(d, a_lo, DESC_HI, b_lo, DESC_HI, idesc, first);
+            umma_bf16_pair(d, a_lo + a_step, DESC_HI, b_lo + b_step, DESC_HI, idesc, 1u);
+            umma_bf16_pair(d, a_lo + 2 * a_step, DESC_HI, b_lo + 2 * b_step, DESC_HI, idesc, 1u);
+            umma_bf16_pair(d, a_lo + 3 * a_step, DESC_HI, b_lo + 3 * b_step, DESC_HI, idesc, 1u);
+          } else {
+            umma_bf16(d, a_lo, DESC_HI, b_lo, DESC_HI, idesc, first);
+            umma_bf16(d, a_lo + a_step, DESC_HI, b_lo + b_step, DESC_HI, idesc, 1u);
+            umma_bf16(d, a_lo + 2 * a_step, DESC_HI, b_lo + 2 * b_step, DESC_HI, idesc, 1u);
+            umma_bf16(d, a_lo + 3 * a_step, DESC_HI, b_lo + 3 * b_step, DESC_HI, idesc, 1u);
+          }
+        };
         for (int ks = t.k_begin; ks < t.k_end && ok; ++ks) {
+          const uint32_t first = ks > t.k_begin ? 1u : 0u;
+          if (p.ncol > 1) {
+            // one A tile, several B tiles (column blocks)
+            if (!(ok = mbar_wait(fullA(sa), pha, abort_flag, prm.status))) break;
+            const uint32_t a_lo = desc_lo(ringA + sa * A_BYTES, a_mn);
+            for (int cb = 0; cb < ncol; ++cb) {
+              if (!(ok = mbar_wait(fullB(sb), phb, abort_flag, prm.status))) break;
+              tc_fence_after();
+              issue4(d_base + cb * bn, a_lo, desc_lo(ringB + sb * B_BYTES, b_mn), first);
+              commit(emptyB(sb));
+              if (++sb == STAGES_B) { sb = 0; phb ^= 1; }
+            }
+            if (!ok) break;
+            commit(emptyA(sa));
+            if (++sa == STAGES_A) { sa = 0; pha ^= 1; }
+            continue;
+          }
           const long long tp1 = PROF_T();
           if (!(ok = mbar_wait(fullB(sb), phb, abort_flag, prm.status))) break;
           PROF_ADD(1, tp1);
           const uint32_t b_lo = desc_lo(ringB + sb * B_BYTES, b_mn);
-          const uint32_t first = ks > t.k_begin ? 1u : 0u;
           for (int mi = 0; mi < nsub; ++mi) {
             const long long tp2 = PROF_T();
             if (!(ok = mbar_wait(fullA(sa), pha, abort_flag, prm.status))) break;
@@ -574,23 +624,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             tc_fence_after();
             PROF_ADD(7, tp7);
             const long long tp3 = PROF_T();
-            const uint32_t a_lo = desc_lo(ringA + sa * A_BYTES, a_mn);
-            const uint32_t d = d_base + mi * bn;
-#ifdef COMPACT_PROFILE
-            if (prm.debug_flags & 1) {
-            } else
-#endif
-            if (kPair) {
-              umma_bf16_pair(d, a_lo, DESC_HI, b_lo, DESC_HI, idesc, first);
-              umma_bf16_pair(d, a_lo + a_step, DESC_HI, b_lo + b_step, DESC_HI, idesc, 1u);
-              umma_bf16_pair(d, a_lo + 2 * a_step, DESC_HI, b_lo + 2 * b_step, DESC_HI, idesc, 1u);
-              umma_bf16_pair(d, a_lo + 3 * a_step, DESC_HI, b_lo + 3 * b_step, DESC_HI, idesc, 1u);
-            } else {
-              umma_bf16(d, a_lo, DESC_HI, b_lo, DESC_HI, idesc, first);
-              umma_bf16(d, a_lo + a_step, DESC_HI, b_lo + b_step, DESC_HI, idesc, 1u);
-              umma_bf16(d, a_lo + 2 * a_step, DESC_HI, b_lo + 2 * b_step, DESC_HI, idesc, 1u);
-              umma_bf16(d, a_lo + 3 * a_step, DESC_HI, b_lo + 3 * b_step, DESC_HI, idesc, 1u);
-            }
+            issue4(d_base + mi * bn, desc_lo(ringA + sa * A_BYTES, a_mn), b_lo, first);
             commit(emptyA(sa));
             PROF_ADD(3, tp3);
             if (++sa == STAGES_A) { sa = 0; pha ^= 1; }
@@ -609,17 +643,28 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       unsigned long long ns1;
       asm volatile("mov.u64 %0, %globaltimer;" : "=l"(ns1));
       prof[5] = ns1 - ns0;
-      for (int i = 0; i < 8; ++i) atomicAdd(&g_prof[i], prof[i]);
+#ifndef COMPACT_PROFILE_EPI
+      for (int i = 0; i < 6; ++i) atomicAdd(&g_prof[i], prof[i]);
+#endif
 #endif
     }
   } else if (warp < 2 + NUM_EPI_WARPS) {
     // ------------------------------ epilogue ------------------------------------
-    // TMEM -> registers -> 128B-swizzled staging tile (32 rows x 128 bytes per warp) -> TMA store.
+    // TMEM -> registers -> 128B-swizzled staging tile (32 rows x 128 bytes, two per warp) -> TMA store.
+    // The chunks of an item (accumulator by accumulator, 64 bf16 or 32 fp32 columns at a time) are
+    // walked as one flat sequence so that the W tile of the next chunk (update) is already on its way
+    // while the current one is processed.
     const int q = warp & 3;                 // TMEM lane quarter this warp may read
-    const uint32_t stg = staging + (warp - 2) * STAGING_BYTES;
-    uint8_t* stg_gen = smem_gen + RING_BYTES + (warp - 2) * STAGING_BYTES;
-    const uint32_t my_wbar = wbar(warp - 2);
-    uint32_t wph = 0;
+    const uint32_t stg0 = staging + (warp - 2) * STAGING_BUFS * STAGING_BYTES;
+    uint8_t* stg_gen0 = smem_gen + RING_BYTES + (warp - 2) * STAGING_BUFS * STAGING_BYTES;
+    uint32_t wph[STAGING_BUFS] = {0, 0};
+    int buf = 0;
+#ifdef COMPACT_PROFILE
+    long long eprof_drain = 0, eprof_wait = 0;
+#endif
+#ifdef COMPACT_PROFILE_EPI
+    long long ep[4] = {0, 0, 0, 0};
+#endif
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
@@ -630,8 +675,42 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       const TileCoord t = decode_tile(prm, tile);
       const Problem& p = prm.prob[t.prob];
       const CUtensorMap* mapC = &prm.tmC[t.prob];
-      const int slots = (p.nsub * p.bn + BN_MAX - 1) / BN_MAX;
-      const int sub_per_slot = BN_MAX / p.bn > p.nsub ? p.nsub : BN_MAX / p.bn;
+      const int naccs = p.nsub * p.ncol;
+      const int slots = (naccs * p.bn + BN_MAX - 1) / BN_MAX;
+      const int sub_per_slot = BN_MAX / p.bn > naccs ? naccs : BN_MAX / p.bn;
+      const int cw = p.epi_mode == EPI_F32 ? 32 : 64;          // columns per staged chunk
+      const int cpa = p.bn / cw;                               // chunks per accumulator
+      // Cursor over the chunks this warp writes: accumulator ai (slot sl, position su in the slot), chunk ci.
+      struct Cur { int ai, sl, su, ci; };
+      const int row_q = (int)rank * BM + q * 32;
+      auto acc_valid = [&](int ai) -> bool {       // does accumulator ai hold rows/columns this warp writes?
+        const int mi = p.ncol > 1 ? 0 : ai, cb = p.ncol > 1 ? ai : 0;
+        return mi < t.nsub && cb < t.ncol && t.m0 + mi * p.rows_per_block + row_q < p.M && t.n0 + cb * p.bn < p.N;
+      };
+      auto cur_col = [&](const Cur& c) -> int { return t.n0 + (p.ncol > 1 ? c.ai : 0) * p.bn + c.ci * cw; };
+      auto cur_row = [&](const Cur& c) -> int { return t.m0 + (p.ncol > 1 ? 0 : c.ai) * p.rows_per_block + row_q; };
+      // first valid chunk at or after (ai, ci = 0)
+      auto seek = [&](Cur c) -> Cur {
+        while (c.ai < naccs && !acc_valid(c.ai)) {
+          ++c.ai;
+          if (++c.su == sub_per_slot) { c.su = 0; ++c.sl; }
+        }
+        c.ci = 0;
+        return c;
+      };
+      auto advance = [&](Cur c) -> Cur {
+        ++c.ci;
+        if (c.ci < cpa && cur_col(c) < p.N) return c;
+        ++c.ai;
+        if (++c.su == sub_per_slot) { c.su = 0; ++c.sl; }
+        return seek(c);
+      };
+      auto load_w = [&](const Cur& c, int b) {      // update: W tile of chunk c into staging buffer b
+        if (lane == 0) {
+          mbar_arrive_expect_tx(wbar((warp - 2) * STAGING_BUFS + b), STAGING_BYTES);
+          tma_load_2d(stg0 + b * STAGING_BYTES, mapC, wbar((warp - 2) * STAGING_BUFS + b), cur_col(c), cur_row(c));
+        }
+      };
       if (slots == 2 && acc == 1) {
         if (!(ok = mbar_wait(tfull_bar(1), acc_phase, abort_flag, prm.status))) break;
         __syncwarp();
@@ -639,100 +718,152 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         acc = 0;
         acc_phase ^= 1;
       }
-      for (int sl = 0; sl < slots && ok; ++sl) {
-        if (!(ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, prm.status))) break;
-        tc_fence_after();
-        for (int su = 0; su < sub_per_slot && ok; ++su) {
-          const int mi = sl * sub_per_slot + su;
-          if (mi >= t.nsub) break;
-          const int row0 = t.m0 + mi * p.rows_per_block + (int)rank * BM + q * 32;
-          if (row0 >= p.M) continue;          // this warp's 32 rows are all padding
-          const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN_MAX + su * p.bn;
-          if (p.epi_mode == EPI_F32) {
-            // fp32 output: 32 columns (128 bytes) per staged tile
-            for (int c0 = 0; c0 < p.bn; c0 += 32) {
-              const int col = t.n0 + c0;
-              if (col >= p.N) break;
-              uint32_t v[32];
-              tmem_ld32(tcol + c0, v);
-              if (lane == 0) tma_store_wait_read();
-              __syncwarp();
-              tmem_ld_wait();
+      Cur cur = seek(Cur{0, 0, 0, 0});
+#if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
+      if (prm.debug_flags & 4) cur.ai = naccs;       // write nothing: hand the accumulators straight back
+#endif
+      if (p.epi_mode == EPI_UPDATE_W && cur.ai < naccs) {
+        if (lane == 0) tma_store_wait_read();          // both staging buffers are free
+        __syncwarp();
+        load_w(cur, buf);
+      }
+      int cur_slot = -1;
+#ifdef COMPACT_PROFILE
+      long long t_slot = 0;
+#endif
+      // enter accumulator slot `want` (waiting for its MMAs), handing back the slots passed on the way
+      auto enter_slot = [&](int want) -> bool {
+        while (cur_slot < want) {
+          if (cur_slot >= 0) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) arrive_leader(tempty_bar(acc));
+            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+          }
+          ++cur_slot;
+#ifdef COMPACT_PROFILE
+          const long long tw0 = clock64();
+          if (t_slot) eprof_drain += tw0 - t_slot;
+#endif
+          if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, prm.status)) return false;
+#ifdef COMPACT_PROFILE
+          t_slot = clock64();
+          eprof_wait += t_slot - tw0;
+#endif
+          tc_fence_after();
+        }
+        return true;
+      };
+      while (cur.ai < naccs && ok) {
+        const int sl = cur.sl, tc = cur.su * p.bn + cur.ci * cw, col = cur_col(cur), row0 = cur_row(cur);
+        const Cur nxt = advance(cur);
+        uint8_t* stg_gen = stg_gen0 + buf * STAGING_BYTES;
+        const uint32_t stg = stg0 + buf * STAGING_BYTES;
+        if (p.epi_mode == EPI_UPDATE_W) {
+          if (nxt.ai < naccs) {
+            if (lane == 0) tma_store_wait_read();      // the other buffer's store has read it
+            __syncwarp();
+            load_w(nxt, buf ^ 1);
+          }
+        } else {
+#ifdef COMPACT_PROFILE_EPI
+          const long long te0 = clock64();
+#endif
+          if (lane == 0) tma_store_wait_read1();       // this buffer's previous store has read it
+          __syncwarp();
+#ifdef COMPACT_PROFILE_EPI
+          ep[0] += clock64() - te0;
+#endif
+        }
+        if (!(ok = enter_slot(sl))) break;
+#ifdef COMPACT_PROFILE_EPI
+        const long long te1 = clock64();
+#endif
+        const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN_MAX + tc;
+        if (p.epi_mode == EPI_F32) {
+          uint32_t v[32];
+          tmem_ld32(tcol, v);
+          tmem_ld_wait();
 #pragma unroll
-              for (int j = 0; j < 8; ++j)
-                *reinterpret_cast<uint4*>(stg_gen + lane * 128 + ((j ^ sw) << 4)) =
-                    make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-              fence_proxy_async_smem();
-              __syncwarp();
-              if (lane == 0) {
-                tma_store_3d(mapC, stg, col, row0, t.split);
-                tma_store_commit();
+          for (int j = 0; j < 8; ++j)
+            *reinterpret_cast<uint4*>(stg_gen + lane * 128 + ((j ^ sw) << 4)) =
+                make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_3d(mapC, stg, col, row0, t.split);
+            tma_store_commit();
+          }
+        } else {
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            uint32_t v[32];
+            tmem_ld32(tcol + 32 * h, v);
+            tmem_ld_wait();
+            if (p.epi_mode == EPI_UPDATE_W) {
+              // W <- W - (eta alpha) (P N), one rounding of the result (Algorithm 3 line 9)
+              if (h == 0) {
+                if (!(ok = mbar_wait(wbar((warp - 2) * STAGING_BUFS + buf), wph[buf], abort_flag, prm.status))) break;
+                wph[buf] ^= 1;
               }
-            }
-          } else {
-            // bf16 output: 64 columns (128 bytes) per staged tile
-            for (int c0 = 0; c0 < p.bn; c0 += 64) {
-              const int col = t.n0 + c0;
-              if (col >= p.N) break;
-              if (lane == 0) tma_store_wait_read();
-              __syncwarp();
-              if (p.epi_mode == EPI_UPDATE_W) {
-                // bring the W tile in first: W <- W - (eta alpha) (P N), one rounding (Algorithm 3 line 9)
-                if (lane == 0) {
-                  mbar_arrive_expect_tx(my_wbar, STAGING_BYTES);
-                  tma_load_2d(stg, mapC, my_wbar, col, row0);
-                }
+              const float sc = -p.scale;
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                uint4* cell = reinterpret_cast<uint4*>(stg_gen + lane * 128 + (((4 * h + j) ^ sw) << 4));
+                uint4 w = *cell;
+                w.x = pack_bf16x2(fmaf(sc, __uint_as_float(v[8 * j + 0]), bf16lo(w.x)), fmaf(sc, __uint_as_float(v[8 * j + 1]), bf16hi(w.x)));
+                w.y = pack_bf16x2(fmaf(sc, __uint_as_float(v[8 * j + 2]), bf16lo(w.y)), fmaf(sc, __uint_as_float(v[8 * j + 3]), bf16hi(w.y)));
+                w.z = pack_bf16x2(fmaf(sc, __uint_as_float(v[8 * j + 4]), bf16lo(w.z)), fmaf(sc, __uint_as_float(v[8 * j + 5]), bf16hi(w.z)));
+                w.w = pack_bf16x2(fmaf(sc, __uint_as_float(v[8 * j + 6]), bf16lo(w.w)), fmaf(sc, __uint_as_float(v[8 * j + 7]), bf16hi(w.w)));
+                *cell = w;
               }
+            } else {
 #pragma unroll
-              for (int h = 0; h < 2; ++h) {
-                uint32_t v[32];
-                tmem_ld32(tcol + c0 + 32 * h, v);
-                tmem_ld_wait();
-                if (p.epi_mode == EPI_UPDATE_W) {
-                  if (h == 0) {
-                    if (!(ok = mbar_wait(my_wbar, wph, abort_flag, prm.status))) break;
-                    wph ^= 1;
-                  }
-                  const float s = -p.scale;
-#pragma unroll
-                  for (int j = 0; j < 4; ++j) {
-                    uint4* cell = reinterpret_cast<uint4*>(stg_gen + lane * 128 + (((4 * h + j) ^ sw) << 4));
-                    uint4 w = *cell;
-                    w.x = pack_bf16x2(fmaf(s, __uint_as_float(v[8 * j + 0]), bf16lo(w.x)), fmaf(s, __uint_as_float(v[8 * j + 1]), bf16hi(w.x)));
-                    w.y = pack_bf16x2(fmaf(s, __uint_as_float(v[8 * j + 2]), bf16lo(w.y)), fmaf(s, __uint_as_float(v[8 * j + 3]), bf16hi(w.y)));
-                    w.z = pack_bf16x2(fmaf(s, __uint_as_float(v[8 * j + 4]), bf16lo(w.z)), fmaf(s, __uint_as_float(v[8 * j + 5]), bf16hi(w.z)));
-                    w.w = pack_bf16x2(fmaf(s, __uint_as_float(v[8 * j + 6]), bf16lo(w.w)), fmaf(s, __uint_as_float(v[8 * j + 7]), bf16hi(w.w)));
-                    *cell = w;
-                  }
-                } else {
-#pragma unroll
-                  for (int j = 0; j < 4; ++j) {
-                    uint4 o;
-                    o.x = pack_bf16x2(__uint_as_float(v[8 * j + 0]), __uint_as_float(v[8 * j + 1]));
-                    o.y = pack_bf16x2(__uint_as_float(v[8 * j + 2]), __uint_as_float(v[8 * j + 3]));
-                    o.z = pack_bf16x2(__uint_as_float(v[8 * j + 4]), __uint_as_float(v[8 * j + 5]));
-                    o.w = pack_bf16x2(__uint_as_float(v[8 * j + 6]), __uint_as_float(v[8 * j + 7]));
-                    *reinterpret_cast<uint4*>(stg_gen + lane * 128 + (((4 * h + j) ^ sw) << 4)) = o;
-                  }
-                }
-              }
-              if (!ok) break;
-              fence_proxy_async_smem();
-              __syncwarp();
-              if (lane == 0) {
-                tma_store_2d(mapC, stg, col, row0);
-                tma_store_commit();
+              for (int j = 0; j < 4; ++j) {
+                uint4 o;
+                o.x = pack_bf16x2(__uint_as_float(v[8 * j + 0]), __uint_as_float(v[8 * j + 1]));
+                o.y = pack_bf16x2(__uint_as_float(v[8 * j + 2]), __uint_as_float(v[8 * j + 3]));
+                o.z = pack_bf16x2(__uint_as_float(v[8 * j + 4]), __uint_as_float(v[8 * j + 5]));
+                o.w = pack_bf16x2(__uint_as_float(v[8 * j + 6]), __uint_as_float(v[8 * j + 7]));
+                *reinterpret_cast<uint4*>(stg_gen + lane * 128 + (((4 * h + j) ^ sw) << 4)) = o;
               }
             }
           }
+          if (!ok) break;
+#ifdef COMPACT_PROFILE_EPI
+          const long long te2 = clock64();
+          ep[1] += te2 - te1;
+#endif
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_2d(mapC, stg, col, row0);
+            tma_store_commit();
+          }
+#ifdef COMPACT_PROFILE_EPI
+          ep[2] += clock64() - te2;
+          ep[3] += 1;
+#endif
         }
-        if (!ok) break;
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) arrive_leader(tempty_bar(acc));
-        if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+        buf ^= 1;
+        cur = nxt;
       }
+      if (!ok) break;
+      if (!(ok = enter_slot(slots - 1))) break;      // slots this warp had nothing to write for
+      tc_fence_before();
+      __syncwarp();
+#ifdef COMPACT_PROFILE
+      eprof_drain += clock64() - t_slot;
+#endif
+      if (lane == 0) arrive_leader(tempty_bar(acc));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1; }
     }
+#ifdef COMPACT_PROFILE_EPI
+    if (warp == 2 && lane == 0 && leader) for (int i = 0; i < 4; ++i) atomicAdd(&g_prof[i], (unsigned long long)ep[i]);
+#endif
+#ifdef COMPACT_PROFILE
+    if (warp == 2 && lane == 0 && leader) { atomicAdd(&g_prof[6], (unsigned long long)eprof_drain); atomicAdd(&g_prof[7], (unsigned long long)eprof_wait); }
+#endif
     if (lane == 0) tma_store_wait_all();
   } else if (prodA >= 0) {
     // ------------------------------ producers of A tiles ------------------------
@@ -754,6 +885,12 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             if (!(ok = mbar_wait(emptyA(sa), pha ^ 1, abort_flag, prm.status))) break;
             const uint32_t dst = ringA + sa * A_BYTES, fa = fullA(sa);
             const int m0 = t.m0 + mi * p.rows_per_block + (int)rank * BM;
+#if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
+            if ((prm.debug_flags & 2) && p.a_mode != GENERATED) {
+              if (leader) mbar_arrive_n(fa, 1 + (prm.gen_ring == GEN_A ? GEN_ARRIVALS : 0));
+              continue;
+            }
+#endif
             if (p.a_mode == GENERATED) {
               if (leader) mbar_arrive(fa);
             } else {
@@ -812,7 +949,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       const Problem& p = prm.prob[t.prob];
       const int klen = t.k_end - t.k_begin;
       if (prm.gen_ring == GEN_B) {
-        if (p.b_mode != GENERATED) { it += klen; continue; }      // the producer arrives for this item
+        if (p.b_mode != GENERATED) { it += klen * t.ncol; continue; }      // the producer arrives for this item
         const int bn_cta = p.bn / NCTA;
         const int n0 = t.n0 + (int)rank * bn_cta;
         const int chunks = bn_cta >> 3;
@@ -991,8 +1128,9 @@ inline void finish_problem(Problem& p, int splits_wanted, bool pair) {
   // single CTA: two row blocks share each B tile (256 x 256 items halve the shared-memory refill per flop);
   // CTA pair: one 256-row block per item, accumulators double-buffered
   if (p.nsub == 0) p.nsub = pair ? 1 : (p.M > BM ? CFG_NSUB : 1);
+  if (p.ncol == 0) p.ncol = 1;
   p.tiles_m = (p.M + p.rows_per_block * p.nsub - 1) / (p.rows_per_block * p.nsub);
-  p.tiles_n = (p.N + p.bn - 1) / p.bn;
+  p.tiles_n = (p.N + p.bn * p.ncol - 1) / (p.bn * p.ncol);
   p.ksteps_total = (p.K + BK - 1) / BK;
   int s = splits_wanted < 1 ? 1 : splits_wanted;
   if (s > p.ksteps_total) s = p.ksteps_total;
@@ -1043,8 +1181,8 @@ inline compact_status_t launch_t(const LaunchInfo& li, Params& prm) {
   prm.total_tiles = t;
   prm.status = li.status;
   prm.sched = li.sched;
-#ifdef COMPACT_PROFILE
-  prm.debug_flags = getenv("COMPACT_SKIP_MMA") ? 1 : 0;
+#if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
+  prm.debug_flags = (getenv("COMPACT_SKIP_MMA") ? 1 : 0) | (getenv("COMPACT_SKIP_LOADS") ? 2 : 0) | (getenv("COMPACT_SKIP_EPI") ? 4 : 0);
 #endif
   const int threads = prm.gen_ring != GEN_NONE ? THREADS_GEN : THREADS_BASE;
   cudaLaunchConfig_t cfg;
@@ -1176,7 +1314,8 @@ inline compact_status_t update(const LaunchInfo& li, const ProjectionParams& pp,
   prm.gen_ring = GEN_A;
   Problem& pu = prm.prob[0];
   pu.M = n; pu.N = m; pu.K = r;
-  pu.nsub = 1;     // one accumulator slot per item keeps the W read-modify-write overlapped with the next item
+  pu.nsub = 1;
+  pu.ncol = m > BN_MAX ? 2 : 1;     // the generator is the bound here: one generated tile of P feeds two column blocks
   pu.a_mode = GENERATED; pu.b_mode = TMA_MNMAJOR; pu.epi_mode = EPI_UPDATE_W;
   pu.scale = scale;
   finish_problem(pu, 1, false);
