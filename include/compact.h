@@ -181,9 +181,7 @@ compact_status_t compact_debug_projection(const compact_layer_t* layer, uint32_t
 
 /* Selects the kernel family: 0 = automatic (tensor-core kernels for bf16 where
  * the shape allows, SIMT otherwise), 1 = force the SIMT kernels (used by the
- * tests as an on-device cross-check), 2 = same as 0, 3 = tensor-core kernels
- * with CTA pairs (tcgen05 cta_group::2) for the forward and backward.
- * Returns the previous value. */
+ * tests as an on-device cross-check).  Returns the previous value. */
 int compact_set_kernel_family(int family);
 
 /* Number of kernels this library has launched since it was loaded. */

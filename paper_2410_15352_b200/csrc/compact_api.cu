@@ -90,9 +90,6 @@ void simt_gemm(int M, int N, int K, AF a, BF b, EP ep, cudaStream_t st) {
   g_launches++;
 }
 
-// CTA pairs (tcgen05 cta_group::2) are opt-in (family 3): at today's tuning the one-CTA items are faster.
-inline bool use_pair(int64_t tokens) { return g_family.load() == 3 && tokens > 128; }
-
 inline bool pitch_ok(int64_t ld, int64_t min_cols, size_t es) { return ld >= min_cols && (ld * (int64_t)es) % 16 == 0; }
 
 // ---- forward ---------------------------------------------------------------------------
@@ -220,7 +217,7 @@ compact_status_t compact_linear_fwd(compact_layer_t* L, int64_t tokens, const vo
     typedef __nv_bfloat16 T;
     if (g_family.load() != 1) {
       tc::LaunchInfo li{st, status_word(L), sched_words(L), &g_launches};
-      s = tc::forward(li, use_pair(tokens), make_pp(L, L->epoch), tokens, L->cfg.m, (const T*)X, ldx, (const T*)W, ldw, (T*)Y, ldy, (T*)Z, ldz,
+      s = tc::forward(li, make_pp(L, L->epoch), tokens, L->cfg.m, (const T*)X, ldx, (const T*)W, ldw, (T*)Y, ldy, (T*)Z, ldz,
                       (int)compact_z_ld(L));
       if (s != COMPACT_ERR_SHAPE) return s;   // SHAPE: the tensor-core kernel does not take it
     }
@@ -262,7 +259,7 @@ compact_status_t compact_linear_bwd(compact_layer_t* L, int64_t tokens, const vo
     typedef __nv_bfloat16 T;
     if (g_family.load() != 1) {
       tc::LaunchInfo li{st, status_word(L), sched_words(L), &g_launches};
-      s = tc::backward(li, use_pair(tokens), tokens, L->cfg.n, L->cfg.m, L->cfg.r, (int)compact_z_ld(L), (const T*)dY, lddy, (const T*)Z, ldz, (const T*)W,
+      s = tc::backward(li, tokens, L->cfg.n, L->cfg.m, L->cfg.r, (int)compact_z_ld(L), (const T*)dY, lddy, (const T*)Z, ldz, (const T*)W,
                        ldw, (T*)dX, lddx, Gc, ldg, accumulate, workspace, workspace_bytes);
       if (s != COMPACT_ERR_SHAPE) return s;
     }
@@ -420,7 +417,7 @@ compact_status_t compact_debug_projection(const compact_layer_t* L, uint32_t epo
 }
 
 int compact_set_kernel_family(int family) {
-  if (family < 0 || family > 3) return g_family.load();
+  if (family < 0 || family > 1) return g_family.load();
   return g_family.exchange(family);
 }
 

@@ -34,40 +34,31 @@ constexpr int BM = 128;              // rows of one accumulator (TMEM lanes)
 constexpr int BK = 64;               // K elements per pipeline stage (one 128-byte swizzle row)
 constexpr int BN_MAX = 256;          // columns of one accumulator slot (TMEM has two slots)
 constexpr int A_BYTES = BM * BK * 2;
+constexpr int B_BYTES = BN_MAX * BK * 2;
+// One pipeline stage holds a B tile and two A tiles under ONE full/empty barrier pair: every
+// mbarrier operation of the MMA-issuing thread costs ~150 clocks of its serial time, so a stage
+// carries as many MMAs (8) as fit.
+constexpr int STAGE_B_OFF = 0, STAGE_A0_OFF = B_BYTES, STAGE_A1_OFF = B_BYTES + A_BYTES;
+constexpr int STAGE_BYTES = B_BYTES + 2 * A_BYTES;
+#ifndef CFG_NS
+#define CFG_NS 3
+#endif
+constexpr int NS = CFG_NS;               // stages in the ring
+constexpr int RING_BYTES = NS * STAGE_BYTES;
 constexpr int STAGING_BYTES = 4096;      // one staged tile: 32 rows x 128 bytes
 constexpr int STAGING_BUFS = 2;          // staged tiles per epilogue warp
 constexpr int QDEPTH = 4;                // work items the scheduler may run ahead
 constexpr int NUM_EPI_WARPS = 4;
 constexpr int NUM_GEN_WARPS = 16;
-constexpr int NUM_PROD = 2;              // producer threads per operand ring (each in its own warp)
-constexpr int THREADS_BASE = 64 + 32 * NUM_EPI_WARPS + 32 * (2 * NUM_PROD - 1);   // scheduler + B producer, MMA, epilogue, other producers
+constexpr int NUM_LOADERS = 3;           // loader threads besides the stage owner: A0, A1, upper half of B
+constexpr int THREADS_BASE = 64 + 32 * NUM_EPI_WARPS + 32 * NUM_LOADERS;   // owner/scheduler, MMA, epilogue, loaders
 constexpr int THREADS_GEN = THREADS_BASE + 32 * NUM_GEN_WARPS;
+constexpr int NUM_BARRIERS = 2 * NS + 4 + 2 * QDEPTH + NUM_EPI_WARPS * STAGING_BUFS;
+constexpr int TAIL_BYTES = 8 * NUM_BARRIERS + 4 * QDEPTH + 16;
+constexpr int SMEM_BYTES = 1024 + RING_BYTES + NUM_EPI_WARPS * STAGING_BUFS * STAGING_BYTES + ((TAIL_BYTES + 127) / 128) * 128;
 constexpr int NUM_SMS = 148;
-#ifndef CFG_ZSUB
-#define CFG_ZSUB 4
-#endif
-constexpr int MAX_SUB = CFG_ZSUB;    // row blocks that share one generated B tile
-
-// Shared-memory plan.  kPair = false: one CTA per item, B tiles up to 256 columns (32 KB).
-// kPair = true: two CTAs (one cluster) per item, tcgen05 cta_group::2; each CTA holds its own
-// 128 rows of A and its half of the B tile (16 KB), so the rings are deeper.
-template <bool kPair> struct Plan {
-#ifndef CFG_SA
-#define CFG_SA 4
-#endif
-#ifndef CFG_SB
-#define CFG_SB 4
-#endif
-  static constexpr int STAGES_A = kPair ? 6 : CFG_SA;
-  static constexpr int STAGES_B = kPair ? 6 : CFG_SB;
-  static constexpr int B_BYTES = (kPair ? BN_MAX / 2 : BN_MAX) * BK * 2;
-  static constexpr int RING_BYTES = STAGES_A * A_BYTES + STAGES_B * B_BYTES;
-  static constexpr int NUM_BARRIERS = 2 * STAGES_A + 2 * STAGES_B + 4 + 2 * QDEPTH + NUM_EPI_WARPS * STAGING_BUFS;
-  static constexpr int TAIL_BYTES = 8 * NUM_BARRIERS + 4 * QDEPTH + 16;
-  static constexpr int SMEM_BYTES = 1024 + RING_BYTES + NUM_EPI_WARPS * STAGING_BUFS * STAGING_BYTES + ((TAIL_BYTES + 127) / 128) * 128;
-  static constexpr int CTAS = kPair ? 2 : 1;
-};
-static_assert(Plan<false>::SMEM_BYTES <= 232448 && Plan<true>::SMEM_BYTES <= 232448, "shared memory budget");
+constexpr int MAX_SUB = 4;           // row blocks that share one generated B tile
+static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 
 enum OperandMode { TMA_KMAJOR = 0, TMA_MNMAJOR = 1, GENERATED = 2 };
 enum EpiMode { EPI_BF16 = 0, EPI_F32 = 1, EPI_UPDATE_W = 2 };
@@ -88,7 +79,6 @@ __device__ unsigned long long g_prof[8];
 // side by side in TMEM (nsub * ncol * bn <= 512 columns).
 struct Problem {
   int M, N, K;
-  int rows_per_block;   // 128, or 256 when a CTA pair shares the item
   int tiles_m, tiles_n, splits, ksteps_total, ksteps_per_split;
   int bn;
   int nsub;
@@ -129,21 +119,6 @@ __device__ __forceinline__ void mbar_arrive_n(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// the generator warps meet on hardware barrier 1 (barrier 0 is __syncthreads)
-// and agree on one answer (true only if every thread's `ok` is true), so that a thread whose
-// bounded wait expired takes the whole group out with it instead of leaving the rest at the barrier
-__device__ __forceinline__ bool gen_group_all(bool ok) {
-  uint32_t r;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\t"
-      "setp.ne.u32 q, %1, 0;\n\t"
-      "bar.red.and.pred p, 1, %2, q;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(r)
-      : "r"((uint32_t)ok), "r"(32 * 16)
-      : "memory");
-  return r != 0;
-}
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
@@ -163,80 +138,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   if (mbar_try_wait(bar, parity)) return true;
   for (uint32_t it = 0; it < 8000000u; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (it > 128) {
-      __nanosleep(100);
-      if (*abort_flag) return false;
-    }
-  }
-  *abort_flag = 1;
-  atomicOr(status, STATUS_TIMEOUT);
-  return false;
-}
-
-// ---- cluster (CTA pair) helpers ----
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
-  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// TMA load issued by either CTA of a pair; completes on the barrier `bar_cluster` (a shared::cluster
-// address, normally the leader's) and writes this CTA's own shared memory.  No multicast.
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster, int x, int y) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
-      "l"(map), "r"(bar_cluster), "r"(x), "r"(y)
-      : "memory");
-}
-__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
-                                               uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-      "mov.b64 da, {%1, %2};\n\t"
-      "mov.b64 db, {%3, %4};\n\t"
-      "setp.ne.b32 p, %6, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
-      "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// Completion of all earlier MMAs of this thread arrives on the barrier at this offset in both CTAs of the pair.
-__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
-               "h"((uint16_t)3)
-               : "memory");
-}
-
-template <bool kCluster>
-__device__ __forceinline__ bool mbar_wait_t(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned int* status) {
-  if (!kCluster) return mbar_wait(bar, parity, abort_flag, status);
-  if (mbar_try_wait_cluster(bar, parity)) return true;
-  for (uint32_t it = 0; it < 8000000u; ++it) {
-    if (mbar_try_wait_cluster(bar, parity)) return true;
     if (it > 128) {
       __nanosleep(100);
       if (*abort_flag) return false;
@@ -338,7 +239,7 @@ __device__ __forceinline__ uint4 projection8_bf16(const ProjectionParams& pp, in
 }
 
 struct TileCoord {
-  int prob, m0, n0, k_begin, k_end, split, nsub, ncol;
+  int prob, m0, n0, k_begin, k_end, split, nsub, ncol, nst;
 };
 
 __device__ __forceinline__ TileCoord decode_tile(const Params& prm, int tile) {
@@ -350,49 +251,43 @@ __device__ __forceinline__ TileCoord decode_tile(const Params& prm, int tile) {
   local /= p.tiles_n;
   const int mb = local % p.tiles_m;
   t.split = local / p.tiles_m;
-  t.m0 = mb * p.rows_per_block * p.nsub;
+  t.m0 = mb * BM * p.nsub;
   t.n0 = nb * p.bn * p.ncol;
   t.k_begin = t.split * p.ksteps_per_split;
   t.k_end = min(p.ksteps_total, t.k_begin + p.ksteps_per_split);
-  t.nsub = min(p.nsub, (p.M - t.m0 + p.rows_per_block - 1) / p.rows_per_block);   // row blocks with a valid row
-  t.ncol = min(p.ncol, (p.N - t.n0 + p.bn - 1) / p.bn);                            // column blocks with a valid column
+  t.nsub = min(p.nsub, (p.M - t.m0 + BM - 1) / BM);          // row blocks with a valid row
+  t.ncol = min(p.ncol, (p.N - t.n0 + p.bn - 1) / p.bn);      // column blocks with a valid column
+  // Stages per k-step.  Row blocks come two to a stage and share the B tile of the first stage;
+  // column blocks come one to a stage and share the A tile of the first stage.
+  t.nst = p.ncol > 1 ? t.ncol : (t.nsub + 1) / 2;
   return t;
 }
 
 // --------------------------------------------------------------------------------------
-// The kernel.  kPair = true runs two CTAs (a cluster of 2) per item with tcgen05 cta_group::2:
-// the leader CTA (cluster rank 0) issues the MMAs over 256 rows; each CTA loads or generates its
-// own 128 rows of A and its own half of the B columns into its own shared memory and drains its
-// own half of the accumulator.  Full barriers and the item queue's hand-back barrier live in the
-// leader; empty and accumulator-full barriers are signalled in both CTAs by multicast commits.
+// The kernel.  Warp roles:
+//   0      item scheduler and stage owner: waits for a free stage, declares the bytes that will land
+//          on its full barrier, arrives, and loads the (lower half of the) B tile
+//   1      tcgen05.mma issuer (one thread), owner of TMEM
+//   2..5   epilogue
+//   6,7,8  loaders: A tile 0, A tile 1, upper half of an MN-major B tile (each only issues TMA)
+//   9..24  generators of P (launches with a generated operand only)
 // --------------------------------------------------------------------------------------
-template <bool kPair>
 __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __grid_constant__ Params prm) {
-  using PL = Plan<kPair>;
-  constexpr int STAGES_A = PL::STAGES_A, STAGES_B = PL::STAGES_B, B_BYTES = PL::B_BYTES, RING_BYTES = PL::RING_BYTES;
-  constexpr int NCTA = PL::CTAS;
-  // generator arrivals on a barrier of the leader: one per local warp, plus one for the whole group of the
-  // second CTA (arrivals across the cluster are slow, so that group meets on a hardware barrier first)
-  constexpr int GEN_ARRIVALS = NUM_GEN_WARPS + (kPair ? 1 : 0);
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));   // generic pointer to the aligned base
-  const uint32_t ringA = smem_base, ringB = smem_base + STAGES_A * A_BYTES;
   const uint32_t staging = smem_base + RING_BYTES;
   const uint32_t bars = staging + NUM_EPI_WARPS * STAGING_BUFS * STAGING_BYTES;
   // barrier slots (8 bytes each)
-  auto fullA = [&](int s) { return bars + 8u * s; };
-  auto emptyA = [&](int s) { return bars + 8u * (STAGES_A + s); };
-  auto fullB = [&](int s) { return bars + 8u * (2 * STAGES_A + s); };
-  auto emptyB = [&](int s) { return bars + 8u * (2 * STAGES_A + STAGES_B + s); };
-  constexpr int kT = 2 * STAGES_A + 2 * STAGES_B;
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (NS + s); };
+  constexpr int kT = 2 * NS;
   auto tfull_bar = [&](int a) { return bars + 8u * (kT + a); };
   auto tempty_bar = [&](int a) { return bars + 8u * (kT + 2 + a); };
   auto qfull = [&](int s) { return bars + 8u * (kT + 4 + s); };
   auto qempty = [&](int s) { return bars + 8u * (kT + 4 + QDEPTH + s); };
   auto wbar = [&](int w) { return bars + 8u * (kT + 4 + 2 * QDEPTH + w); };
-  const uint32_t tail_u32 = bars + 8 * PL::NUM_BARRIERS;
-  uint8_t* tail = smem_gen + RING_BYTES + NUM_EPI_WARPS * STAGING_BUFS * STAGING_BYTES + 8 * PL::NUM_BARRIERS;
+  uint8_t* tail = smem_gen + RING_BYTES + NUM_EPI_WARPS * STAGING_BUFS * STAGING_BYTES + 8 * NUM_BARRIERS;
   volatile int* tile_q = reinterpret_cast<volatile int*>(tail);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail + 4 * QDEPTH);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 4 * QDEPTH + 8);
@@ -400,33 +295,19 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const bool has_gen = prm.gen_ring != GEN_NONE;
-  const uint32_t rank = kPair ? cluster_ctarank() : 0u;        // 0 = leader
-  const bool leader = rank == 0;
-  // arrive on a barrier that lives in the leader CTA
-  auto arrive_leader = [&](uint32_t bar) {
-    if (!kPair || leader) mbar_arrive(bar);
-    else mbar_arrive_cluster(map_to_cta(bar, 0));
-  };
-  auto commit = [&](uint32_t bar) {
-    if (kPair) umma_commit_pair(bar); else umma_commit(bar);
-  };
+  constexpr int GEN_ARRIVALS = NUM_GEN_WARPS;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES_A; ++s) {
-      mbar_init(fullA(s), 1 + (prm.gen_ring == GEN_A ? GEN_ARRIVALS : 0));
-      mbar_init(emptyA(s), 1);
-    }
-    for (int s = 0; s < STAGES_B; ++s) {
-      mbar_init(fullB(s), 1 + (prm.gen_ring == GEN_B ? GEN_ARRIVALS : 0));
-      mbar_init(emptyB(s), 1);
+    for (int s = 0; s < NS; ++s) {
+      mbar_init(full_bar(s), 1 + (has_gen ? GEN_ARRIVALS : 0));   // the stage owner, and the generator warps
+      mbar_init(empty_bar(s), 1);
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);
-      mbar_init(tempty_bar(a), NCTA * NUM_EPI_WARPS);
+      mbar_init(tempty_bar(a), NUM_EPI_WARPS);
     }
-    // consumers of the item queue: the MMA thread (leader); the producers other than the scheduler,
-    // the epilogue warps and the generator group (one arrival) of each CTA; the second CTA's first B producer
-    const int consumers = 1 + NCTA * (2 * NUM_PROD - 1 + NUM_EPI_WARPS) + (has_gen ? GEN_ARRIVALS : 0) + (kPair ? 1 : 0);
+    // consumers of the item queue: MMA thread, loaders, epilogue warps, generator warps
+    const int consumers = 1 + NUM_LOADERS + NUM_EPI_WARPS + (has_gen ? NUM_GEN_WARPS : 0);
     for (int s = 0; s < QDEPTH; ++s) {
       mbar_init(qfull(s), 1);
       mbar_init(qempty(s), consumers);
@@ -442,94 +323,121 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
   }
   tc_fence_before();
   __syncthreads();
-  if (kPair) cluster_sync_all();          // both CTAs' barriers exist before anyone signals across
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  // Every consumer role reads the next item from the queue the (leader's) producer fills.
+  // Every consumer role reads the next item from the queue the scheduler fills.
   int qs = 0;
   uint32_t qph = 0;
   auto next_tile = [&](bool whole_warp, bool elected) -> int {
-    // the second CTA's slot is written by the leader from across the cluster: acquire at cluster scope there
-    const bool got = (kPair && !leader) ? mbar_wait_t<true>(qfull(qs), qph, abort_flag, prm.status)
-                                        : mbar_wait(qfull(qs), qph, abort_flag, prm.status);
-    if (!got) return -1;
+    if (!mbar_wait(qfull(qs), qph, abort_flag, prm.status)) return -1;
     const int tile = tile_q[qs];
     if (whole_warp) __syncwarp();           // every lane has read the slot before it is handed back
-    if (elected) arrive_leader(qempty(qs));
+    if (elected) mbar_arrive(qempty(qs));
     if (++qs == QDEPTH) { qs = 0; qph ^= 1; }
     return tile;
   };
+  // what stage j of a k-step of item t holds
+  auto stage_has_b = [&](const Problem& p, int j) { return p.ncol > 1 || j == 0; };
+  auto stage_num_a = [&](const Problem& p, const TileCoord& t, int j) {
+    if (p.ncol > 1) return j == 0 ? 1 : 0;
+    return min(2, t.nsub - 2 * j);
+  };
 
-  // Producer threads: NUM_PROD per operand ring, each lane 0 of its own warp.  Thread j of a ring
-  // loads the tiles whose running index is j modulo NUM_PROD: every barrier wait / expect / TMA issue
-  // is a dependent long-latency step, and several threads overlap them.
-  const int prodB = warp == 0 ? 0 : ((warp >= 2 + NUM_EPI_WARPS && warp < 2 + NUM_EPI_WARPS + 2 * NUM_PROD - 1 && ((warp - 2 - NUM_EPI_WARPS) & 1)) ? (warp - 2 - NUM_EPI_WARPS + 1) / 2 : -1);
-  const int prodA = (warp >= 2 + NUM_EPI_WARPS && warp < 2 + NUM_EPI_WARPS + 2 * NUM_PROD - 1 && !((warp - 2 - NUM_EPI_WARPS) & 1)) ? (warp - 2 - NUM_EPI_WARPS) / 2 : -1;
-  if (prodB >= 0) {
-    // ------------------------- producers of B tiles (thread 0 is also the scheduler) ----------
+  const int loader = (warp >= 2 + NUM_EPI_WARPS && warp < 2 + NUM_EPI_WARPS + NUM_LOADERS) ? warp - 2 - NUM_EPI_WARPS : -1;
+  if (warp == 0) {
+    // ------------------------- scheduler + stage owner --------------------------
     if (lane == 0) {
-      uint32_t ib = 0;                     // running index of B tiles in this CTA
+      uint32_t is = 0;                     // running stage index
       bool ok = true;
       while (ok) {
-        int tile;
-        if (prodB == 0 && leader) {
-          if (!(ok = mbar_wait(qempty(qs), qph ^ 1, abort_flag, prm.status))) break;
-          tile = (int)atomicAdd(prm.sched, 1u);
-          if (tile >= prm.total_tiles) tile = -1;
-          tile_q[qs] = tile;
-          mbar_arrive(qfull(qs));
-          if (kPair) {
-            st_cluster_u32(map_to_cta(tail_u32 + 4u * qs, 1), (uint32_t)tile);
-            mbar_arrive_cluster(map_to_cta(qfull(qs), 1));
-          }
-          if (++qs == QDEPTH) { qs = 0; qph ^= 1; }
-        } else {
-          tile = next_tile(false, true);
-        }
+        if (!(ok = mbar_wait(qempty(qs), qph ^ 1, abort_flag, prm.status))) break;
+        int tile = (int)atomicAdd(prm.sched, 1u);
+        if (tile >= prm.total_tiles) tile = -1;
+        tile_q[qs] = tile;
+        mbar_arrive(qfull(qs));
+        if (++qs == QDEPTH) { qs = 0; qph ^= 1; }
         if (tile < 0) break;
         const TileCoord t = decode_tile(prm, tile);
         const Problem& p = prm.prob[t.prob];
         const CUtensorMap* mapB = &prm.tmB[t.prob];
-        const int bn_cta = p.bn / NCTA;                 // B columns this CTA holds
-        const int n_first = t.n0 + (int)rank * bn_cta;
-        for (int kc = 0; kc < (t.k_end - t.k_begin) * t.ncol && ok; ++kc, ++ib) {
-          if ((int)(ib % NUM_PROD) != prodB) continue;
-          const int sb = (int)(ib % STAGES_B);
-          const uint32_t phb = (ib / STAGES_B) & 1u;
-          const int k0 = (t.k_begin + kc / t.ncol) * BK;
-          const int n0 = n_first + (kc % t.ncol) * p.bn;
-          // B tile of this k-step (shared by all row blocks of the item)
-          if (!(ok = mbar_wait(emptyB(sb), phb ^ 1, abort_flag, prm.status))) break;
-          const uint32_t dst = ringB + sb * B_BYTES, fb = fullB(sb);
+        const bool a_tma = p.a_mode != GENERATED, b_tma = p.b_mode != GENERATED;
+        for (int ks = t.k_begin; ks < t.k_end && ok; ++ks) {
+          const int k0 = ks * BK;
+          for (int j = 0; j < t.nst; ++j, ++is) {
+            const int s = (int)(is % NS);
+            if (!(ok = mbar_wait(empty_bar(s), ((is / NS) & 1u) ^ 1, abort_flag, prm.status))) break;
+            const bool hb = stage_has_b(p, j);
+            const int na = stage_num_a(p, t, j);
+            uint32_t tx = 0;
+            bool gen_here = false;
+            if (hb) { if (b_tma) tx += p.bn * BK * 2; else gen_here = true; }
+            if (na > 0) { if (a_tma) tx += na * A_BYTES; else gen_here = true; }
 #if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
-          if ((prm.debug_flags & 2) && p.b_mode != GENERATED) {          // no loads: MMAs run on whatever is in the ring
-            if (leader) mbar_arrive_n(fb, 1 + (prm.gen_ring == GEN_B ? GEN_ARRIVALS : 0));
-            continue;
-          }
+            if (prm.debug_flags & 2) tx = 0;
 #endif
-          if (p.b_mode == GENERATED) {
-            if (leader) mbar_arrive(fb);                                 // the generator groups arrive for the data
-          } else {
-            if (leader) {
-              // both CTAs' halves land on this barrier; the generators sit this item out, so arrive for them too
-              mbar_expect_tx(fb, p.bn * BK * 2);
-              mbar_arrive_n(fb, 1 + (prm.gen_ring == GEN_B ? GEN_ARRIVALS : 0));
-            }
-            if (!kPair || leader) {
-              // ordinary loads onto this CTA's own barrier
+            const uint32_t fb = full_bar(s);
+            if (tx) mbar_expect_tx(fb, tx);
+            // arrive for this thread, and for the generator warps when they have nothing to write here
+            mbar_arrive_n(fb, 1 + ((has_gen && !gen_here) ? GEN_ARRIVALS : 0));
+            if (hb && b_tma && tx) {
+              const uint32_t dst = smem_base + s * STAGE_BYTES + STAGE_B_OFF;
+              const int n0 = t.n0 + (p.ncol > 1 ? j : 0) * p.bn;
               if (p.b_mode == TMA_KMAJOR) {
                 tma_load_2d(dst, mapB, fb, k0, n0);
               } else {
-                for (int b = 0; b < bn_cta / 64; ++b) tma_load_2d(dst + b * 8192, mapB, fb, n0 + 64 * b, k0);
+                const int nblk = p.bn / 64, lower = nblk > 2 ? 2 : nblk;   // the upper blocks go to a loader
+                for (int b = 0; b < lower; ++b) tma_load_2d(dst + b * 8192, mapB, fb, n0 + 64 * b, k0);
               }
+            }
+          }
+        }
+      }
+    }
+  } else if (loader >= 0) {
+    // ------------------------------ loaders --------------------------------------
+    // 0: A tile in slot 0, 1: A tile in slot 1, 2: blocks 2.. of an MN-major B tile.  They only issue
+    // TMA; the bytes were declared by the stage owner.
+    if (lane == 0) {
+      uint32_t is = 0;
+      bool ok = true;
+      while (ok) {
+        const int tile = next_tile(false, true);
+        if (tile < 0) break;
+        const TileCoord t = decode_tile(prm, tile);
+        const Problem& p = prm.prob[t.prob];
+        const CUtensorMap* mapA = &prm.tmA[t.prob];
+        const CUtensorMap* mapB = &prm.tmB[t.prob];
+        bool mine;
+        if (loader == 2) mine = p.b_mode == TMA_MNMAJOR && p.bn > 128;
+        else mine = p.a_mode != GENERATED;
+#if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
+        if (prm.debug_flags & 2) mine = false;
+#endif
+        const int klen = t.k_end - t.k_begin;
+        if (!mine) { is += klen * t.nst; continue; }
+        for (int ks = t.k_begin; ks < t.k_end && ok; ++ks) {
+          const int k0 = ks * BK;
+          for (int j = 0; j < t.nst; ++j, ++is) {
+            const int s = (int)(is % NS);
+            const uint32_t fb = full_bar(s);
+            const uint32_t stage = smem_base + s * STAGE_BYTES;
+            if (loader == 2) {
+              if (!stage_has_b(p, j)) continue;
+              if (!(ok = mbar_wait(empty_bar(s), ((is / NS) & 1u) ^ 1, abort_flag, prm.status))) break;
+              const int n0 = t.n0 + (p.ncol > 1 ? j : 0) * p.bn;
+              for (int b = 2; b < p.bn / 64; ++b) tma_load_2d(stage + STAGE_B_OFF + b * 8192, mapB, fb, n0 + 64 * b, k0);
             } else {
-              // second CTA: data into its own shared memory, completion onto the leader's barrier
-              const uint32_t fb_sig = map_to_cta(fb, 0);
-              if (p.b_mode == TMA_KMAJOR) {
-                tma_load_2d_pair(dst, mapB, fb_sig, k0, n0);
+              if (loader >= stage_num_a(p, t, j)) continue;
+              if (!(ok = mbar_wait(empty_bar(s), ((is / NS) & 1u) ^ 1, abort_flag, prm.status))) break;
+              const int mi = p.ncol > 1 ? 0 : 2 * j + loader;
+              const int m0 = t.m0 + mi * BM;
+              const uint32_t dst = stage + (loader == 0 ? STAGE_A0_OFF : STAGE_A1_OFF);
+              if (p.a_mode == TMA_KMAJOR) {
+                tma_load_2d(dst, mapA, fb, k0, m0);
               } else {
-                for (int b = 0; b < bn_cta / 64; ++b) tma_load_2d_pair(dst + b * 8192, mapB, fb_sig, n0 + 64 * b, k0);
+                tma_load_2d(dst, mapA, fb, m0, k0);
+                tma_load_2d(dst + 8192, mapA, fb, m0 + 64, k0);
               }
             }
           }
@@ -537,17 +445,12 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       }
     }
   } else if (warp == 1) {
-    // ------------------------------ MMA issuer (leader CTA only) ----------------
-    if (lane == 0 && leader) {
-      int sa = 0, sb = 0, acc = 0;
-      uint32_t pha = 0, phb = 0, acc_phase = 0;
+    // ------------------------------ MMA issuer ---------------------------------
+    if (lane == 0) {
+      uint32_t is = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
       bool ok = true;
-#ifdef COMPACT_PROFILE
-      unsigned long long prof[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-      const long long t_start = clock64();
-      unsigned long long ns0;
-      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(ns0));
-#endif
       while (ok) {
         const int tile = next_tile(false, true);
         if (tile < 0) break;
@@ -556,13 +459,12 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const bool a_mn = p.a_mode == TMA_MNMAJOR;
         const bool b_mn = p.b_mode != TMA_KMAJOR;          // generated B tiles are written MN-major
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
-                               ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)((NCTA * BM) >> 4) << 24);
+                               ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
         const int slots = (p.nsub * p.ncol * p.bn + BN_MAX - 1) / BN_MAX;   // accumulator slots this item occupies
-        const long long tp0 = PROF_T();
         if (slots == 2 && acc == 1) {
           // a two-slot item starts at slot 0: pass slot 1 through unused
           if (!(ok = mbar_wait(tempty_bar(1), acc_phase ^ 1, abort_flag, prm.status))) break;
-          commit(tfull_bar(1));
+          umma_commit(tfull_bar(1));
           acc = 0;
           acc_phase ^= 1;
         }
@@ -571,100 +473,58 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
           ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag, prm.status);
           if (++acc == 2) { acc = 0; acc_phase ^= 1; }
         }
-        PROF_ADD(0, tp0);
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_base = tmem_base + acc0 * BN_MAX;
         // one UMMA consumes K = 16: 32 bytes along a K-major row, or two 8-row groups (2048 bytes) MN-major
         const uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4), b_step = b_mn ? (2048u >> 4) : (32u >> 4);
-        const int nsub = t.nsub, ncol = t.ncol, bn = p.bn;
+        const int bn = p.bn, nst = t.nst;
         auto issue4 = [&](uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t first) {
 #if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
           if (prm.debug_flags & 1) return;
 #endif
-          if (kPair) {
-            umma_bf16_pair(d, a_lo, DESC_HI, b_lo, DESC_HI, idesc, first);
-            umma_bf16_pair(d, a_lo + a_step, DESC_HI, b_lo + b_step, DESC_HI, idesc, 1u);
-            umma_bf16_pair(d, a_lo + 2 * a_step, DESC_HI, b_lo + 2 * b_step, DESC_HI, idesc, 1u);
-            umma_bf16_pair(d, a_lo + 3 * a_step, DESC_HI, b_lo + 3 * b_step, DESC_HI, idesc, 1u);
-          } else {
-            umma_bf16(d, a_lo, DESC_HI, b_lo, DESC_HI, idesc, first);
-            umma_bf16(d, a_lo + a_step, DESC_HI, b_lo + b_step, DESC_HI, idesc, 1u);
-            umma_bf16(d, a_lo + 2 * a_step, DESC_HI, b_lo + 2 * b_step, DESC_HI, idesc, 1u);
-            umma_bf16(d, a_lo + 3 * a_step, DESC_HI, b_lo + 3 * b_step, DESC_HI, idesc, 1u);
-          }
+          umma_bf16(d, a_lo, DESC_HI, b_lo, DESC_HI, idesc, first);
+          umma_bf16(d, a_lo + a_step, DESC_HI, b_lo + b_step, DESC_HI, idesc, 1u);
+          umma_bf16(d, a_lo + 2 * a_step, DESC_HI, b_lo + 2 * b_step, DESC_HI, idesc, 1u);
+          umma_bf16(d, a_lo + 3 * a_step, DESC_HI, b_lo + 3 * b_step, DESC_HI, idesc, 1u);
         };
         for (int ks = t.k_begin; ks < t.k_end && ok; ++ks) {
           const uint32_t first = ks > t.k_begin ? 1u : 0u;
-          if (p.ncol > 1) {
-            // one A tile, several B tiles (column blocks)
-            if (!(ok = mbar_wait(fullA(sa), pha, abort_flag, prm.status))) break;
-            const uint32_t a_lo = desc_lo(ringA + sa * A_BYTES, a_mn);
-            for (int cb = 0; cb < ncol; ++cb) {
-              if (!(ok = mbar_wait(fullB(sb), phb, abort_flag, prm.status))) break;
-              tc_fence_after();
-              issue4(d_base + cb * bn, a_lo, desc_lo(ringB + sb * B_BYTES, b_mn), first);
-              commit(emptyB(sb));
-              if (++sb == STAGES_B) { sb = 0; phb ^= 1; }
-            }
-            if (!ok) break;
-            commit(emptyA(sa));
-            if (++sa == STAGES_A) { sa = 0; pha ^= 1; }
-            continue;
-          }
-          const long long tp1 = PROF_T();
-          if (!(ok = mbar_wait(fullB(sb), phb, abort_flag, prm.status))) break;
-          PROF_ADD(1, tp1);
-          const uint32_t b_lo = desc_lo(ringB + sb * B_BYTES, b_mn);
-          for (int mi = 0; mi < nsub; ++mi) {
-            const long long tp2 = PROF_T();
-            if (!(ok = mbar_wait(fullA(sa), pha, abort_flag, prm.status))) break;
-            PROF_ADD(2, tp2);
-            const long long tp7 = PROF_T();
+          const uint32_t is0 = is;
+          const uint32_t stage0 = smem_base + (is0 % NS) * STAGE_BYTES;       // holds the shared operand
+          for (int j = 0; j < nst; ++j, ++is) {
+            const int s = (int)(is % NS);
+            if (!(ok = mbar_wait(full_bar(s), (is / NS) & 1u, abort_flag, prm.status))) break;
             tc_fence_after();
-            PROF_ADD(7, tp7);
-            const long long tp3 = PROF_T();
-            issue4(d_base + mi * bn, desc_lo(ringA + sa * A_BYTES, a_mn), b_lo, first);
-            commit(emptyA(sa));
-            PROF_ADD(3, tp3);
-            if (++sa == STAGES_A) { sa = 0; pha ^= 1; }
+            const uint32_t stage = smem_base + s * STAGE_BYTES;
+            if (p.ncol > 1) {
+              issue4(d_base + j * bn, desc_lo(stage0 + STAGE_A0_OFF, a_mn), desc_lo(stage + STAGE_B_OFF, b_mn), first);
+            } else {
+              const uint32_t b_lo = desc_lo(stage0 + STAGE_B_OFF, b_mn);
+              issue4(d_base + (2 * j) * bn, desc_lo(stage + STAGE_A0_OFF, a_mn), b_lo, first);
+              if (2 * j + 1 < t.nsub) issue4(d_base + (2 * j + 1) * bn, desc_lo(stage + STAGE_A1_OFF, a_mn), b_lo, first);
+            }
+            // a stage that holds nothing shared goes back at once; the first stage of the k-step goes last
+            if (j > 0) umma_commit(empty_bar(s));
           }
           if (!ok) break;
-          const long long tp6 = PROF_T();
-          commit(emptyB(sb));
-          PROF_ADD(6, tp6);
-          if (++sb == STAGES_B) { sb = 0; phb ^= 1; }
+          umma_commit(empty_bar((int)(is0 % NS)));
         }
         if (!ok) break;
-        for (int sl = 0; sl < slots; ++sl) commit(tfull_bar((acc0 + sl) & 1));
+        for (int sl = 0; sl < slots; ++sl) umma_commit(tfull_bar((acc0 + sl) & 1));
       }
-#ifdef COMPACT_PROFILE
-      prof[4] = clock64() - t_start;
-      unsigned long long ns1;
-      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(ns1));
-      prof[5] = ns1 - ns0;
-#ifndef COMPACT_PROFILE_EPI
-      for (int i = 0; i < 6; ++i) atomicAdd(&g_prof[i], prof[i]);
-#endif
-#endif
     }
   } else if (warp < 2 + NUM_EPI_WARPS) {
     // ------------------------------ epilogue ------------------------------------
     // TMEM -> registers -> 128B-swizzled staging tile (32 rows x 128 bytes, two per warp) -> TMA store.
     // The chunks of an item (accumulator by accumulator, 64 bf16 or 32 fp32 columns at a time) are
-    // walked as one flat sequence so that the W tile of the next chunk (update) is already on its way
+    // walked as one sequence so that the W tile of the next chunk (update) is already on its way
     // while the current one is processed.
     const int q = warp & 3;                 // TMEM lane quarter this warp may read
     const uint32_t stg0 = staging + (warp - 2) * STAGING_BUFS * STAGING_BYTES;
     uint8_t* stg_gen0 = smem_gen + RING_BYTES + (warp - 2) * STAGING_BUFS * STAGING_BYTES;
     uint32_t wph[STAGING_BUFS] = {0, 0};
     int buf = 0;
-#ifdef COMPACT_PROFILE
-    long long eprof_drain = 0, eprof_wait = 0;
-#endif
-#ifdef COMPACT_PROFILE_EPI
-    long long ep[4] = {0, 0, 0, 0};
-#endif
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
@@ -682,15 +542,14 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       const int cpa = p.bn / cw;                               // chunks per accumulator
       // Cursor over the chunks this warp writes: accumulator ai (slot sl, position su in the slot), chunk ci.
       struct Cur { int ai, sl, su, ci; };
-      const int row_q = (int)rank * BM + q * 32;
+      const int row_q = q * 32;
       auto acc_valid = [&](int ai) -> bool {       // does accumulator ai hold rows/columns this warp writes?
         const int mi = p.ncol > 1 ? 0 : ai, cb = p.ncol > 1 ? ai : 0;
-        return mi < t.nsub && cb < t.ncol && t.m0 + mi * p.rows_per_block + row_q < p.M && t.n0 + cb * p.bn < p.N;
+        return mi < t.nsub && cb < t.ncol && t.m0 + mi * BM + row_q < p.M && t.n0 + cb * p.bn < p.N;
       };
       auto cur_col = [&](const Cur& c) -> int { return t.n0 + (p.ncol > 1 ? c.ai : 0) * p.bn + c.ci * cw; };
-      auto cur_row = [&](const Cur& c) -> int { return t.m0 + (p.ncol > 1 ? 0 : c.ai) * p.rows_per_block + row_q; };
-      // first valid chunk at or after (ai, ci = 0)
-      auto seek = [&](Cur c) -> Cur {
+      auto cur_row = [&](const Cur& c) -> int { return t.m0 + (p.ncol > 1 ? 0 : c.ai) * BM + row_q; };
+      auto seek = [&](Cur c) -> Cur {              // first valid chunk at or after (ai, 0)
         while (c.ai < naccs && !acc_valid(c.ai)) {
           ++c.ai;
           if (++c.su == sub_per_slot) { c.su = 0; ++c.sl; }
@@ -714,7 +573,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       if (slots == 2 && acc == 1) {
         if (!(ok = mbar_wait(tfull_bar(1), acc_phase, abort_flag, prm.status))) break;
         __syncwarp();
-        if (lane == 0) arrive_leader(tempty_bar(1));
+        if (lane == 0) mbar_arrive(tempty_bar(1));
         acc = 0;
         acc_phase ^= 1;
       }
@@ -728,28 +587,17 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         load_w(cur, buf);
       }
       int cur_slot = -1;
-#ifdef COMPACT_PROFILE
-      long long t_slot = 0;
-#endif
       // enter accumulator slot `want` (waiting for its MMAs), handing back the slots passed on the way
       auto enter_slot = [&](int want) -> bool {
         while (cur_slot < want) {
           if (cur_slot >= 0) {
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) arrive_leader(tempty_bar(acc));
+            if (lane == 0) mbar_arrive(tempty_bar(acc));
             if (++acc == 2) { acc = 0; acc_phase ^= 1; }
           }
           ++cur_slot;
-#ifdef COMPACT_PROFILE
-          const long long tw0 = clock64();
-          if (t_slot) eprof_drain += tw0 - t_slot;
-#endif
           if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, prm.status)) return false;
-#ifdef COMPACT_PROFILE
-          t_slot = clock64();
-          eprof_wait += t_slot - tw0;
-#endif
           tc_fence_after();
         }
         return true;
@@ -766,19 +614,10 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             load_w(nxt, buf ^ 1);
           }
         } else {
-#ifdef COMPACT_PROFILE_EPI
-          const long long te0 = clock64();
-#endif
           if (lane == 0) tma_store_wait_read1();       // this buffer's previous store has read it
           __syncwarp();
-#ifdef COMPACT_PROFILE_EPI
-          ep[0] += clock64() - te0;
-#endif
         }
         if (!(ok = enter_slot(sl))) break;
-#ifdef COMPACT_PROFILE_EPI
-        const long long te1 = clock64();
-#endif
         const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN_MAX + tc;
         if (p.epi_mode == EPI_F32) {
           uint32_t v[32];
@@ -830,20 +669,12 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             }
           }
           if (!ok) break;
-#ifdef COMPACT_PROFILE_EPI
-          const long long te2 = clock64();
-          ep[1] += te2 - te1;
-#endif
           fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) {
             tma_store_2d(mapC, stg, col, row0);
             tma_store_commit();
           }
-#ifdef COMPACT_PROFILE_EPI
-          ep[2] += clock64() - te2;
-          ep[3] += 1;
-#endif
         }
         buf ^= 1;
         cur = nxt;
@@ -852,150 +683,58 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       if (!(ok = enter_slot(slots - 1))) break;      // slots this warp had nothing to write for
       tc_fence_before();
       __syncwarp();
-#ifdef COMPACT_PROFILE
-      eprof_drain += clock64() - t_slot;
-#endif
-      if (lane == 0) arrive_leader(tempty_bar(acc));
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
       if (++acc == 2) { acc = 0; acc_phase ^= 1; }
     }
-#ifdef COMPACT_PROFILE_EPI
-    if (warp == 2 && lane == 0 && leader) for (int i = 0; i < 4; ++i) atomicAdd(&g_prof[i], (unsigned long long)ep[i]);
-#endif
-#ifdef COMPACT_PROFILE
-    if (warp == 2 && lane == 0 && leader) { atomicAdd(&g_prof[6], (unsigned long long)eprof_drain); atomicAdd(&g_prof[7], (unsigned long long)eprof_wait); }
-#endif
     if (lane == 0) tma_store_wait_all();
-  } else if (prodA >= 0) {
-    // ------------------------------ producers of A tiles ------------------------
-    if (lane == 0) {
-      uint32_t ia = 0;                     // running index of A tiles in this CTA
-      bool ok = true;
-      while (ok) {
-        const int tile = next_tile(false, true);
-        if (tile < 0) break;
-        const TileCoord t = decode_tile(prm, tile);
-        const Problem& p = prm.prob[t.prob];
-        const CUtensorMap* mapA = &prm.tmA[t.prob];
-        for (int ks = t.k_begin; ks < t.k_end && ok; ++ks) {
-          const int k0 = ks * BK;
-          for (int mi = 0; mi < t.nsub; ++mi, ++ia) {
-            if ((int)(ia % NUM_PROD) != prodA) continue;
-            const int sa = (int)(ia % STAGES_A);
-            const uint32_t pha = (ia / STAGES_A) & 1u;
-            if (!(ok = mbar_wait(emptyA(sa), pha ^ 1, abort_flag, prm.status))) break;
-            const uint32_t dst = ringA + sa * A_BYTES, fa = fullA(sa);
-            const int m0 = t.m0 + mi * p.rows_per_block + (int)rank * BM;
-#if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
-            if ((prm.debug_flags & 2) && p.a_mode != GENERATED) {
-              if (leader) mbar_arrive_n(fa, 1 + (prm.gen_ring == GEN_A ? GEN_ARRIVALS : 0));
-              continue;
-            }
-#endif
-            if (p.a_mode == GENERATED) {
-              if (leader) mbar_arrive(fa);
-            } else {
-              if (leader) {
-                mbar_expect_tx(fa, NCTA * A_BYTES);
-                mbar_arrive_n(fa, 1 + (prm.gen_ring == GEN_A ? GEN_ARRIVALS : 0));
-              }
-              if (!kPair || leader) {
-                if (p.a_mode == TMA_KMAJOR) {
-                  tma_load_2d(dst, mapA, fa, k0, m0);
-                } else {
-                  tma_load_2d(dst, mapA, fa, m0, k0);
-                  tma_load_2d(dst + 8192, mapA, fa, m0 + 64, k0);
-                }
-              } else {
-                const uint32_t fa_sig = map_to_cta(fa, 0);
-                if (p.a_mode == TMA_KMAJOR) {
-                  tma_load_2d_pair(dst, mapA, fa_sig, k0, m0);
-                } else {
-                  tma_load_2d_pair(dst, mapA, fa_sig, m0, k0);
-                  tma_load_2d_pair(dst + 8192, mapA, fa_sig, m0 + 64, k0);
-                }
-              }
-            }
-          }
-        }
-      }
-    }
   } else {
     // ------------------------------ P generators --------------------------------
-    // Write bf16 tiles of P straight into the swizzled operand layout the MMA reads.  The group
-    // meets on a hardware barrier and signals each tile (and each item hand-back) once.
+    // Write bf16 tiles of P straight into the swizzled operand layout the MMA reads: as the B tile
+    // of the first stage of a k-step (forward) or as its A tile 0 (update).
     const int gtid = threadIdx.x - THREADS_BASE;
-    uint32_t it = 0;                       // running index of tiles in the ring this launch generates into
+    uint32_t is = 0;
     bool ok = true;
-    // Signal `bar` of the leader once this thread's warp (leader CTA) or the whole group (second CTA)
-    // is done; returns false if some participant's wait had expired.
-    auto signal = [&](uint32_t bar, bool w) -> bool {
-      if (!kPair || leader) {
-        const bool all = __all_sync(0xffffffffu, w);
-        if (all && lane == 0) mbar_arrive(bar);
-        return all;
-      }
-      const bool all = gen_group_all(w);
-      if (all && gtid == 0) mbar_arrive_cluster(map_to_cta(bar, 0));
-      return all;
-    };
     while (ok) {
-      const bool got = (kPair && !leader) ? mbar_wait_t<true>(qfull(qs), qph, abort_flag, prm.status)
-                                          : mbar_wait(qfull(qs), qph, abort_flag, prm.status);
-      const int tile = got ? tile_q[qs] : -1;
-      if (!(ok = signal(qempty(qs), got))) break;     // every participating thread has read the slot
-      if (++qs == QDEPTH) { qs = 0; qph ^= 1; }
+      const int tile = next_tile(true, lane == 0);
       if (tile < 0) break;
       const TileCoord t = decode_tile(prm, tile);
       const Problem& p = prm.prob[t.prob];
       const int klen = t.k_end - t.k_begin;
-      if (prm.gen_ring == GEN_B) {
-        if (p.b_mode != GENERATED) { it += klen * t.ncol; continue; }      // the producer arrives for this item
-        const int bn_cta = p.bn / NCTA;
-        const int n0 = t.n0 + (int)rank * bn_cta;
-        const int chunks = bn_cta >> 3;
-        for (int ks = t.k_begin; ks < t.k_end; ++ks, ++it) {
-          const int st = (int)(it % STAGES_B);
-          const bool w = mbar_wait(emptyB(st), ((it / STAGES_B) & 1u) ^ 1, abort_flag, prm.status);
-          if (w) {
-            // B[k = row i of P][n = column j of P], MN-major: 64-column blocks of [64 k][128 B]
-            uint8_t* sbp = smem_gen + STAGES_A * A_BYTES + st * B_BYTES;
-            const int k0 = ks * BK;
-            for (int id = gtid; id < BK * chunks; id += 32 * NUM_GEN_WARPS) {
-              const int c = id % chunks, kr = id / chunks;
-              const uint4 val = projection8_bf16(prm.pp, k0 + kr, n0 + c * 8);
-              *reinterpret_cast<uint4*>(sbp + (c >> 3) * 8192 + kr * 128 + (((c & 7) ^ (kr & 7)) << 4)) = val;
-            }
-            fence_proxy_async_smem();
-          }
-          if (!(ok = signal(fullB(st), w))) break;
-        }
-      } else {
-        if (p.a_mode != GENERATED) { it += klen * t.nsub; continue; }
-        for (int ks = t.k_begin; ks < t.k_end && ok; ++ks) {
-          for (int mi = 0; mi < t.nsub; ++mi, ++it) {
-            const int st = (int)(it % STAGES_A);
-            const bool w = mbar_wait(emptyA(st), ((it / STAGES_A) & 1u) ^ 1, abort_flag, prm.status);
-            if (w) {
-              // A[m = row i of P][k = column j of P], K-major: [128 rows][128 B]
-              uint8_t* sap = smem_gen + st * A_BYTES;
-              const int k0 = ks * BK, m0 = t.m0 + mi * p.rows_per_block + (int)rank * BM;
-              for (int id = gtid; id < BM * 8; id += 32 * NUM_GEN_WARPS) {
-                const int c = id & 7, rr = id >> 3;
-                const uint4 val = projection8_bf16(prm.pp, m0 + rr, k0 + c * 8);
-                *reinterpret_cast<uint4*>(sap + rr * 128 + ((c ^ (rr & 7)) << 4)) = val;
-              }
-              fence_proxy_async_smem();
-            }
-            if (!(ok = signal(fullA(st), w))) break;
+      const bool gen_b = p.b_mode == GENERATED, gen_a = p.a_mode == GENERATED;
+      if (!gen_a && !gen_b) { is += klen * t.nst; continue; }      // the stage owner arrives for this item
+      for (int ks = t.k_begin; ks < t.k_end && ok; ++ks, is += t.nst) {
+        const int s = (int)(is % NS);
+        const bool w = mbar_wait(empty_bar(s), ((is / NS) & 1u) ^ 1, abort_flag, prm.status);
+        const int k0 = ks * BK;
+        if (w && gen_b) {
+          // B[k = row i of P][n = column j of P], MN-major: 64-column blocks of [64 k][128 B]
+          uint8_t* sbp = smem_gen + s * STAGE_BYTES + STAGE_B_OFF;
+          const int chunks = p.bn >> 3;
+          for (int id = gtid; id < BK * chunks; id += 32 * NUM_GEN_WARPS) {
+            const int c = id % chunks, kr = id / chunks;
+            const uint4 val = projection8_bf16(prm.pp, k0 + kr, t.n0 + c * 8);
+            *reinterpret_cast<uint4*>(sbp + (c >> 3) * 8192 + kr * 128 + (((c & 7) ^ (kr & 7)) << 4)) = val;
           }
         }
+        if (w && gen_a) {
+          // A[m = row i of P][k = column j of P], K-major: [128 rows][128 B]
+          uint8_t* sap = smem_gen + s * STAGE_BYTES + STAGE_A0_OFF;
+          for (int id = gtid; id < BM * 8; id += 32 * NUM_GEN_WARPS) {
+            const int c = id & 7, rr = id >> 3;
+            const uint4 val = projection8_bf16(prm.pp, t.m0 + rr, k0 + c * 8);
+            *reinterpret_cast<uint4*>(sap + rr * 128 + ((c ^ (rr & 7)) << 4)) = val;
+          }
+        }
+        fence_proxy_async_smem();
+        ok = __all_sync(0xffffffffu, w);
+        if (ok && lane == 0) mbar_arrive(full_bar(s));
+        // later stages of the k-step hold no generated data: the stage owner arrives for the generators there
       }
     }
   }
 
   tc_fence_before();
   __syncthreads();
-  if (kPair) cluster_sync_all();          // the partner may still signal into this CTA until it is done too
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
@@ -1111,25 +850,20 @@ inline bool make_map_f32_3d(CUtensorMap* map, const void* base, int64_t inner, i
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Tile width: up to 256 columns; a CTA pair splits it in two halves of whole 64-column blocks.
-inline int pick_bn(int N, bool pair) {
-  if (N >= BN_MAX) return BN_MAX;
-  const int g = pair ? 128 : 64;
-  return (int)((N + g - 1) / g * g);
-}
+// Tile width: up to 256 columns, in whole 64-column blocks.
+inline int pick_bn(int N) { return N >= BN_MAX ? BN_MAX : (int)((N + 63) / 64 * 64); }
 
 #ifndef CFG_NSUB
 #define CFG_NSUB 2
 #endif
 
-inline void finish_problem(Problem& p, int splits_wanted, bool pair) {
-  p.rows_per_block = pair ? 2 * BM : BM;
-  if (p.bn == 0) p.bn = pick_bn(p.N, pair);
-  // single CTA: two row blocks share each B tile (256 x 256 items halve the shared-memory refill per flop);
-  // CTA pair: one 256-row block per item, accumulators double-buffered
-  if (p.nsub == 0) p.nsub = pair ? 1 : (p.M > BM ? CFG_NSUB : 1);
+inline void finish_problem(Problem& p, int splits_wanted) {
+  if (p.bn == 0) p.bn = pick_bn(p.N);
+  // two row blocks share each B tile: 256 x 256 items halve the shared-memory refill per flop and
+  // put eight MMAs behind every barrier wait
+  if (p.nsub == 0) p.nsub = p.M > BM ? CFG_NSUB : 1;
   if (p.ncol == 0) p.ncol = 1;
-  p.tiles_m = (p.M + p.rows_per_block * p.nsub - 1) / (p.rows_per_block * p.nsub);
+  p.tiles_m = (p.M + BM * p.nsub - 1) / (BM * p.nsub);
   p.tiles_n = (p.N + p.bn * p.ncol - 1) / (p.bn * p.ncol);
   p.ksteps_total = (p.K + BK - 1) / BK;
   int s = splits_wanted < 1 ? 1 : splits_wanted;
@@ -1142,7 +876,7 @@ inline void finish_problem(Problem& p, int splits_wanted, bool pair) {
 // (m / 64 k-steps) so that the dynamic scheduler balances well, and there should be enough
 // items to occupy the SMs; at most 32.
 inline int plan_gc_splits(int64_t tokens, int r, int m) {
-  const int items = ((r + 2 * BM - 1) / (2 * BM)) * ((m + pick_bn(m, false) - 1) / pick_bn(m, false));
+  const int items = ((r + 2 * BM - 1) / (2 * BM)) * ((m + pick_bn(m) - 1) / pick_bn(m));
   const int ksteps = (int)((tokens + BK - 1) / BK);
   if (ksteps < 1) return 1;
   const int dx_ksteps = (m + BK - 1) / BK;
@@ -1162,12 +896,10 @@ inline size_t gc_workspace_bytes(int64_t tokens, int r, int m) {
   return (size_t)plan_gc_splits(tokens, r, m) * r * m * sizeof(float);
 }
 
-template <bool kPair>
-inline compact_status_t launch_t(const LaunchInfo& li, Params& prm) {
+inline compact_status_t launch(const LaunchInfo& li, Params& prm) {
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(compact_gemm_kernel<kPair>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             Plan<kPair>::SMEM_BYTES) != cudaSuccess) {
+    if (cudaFuncSetAttribute(compact_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
       cudaGetLastError();
       return COMPACT_ERR_CUDA;
     }
@@ -1184,39 +916,17 @@ inline compact_status_t launch_t(const LaunchInfo& li, Params& prm) {
 #if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
   prm.debug_flags = (getenv("COMPACT_SKIP_MMA") ? 1 : 0) | (getenv("COMPACT_SKIP_LOADS") ? 2 : 0) | (getenv("COMPACT_SKIP_EPI") ? 4 : 0);
 #endif
+  const int grid = t < NUM_SMS ? t : NUM_SMS;
   const int threads = prm.gen_ring != GEN_NONE ? THREADS_GEN : THREADS_BASE;
-  cudaLaunchConfig_t cfg;
-  memset(&cfg, 0, sizeof(cfg));
-  cfg.blockDim = dim3(threads, 1, 1);
-  cfg.dynamicSmemBytes = Plan<kPair>::SMEM_BYTES;
-  cfg.stream = li.stream;
-  cudaLaunchAttribute attr[1];
-  if (kPair) {
-    int pairs = t < NUM_SMS / 2 ? t : NUM_SMS / 2;
-    cfg.gridDim = dim3(2 * pairs, 1, 1);
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-  } else {
-    cfg.gridDim = dim3(t < NUM_SMS ? t : NUM_SMS, 1, 1);
-  }
-  const cudaError_t e = cudaLaunchKernelEx(&cfg, compact_gemm_kernel<kPair>, prm);
+  compact_gemm_kernel<<<grid, threads, SMEM_BYTES, li.stream>>>(prm);
   (*li.launches)++;
-  if (e != cudaSuccess) { cudaGetLastError(); return COMPACT_ERR_CUDA; }
   return cudaGetLastError() == cudaSuccess ? COMPACT_OK : COMPACT_ERR_CUDA;
-}
-
-inline compact_status_t launch(const LaunchInfo& li, Params& prm, bool pair) {
-  return pair ? launch_t<true>(li, prm) : launch_t<false>(li, prm);
 }
 
 inline bool tc_shape_ok(int64_t tokens, int n, int m) { return tokens >= 1 && n % 8 == 0 && m % 8 == 0; }
 
 // Algorithm 1: problem 0 = Z = X P (generated B operand; longest items go first), problem 1 = Y = X W.
-inline compact_status_t forward(const LaunchInfo& li, bool pair, const ProjectionParams& pp, int64_t tokens, int m,
+inline compact_status_t forward(const LaunchInfo& li, const ProjectionParams& pp, int64_t tokens, int m,
                                 const __nv_bfloat16* X, int64_t ldx, const __nv_bfloat16* W, int64_t ldw,
                                 __nv_bfloat16* Y, int64_t ldy, __nv_bfloat16* Z, int64_t ldz, int zcols) {
   const int n = pp.n;
@@ -1229,28 +939,26 @@ inline compact_status_t forward(const LaunchInfo& li, bool pair, const Projectio
   prm.gen_ring = GEN_B;
   Problem& pz = prm.prob[0];
   pz.M = (int)tokens; pz.N = zcols; pz.K = n;
-  // one generated 64 x 128 tile of P feeds up to four row blocks of X: 512 tokens per CTA,
-  // 1024 per CTA pair (each CTA of a pair generates 64 of the 128 columns)
-  const int rows_pb = pair ? 2 * BM : BM;
-  pz.bn = (zcols >= 512 / MAX_SUB || pair) ? 512 / MAX_SUB : (int)((zcols + 63) / 64 * 64);
-  pz.nsub = (int)((tokens + rows_pb - 1) / rows_pb) < MAX_SUB ? (int)((tokens + rows_pb - 1) / rows_pb) : MAX_SUB;
+  // one generated 64 x 128 tile of P feeds up to four row blocks of X (512 tokens)
+  pz.bn = zcols >= 512 / MAX_SUB ? 512 / MAX_SUB : (int)((zcols + 63) / 64 * 64);
+  pz.nsub = (int)((tokens + BM - 1) / BM) < MAX_SUB ? (int)((tokens + BM - 1) / BM) : MAX_SUB;
   pz.a_mode = TMA_KMAJOR; pz.b_mode = GENERATED; pz.epi_mode = EPI_BF16;
-  finish_problem(pz, 1, pair);
+  finish_problem(pz, 1);
   Problem& py = prm.prob[1];
   py.M = (int)tokens; py.N = m; py.K = n;
   py.a_mode = TMA_KMAJOR; py.b_mode = TMA_MNMAJOR; py.epi_mode = EPI_BF16;
-  finish_problem(py, 1, pair);
+  finish_problem(py, 1);
   if (!make_map(&prm.tmA[0], X, n, tokens, ldx, BK, BM)) return COMPACT_ERR_CUDA;
   prm.tmA[1] = prm.tmA[0];
   if (!make_map(&prm.tmB[1], W, m, n, ldw, 64, BK)) return COMPACT_ERR_CUDA;
   prm.tmB[0] = prm.tmB[1];   // unused by the generated operand
   if (!make_map(&prm.tmC[0], Z, zcols, tokens, ldz, 64, 32)) return COMPACT_ERR_CUDA;
   if (!make_map(&prm.tmC[1], Y, m, tokens, ldy, 64, 32)) return COMPACT_ERR_CUDA;
-  return launch(li, prm, pair);
+  return launch(li, prm);
 }
 
 // Algorithm 2: problem 0 = Gc = Z^T dY (both operands MN-major, split over tokens), problem 1 = dX = dY W^T.
-inline compact_status_t backward(const LaunchInfo& li, bool pair, int64_t tokens, int n, int m, int r, int zcols,
+inline compact_status_t backward(const LaunchInfo& li, int64_t tokens, int n, int m, int r, int zcols,
                                  const __nv_bfloat16* dY, int64_t lddy, const __nv_bfloat16* Z, int64_t ldz,
                                  const __nv_bfloat16* W, int64_t ldw, __nv_bfloat16* dX, int64_t lddx, float* Gc,
                                  int64_t ldg, int accumulate, void* workspace, size_t workspace_bytes) {
@@ -1266,7 +974,7 @@ inline compact_status_t backward(const LaunchInfo& li, bool pair, int64_t tokens
   Problem& pg = prm.prob[0];
   pg.M = r; pg.N = m; pg.K = (int)tokens;
   pg.a_mode = TMA_MNMAJOR; pg.b_mode = TMA_MNMAJOR; pg.epi_mode = EPI_F32;
-  finish_problem(pg, splits, pair);
+  finish_problem(pg, splits);
   if (staged) {
     if (!make_map_f32_3d(&prm.tmC[0], workspace, m, r, pg.splits, m, (int64_t)r * m)) return COMPACT_ERR_CUDA;
   } else {
@@ -1278,12 +986,12 @@ inline compact_status_t backward(const LaunchInfo& li, bool pair, int64_t tokens
     Problem& px = prm.prob[1];
     px.M = (int)tokens; px.N = n; px.K = m;
     px.a_mode = TMA_KMAJOR; px.b_mode = TMA_KMAJOR; px.epi_mode = EPI_BF16;
-    finish_problem(px, 1, pair);
+    finish_problem(px, 1);
     if (!make_map(&prm.tmA[1], dY, m, tokens, lddy, BK, BM)) return COMPACT_ERR_CUDA;
-    if (!make_map(&prm.tmB[1], W, m, n, ldw, BK, pair ? px.bn / 2 : px.bn)) return COMPACT_ERR_CUDA;
+    if (!make_map(&prm.tmB[1], W, m, n, ldw, BK, px.bn)) return COMPACT_ERR_CUDA;
     if (!make_map(&prm.tmC[1], dX, n, tokens, lddx, 64, 32)) return COMPACT_ERR_CUDA;
   }
-  compact_status_t s = launch(li, prm, pair);
+  compact_status_t s = launch(li, prm);
   if (s != COMPACT_OK) return s;
   if (staged) {
     const long long cnt = (long long)r * (m / 4);
@@ -1318,11 +1026,11 @@ inline compact_status_t update(const LaunchInfo& li, const ProjectionParams& pp,
   pu.ncol = m > BN_MAX ? 2 : 1;     // the generator is the bound here: one generated tile of P feeds two column blocks
   pu.a_mode = GENERATED; pu.b_mode = TMA_MNMAJOR; pu.epi_mode = EPI_UPDATE_W;
   pu.scale = scale;
-  finish_problem(pu, 1, false);
+  finish_problem(pu, 1);
   if (!make_map(&prm.tmB[0], Nbuf, m, r, m, 64, BK)) return COMPACT_ERR_CUDA;
   prm.tmA[0] = prm.tmB[0];
   if (!make_map(&prm.tmC[0], W, m, n, ldw, 64, 32)) return COMPACT_ERR_CUDA;
-  return launch(li, prm, false);
+  return launch(li, prm);
 }
 
 }  // namespace tc

@@ -88,27 +88,11 @@ def test_full_size_sampled(cfg, li):
         assert v <= TOL["bf16"], (cfg, li, k, v)
 
 
-@pytest.mark.parametrize("fam", [0, 3], ids=["auto", "pair"])
-def test_config5_reduced_tokens_trajectory(fam):
+def test_config5_reduced_tokens_trajectory():
     # whole-tensor parity over 3 steps at the 7B layer shape with fewer tokens
-    cb.set_kernel_family(fam)
-    try:
-        wl = wlm.config5().with_tokens(2048)
-        errs, epochs, _ = run_layer_trajectory(wl, 0, steps=3)
-    finally:
-        cb.set_kernel_family(0)
+    wl = wlm.config5().with_tokens(2048)
+    errs, epochs, _ = run_layer_trajectory(wl, 0, steps=3)
     assert epochs == [0, 0, 0]
-    for k, v in errs.items():
-        assert v <= TOL["bf16"], (k, v)
-
-
-def test_pair_kernels_full_size_down_proj():
-    # the CTA-pair kernels on the largest ragged shape (r = 1376 -> eleven 128-column P blocks)
-    cb.set_kernel_family(3)
-    try:
-        errs = _sampled_step(wlm.config5(), 6, 16384, np.random.default_rng(0))
-    finally:
-        cb.set_kernel_family(0)
     for k, v in errs.items():
         assert v <= TOL["bf16"], (k, v)
 

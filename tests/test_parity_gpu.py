@@ -25,7 +25,7 @@ def _built():
     cb.set_kernel_family(0)
 
 
-@pytest.fixture(params=[0, 1, 3], ids=["auto", "simt", "pair"])
+@pytest.fixture(params=[0, 1], ids=["auto", "simt"])
 def family(request):
     cb.set_kernel_family(request.param)
     yield request.param
