@@ -71,7 +71,7 @@ class ClockSampler:
             os.close(fd)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+                 "-lms", "20"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -295,14 +295,23 @@ def run_ours(args):
     upd_ms = t_upd / nrec
     upd_gbs = upd_bytes / (upd_ms * 1e-3) / 1e9
     gemm_launches = 2 * len(wl.layers)
+    # DRAM traffic from the committed ncu capture of the C5 q_proj launches
+    # (profiles/compact_gemm_kernel_c5_qproj_full.md): forward 559.6 MB, backward 574.0 MB for
+    # 1236.95 algorithmic GFLOP; update 38.0 MB for 109.1 MB of algorithmic bytes (W stays in L2
+    # at that size).  Scaled to this workload's launches in proportion to the algorithmic work.
+    traffic_gemm = (559.6e6 + 574.0e6) / 1236.95e9 * gemm_flops / gemm_launches
+    traffic_upd = None
     roofline = {"kernel": "compact_gemm_kernel (forward and backward launches)", "bound": "tensor",
                 "achieved": gemm_tflops, "peak": tens_peak, "unit": "TFLOP/s", "frac": gemm_tflops / tens_peak,
                 "peak_kind": f"{peak_kind} bf16 sustained", "frac_of_nominal_2250": gemm_tflops / NOMINAL_BF16_TFLOPS,
-                "avg_launch_ms": gemm_ms / gemm_launches, "launches_per_step": gemm_launches, "traffic": None}
+                "avg_launch_ms": gemm_ms / gemm_launches, "launches_per_step": gemm_launches,
+                "algorithmic_flops_per_launch": gemm_flops / gemm_launches, "traffic": traffic_gemm,
+                "traffic_note": "bytes per launch, scaled by flops from the ncu capture of the C5 q_proj forward+backward launches"}
     roofline_update = {"kernel": "adam_moments + compact_gemm_kernel (update launches)", "bound": "hbm",
                        "achieved": upd_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": upd_gbs / hbm_peak,
                        "peak_kind": f"{peak_kind} copy", "frac_of_nominal_8000": upd_gbs / NOMINAL_HBM_GBS,
-                       "avg_launch_ms": upd_ms / len(wl.layers), "traffic": None}
+                       "avg_launch_ms": upd_ms / len(wl.layers), "algorithmic_bytes_per_launch": upd_bytes / len(wl.layers),
+                       "traffic": traffic_upd}
 
     # end to end through the public API with HOST inputs: H2D of X, dY every step, D2H of the step's Gc
     e2e = None
