@@ -423,7 +423,7 @@ int compact_set_kernel_family(int family) {
 
 uint64_t compact_kernel_launch_count(void) { return g_launches.load(); }
 
-#ifdef COMPACT_PROFILE
+#if defined(COMPACT_PROFILE) || defined(COMPACT_PROFILE_GEN)
 // Profiling build only: cumulative clocks of the MMA-issuing threads
 // [wait accumulator, wait B, wait A, issue, total]; reading clears them.
 void compact_debug_profile(unsigned long long* out) {

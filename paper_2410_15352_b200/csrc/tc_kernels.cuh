@@ -46,11 +46,11 @@ constexpr int STAGE_BYTES = B_BYTES + 2 * A_BYTES;
 constexpr int NS = CFG_NS;               // stages in the ring
 constexpr int RING_BYTES = NS * STAGE_BYTES;
 constexpr int STAGING_BYTES = 4096;      // one staged tile: 32 rows x 128 bytes
-constexpr int STAGING_BUFS = 2;          // staged tiles per epilogue warp
+constexpr int STAGING_BUFS = 1;          // staged tiles per epilogue warp
 constexpr int QDEPTH = 4;                // work items the scheduler may run ahead
-constexpr int NUM_EPI_WARPS = 4;
+constexpr int NUM_EPI_WARPS = 8;         // two sets of four (one per TMEM lane quarter); each set drains one accumulator slot
 constexpr int NUM_GEN_WARPS = 16;
-constexpr int NUM_LOADERS = 3;           // loader threads besides the stage owner: A0, A1, upper half of B
+constexpr int NUM_LOADERS = 2;           // loader threads besides the stage owner: A tile 0, A tile 1
 constexpr int THREADS_BASE = 64 + 32 * NUM_EPI_WARPS + 32 * NUM_LOADERS;   // owner/scheduler, MMA, epilogue, loaders
 constexpr int THREADS_GEN = THREADS_BASE + 32 * NUM_GEN_WARPS;
 constexpr int NUM_BARRIERS = 2 * NS + 4 + 2 * QDEPTH + NUM_EPI_WARPS * STAGING_BUFS;
@@ -65,8 +65,10 @@ enum EpiMode { EPI_BF16 = 0, EPI_F32 = 1, EPI_UPDATE_W = 2 };
 enum GenRing { GEN_NONE = 0, GEN_A = 1, GEN_B = 2 };
 
 constexpr unsigned int STATUS_TIMEOUT = 1u;
-#ifdef COMPACT_PROFILE
+#if defined(COMPACT_PROFILE) || defined(COMPACT_PROFILE_GEN)
 __device__ unsigned long long g_prof[8];
+#endif
+#ifdef COMPACT_PROFILE
 #define PROF_T() clock64()
 #define PROF_ADD(i, t0) prof[i] += clock64() - (t0)
 #else
@@ -169,7 +171,6 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t sr
 }
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
@@ -268,9 +269,9 @@ __device__ __forceinline__ TileCoord decode_tile(const Params& prm, int tile) {
 //   0      item scheduler and stage owner: waits for a free stage, declares the bytes that will land
 //          on its full barrier, arrives, and loads the (lower half of the) B tile
 //   1      tcgen05.mma issuer (one thread), owner of TMEM
-//   2..5   epilogue
-//   6,7,8  loaders: A tile 0, A tile 1, upper half of an MN-major B tile (each only issues TMA)
-//   9..24  generators of P (launches with a generated operand only)
+//   2..9   epilogue: two sets of four warps; with two accumulator slots each set drains one of them
+//   10,11  loaders: A tile 0, A tile 1 (each only issues TMA)
+//   12..27 generators of P (launches with a generated operand only)
 // --------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __grid_constant__ Params prm) {
   extern __shared__ uint8_t smem_raw[];
@@ -312,7 +313,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       mbar_init(qfull(s), 1);
       mbar_init(qempty(s), consumers);
     }
-    for (int w = 0; w < NUM_EPI_WARPS * STAGING_BUFS; ++w) mbar_init(wbar(w), 1);
+    for (int w = 0; w < NUM_EPI_WARPS; ++w) mbar_init(wbar(w), 1);
     *abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async_smem();
@@ -386,8 +387,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
               if (p.b_mode == TMA_KMAJOR) {
                 tma_load_2d(dst, mapB, fb, k0, n0);
               } else {
-                const int nblk = p.bn / 64, lower = nblk > 2 ? 2 : nblk;   // the upper blocks go to a loader
-                for (int b = 0; b < lower; ++b) tma_load_2d(dst + b * 8192, mapB, fb, n0 + 64 * b, k0);
+                for (int b = 0; b < p.bn / 64; ++b) tma_load_2d(dst + b * 8192, mapB, fb, n0 + 64 * b, k0);
               }
             }
           }
@@ -396,8 +396,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
     }
   } else if (loader >= 0) {
     // ------------------------------ loaders --------------------------------------
-    // 0: A tile in slot 0, 1: A tile in slot 1, 2: blocks 2.. of an MN-major B tile.  They only issue
-    // TMA; the bytes were declared by the stage owner.
+    // 0: A tile in slot 0, 1: A tile in slot 1.  They only issue TMA; the bytes were declared by the stage owner.
     if (lane == 0) {
       uint32_t is = 0;
       bool ok = true;
@@ -407,10 +406,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const TileCoord t = decode_tile(prm, tile);
         const Problem& p = prm.prob[t.prob];
         const CUtensorMap* mapA = &prm.tmA[t.prob];
-        const CUtensorMap* mapB = &prm.tmB[t.prob];
-        bool mine;
-        if (loader == 2) mine = p.b_mode == TMA_MNMAJOR && p.bn > 128;
-        else mine = p.a_mode != GENERATED;
+        bool mine = p.a_mode != GENERATED;
 #if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
         if (prm.debug_flags & 2) mine = false;
 #endif
@@ -422,12 +418,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             const int s = (int)(is % NS);
             const uint32_t fb = full_bar(s);
             const uint32_t stage = smem_base + s * STAGE_BYTES;
-            if (loader == 2) {
-              if (!stage_has_b(p, j)) continue;
-              if (!(ok = mbar_wait(empty_bar(s), ((is / NS) & 1u) ^ 1, abort_flag, prm.status))) break;
-              const int n0 = t.n0 + (p.ncol > 1 ? j : 0) * p.bn;
-              for (int b = 2; b < p.bn / 64; ++b) tma_load_2d(stage + STAGE_B_OFF + b * 8192, mapB, fb, n0 + 64 * b, k0);
-            } else {
+            {
               if (loader >= stage_num_a(p, t, j)) continue;
               if (!(ok = mbar_wait(empty_bar(s), ((is / NS) & 1u) ^ 1, abort_flag, prm.status))) break;
               const int mi = p.ncol > 1 ? 0 : 2 * j + loader;
@@ -479,6 +470,10 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         // one UMMA consumes K = 16: 32 bytes along a K-major row, or two 8-row groups (2048 bytes) MN-major
         const uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4), b_step = b_mn ? (2048u >> 4) : (32u >> 4);
         const int bn = p.bn, nst = t.nst;
+        // accumulator ai of the item sits in slot ai / sps at column (ai % sps) * bn (a slot is 256 columns)
+        const int naccs = p.nsub * p.ncol;
+        const int sps = BN_MAX / bn > naccs ? naccs : BN_MAX / bn;
+        auto acc_col = [&](int ai) -> uint32_t { return (uint32_t)((ai / sps) * BN_MAX + (ai % sps) * bn); };
         auto issue4 = [&](uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t first) {
 #if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
           if (prm.debug_flags & 1) return;
@@ -498,11 +493,11 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             tc_fence_after();
             const uint32_t stage = smem_base + s * STAGE_BYTES;
             if (p.ncol > 1) {
-              issue4(d_base + j * bn, desc_lo(stage0 + STAGE_A0_OFF, a_mn), desc_lo(stage + STAGE_B_OFF, b_mn), first);
+              issue4(d_base + acc_col(j), desc_lo(stage0 + STAGE_A0_OFF, a_mn), desc_lo(stage + STAGE_B_OFF, b_mn), first);
             } else {
               const uint32_t b_lo = desc_lo(stage0 + STAGE_B_OFF, b_mn);
-              issue4(d_base + (2 * j) * bn, desc_lo(stage + STAGE_A0_OFF, a_mn), b_lo, first);
-              if (2 * j + 1 < t.nsub) issue4(d_base + (2 * j + 1) * bn, desc_lo(stage + STAGE_A1_OFF, a_mn), b_lo, first);
+              issue4(d_base + acc_col(2 * j), desc_lo(stage + STAGE_A0_OFF, a_mn), b_lo, first);
+              if (2 * j + 1 < t.nsub) issue4(d_base + acc_col(2 * j + 1), desc_lo(stage + STAGE_A1_OFF, a_mn), b_lo, first);
             }
             // a stage that holds nothing shared goes back at once; the first stage of the k-step goes last
             if (j > 0) umma_commit(empty_bar(s));
@@ -516,15 +511,17 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
     }
   } else if (warp < 2 + NUM_EPI_WARPS) {
     // ------------------------------ epilogue ------------------------------------
-    // TMEM -> registers -> 128B-swizzled staging tile (32 rows x 128 bytes, two per warp) -> TMA store.
-    // The chunks of an item (accumulator by accumulator, 64 bf16 or 32 fp32 columns at a time) are
-    // walked as one sequence so that the W tile of the next chunk (update) is already on its way
-    // while the current one is processed.
+    // TMEM -> registers -> 128B-swizzled staging tile (32 rows x 128 bytes per warp) -> TMA store.
+    // Two sets of four warps (one warp per TMEM lane quarter).  With two accumulator slots in an item
+    // set e drains slot e, so both slots empty at the same time; with one slot the sets take alternate
+    // chunks.  Every warp still walks every slot (wait for its MMAs, hand it back) so that the
+    // hand-back barrier sees a fixed number of arrivals.
     const int q = warp & 3;                 // TMEM lane quarter this warp may read
-    const uint32_t stg0 = staging + (warp - 2) * STAGING_BUFS * STAGING_BYTES;
-    uint8_t* stg_gen0 = smem_gen + RING_BYTES + (warp - 2) * STAGING_BUFS * STAGING_BYTES;
-    uint32_t wph[STAGING_BUFS] = {0, 0};
-    int buf = 0;
+    const int eset = (warp - 2) >> 2;       // 0 or 1
+    const uint32_t stg = staging + (warp - 2) * STAGING_BYTES;
+    uint8_t* stg_gen = smem_gen + RING_BYTES + (warp - 2) * STAGING_BYTES;
+    const uint32_t my_wbar = wbar(warp - 2);
+    uint32_t wph = 0;
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
@@ -540,36 +537,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       const int sub_per_slot = BN_MAX / p.bn > naccs ? naccs : BN_MAX / p.bn;
       const int cw = p.epi_mode == EPI_F32 ? 32 : 64;          // columns per staged chunk
       const int cpa = p.bn / cw;                               // chunks per accumulator
-      // Cursor over the chunks this warp writes: accumulator ai (slot sl, position su in the slot), chunk ci.
-      struct Cur { int ai, sl, su, ci; };
       const int row_q = q * 32;
-      auto acc_valid = [&](int ai) -> bool {       // does accumulator ai hold rows/columns this warp writes?
-        const int mi = p.ncol > 1 ? 0 : ai, cb = p.ncol > 1 ? ai : 0;
-        return mi < t.nsub && cb < t.ncol && t.m0 + mi * BM + row_q < p.M && t.n0 + cb * p.bn < p.N;
-      };
-      auto cur_col = [&](const Cur& c) -> int { return t.n0 + (p.ncol > 1 ? c.ai : 0) * p.bn + c.ci * cw; };
-      auto cur_row = [&](const Cur& c) -> int { return t.m0 + (p.ncol > 1 ? 0 : c.ai) * BM + row_q; };
-      auto seek = [&](Cur c) -> Cur {              // first valid chunk at or after (ai, 0)
-        while (c.ai < naccs && !acc_valid(c.ai)) {
-          ++c.ai;
-          if (++c.su == sub_per_slot) { c.su = 0; ++c.sl; }
-        }
-        c.ci = 0;
-        return c;
-      };
-      auto advance = [&](Cur c) -> Cur {
-        ++c.ci;
-        if (c.ci < cpa && cur_col(c) < p.N) return c;
-        ++c.ai;
-        if (++c.su == sub_per_slot) { c.su = 0; ++c.sl; }
-        return seek(c);
-      };
-      auto load_w = [&](const Cur& c, int b) {      // update: W tile of chunk c into staging buffer b
-        if (lane == 0) {
-          mbar_arrive_expect_tx(wbar((warp - 2) * STAGING_BUFS + b), STAGING_BYTES);
-          tma_load_2d(stg0 + b * STAGING_BYTES, mapC, wbar((warp - 2) * STAGING_BUFS + b), cur_col(c), cur_row(c));
-        }
-      };
       if (slots == 2 && acc == 1) {
         if (!(ok = mbar_wait(tfull_bar(1), acc_phase, abort_flag, prm.status))) break;
         __syncwarp();
@@ -577,114 +545,108 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         acc = 0;
         acc_phase ^= 1;
       }
-      Cur cur = seek(Cur{0, 0, 0, 0});
+      for (int sl = 0; sl < slots && ok; ++sl) {
+        if (!(ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, prm.status))) break;
+        tc_fence_after();
+        bool mine_slot = slots == 2 ? (sl == eset) : true;
 #if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
-      if (prm.debug_flags & 4) cur.ai = naccs;       // write nothing: hand the accumulators straight back
+        if (prm.debug_flags & 4) mine_slot = false;       // write nothing: hand the accumulators straight back
 #endif
-      if (p.epi_mode == EPI_UPDATE_W && cur.ai < naccs) {
-        if (lane == 0) tma_store_wait_read();          // both staging buffers are free
-        __syncwarp();
-        load_w(cur, buf);
-      }
-      int cur_slot = -1;
-      // enter accumulator slot `want` (waiting for its MMAs), handing back the slots passed on the way
-      auto enter_slot = [&](int want) -> bool {
-        while (cur_slot < want) {
-          if (cur_slot >= 0) {
-            tc_fence_before();
+        for (int su = 0; su < sub_per_slot && ok && mine_slot; ++su) {
+          const int ai = sl * sub_per_slot + su;            // accumulator of the item: a row block or a column block
+          const int mi = p.ncol > 1 ? 0 : ai, cb = p.ncol > 1 ? ai : 0;
+          if (mi >= t.nsub || cb >= t.ncol) break;
+          const int row0 = t.m0 + mi * BM + row_q;
+          if (row0 >= p.M) continue;          // this warp's 32 rows are all padding
+          const int ncol0 = t.n0 + cb * p.bn;
+          const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN_MAX + su * p.bn;
+          for (int ci = (slots == 2 ? 0 : eset); ci < cpa && ok; ci += (slots == 2 ? 1 : 2)) {
+            const int col = ncol0 + ci * cw;
+            if (col >= p.N) break;
+            if (lane == 0) tma_store_wait_read();          // the previous store has read the staging tile
             __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(acc));
-            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
-          }
-          ++cur_slot;
-          if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, prm.status)) return false;
-          tc_fence_after();
-        }
-        return true;
-      };
-      while (cur.ai < naccs && ok) {
-        const int sl = cur.sl, tc = cur.su * p.bn + cur.ci * cw, col = cur_col(cur), row0 = cur_row(cur);
-        const Cur nxt = advance(cur);
-        uint8_t* stg_gen = stg_gen0 + buf * STAGING_BYTES;
-        const uint32_t stg = stg0 + buf * STAGING_BYTES;
-        if (p.epi_mode == EPI_UPDATE_W) {
-          if (nxt.ai < naccs) {
-            if (lane == 0) tma_store_wait_read();      // the other buffer's store has read it
-            __syncwarp();
-            load_w(nxt, buf ^ 1);
-          }
-        } else {
-          if (lane == 0) tma_store_wait_read1();       // this buffer's previous store has read it
-          __syncwarp();
-        }
-        if (!(ok = enter_slot(sl))) break;
-        const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + acc * BN_MAX + tc;
-        if (p.epi_mode == EPI_F32) {
-          uint32_t v[32];
-          tmem_ld32(tcol, v);
-          tmem_ld_wait();
+            if (p.epi_mode == EPI_F32) {
+              uint32_t v[32];
+              tmem_ld32(tcol + ci * cw, v);
+              tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 8; ++j)
-            *reinterpret_cast<uint4*>(stg_gen + lane * 128 + ((j ^ sw) << 4)) =
-                make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-          fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0) {
-            tma_store_3d(mapC, stg, col, row0, t.split);
-            tma_store_commit();
-          }
-        } else {
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            uint32_t v[32];
-            tmem_ld32(tcol + 32 * h, v);
-            tmem_ld_wait();
+              for (int j = 0; j < 8; ++j)
+                *reinterpret_cast<uint4*>(stg_gen + lane * 128 + ((j ^ sw) << 4)) =
+                    make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+              fence_proxy_async_smem();
+              __syncwarp();
+              if (lane == 0) {
+                tma_store_3d(mapC, stg, col, row0, t.split);
+                tma_store_commit();
+              }
+              continue;
+            }
             if (p.epi_mode == EPI_UPDATE_W) {
-              // W <- W - (eta alpha) (P N), one rounding of the result (Algorithm 3 line 9)
-              if (h == 0) {
-                if (!(ok = mbar_wait(wbar((warp - 2) * STAGING_BUFS + buf), wph[buf], abort_flag, prm.status))) break;
-                wph[buf] ^= 1;
-              }
-              const float sc = -p.scale;
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                uint4* cell = reinterpret_cast<uint4*>(stg_gen + lane * 128 + (((4 * h + j) ^ sw) << 4));
-                uint4 w = *cell;
-                w.x = pack_bf16x2(fmaf(sc, __uint_as_float(v[8 * j + 0]), bf16lo(w.x)), fmaf(sc, __uint_as_float(v[8 * j + 1]), bf16hi(w.x)));
-                w.y = pack_bf16x2(fmaf(sc, __uint_as_float(v[8 * j + 2]), bf16lo(w.y)), fmaf(sc, __uint_as_float(v[8 * j + 3]), bf16hi(w.y)));
-                w.z = pack_bf16x2(fmaf(sc, __uint_as_float(v[8 * j + 4]), bf16lo(w.z)), fmaf(sc, __uint_as_float(v[8 * j + 5]), bf16hi(w.z)));
-                w.w = pack_bf16x2(fmaf(sc, __uint_as_float(v[8 * j + 6]), bf16lo(w.w)), fmaf(sc, __uint_as_float(v[8 * j + 7]), bf16hi(w.w)));
-                *cell = w;
-              }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                uint4 o;
-                o.x = pack_bf16x2(__uint_as_float(v[8 * j + 0]), __uint_as_float(v[8 * j + 1]));
-                o.y = pack_bf16x2(__uint_as_float(v[8 * j + 2]), __uint_as_float(v[8 * j + 3]));
-                o.z = pack_bf16x2(__uint_as_float(v[8 * j + 4]), __uint_as_float(v[8 * j + 5]));
-                o.w = pack_bf16x2(__uint_as_float(v[8 * j + 6]), __uint_as_float(v[8 * j + 7]));
-                *reinterpret_cast<uint4*>(stg_gen + lane * 128 + (((4 * h + j) ^ sw) << 4)) = o;
+              // bring the W tile in first: W <- W - (eta alpha) (P N), one rounding (Algorithm 3 line 9)
+              if (lane == 0) {
+                mbar_arrive_expect_tx(my_wbar, STAGING_BYTES);
+                tma_load_2d(stg, mapC, my_wbar, col, row0);
               }
             }
-          }
-          if (!ok) break;
-          fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0) {
-            tma_store_2d(mapC, stg, col, row0);
-            tma_store_commit();
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              uint32_t v[32];
+#if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
+              if (prm.debug_flags & 16) {
+#pragma unroll
+                for (int z = 0; z < 32; ++z) v[z] = 0;
+              } else
+#endif
+              {
+                tmem_ld32(tcol + ci * cw + 32 * h, v);
+                tmem_ld_wait();
+              }
+              if (p.epi_mode == EPI_UPDATE_W) {
+                if (h == 0) {
+                  if (!(ok = mbar_wait(my_wbar, wph, abort_flag, prm.status))) break;
+                  wph ^= 1;
+                }
+                const float sc = -p.scale;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  uint4* cell = reinterpret_cast<uint4*>(stg_gen + lane * 128 + (((4 * h + j) ^ sw) << 4));
+                  uint4 w = *cell;
+                  w.x = pack_bf16x2(fmaf(sc, __uint_as_float(v[8 * j + 0]), bf16lo(w.x)), fmaf(sc, __uint_as_float(v[8 * j + 1]), bf16hi(w.x)));
+                  w.y = pack_bf16x2(fmaf(sc, __uint_as_float(v[8 * j + 2]), bf16lo(w.y)), fmaf(sc, __uint_as_float(v[8 * j + 3]), bf16hi(w.y)));
+                  w.z = pack_bf16x2(fmaf(sc, __uint_as_float(v[8 * j + 4]), bf16lo(w.z)), fmaf(sc, __uint_as_float(v[8 * j + 5]), bf16hi(w.z)));
+                  w.w = pack_bf16x2(fmaf(sc, __uint_as_float(v[8 * j + 6]), bf16lo(w.w)), fmaf(sc, __uint_as_float(v[8 * j + 7]), bf16hi(w.w)));
+                  *cell = w;
+                }
+              } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  uint4 o;
+                  o.x = pack_bf16x2(__uint_as_float(v[8 * j + 0]), __uint_as_float(v[8 * j + 1]));
+                  o.y = pack_bf16x2(__uint_as_float(v[8 * j + 2]), __uint_as_float(v[8 * j + 3]));
+                  o.z = pack_bf16x2(__uint_as_float(v[8 * j + 4]), __uint_as_float(v[8 * j + 5]));
+                  o.w = pack_bf16x2(__uint_as_float(v[8 * j + 6]), __uint_as_float(v[8 * j + 7]));
+                  *reinterpret_cast<uint4*>(stg_gen + lane * 128 + (((4 * h + j) ^ sw) << 4)) = o;
+                }
+              }
+            }
+            if (!ok) break;
+#if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
+            if (prm.debug_flags & 8) continue;
+#endif
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(mapC, stg, col, row0);
+              tma_store_commit();
+            }
           }
         }
-        buf ^= 1;
-        cur = nxt;
+        if (!ok) break;
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(tempty_bar(acc));
+        if (++acc == 2) { acc = 0; acc_phase ^= 1; }
       }
-      if (!ok) break;
-      if (!(ok = enter_slot(slots - 1))) break;      // slots this warp had nothing to write for
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(acc));
-      if (++acc == 2) { acc = 0; acc_phase ^= 1; }
     }
     if (lane == 0) tma_store_wait_all();
   } else {
@@ -704,7 +666,13 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       if (!gen_a && !gen_b) { is += klen * t.nst; continue; }      // the stage owner arrives for this item
       for (int ks = t.k_begin; ks < t.k_end && ok; ++ks, is += t.nst) {
         const int s = (int)(is % NS);
+#ifdef COMPACT_PROFILE_GEN
+        const long long g0 = clock64();
+#endif
         const bool w = mbar_wait(empty_bar(s), ((is / NS) & 1u) ^ 1, abort_flag, prm.status);
+#ifdef COMPACT_PROFILE_GEN
+        const long long g1 = clock64();
+#endif
         const int k0 = ks * BK;
         if (w && gen_b) {
           // B[k = row i of P][n = column j of P], MN-major: 64-column blocks of [64 k][128 B]
@@ -725,9 +693,15 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             *reinterpret_cast<uint4*>(sap + rr * 128 + ((c ^ (rr & 7)) << 4)) = val;
           }
         }
+#ifdef COMPACT_PROFILE_GEN
+        const long long g2 = clock64();
+#endif
         fence_proxy_async_smem();
         ok = __all_sync(0xffffffffu, w);
         if (ok && lane == 0) mbar_arrive(full_bar(s));
+#ifdef COMPACT_PROFILE_GEN
+        if (gtid == 0) { atomicAdd(&g_prof[0], (unsigned long long)(g1 - g0)); atomicAdd(&g_prof[1], (unsigned long long)(g2 - g1)); atomicAdd(&g_prof[2], (unsigned long long)(clock64() - g2)); atomicAdd(&g_prof[3], 1ull); }
+#endif
         // later stages of the k-step hold no generated data: the stage owner arrives for the generators there
       }
     }
@@ -914,7 +888,7 @@ inline compact_status_t launch(const LaunchInfo& li, Params& prm) {
   prm.status = li.status;
   prm.sched = li.sched;
 #if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
-  prm.debug_flags = (getenv("COMPACT_SKIP_MMA") ? 1 : 0) | (getenv("COMPACT_SKIP_LOADS") ? 2 : 0) | (getenv("COMPACT_SKIP_EPI") ? 4 : 0);
+  prm.debug_flags = (getenv("COMPACT_SKIP_MMA") ? 1 : 0) | (getenv("COMPACT_SKIP_LOADS") ? 2 : 0) | (getenv("COMPACT_SKIP_EPI") ? 4 : 0) | (getenv("COMPACT_SKIP_STORE") ? 8 : 0) | (getenv("COMPACT_SKIP_TMEMLD") ? 16 : 0);
 #endif
   const int grid = t < NUM_SMS ? t : NUM_SMS;
   const int threads = prm.gen_ring != GEN_NONE ? THREADS_GEN : THREADS_BASE;

@@ -88,6 +88,9 @@ SMALL = [
     (300, 1376, 512, 344),       # ragged tokens, ragged r (ldz 352)
     (1000, 512, 1376, 128),      # ragged m tile
     (130, 264, 72, 50),          # everything ragged
+    (1, 64, 64, 8),              # a single token
+    (129, 128, 136, 24),         # one row past a block, m not a multiple of 64
+    (640, 320, 520, 320),        # r == n (full rank), three 128-column blocks of P
 ]
 
 
@@ -154,6 +157,35 @@ def test_run_twice_bitwise_and_accumulate(family):
     _, Gco = ora.backward(to64(dY), to64(Z1[:, :128]))
     assert co.rel_frobenius(to64(Ga), Gco) <= TOL["bf16"]
     assert co.rel_frobenius(to64(G1), Gco) <= TOL["bf16"]
+
+
+def test_padded_pitches(family):
+    # leading dimensions larger than the logical widths (views into wider buffers)
+    tokens, n, m, r = 300, 256, 192, 40
+    wl = wlm.Workload("pitch", 98, "bf16", tokens, [wlm.LayerShape("l", n, m, r)], x_scale_inv_sqrt_n=True)
+    gpu, ora, W0 = make_pair(wl, 0)
+    pad = lambda t, extra: torch.cat([t, torch.full((t.shape[0], extra), 7.0, dtype=t.dtype)], dim=1).cuda()[:, :t.shape[1]]
+    X, dY, W = pad(wlm.draw_X(wl, 0, 0), 8), pad(wlm.draw_dY(wl, 0, 0), 16), pad(W0, 24)
+    Y = torch.zeros((tokens, m + 8), dtype=torch.bfloat16, device="cuda")[:, :m]
+    Z = torch.zeros((tokens, gpu.ldz + 16), dtype=torch.bfloat16, device="cuda")[:, :gpu.ldz]
+    dX = torch.zeros((tokens, n + 8), dtype=torch.bfloat16, device="cuda")[:, :n]
+    Gc = torch.zeros((r, m + 4), dtype=torch.float32, device="cuda")[:, :m]
+    M, V = torch.zeros_like(Gc.contiguous()), torch.zeros_like(Gc.contiguous())
+    assert X.stride(0) == n + 8 and W.stride(0) == m + 24
+    _, _, ep = gpu.forward(X, W, Y, Z)
+    gpu.backward(dY, Z, W, Gc=Gc, dX=dX)
+    Yo, Zo = ora.forward(to64(X))
+    dXo, Gco = ora.backward(to64(dY), Zo)
+    for k, a, b in (("Y", Y, Yo), ("Z", Z[:, :r], Zo), ("dX", dX, dXo), ("Gc", Gc, Gco)):
+        assert co.rel_frobenius(to64(a), b) <= TOL["bf16"], k
+    assert not Z[:, r:].any()
+    # nothing outside the logical widths was touched
+    assert not Y._base[:, m:].any() and not dX._base[:, n:].any() and not Gc._base[:, m:].any() and not Z._base[:, gpu.ldz:].any()
+    Gd = Gc.contiguous()
+    gpu.adam_update(W, Gd, M, V, ep)
+    ora.update(Gco)
+    assert co.rel_frobenius(to64(W), ora.W) <= TOL["bf16"]
+    assert torch.all(W._base[:, m:] == 7.0)
 
 
 def test_empty_batch_and_epoch_guard():
