@@ -71,6 +71,11 @@ ProjectionParams make_pp(const compact_layer_t* L, uint32_t epoch) {
   ProjectionParams pp;
   pp.key = make_philox_key(L->cfg.seed);
   pp.layer_id = L->cfg.layer_id;
+  {
+    const uint64_t pl = (uint64_t)0xCD9E8D57u * (uint64_t)L->cfg.layer_id;
+    pp.layer_hi = (uint32_t)(pl >> 32);
+    pp.layer_lo = (uint32_t)pl;
+  }
   pp.epoch = epoch;
   pp.n = L->cfg.n;
   pp.r = L->cfg.r;

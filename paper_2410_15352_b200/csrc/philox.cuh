@@ -26,10 +26,11 @@ __host__ __device__ inline PhiloxKey make_philox_key(uint64_t seed) {
   return k;
 }
 
-__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                               const PhiloxKey& key) {
+// Ten rounds starting from the state after `first` rounds.
+template <int kFirst>
+__device__ __forceinline__ uint4 philox_rounds(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, const PhiloxKey& key) {
 #pragma unroll
-  for (int i = 0; i < 10; ++i) {
+  for (int i = kFirst; i < 10; ++i) {
     const uint64_t p0 = (uint64_t)0xD2511F53u * c0;   // one wide multiply each
     const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
     c0 = (uint32_t)(p1 >> 32) ^ c1 ^ key.k0[i];
@@ -38,6 +39,24 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
     c3 = (uint32_t)p0;
   }
   return make_uint4(c0, c1, c2, c3);
+}
+
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                               const PhiloxKey& key) {
+  return philox_rounds<0>(c0, c1, c2, c3, key);
+}
+
+// Same function for the projection's counter (q, i, layer_id, epoch): the third counter word is
+// the same for every entry of a layer, so its first-round product 0xCD9E8D57 * layer_id is
+// computed once on the host (hi, lo) and the first round needs one wide multiply instead of two.
+__device__ __forceinline__ uint4 philox4x32_10_layer(uint32_t q, uint32_t i, uint32_t epoch, uint32_t layer_hi,
+                                                     uint32_t layer_lo, const PhiloxKey& key) {
+  const uint64_t p0 = (uint64_t)0xD2511F53u * q;
+  const uint32_t c0 = layer_hi ^ i ^ key.k0[0];
+  const uint32_t c1 = layer_lo;
+  const uint32_t c2 = (uint32_t)(p0 >> 32) ^ epoch ^ key.k1[0];
+  const uint32_t c3 = (uint32_t)p0;
+  return philox_rounds<1>(c0, c1, c2, c3, key);
 }
 
 // Four consecutive entries P[i, 4q .. 4q+3] before the 1/sqrt(r) scale.
@@ -85,6 +104,7 @@ __device__ __forceinline__ float4 gaussian4_fast_scaled(uint4 x, float neg2ln2_o
 struct ProjectionParams {
   PhiloxKey key;
   uint32_t layer_id;
+  uint32_t layer_hi, layer_lo;   // 0xCD9E8D57 * layer_id, high and low words
   uint32_t epoch;
   int32_t n;
   int32_t r;
@@ -97,7 +117,7 @@ struct ProjectionParams {
 template <bool kFast>
 __device__ __forceinline__ float4 projection4(const ProjectionParams& pp, int i, int q) {
   if (i >= pp.n || 4 * q >= pp.r) return make_float4(0.f, 0.f, 0.f, 0.f);
-  const uint4 x = philox4x32_10((uint32_t)q, (uint32_t)i, pp.layer_id, pp.epoch, pp.key);
+  const uint4 x = philox4x32_10_layer((uint32_t)q, (uint32_t)i, pp.epoch, pp.layer_hi, pp.layer_lo, pp.key);
   float4 g;
   if (kFast) {
     g = gaussian4_fast_scaled(x, pp.neg2ln2_over_r);

@@ -677,9 +677,10 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         if (w && gen_b) {
           // B[k = row i of P][n = column j of P], MN-major: 64-column blocks of [64 k][128 B]
           uint8_t* sbp = smem_gen + s * STAGE_BYTES + STAGE_B_OFF;
-          const int chunks = p.bn >> 3;
+          // bn is 64, 128 or 256 here: 8, 16 or 32 eight-column chunks per row of P
+          const int chunks = p.bn >> 3, cshift = 31 - __clz(chunks);
           for (int id = gtid; id < BK * chunks; id += 32 * NUM_GEN_WARPS) {
-            const int c = id % chunks, kr = id / chunks;
+            const int c = id & (chunks - 1), kr = id >> cshift;
             const uint4 val = projection8_bf16(prm.pp, k0 + kr, t.n0 + c * 8);
             *reinterpret_cast<uint4*>(sbp + (c >> 3) * 8192 + kr * 128 + (((c & 7) ^ (kr & 7)) << 4)) = val;
           }
