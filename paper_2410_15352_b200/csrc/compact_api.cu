@@ -27,6 +27,9 @@ struct compact_layer {
 namespace {
 
 std::atomic<uint64_t> g_launches{0};
+#ifndef CFG_CS
+#define CFG_CS 2   // CTAs of a cluster that share each generated tile of P
+#endif
 std::atomic<int> g_family{0};
 std::atomic<int> g_next_slot{0};
 
@@ -221,7 +224,7 @@ compact_status_t compact_linear_fwd(compact_layer_t* L, int64_t tokens, const vo
   if (L->cfg.dtype == COMPACT_BF16) {
     typedef __nv_bfloat16 T;
     if (g_family.load() != 1) {
-      tc::LaunchInfo li{st, status_word(L), sched_words(L), &g_launches};
+      tc::LaunchInfo li{g_family.load() == 2 ? 1 : CFG_CS, st, status_word(L), sched_words(L), &g_launches};
       s = tc::forward(li, make_pp(L, L->epoch), tokens, L->cfg.m, (const T*)X, ldx, (const T*)W, ldw, (T*)Y, ldy, (T*)Z, ldz,
                       (int)compact_z_ld(L));
       if (s != COMPACT_ERR_SHAPE) return s;   // SHAPE: the tensor-core kernel does not take it
@@ -263,7 +266,7 @@ compact_status_t compact_linear_bwd(compact_layer_t* L, int64_t tokens, const vo
   if (L->cfg.dtype == COMPACT_BF16) {
     typedef __nv_bfloat16 T;
     if (g_family.load() != 1) {
-      tc::LaunchInfo li{st, status_word(L), sched_words(L), &g_launches};
+      tc::LaunchInfo li{g_family.load() == 2 ? 1 : CFG_CS, st, status_word(L), sched_words(L), &g_launches};
       s = tc::backward(li, tokens, L->cfg.n, L->cfg.m, L->cfg.r, (int)compact_z_ld(L), (const T*)dY, lddy, (const T*)Z, ldz, (const T*)W,
                        ldw, (T*)dX, lddx, Gc, ldg, accumulate, workspace, workspace_bytes);
       if (s != COMPACT_ERR_SHAPE) return s;
@@ -293,7 +296,7 @@ compact_status_t compact_adam_update(compact_layer_t* L, void* W, int64_t ldw, c
     typedef __nv_bfloat16 T;
     s = COMPACT_ERR_SHAPE;
     if (g_family.load() != 1) {
-      tc::LaunchInfo li{st, status_word(L), sched_words(L), &g_launches};
+      tc::LaunchInfo li{g_family.load() == 2 ? 1 : CFG_CS, st, status_word(L), sched_words(L), &g_launches};
       s = tc::update(li, make_pp(L, L->epoch), adam_scalars(L, L->step + 1), L->cfg.n, L->cfg.m, L->cfg.r, (T*)W, ldw,
                      Gc, ldg, M, V, lr * L->cfg.alpha, workspace, workspace_bytes);
     }
@@ -422,7 +425,7 @@ compact_status_t compact_debug_projection(const compact_layer_t* L, uint32_t epo
 }
 
 int compact_set_kernel_family(int family) {
-  if (family < 0 || family > 1) return g_family.load();
+  if (family < 0 || family > 2) return g_family.load();
   return g_family.exchange(family);
 }
 

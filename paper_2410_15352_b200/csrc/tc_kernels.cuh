@@ -24,6 +24,7 @@ namespace compact {
 namespace tc {
 
 struct LaunchInfo {
+  int cluster;            // CTAs that share each generated tile of P (1 or 2)
   cudaStream_t stream;
   unsigned int* status;   // device word: kernels OR error bits into it
   unsigned int* sched;    // two device words, zero between launches: next item, finished CTAs
@@ -38,13 +39,20 @@ constexpr int B_BYTES = BN_MAX * BK * 2;
 // One pipeline stage holds a B tile and two A tiles under ONE full/empty barrier pair: every
 // mbarrier operation of the MMA-issuing thread costs ~150 clocks of its serial time, so a stage
 // carries as many MMAs (8) as fit.
+//
+// The ring memory is cut in one of two ways, chosen per problem:
+//   geometry 0: three stages of [B | A0 | A1] (64 KB) for items with two row blocks per stage;
+//   geometry 1: four stages of [B | A0] (48 KB) for items with one row block, whose k-steps take two
+//               stages when they have two column blocks -- the fourth stage gives them two whole
+//               k-steps of look-ahead, which the latency of a generated tile needs.
+// Each geometry has its own barriers.  A CTA meets the problems of a launch in order, so it changes
+// geometry at most once; the roles that write into the ring first wait until the old ring has drained.
 constexpr int STAGE_B_OFF = 0, STAGE_A0_OFF = B_BYTES, STAGE_A1_OFF = B_BYTES + A_BYTES;
-constexpr int STAGE_BYTES = B_BYTES + 2 * A_BYTES;
-#ifndef CFG_NS
-#define CFG_NS 3
-#endif
-constexpr int NS = CFG_NS;               // stages in the ring
-constexpr int RING_BYTES = NS * STAGE_BYTES;
+constexpr int NS0 = 3, STAGE0_BYTES = B_BYTES + 2 * A_BYTES;
+constexpr int NS1 = 4, STAGE1_BYTES = B_BYTES + A_BYTES;
+constexpr int RING_BYTES = NS0 * STAGE0_BYTES;
+static_assert(NS1 * STAGE1_BYTES <= RING_BYTES, "both geometries share the ring memory");
+constexpr int NUM_RING_BARS = 2 * (NS0 + NS1);
 constexpr int STAGING_BYTES = 4096;      // one staged tile: 32 rows x 128 bytes
 constexpr int STAGING_BUFS = 1;          // staged tiles per epilogue warp
 constexpr int QDEPTH = 4;                // work items the scheduler may run ahead
@@ -53,15 +61,19 @@ constexpr int NUM_GEN_WARPS = 16;
 constexpr int NUM_LOADERS = 2;           // loader threads besides the stage owner: A tile 0, A tile 1
 constexpr int THREADS_BASE = 64 + 32 * NUM_EPI_WARPS + 32 * NUM_LOADERS;   // owner/scheduler, MMA, epilogue, loaders
 constexpr int THREADS_GEN = THREADS_BASE + 32 * NUM_GEN_WARPS;
-constexpr int NUM_BARRIERS = 2 * NS + 4 + 2 * QDEPTH + NUM_EPI_WARPS * STAGING_BUFS;
+constexpr int NUM_BARRIERS = NUM_RING_BARS + 4 + 2 * QDEPTH + NUM_EPI_WARPS * STAGING_BUFS;
 constexpr int TAIL_BYTES = 8 * NUM_BARRIERS + 4 * QDEPTH + 16;
 constexpr int SMEM_BYTES = 1024 + RING_BYTES + NUM_EPI_WARPS * STAGING_BUFS * STAGING_BYTES + ((TAIL_BYTES + 127) / 128) * 128;
 constexpr int NUM_SMS = 148;
 constexpr int MAX_SUB = 4;           // row blocks that share one generated B tile
 static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 
-enum OperandMode { TMA_KMAJOR = 0, TMA_MNMAJOR = 1, GENERATED = 2 };
-enum EpiMode { EPI_BF16 = 0, EPI_F32 = 1, EPI_UPDATE_W = 2 };
+// GENERATED: tiles of P with the tile's M (or N) index running over rows of P; as the A operand they are
+// written K-major.  GENERATED_T (A operand only): the M index runs over columns of P and the K index
+// over its rows, written MN-major -- the operand of Z^T = P^T X^T.
+enum OperandMode { TMA_KMAJOR = 0, TMA_MNMAJOR = 1, GENERATED = 2, GENERATED_T = 3 };
+// EPI_BF16_T stores the transpose of the accumulator (lanes become columns of the output).
+enum EpiMode { EPI_BF16 = 0, EPI_F32 = 1, EPI_UPDATE_W = 2, EPI_BF16_T = 3 };
 enum GenRing { GEN_NONE = 0, GEN_A = 1, GEN_B = 2 };
 
 constexpr unsigned int STATUS_TIMEOUT = 1u;
@@ -86,6 +98,7 @@ struct Problem {
   int nsub;
   int ncol;
   int a_mode, b_mode, epi_mode;
+  int geo;                // ring geometry its items use (0 or 1)
   int tile_begin;
   float scale;
 };
@@ -98,6 +111,13 @@ struct alignas(64) Params {
   int num_problems;
   int total_tiles;
   int gen_ring;
+  // Cluster-shared generation: the `cs` CTAs of a cluster take items that need the same tiles of P
+  // (same columns of P, different tokens in the forward; same rows of P, different columns of W in
+  // the update), each generates 1/cs of every tile and writes it into all cs shared memories.
+  int cs;                 // CTAs per cluster (1: every CTA generates for itself)
+  int share_n;            // 0: the cs items of a group are neighbours along M, 1: along N
+  int gen_groups;         // groups of cs generated items; handed out statically, cluster by cluster
+  int dyn_begin;          // first item handed out dynamically (0 when cs == 1)
   int debug_flags;        // profiling builds only: bit 0 = issue no MMAs (measures the load path alone)
   ProjectionParams pp;
   unsigned int* status;
@@ -201,6 +221,33 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+// Commit that arrives on the barrier at the same offset in every CTA of `mask`.
+__device__ __forceinline__ void umma_commit_mc(uint32_t bar, uint16_t mask) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+               "h"(mask)
+               : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address of the same shared-memory location in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+// 16-byte store into another CTA's shared memory; its bytes complete on that CTA's barrier `rbar`.
+__device__ __forceinline__ void st_async_16(uint32_t raddr, uint4 v, uint32_t rbar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(raddr),
+               "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"(rbar)
+               : "memory");
+}
+
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -239,6 +286,20 @@ __device__ __forceinline__ uint4 projection8_bf16(const ProjectionParams& pp, in
   return make_uint4(pack_bf16x2(a.x, a.y), pack_bf16x2(a.z, a.w), pack_bf16x2(b.x, b.y), pack_bf16x2(b.z, b.w));
 }
 
+// Position in a stage ring: the next stage and the parity of the round it is in.
+struct Ring {
+  int s;
+  uint32_t ph;
+};
+__device__ __forceinline__ void ring_next(Ring& r, int ns) {
+  if (++r.s == ns) { r.s = 0; r.ph ^= 1u; }
+}
+__device__ __forceinline__ void ring_skip(Ring& r, int ns, int count) {
+  const int x = r.s + count;
+  r.ph ^= (uint32_t)(x / ns) & 1u;
+  r.s = x % ns;
+}
+
 struct TileCoord {
   int prob, m0, n0, k_begin, k_end, split, nsub, ncol, nst;
 };
@@ -256,8 +317,15 @@ __device__ __forceinline__ TileCoord decode_tile(const Params& prm, int tile) {
   t.n0 = nb * p.bn * p.ncol;
   t.k_begin = t.split * p.ksteps_per_split;
   t.k_end = min(p.ksteps_total, t.k_begin + p.ksteps_per_split);
-  t.nsub = min(p.nsub, (p.M - t.m0 + BM - 1) / BM);          // row blocks with a valid row
-  t.ncol = min(p.ncol, (p.N - t.n0 + p.bn - 1) / p.bn);      // column blocks with a valid column
+  if (prm.cs > 1 && t.prob == 0) {
+    // items of a cluster walk the stage ring in step: all of them take the full shape, the rows and
+    // columns past the edge load as zeros and are never stored
+    t.nsub = p.nsub;
+    t.ncol = p.ncol;
+  } else {
+    t.nsub = min(p.nsub, (p.M - t.m0 + BM - 1) / BM);          // row blocks with a valid row
+    t.ncol = min(p.ncol, (p.N - t.n0 + p.bn - 1) / p.bn);      // column blocks with a valid column
+  }
   // Stages per k-step.  Row blocks come two to a stage and share the B tile of the first stage;
   // column blocks come one to a stage and share the A tile of the first stage.
   t.nst = p.ncol > 1 ? t.ncol : (t.nsub + 1) / 2;
@@ -280,9 +348,10 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
   const uint32_t staging = smem_base + RING_BYTES;
   const uint32_t bars = staging + NUM_EPI_WARPS * STAGING_BUFS * STAGING_BYTES;
   // barrier slots (8 bytes each)
-  auto full_bar = [&](int s) { return bars + 8u * s; };
-  auto empty_bar = [&](int s) { return bars + 8u * (NS + s); };
-  constexpr int kT = 2 * NS;
+  auto full_bar = [&](int g, int s) { return bars + 8u * ((g ? 2 * NS0 : 0) + s); };
+  auto empty_bar = [&](int g, int s) { return bars + 8u * ((g ? 2 * NS0 + NS1 : NS0) + s); };
+  auto stage_addr = [&](int g, int s) { return smem_base + (uint32_t)s * (g ? STAGE1_BYTES : STAGE0_BYTES); };
+  constexpr int kT = NUM_RING_BARS;
   auto tfull_bar = [&](int a) { return bars + 8u * (kT + a); };
   auto tempty_bar = [&](int a) { return bars + 8u * (kT + 2 + a); };
   auto qfull = [&](int s) { return bars + 8u * (kT + 4 + s); };
@@ -297,12 +366,17 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
   const int lane = threadIdx.x & 31;
   const bool has_gen = prm.gen_ring != GEN_NONE;
   constexpr int GEN_ARRIVALS = NUM_GEN_WARPS;
+  const int cs = prm.cs;
+  const uint32_t crank = cs > 1 ? cluster_ctarank() : 0u;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < NS; ++s) {
-      mbar_init(full_bar(s), 1 + (has_gen ? GEN_ARRIVALS : 0));   // the stage owner, and the generator warps
-      mbar_init(empty_bar(s), 1);
-    }
+    for (int g = 0; g < 2; ++g)
+      for (int s = 0; s < (g ? NS1 : NS0); ++s) {
+        mbar_init(full_bar(g, s), 1 + (has_gen ? GEN_ARRIVALS : 0));   // the stage owner, and the generator warps
+        // in an item with a generated operand a stage is free once the MMAs of all cs CTAs have read
+        // it; in every other item the owner supplies the cs - 1 arrivals that will not come
+        mbar_init(empty_bar(g, s), cs);
+      }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);
       mbar_init(tempty_bar(a), NUM_EPI_WARPS);
@@ -325,6 +399,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if (cs > 1) cluster_sync_all();          // every CTA's barriers exist before anything crosses CTAs
   const uint32_t tmem_base = *tmem_slot;
 
   // Every consumer role reads the next item from the queue the scheduler fills.
@@ -338,6 +413,12 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
     if (++qs == QDEPTH) { qs = 0; qph ^= 1; }
     return tile;
   };
+  // Before the first write into a new geometry: every stage of the old one has been handed back.
+  auto drain = [&](int g, const Ring& ro) -> bool {
+    for (int s = 0; s < (g ? NS1 : NS0); ++s)
+      if (!mbar_wait(empty_bar(g, s), s < ro.s ? ro.ph : ro.ph ^ 1u, abort_flag, prm.status)) return false;
+    return true;
+  };
   // what stage j of a k-step of item t holds
   auto stage_has_b = [&](const Problem& p, int j) { return p.ncol > 1 || j == 0; };
   auto stage_num_a = [&](const Problem& p, const TileCoord& t, int j) {
@@ -349,12 +430,31 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
   if (warp == 0) {
     // ------------------------- scheduler + stage owner --------------------------
     if (lane == 0) {
-      uint32_t is = 0;                     // running stage index
+      Ring r0 = {0, 0u}, r1 = {0, 0u};     // position in each geometry's ring
+      int cur_geo = -1;
       bool ok = true;
+      int group = (int)(blockIdx.x / cs);  // static part: cluster c takes groups c, c + clusters, ...
+      const int group_step = (int)(gridDim.x / cs);
       while (ok) {
         if (!(ok = mbar_wait(qempty(qs), qph ^ 1, abort_flag, prm.status))) break;
-        int tile = (int)atomicAdd(prm.sched, 1u);
-        if (tile >= prm.total_tiles) tile = -1;
+        int tile;
+        if (cs > 1 && group < prm.gen_groups) {
+          const Problem& p0 = prm.prob[0];
+          int mb, nb;
+          if (prm.share_n) {
+            const int per_row = p0.tiles_n / cs;
+            mb = group / per_row;
+            nb = (group % per_row) * cs + (int)crank;
+          } else {
+            nb = group % p0.tiles_n;
+            mb = (group / p0.tiles_n) * cs + (int)crank;
+          }
+          tile = mb * p0.tiles_n + nb;
+          group += group_step;
+        } else {
+          tile = prm.dyn_begin + (int)atomicAdd(prm.sched, 1u);
+          if (tile >= prm.total_tiles) tile = -1;
+        }
         tile_q[qs] = tile;
         mbar_arrive(qfull(qs));
         if (++qs == QDEPTH) { qs = 0; qph ^= 1; }
@@ -362,27 +462,37 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const TileCoord t = decode_tile(prm, tile);
         const Problem& p = prm.prob[t.prob];
         const CUtensorMap* mapB = &prm.tmB[t.prob];
-        const bool a_tma = p.a_mode != GENERATED, b_tma = p.b_mode != GENERATED;
+        const bool a_tma = p.a_mode < GENERATED, b_tma = p.b_mode < GENERATED;
+        const int geo = p.geo, ns = geo ? NS1 : NS0;
+        if (cur_geo >= 0 && geo != cur_geo && !(ok = drain(cur_geo, cur_geo ? r1 : r0))) break;
+        cur_geo = geo;
+        Ring r = geo ? r1 : r0;
         for (int ks = t.k_begin; ks < t.k_end && ok; ++ks) {
           const int k0 = ks * BK;
-          for (int j = 0; j < t.nst; ++j, ++is) {
-            const int s = (int)(is % NS);
-            if (!(ok = mbar_wait(empty_bar(s), ((is / NS) & 1u) ^ 1, abort_flag, prm.status))) break;
+          for (int j = 0; j < t.nst; ++j, ring_next(r, ns)) {
+            const int s = r.s;
+            if (!(ok = mbar_wait(empty_bar(geo, s), r.ph ^ 1u, abort_flag, prm.status))) break;
             const bool hb = stage_has_b(p, j);
             const int na = stage_num_a(p, t, j);
             uint32_t tx = 0;
             bool gen_here = false;
-            if (hb) { if (b_tma) tx += p.bn * BK * 2; else gen_here = true; }
-            if (na > 0) { if (a_tma) tx += na * A_BYTES; else gen_here = true; }
+            // of a generated tile, the shares of the other CTAs arrive as counted bytes
+            if (hb) { if (b_tma) tx += p.bn * BK * 2; else { gen_here = true; tx += (p.bn * BK * 2 / cs) * (cs - 1); } }
+            if (na > 0) { if (a_tma) tx += na * A_BYTES; else { gen_here = true; tx += (A_BYTES / cs) * (cs - 1); } }
+            // Items with a generated operand hand every stage back with a commit from each CTA of the
+            // cluster, so that no CTA writes its share of the next tile (or counts its bytes) into a
+            // stage that its neighbour has not finished with.  Other items hand stages back locally
+            // and the owner supplies the arrivals that will not come.
+            if (cs > 1 && a_tma && b_tma) mbar_arrive_n(empty_bar(geo, s), cs - 1);
 #if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
             if (prm.debug_flags & 2) tx = 0;
 #endif
-            const uint32_t fb = full_bar(s);
+            const uint32_t fb = full_bar(geo, s);
             if (tx) mbar_expect_tx(fb, tx);
             // arrive for this thread, and for the generator warps when they have nothing to write here
             mbar_arrive_n(fb, 1 + ((has_gen && !gen_here) ? GEN_ARRIVALS : 0));
             if (hb && b_tma && tx) {
-              const uint32_t dst = smem_base + s * STAGE_BYTES + STAGE_B_OFF;
+              const uint32_t dst = stage_addr(geo, s) + STAGE_B_OFF;
               const int n0 = t.n0 + (p.ncol > 1 ? j : 0) * p.bn;
               if (p.b_mode == TMA_KMAJOR) {
                 tma_load_2d(dst, mapB, fb, k0, n0);
@@ -392,13 +502,15 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             }
           }
         }
+        if (geo) r1 = r; else r0 = r;
       }
     }
   } else if (loader >= 0) {
     // ------------------------------ loaders --------------------------------------
     // 0: A tile in slot 0, 1: A tile in slot 1.  They only issue TMA; the bytes were declared by the stage owner.
     if (lane == 0) {
-      uint32_t is = 0;
+      Ring r0 = {0, 0u}, r1 = {0, 0u};
+      int cur_geo = -1;
       bool ok = true;
       while (ok) {
         const int tile = next_tile(false, true);
@@ -406,21 +518,27 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const TileCoord t = decode_tile(prm, tile);
         const Problem& p = prm.prob[t.prob];
         const CUtensorMap* mapA = &prm.tmA[t.prob];
-        bool mine = p.a_mode != GENERATED;
+        const int geo = p.geo, ns = geo ? NS1 : NS0;
+        if (cur_geo >= 0 && geo != cur_geo && !(ok = drain(cur_geo, cur_geo ? r1 : r0))) break;
+        cur_geo = geo;
+        Ring r = geo ? r1 : r0;
+        bool mine = p.a_mode < GENERATED;
 #if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
         if (prm.debug_flags & 2) mine = false;
 #endif
         const int klen = t.k_end - t.k_begin;
-        if (!mine) { is += klen * t.nst; continue; }
-        for (int ks = t.k_begin; ks < t.k_end && ok; ++ks) {
+        if (!mine) ring_skip(r, ns, klen * t.nst);
+        for (int ks = t.k_begin; ks < t.k_end && ok && mine; ++ks) {
           const int k0 = ks * BK;
-          for (int j = 0; j < t.nst; ++j, ++is) {
-            const int s = (int)(is % NS);
-            const uint32_t fb = full_bar(s);
-            const uint32_t stage = smem_base + s * STAGE_BYTES;
+          for (int j = 0; j < t.nst; ++j) {
+            const int s = r.s;
+            const uint32_t eph = r.ph ^ 1u;
+            ring_next(r, ns);
+            const uint32_t fb = full_bar(geo, s);
+            const uint32_t stage = stage_addr(geo, s);
             {
               if (loader >= stage_num_a(p, t, j)) continue;
-              if (!(ok = mbar_wait(empty_bar(s), ((is / NS) & 1u) ^ 1, abort_flag, prm.status))) break;
+              if (!(ok = mbar_wait(empty_bar(geo, s), eph, abort_flag, prm.status))) break;
               const int mi = p.ncol > 1 ? 0 : 2 * j + loader;
               const int m0 = t.m0 + mi * BM;
               const uint32_t dst = stage + (loader == 0 ? STAGE_A0_OFF : STAGE_A1_OFF);
@@ -433,12 +551,13 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             }
           }
         }
+        if (geo) r1 = r; else r0 = r;
       }
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ---------------------------------
     if (lane == 0) {
-      uint32_t is = 0;
+      Ring r0 = {0, 0u}, r1 = {0, 0u};
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
@@ -447,7 +566,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         if (tile < 0) break;
         const TileCoord t = decode_tile(prm, tile);
         const Problem& p = prm.prob[t.prob];
-        const bool a_mn = p.a_mode == TMA_MNMAJOR;
+        const bool a_mn = p.a_mode == TMA_MNMAJOR || p.a_mode == GENERATED_T;
         const bool b_mn = p.b_mode != TMA_KMAJOR;          // generated B tiles are written MN-major
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
                                ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
@@ -460,16 +579,27 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
           acc_phase ^= 1;
         }
         const int acc0 = acc;
+#ifdef COMPACT_PROFILE_GEN
+        const long long m0c = clock64();
+        long long mwait = 0, missue = 0;
+#endif
         for (int sl = 0; sl < slots && ok; ++sl) {
           ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag, prm.status);
           if (++acc == 2) { acc = 0; acc_phase ^= 1; }
         }
         if (!ok) break;
         tc_fence_after();
+#ifdef COMPACT_PROFILE_GEN
+        const long long m1c = clock64();
+#endif
         const uint32_t d_base = tmem_base + acc0 * BN_MAX;
         // one UMMA consumes K = 16: 32 bytes along a K-major row, or two 8-row groups (2048 bytes) MN-major
         const uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4), b_step = b_mn ? (2048u >> 4) : (32u >> 4);
         const int bn = p.bn, nst = t.nst;
+        const int geo = p.geo, ns = geo ? NS1 : NS0;
+        Ring r = geo ? r1 : r0;
+        // items with a generated operand walk the ring in step with the other CTAs of the cluster
+        const bool gen_shared = cs > 1 && (p.a_mode >= GENERATED || p.b_mode >= GENERATED);
         // accumulator ai of the item sits in slot ai / sps at column (ai % sps) * bn (a slot is 256 columns)
         const int naccs = p.nsub * p.ncol;
         const int sps = BN_MAX / bn > naccs ? naccs : BN_MAX / bn;
@@ -485,13 +615,22 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         };
         for (int ks = t.k_begin; ks < t.k_end && ok; ++ks) {
           const uint32_t first = ks > t.k_begin ? 1u : 0u;
-          const uint32_t is0 = is;
-          const uint32_t stage0 = smem_base + (is0 % NS) * STAGE_BYTES;       // holds the shared operand
-          for (int j = 0; j < nst; ++j, ++is) {
-            const int s = (int)(is % NS);
-            if (!(ok = mbar_wait(full_bar(s), (is / NS) & 1u, abort_flag, prm.status))) break;
+          const int s0 = r.s;
+          const uint32_t stage0 = stage_addr(geo, s0);       // holds the shared operand
+          for (int j = 0; j < nst; ++j, ring_next(r, ns)) {
+            const int s = r.s;
+#ifdef COMPACT_PROFILE_GEN
+            const long long w0c = clock64();
+#endif
+            if (!(ok = mbar_wait(full_bar(geo, s), r.ph, abort_flag, prm.status))) break;
+#ifdef COMPACT_PROFILE_GEN
+            mwait += clock64() - w0c;
+#endif
             tc_fence_after();
-            const uint32_t stage = smem_base + s * STAGE_BYTES;
+#ifdef COMPACT_PROFILE_GEN
+            const long long i0c = clock64();
+#endif
+            const uint32_t stage = stage_addr(geo, s);
             if (p.ncol > 1) {
               issue4(d_base + acc_col(j), desc_lo(stage0 + STAGE_A0_OFF, a_mn), desc_lo(stage + STAGE_B_OFF, b_mn), first);
             } else {
@@ -499,13 +638,34 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
               issue4(d_base + acc_col(2 * j), desc_lo(stage + STAGE_A0_OFF, a_mn), b_lo, first);
               if (2 * j + 1 < t.nsub) issue4(d_base + acc_col(2 * j + 1), desc_lo(stage + STAGE_A1_OFF, a_mn), b_lo, first);
             }
+#ifdef COMPACT_PROFILE_GEN
+            missue += clock64() - i0c;
+#endif
             // a stage that holds nothing shared goes back at once; the first stage of the k-step goes last
-            if (j > 0) umma_commit(empty_bar(s));
+            if (j > 0) {
+              if (gen_shared) umma_commit_mc(empty_bar(geo, s), (uint16_t)((1u << cs) - 1u));
+              else umma_commit(empty_bar(geo, s));
+            }
           }
           if (!ok) break;
-          umma_commit(empty_bar((int)(is0 % NS)));
+          if (gen_shared) umma_commit_mc(empty_bar(geo, s0), (uint16_t)((1u << cs) - 1u));
+          else umma_commit(empty_bar(geo, s0));
         }
         if (!ok) break;
+        if (geo) r1 = r; else r0 = r;
+#ifdef COMPACT_PROFILE_GEN
+        if (p.a_mode >= GENERATED || p.b_mode >= GENERATED) {
+          atomicAdd(&g_prof[4], (unsigned long long)mwait);                 // waiting for full stages
+          atomicAdd(&g_prof[5], (unsigned long long)missue);               // issuing MMAs
+          atomicAdd(&g_prof[6], (unsigned long long)(clock64() - m1c));    // whole k loop
+          atomicAdd(&g_prof[7], (unsigned long long)(t.k_end - t.k_begin));
+        } else if (!has_gen) {
+          atomicAdd(&g_prof[0], (unsigned long long)mwait);
+          atomicAdd(&g_prof[1], (unsigned long long)missue);
+          atomicAdd(&g_prof[2], (unsigned long long)(clock64() - m1c));
+          atomicAdd(&g_prof[3], (unsigned long long)(t.k_end - t.k_begin));
+        }
+#endif
         for (int sl = 0; sl < slots; ++sl) umma_commit(tfull_bar((acc0 + sl) & 1));
       }
     }
@@ -601,7 +761,14 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
                 tmem_ld32(tcol + ci * cw + 32 * h, v);
                 tmem_ld_wait();
               }
-              if (p.epi_mode == EPI_UPDATE_W) {
+              if (p.epi_mode == EPI_BF16_T) {
+                // lane = output column (row0 + lane), v[z] = output row col + 32 h + z: the staged tile is
+                // [64 output rows][32 output columns] of bf16, unswizzled
+#pragma unroll
+                for (int z = 0; z < 32; ++z)
+                  *reinterpret_cast<__nv_bfloat16*>(stg_gen + (32 * h + z) * 64 + lane * 2) =
+                      __float2bfloat16_rn(__uint_as_float(v[z]));
+              } else if (p.epi_mode == EPI_UPDATE_W) {
                 if (h == 0) {
                   if (!(ok = mbar_wait(my_wbar, wph, abort_flag, prm.status))) break;
                   wph ^= 1;
@@ -636,7 +803,8 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
-              tma_store_2d(mapC, stg, col, row0);
+              if (p.epi_mode == EPI_BF16_T) tma_store_2d(mapC, stg, row0, col);
+              else tma_store_2d(mapC, stg, col, row0);
               tma_store_commit();
             }
           }
@@ -653,45 +821,67 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
     // ------------------------------ P generators --------------------------------
     // Write bf16 tiles of P straight into the swizzled operand layout the MMA reads: as the B tile
     // of the first stage of a k-step (forward) or as its A tile 0 (update).
+#ifdef CFG_GEN_SKIP1
+    // experiment: the four generator warps that share a scheduler with the MMA warp do no work
+    const int gw_ = warp - (THREADS_BASE >> 5), sc_ = gw_ & 3;
+    const int gtid = sc_ == 1 ? (1 << 20) : (((gw_ >> 2) * 3 + (sc_ == 0 ? 0 : sc_ - 1)) * 32 + lane);
+    constexpr int GSTRIDE = 32 * NUM_GEN_WARPS * 3 / 4;
+#else
     const int gtid = threadIdx.x - THREADS_BASE;
-    uint32_t is = 0;
+    constexpr int GSTRIDE = 32 * NUM_GEN_WARPS;
+#endif
+    Ring r0 = {0, 0u}, r1 = {0, 0u};
     bool ok = true;
+    const int csh = cs - 1;                                 // log2(cs), cs is 1 or 2
+    // the other CTA's window onto the same addresses
+    const uint32_t peer_base = cs > 1 ? map_to_cta(smem_base, crank ^ 1u) : 0u;
+    const uint32_t peer_full = cs > 1 ? map_to_cta(bars, crank ^ 1u) : 0u;
     while (ok) {
       const int tile = next_tile(true, lane == 0);
       if (tile < 0) break;
       const TileCoord t = decode_tile(prm, tile);
       const Problem& p = prm.prob[t.prob];
       const int klen = t.k_end - t.k_begin;
-      const bool gen_b = p.b_mode == GENERATED, gen_a = p.a_mode == GENERATED;
-      if (!gen_a && !gen_b) { is += klen * t.nst; continue; }      // the stage owner arrives for this item
-      for (int ks = t.k_begin; ks < t.k_end && ok; ++ks, is += t.nst) {
-        const int s = (int)(is % NS);
+      const bool gen_a = p.a_mode == GENERATED, gen_at = p.a_mode == GENERATED_T;
+      const int geo = p.geo, ns = geo ? NS1 : NS0;
+      Ring r = geo ? r1 : r0;
+      // The generated problem is the first of its launch, so the generators never write into a ring
+      // whose geometry has changed.  In other items the stage owner arrives for them.
+      if (!gen_a && !gen_at) ring_skip(r, ns, klen * t.nst);
+      for (int ks = t.k_begin; ks < t.k_end && ok && (gen_a || gen_at); ++ks) {
+        const int s = r.s;
+        const uint32_t eph = r.ph ^ 1u;
+        ring_skip(r, ns, t.nst);
+        const uint32_t stage_off = (uint32_t)s * (geo ? STAGE1_BYTES : STAGE0_BYTES);
+        const uint32_t full_off = full_bar(geo, s) - bars;
 #ifdef COMPACT_PROFILE_GEN
         const long long g0 = clock64();
 #endif
-        const bool w = mbar_wait(empty_bar(s), ((is / NS) & 1u) ^ 1, abort_flag, prm.status);
+        const bool w = mbar_wait(empty_bar(geo, s), eph, abort_flag, prm.status);
 #ifdef COMPACT_PROFILE_GEN
         const long long g1 = clock64();
 #endif
         const int k0 = ks * BK;
-        if (w && gen_b) {
-          // B[k = row i of P][n = column j of P], MN-major: 64-column blocks of [64 k][128 B]
-          uint8_t* sbp = smem_gen + s * STAGE_BYTES + STAGE_B_OFF;
-          // bn is 64, 128 or 256 here: 8, 16 or 32 eight-column chunks per row of P
-          const int chunks = p.bn >> 3, cshift = 31 - __clz(chunks);
-          for (int id = gtid; id < BK * chunks; id += 32 * NUM_GEN_WARPS) {
-            const int c = id & (chunks - 1), kr = id >> cshift;
-            const uint4 val = projection8_bf16(prm.pp, k0 + kr, t.n0 + c * 8);
-            *reinterpret_cast<uint4*>(sbp + (c >> 3) * 8192 + kr * 128 + (((c & 7) ^ (kr & 7)) << 4)) = val;
+        if (w && gen_at) {
+          // A[m = column j of P][k = row i of P], MN-major: two 64-column blocks of [64 k][128 B]
+          const int kr0 = (int)crank * (BK >> csh);           // this CTA's rows of the tile
+          for (int id = gtid; id < (BK >> csh) * 16; id += GSTRIDE) {
+            const int c = id & 15, kr = kr0 + (id >> 4);
+            const uint4 val = projection8_bf16(prm.pp, k0 + kr, t.m0 + c * 8);
+            const uint32_t off = stage_off + STAGE_A0_OFF + (c >> 3) * 8192 + kr * 128 + (((c & 7) ^ (kr & 7)) << 4);
+            *reinterpret_cast<uint4*>(smem_gen + off) = val;
+            if (cs > 1) st_async_16(peer_base + off, val, peer_full + full_off);
           }
         }
         if (w && gen_a) {
           // A[m = row i of P][k = column j of P], K-major: [128 rows][128 B]
-          uint8_t* sap = smem_gen + s * STAGE_BYTES + STAGE_A0_OFF;
-          for (int id = gtid; id < BM * 8; id += 32 * NUM_GEN_WARPS) {
-            const int c = id & 7, rr = id >> 3;
+          const int rr0 = (int)crank * (BM >> csh);           // this CTA's rows of the tile
+          for (int id = gtid; id < (BM >> csh) * 8; id += GSTRIDE) {
+            const int c = id & 7, rr = rr0 + (id >> 3);
             const uint4 val = projection8_bf16(prm.pp, t.m0 + rr, k0 + c * 8);
-            *reinterpret_cast<uint4*>(sap + rr * 128 + ((c ^ (rr & 7)) << 4)) = val;
+            const uint32_t off = stage_off + STAGE_A0_OFF + rr * 128 + ((c ^ (rr & 7)) << 4);
+            *reinterpret_cast<uint4*>(smem_gen + off) = val;
+            if (cs > 1) st_async_16(peer_base + off, val, peer_full + full_off);
           }
         }
 #ifdef COMPACT_PROFILE_GEN
@@ -699,12 +889,13 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
 #endif
         fence_proxy_async_smem();
         ok = __all_sync(0xffffffffu, w);
-        if (ok && lane == 0) mbar_arrive(full_bar(s));
+        if (ok && lane == 0) mbar_arrive(full_bar(geo, s));
 #ifdef COMPACT_PROFILE_GEN
-        if (gtid == 0) { atomicAdd(&g_prof[0], (unsigned long long)(g1 - g0)); atomicAdd(&g_prof[1], (unsigned long long)(g2 - g1)); atomicAdd(&g_prof[2], (unsigned long long)(clock64() - g2)); atomicAdd(&g_prof[3], 1ull); }
+        if (warp == (THREADS_BASE >> 5) && lane == 0) { atomicAdd(&g_prof[0], (unsigned long long)(g1 - g0)); atomicAdd(&g_prof[1], (unsigned long long)(g2 - g1)); atomicAdd(&g_prof[2], (unsigned long long)(clock64() - g2)); atomicAdd(&g_prof[3], 1ull); }
 #endif
         // later stages of the k-step hold no generated data: the stage owner arrives for the generators there
       }
+      if (geo) r1 = r; else r0 = r;
     }
   }
 
@@ -714,6 +905,8 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
   }
+  // no CTA leaves while another of its cluster may still signal its barriers
+  if (cs > 1) cluster_sync_all();
   // the last CTA to finish re-arms the scheduler words for the next launch
   if (threadIdx.x == 0) {
     __threadfence();
@@ -798,7 +991,7 @@ inline EncodeTiledFn encode_fn() {
 
 // 2-D bf16 map over a row-major matrix: `inner` contiguous elements per row, `rows` rows, pitch in elements.
 inline bool make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t rows, int64_t pitch, int box_inner,
-                     int box_rows) {
+                     int box_rows, bool swizzle = true) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)rows};
@@ -806,7 +999,8 @@ inline bool make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t 
   cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -838,6 +1032,7 @@ inline void finish_problem(Problem& p, int splits_wanted) {
   // put eight MMAs behind every barrier wait
   if (p.nsub == 0) p.nsub = p.M > BM ? CFG_NSUB : 1;
   if (p.ncol == 0) p.ncol = 1;
+  p.geo = p.nsub == 1 ? 1 : 0;
   p.tiles_m = (p.M + BM * p.nsub - 1) / (BM * p.nsub);
   p.tiles_n = (p.N + p.bn * p.ncol - 1) / (p.bn * p.ncol);
   p.ksteps_total = (p.K + BK - 1) / BK;
@@ -880,6 +1075,17 @@ inline compact_status_t launch(const LaunchInfo& li, Params& prm) {
     }
     attr_set = true;
   }
+  const int cs = (prm.gen_ring != GEN_NONE && li.cluster > 1) ? li.cluster : 1;
+  prm.cs = cs;
+  if (cs > 1) {
+    // the generated problem is problem 0; its items come in groups of cs neighbours
+    Problem& p0 = prm.prob[0];
+    prm.share_n = prm.gen_ring == GEN_A ? 1 : 0;
+    if (prm.share_n) p0.tiles_n = (p0.tiles_n + cs - 1) / cs * cs;
+    else p0.tiles_m = (p0.tiles_m + cs - 1) / cs * cs;
+    prm.gen_groups = p0.tiles_m * p0.tiles_n / cs;
+    prm.dyn_begin = p0.tiles_m * p0.tiles_n;
+  }
   int t = 0;
   for (int i = 0; i < prm.num_problems; ++i) {
     prm.prob[i].tile_begin = t;
@@ -891,10 +1097,24 @@ inline compact_status_t launch(const LaunchInfo& li, Params& prm) {
 #if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
   prm.debug_flags = (getenv("COMPACT_SKIP_MMA") ? 1 : 0) | (getenv("COMPACT_SKIP_LOADS") ? 2 : 0) | (getenv("COMPACT_SKIP_EPI") ? 4 : 0) | (getenv("COMPACT_SKIP_STORE") ? 8 : 0) | (getenv("COMPACT_SKIP_TMEMLD") ? 16 : 0);
 #endif
-  const int grid = t < NUM_SMS ? t : NUM_SMS;
+  const int grid = t < NUM_SMS ? (t + cs - 1) / cs * cs : NUM_SMS / cs * cs;
   const int threads = prm.gen_ring != GEN_NONE ? THREADS_GEN : THREADS_BASE;
-  compact_gemm_kernel<<<grid, threads, SMEM_BYTES, li.stream>>>(prm);
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3((unsigned)grid, 1, 1);
+  cfg.blockDim = dim3((unsigned)threads, 1, 1);
+  cfg.dynamicSmemBytes = SMEM_BYTES;
+  cfg.stream = li.stream;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = (unsigned)cs;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, compact_gemm_kernel, prm);
   (*li.launches)++;
+  if (e != cudaSuccess) { cudaGetLastError(); return COMPACT_ERR_CUDA; }
   return cudaGetLastError() == cudaSuccess ? COMPACT_OK : COMPACT_ERR_CUDA;
 }
 
@@ -911,23 +1131,25 @@ inline compact_status_t forward(const LaunchInfo& li, const ProjectionParams& pp
   memset(&prm, 0, sizeof(prm));
   prm.pp = pp;
   prm.num_problems = 2;
-  prm.gen_ring = GEN_B;
+  prm.gen_ring = GEN_A;
+  // Z is computed transposed, Z^T = P^T X^T: the generated tile of P (64 rows of P by 128 of its columns)
+  // is the A operand, and up to 512 tokens of X ride on the N side in two 256-wide accumulators, so the
+  // MMAs run at N = 256 and one generated tile feeds 512 tokens.
   Problem& pz = prm.prob[0];
-  pz.M = (int)tokens; pz.N = zcols; pz.K = n;
-  // one generated 64 x 128 tile of P feeds up to four row blocks of X (512 tokens)
-  pz.bn = zcols >= 512 / MAX_SUB ? 512 / MAX_SUB : (int)((zcols + 63) / 64 * 64);
-  pz.nsub = (int)((tokens + BM - 1) / BM) < MAX_SUB ? (int)((tokens + BM - 1) / BM) : MAX_SUB;
-  pz.a_mode = TMA_KMAJOR; pz.b_mode = GENERATED; pz.epi_mode = EPI_BF16;
+  pz.M = zcols; pz.N = (int)tokens; pz.K = n;
+  pz.nsub = 1;
+  pz.ncol = tokens > BN_MAX ? 2 : 1;
+  pz.a_mode = GENERATED_T; pz.b_mode = TMA_KMAJOR; pz.epi_mode = EPI_BF16_T;
   finish_problem(pz, 1);
   Problem& py = prm.prob[1];
   py.M = (int)tokens; py.N = m; py.K = n;
   py.a_mode = TMA_KMAJOR; py.b_mode = TMA_MNMAJOR; py.epi_mode = EPI_BF16;
   finish_problem(py, 1);
-  if (!make_map(&prm.tmA[0], X, n, tokens, ldx, BK, BM)) return COMPACT_ERR_CUDA;
-  prm.tmA[1] = prm.tmA[0];
+  if (!make_map(&prm.tmA[1], X, n, tokens, ldx, BK, BM)) return COMPACT_ERR_CUDA;
+  prm.tmA[0] = prm.tmA[1];   // unused by the generated operand
+  if (!make_map(&prm.tmB[0], X, n, tokens, ldx, BK, pz.bn)) return COMPACT_ERR_CUDA;
   if (!make_map(&prm.tmB[1], W, m, n, ldw, 64, BK)) return COMPACT_ERR_CUDA;
-  prm.tmB[0] = prm.tmB[1];   // unused by the generated operand
-  if (!make_map(&prm.tmC[0], Z, zcols, tokens, ldz, 64, 32)) return COMPACT_ERR_CUDA;
+  if (!make_map(&prm.tmC[0], Z, zcols, tokens, ldz, 32, 64, false)) return COMPACT_ERR_CUDA;
   if (!make_map(&prm.tmC[1], Y, m, tokens, ldy, 64, 32)) return COMPACT_ERR_CUDA;
   return launch(li, prm);
 }
