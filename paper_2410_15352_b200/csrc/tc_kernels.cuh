@@ -99,6 +99,7 @@ struct Problem {
   int ncol;
   int a_mode, b_mode, epi_mode;
   int geo;                // ring geometry its items use (0 or 1)
+  int a_blocked, b_blocked;   // MN-major operand read through a map that brings a whole tile in one copy
   int tile_begin;
   float scale;
 };
@@ -179,6 +180,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "l"(map), "r"(bar), "r"(x), "r"(y)
       : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
+      "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z)
+      : "memory");
+}
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src), "r"(x),
                "r"(y)
@@ -246,6 +253,17 @@ __device__ __forceinline__ void st_async_16(uint32_t raddr, uint4 v, uint32_t rb
   asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(raddr),
                "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"(rbar)
                : "memory");
+}
+
+// True in exactly one lane of a converged warp.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
 }
 
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
@@ -429,14 +447,16 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
   const int loader = (warp >= 2 + NUM_EPI_WARPS && warp < 2 + NUM_EPI_WARPS + NUM_LOADERS) ? warp - 2 - NUM_EPI_WARPS : -1;
   if (warp == 0) {
     // ------------------------- scheduler + stage owner --------------------------
-    if (lane == 0) {
+    // Like the MMA warp, these warps walk their loops whole (warp-uniform addresses and counters) and
+    // one elected lane touches the barriers and issues the copies.
+    {
       Ring r0 = {0, 0u}, r1 = {0, 0u};     // position in each geometry's ring
       int cur_geo = -1;
       bool ok = true;
       int group = (int)(blockIdx.x / cs);  // static part: cluster c takes groups c, c + clusters, ...
       const int group_step = (int)(gridDim.x / cs);
       while (ok) {
-        if (!(ok = mbar_wait(qempty(qs), qph ^ 1, abort_flag, prm.status))) break;
+        if (!(ok = __all_sync(0xffffffffu, mbar_wait(qempty(qs), qph ^ 1, abort_flag, prm.status)))) break;
         int tile;
         if (cs > 1 && group < prm.gen_groups) {
           const Problem& p0 = prm.prob[0];
@@ -452,11 +472,16 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
           tile = mb * p0.tiles_n + nb;
           group += group_step;
         } else {
-          tile = prm.dyn_begin + (int)atomicAdd(prm.sched, 1u);
+          tile = 0;
+          if (lane == 0) tile = prm.dyn_begin + (int)atomicAdd(prm.sched, 1u);
+          tile = __shfl_sync(0xffffffffu, tile, 0);
           if (tile >= prm.total_tiles) tile = -1;
         }
-        tile_q[qs] = tile;
-        mbar_arrive(qfull(qs));
+        if (lane == 0) {
+          tile_q[qs] = tile;
+          mbar_arrive(qfull(qs));
+        }
+        __syncwarp();
         if (++qs == QDEPTH) { qs = 0; qph ^= 1; }
         if (tile < 0) break;
         const TileCoord t = decode_tile(prm, tile);
@@ -464,14 +489,14 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const CUtensorMap* mapB = &prm.tmB[t.prob];
         const bool a_tma = p.a_mode < GENERATED, b_tma = p.b_mode < GENERATED;
         const int geo = p.geo, ns = geo ? NS1 : NS0;
-        if (cur_geo >= 0 && geo != cur_geo && !(ok = drain(cur_geo, cur_geo ? r1 : r0))) break;
+        if (cur_geo >= 0 && geo != cur_geo && !(ok = __all_sync(0xffffffffu, drain(cur_geo, cur_geo ? r1 : r0)))) break;
         cur_geo = geo;
         Ring r = geo ? r1 : r0;
         for (int ks = t.k_begin; ks < t.k_end && ok; ++ks) {
           const int k0 = ks * BK;
           for (int j = 0; j < t.nst; ++j, ring_next(r, ns)) {
             const int s = r.s;
-            if (!(ok = mbar_wait(empty_bar(geo, s), r.ph ^ 1u, abort_flag, prm.status))) break;
+            if (!(ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(geo, s), r.ph ^ 1u, abort_flag, prm.status)))) break;
             const bool hb = stage_has_b(p, j);
             const int na = stage_num_a(p, t, j);
             uint32_t tx = 0;
@@ -479,27 +504,32 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             // of a generated tile, the shares of the other CTAs arrive as counted bytes
             if (hb) { if (b_tma) tx += p.bn * BK * 2; else { gen_here = true; tx += (p.bn * BK * 2 / cs) * (cs - 1); } }
             if (na > 0) { if (a_tma) tx += na * A_BYTES; else { gen_here = true; tx += (A_BYTES / cs) * (cs - 1); } }
-            // Items with a generated operand hand every stage back with a commit from each CTA of the
-            // cluster, so that no CTA writes its share of the next tile (or counts its bytes) into a
-            // stage that its neighbour has not finished with.  Other items hand stages back locally
-            // and the owner supplies the arrivals that will not come.
-            if (cs > 1 && a_tma && b_tma) mbar_arrive_n(empty_bar(geo, s), cs - 1);
 #if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
             if (prm.debug_flags & 2) tx = 0;
 #endif
-            const uint32_t fb = full_bar(geo, s);
-            if (tx) mbar_expect_tx(fb, tx);
-            // arrive for this thread, and for the generator warps when they have nothing to write here
-            mbar_arrive_n(fb, 1 + ((has_gen && !gen_here) ? GEN_ARRIVALS : 0));
-            if (hb && b_tma && tx) {
-              const uint32_t dst = stage_addr(geo, s) + STAGE_B_OFF;
-              const int n0 = t.n0 + (p.ncol > 1 ? j : 0) * p.bn;
-              if (p.b_mode == TMA_KMAJOR) {
-                tma_load_2d(dst, mapB, fb, k0, n0);
-              } else {
-                for (int b = 0; b < p.bn / 64; ++b) tma_load_2d(dst + b * 8192, mapB, fb, n0 + 64 * b, k0);
+            if (elect_one()) {
+              // Items with a generated operand hand every stage back with a commit from each CTA of the
+              // cluster, so that no CTA writes its share of the next tile (or counts its bytes) into a
+              // stage that its neighbour has not finished with.  Other items hand stages back locally
+              // and the owner supplies the arrivals that will not come.
+              if (cs > 1 && a_tma && b_tma) mbar_arrive_n(empty_bar(geo, s), cs - 1);
+              const uint32_t fb = full_bar(geo, s);
+              if (tx) mbar_expect_tx(fb, tx);
+              // arrive for this thread, and for the generator warps when they have nothing to write here
+              mbar_arrive_n(fb, 1 + ((has_gen && !gen_here) ? GEN_ARRIVALS : 0));
+              if (hb && b_tma && tx) {
+                const uint32_t dst = stage_addr(geo, s) + STAGE_B_OFF;
+                const int n0 = t.n0 + (p.ncol > 1 ? j : 0) * p.bn;
+                if (p.b_mode == TMA_KMAJOR) {
+                  tma_load_2d(dst, mapB, fb, k0, n0);
+                } else if (p.b_blocked) {
+                  tma_load_3d(dst, mapB, fb, 0, k0, n0 >> 6);
+                } else {
+                  for (int b = 0; b < p.bn / 64; ++b) tma_load_2d(dst + b * 8192, mapB, fb, n0 + 64 * b, k0);
+                }
               }
             }
+            __syncwarp();
           }
         }
         if (geo) r1 = r; else r0 = r;
@@ -508,18 +538,18 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
   } else if (loader >= 0) {
     // ------------------------------ loaders --------------------------------------
     // 0: A tile in slot 0, 1: A tile in slot 1.  They only issue TMA; the bytes were declared by the stage owner.
-    if (lane == 0) {
+    {
       Ring r0 = {0, 0u}, r1 = {0, 0u};
       int cur_geo = -1;
       bool ok = true;
       while (ok) {
-        const int tile = next_tile(false, true);
+        const int tile = __shfl_sync(0xffffffffu, next_tile(true, lane == 0), 0);
         if (tile < 0) break;
         const TileCoord t = decode_tile(prm, tile);
         const Problem& p = prm.prob[t.prob];
         const CUtensorMap* mapA = &prm.tmA[t.prob];
         const int geo = p.geo, ns = geo ? NS1 : NS0;
-        if (cur_geo >= 0 && geo != cur_geo && !(ok = drain(cur_geo, cur_geo ? r1 : r0))) break;
+        if (cur_geo >= 0 && geo != cur_geo && !(ok = __all_sync(0xffffffffu, drain(cur_geo, cur_geo ? r1 : r0)))) break;
         cur_geo = geo;
         Ring r = geo ? r1 : r0;
         bool mine = p.a_mode < GENERATED;
@@ -534,21 +564,23 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             const int s = r.s;
             const uint32_t eph = r.ph ^ 1u;
             ring_next(r, ns);
-            const uint32_t fb = full_bar(geo, s);
-            const uint32_t stage = stage_addr(geo, s);
-            {
-              if (loader >= stage_num_a(p, t, j)) continue;
-              if (!(ok = mbar_wait(empty_bar(geo, s), eph, abort_flag, prm.status))) break;
+            if (loader >= stage_num_a(p, t, j)) continue;
+            if (!(ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(geo, s), eph, abort_flag, prm.status)))) break;
+            if (elect_one()) {
+              const uint32_t fb = full_bar(geo, s);
               const int mi = p.ncol > 1 ? 0 : 2 * j + loader;
               const int m0 = t.m0 + mi * BM;
-              const uint32_t dst = stage + (loader == 0 ? STAGE_A0_OFF : STAGE_A1_OFF);
+              const uint32_t dst = stage_addr(geo, s) + (loader == 0 ? STAGE_A0_OFF : STAGE_A1_OFF);
               if (p.a_mode == TMA_KMAJOR) {
                 tma_load_2d(dst, mapA, fb, k0, m0);
+              } else if (p.a_blocked) {
+                tma_load_3d(dst, mapA, fb, 0, k0, m0 >> 6);
               } else {
                 tma_load_2d(dst, mapA, fb, m0, k0);
                 tma_load_2d(dst + 8192, mapA, fb, m0 + 64, k0);
               }
             }
+            __syncwarp();
           }
         }
         if (geo) r1 = r; else r0 = r;
@@ -556,13 +588,16 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ---------------------------------
-    if (lane == 0) {
+    // The whole warp walks the loops, so that addresses, descriptors and counters are warp-uniform
+    // values; one elected lane issues the MMAs and the commits.
+    {
       Ring r0 = {0, 0u}, r1 = {0, 0u};
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
+      const uint16_t cta_mask = (uint16_t)((1u << cs) - 1u);
       while (ok) {
-        const int tile = next_tile(false, true);
+        const int tile = __shfl_sync(0xffffffffu, next_tile(true, lane == 0), 0);
         if (tile < 0) break;
         const TileCoord t = decode_tile(prm, tile);
         const Problem& p = prm.prob[t.prob];
@@ -573,18 +608,18 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const int slots = (p.nsub * p.ncol * p.bn + BN_MAX - 1) / BN_MAX;   // accumulator slots this item occupies
         if (slots == 2 && acc == 1) {
           // a two-slot item starts at slot 0: pass slot 1 through unused
-          if (!(ok = mbar_wait(tempty_bar(1), acc_phase ^ 1, abort_flag, prm.status))) break;
-          umma_commit(tfull_bar(1));
+          if (!(ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(1), acc_phase ^ 1, abort_flag, prm.status)))) break;
+          if (elect_one()) umma_commit(tfull_bar(1));
+          __syncwarp();
           acc = 0;
           acc_phase ^= 1;
         }
         const int acc0 = acc;
 #ifdef COMPACT_PROFILE_GEN
-        const long long m0c = clock64();
         long long mwait = 0, missue = 0;
 #endif
         for (int sl = 0; sl < slots && ok; ++sl) {
-          ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag, prm.status);
+          ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag, prm.status));
           if (++acc == 2) { acc = 0; acc_phase ^= 1; }
         }
         if (!ok) break;
@@ -595,7 +630,8 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const uint32_t d_base = tmem_base + acc0 * BN_MAX;
         // one UMMA consumes K = 16: 32 bytes along a K-major row, or two 8-row groups (2048 bytes) MN-major
         const uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4), b_step = b_mn ? (2048u >> 4) : (32u >> 4);
-        const int bn = p.bn, nst = t.nst;
+        const int bn = p.bn, nst = t.nst, nsub = t.nsub;
+        const bool by_col = p.ncol > 1;
         const int geo = p.geo, ns = geo ? NS1 : NS0;
         Ring r = geo ? r1 : r0;
         // items with a generated operand walk the ring in step with the other CTAs of the cluster
@@ -604,6 +640,12 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const int naccs = p.nsub * p.ncol;
         const int sps = BN_MAX / bn > naccs ? naccs : BN_MAX / bn;
         auto acc_col = [&](int ai) -> uint32_t { return (uint32_t)((ai / sps) * BN_MAX + (ai % sps) * bn); };
+        // TMEM addresses of the (at most four) accumulators, and the descriptor offsets inside a stage
+        const uint32_t d0 = d_base + acc_col(0), d1 = d_base + acc_col(1), d2 = d_base + acc_col(2), d3 = d_base + acc_col(3);
+        const uint32_t lbo = (8192u >> 4) << 16, one = 1u << 16;
+        const uint32_t a_flags = a_mn ? lbo : one, b_flags = b_mn ? lbo : one;
+        const uint32_t stage_step = (uint32_t)(geo ? STAGE1_BYTES : STAGE0_BYTES) >> 4;
+        const uint32_t ring_lo = (smem_base >> 4) & 0x3FFFu;
         auto issue4 = [&](uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t first) {
 #if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
           if (prm.debug_flags & 1) return;
@@ -616,13 +658,13 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         for (int ks = t.k_begin; ks < t.k_end && ok; ++ks) {
           const uint32_t first = ks > t.k_begin ? 1u : 0u;
           const int s0 = r.s;
-          const uint32_t stage0 = stage_addr(geo, s0);       // holds the shared operand
+          const uint32_t base0 = ring_lo + (uint32_t)s0 * stage_step;       // first stage: holds the shared operand
           for (int j = 0; j < nst; ++j, ring_next(r, ns)) {
             const int s = r.s;
 #ifdef COMPACT_PROFILE_GEN
             const long long w0c = clock64();
 #endif
-            if (!(ok = mbar_wait(full_bar(geo, s), r.ph, abort_flag, prm.status))) break;
+            if (!(ok = __all_sync(0xffffffffu, mbar_wait(full_bar(geo, s), r.ph, abort_flag, prm.status)))) break;
 #ifdef COMPACT_PROFILE_GEN
             mwait += clock64() - w0c;
 #endif
@@ -630,43 +672,51 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
 #ifdef COMPACT_PROFILE_GEN
             const long long i0c = clock64();
 #endif
-            const uint32_t stage = stage_addr(geo, s);
-            if (p.ncol > 1) {
-              issue4(d_base + acc_col(j), desc_lo(stage0 + STAGE_A0_OFF, a_mn), desc_lo(stage + STAGE_B_OFF, b_mn), first);
-            } else {
-              const uint32_t b_lo = desc_lo(stage0 + STAGE_B_OFF, b_mn);
-              issue4(d_base + acc_col(2 * j), desc_lo(stage + STAGE_A0_OFF, a_mn), b_lo, first);
-              if (2 * j + 1 < t.nsub) issue4(d_base + acc_col(2 * j + 1), desc_lo(stage + STAGE_A1_OFF, a_mn), b_lo, first);
+            const uint32_t base = ring_lo + (uint32_t)s * stage_step;
+            if (elect_one()) {
+              if (by_col) {
+                issue4(j == 0 ? d0 : d1, (base0 + (STAGE_A0_OFF >> 4)) | a_flags, (base + (STAGE_B_OFF >> 4)) | b_flags, first);
+              } else {
+                const uint32_t b_lo = (base0 + (STAGE_B_OFF >> 4)) | b_flags;
+                issue4(j == 0 ? d0 : d2, (base + (STAGE_A0_OFF >> 4)) | a_flags, b_lo, first);
+                if (2 * j + 1 < nsub) issue4(j == 0 ? d1 : d3, (base + (STAGE_A1_OFF >> 4)) | a_flags, b_lo, first);
+              }
+              // a stage that holds nothing shared goes back at once; the first stage of the k-step goes last
+              if (j > 0) {
+                if (gen_shared) umma_commit_mc(empty_bar(geo, s), cta_mask);
+                else umma_commit(empty_bar(geo, s));
+              }
+              if (j == nst - 1) {
+                if (gen_shared) umma_commit_mc(empty_bar(geo, s0), cta_mask);
+                else umma_commit(empty_bar(geo, s0));
+              }
             }
+            __syncwarp();
 #ifdef COMPACT_PROFILE_GEN
             missue += clock64() - i0c;
 #endif
-            // a stage that holds nothing shared goes back at once; the first stage of the k-step goes last
-            if (j > 0) {
-              if (gen_shared) umma_commit_mc(empty_bar(geo, s), (uint16_t)((1u << cs) - 1u));
-              else umma_commit(empty_bar(geo, s));
-            }
           }
-          if (!ok) break;
-          if (gen_shared) umma_commit_mc(empty_bar(geo, s0), (uint16_t)((1u << cs) - 1u));
-          else umma_commit(empty_bar(geo, s0));
         }
         if (!ok) break;
         if (geo) r1 = r; else r0 = r;
 #ifdef COMPACT_PROFILE_GEN
-        if (p.a_mode >= GENERATED || p.b_mode >= GENERATED) {
-          atomicAdd(&g_prof[4], (unsigned long long)mwait);                 // waiting for full stages
-          atomicAdd(&g_prof[5], (unsigned long long)missue);               // issuing MMAs
-          atomicAdd(&g_prof[6], (unsigned long long)(clock64() - m1c));    // whole k loop
-          atomicAdd(&g_prof[7], (unsigned long long)(t.k_end - t.k_begin));
-        } else if (!has_gen) {
-          atomicAdd(&g_prof[0], (unsigned long long)mwait);
-          atomicAdd(&g_prof[1], (unsigned long long)missue);
-          atomicAdd(&g_prof[2], (unsigned long long)(clock64() - m1c));
-          atomicAdd(&g_prof[3], (unsigned long long)(t.k_end - t.k_begin));
+        if (lane == 0) {
+          if (p.a_mode >= GENERATED || p.b_mode >= GENERATED) {
+            atomicAdd(&g_prof[4], (unsigned long long)mwait);                 // waiting for full stages
+            atomicAdd(&g_prof[5], (unsigned long long)missue);               // issuing MMAs and commits
+            atomicAdd(&g_prof[6], (unsigned long long)(clock64() - m1c));    // whole k loop
+            atomicAdd(&g_prof[7], (unsigned long long)(t.k_end - t.k_begin));
+          } else if (!has_gen) {
+            atomicAdd(&g_prof[0], (unsigned long long)mwait);
+            atomicAdd(&g_prof[1], (unsigned long long)missue);
+            atomicAdd(&g_prof[2], (unsigned long long)(clock64() - m1c));
+            atomicAdd(&g_prof[3], (unsigned long long)(t.k_end - t.k_begin));
+          }
         }
 #endif
-        for (int sl = 0; sl < slots; ++sl) umma_commit(tfull_bar((acc0 + sl) & 1));
+        if (elect_one())
+          for (int sl = 0; sl < slots; ++sl) umma_commit(tfull_bar((acc0 + sl) & 1));
+        __syncwarp();
       }
     }
   } else if (warp < 2 + NUM_EPI_WARPS) {
@@ -1004,6 +1054,22 @@ inline bool make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t 
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// MN-major operand tiles: the matrix (rows x cols, cols a multiple of 64) seen as [cols / 64][rows][64], so
+// that one copy of a {64, box_rows, blocks} box lands as `blocks` consecutive swizzled [box_rows][128 B]
+// pieces -- the layout the MMA descriptor of an MN-major operand walks.
+inline bool make_map_blocked(CUtensorMap* map, const void* base, int64_t cols, int64_t rows, int64_t pitch, int box_rows,
+                             int blocks) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {64, (cuuint64_t)rows, (cuuint64_t)(cols / 64)};
+  cuuint64_t strides[2] = {(cuuint64_t)pitch * 2, 128};
+  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, (cuuint32_t)blocks};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // 3-D fp32 map over `planes` row-major matrices of rows x inner (pitch and plane stride in elements);
 // boxes are 32 columns x 32 rows of one plane.
 inline bool make_map_f32_3d(CUtensorMap* map, const void* base, int64_t inner, int64_t rows, int64_t planes, int64_t pitch,
@@ -1148,7 +1214,9 @@ inline compact_status_t forward(const LaunchInfo& li, const ProjectionParams& pp
   if (!make_map(&prm.tmA[1], X, n, tokens, ldx, BK, BM)) return COMPACT_ERR_CUDA;
   prm.tmA[0] = prm.tmA[1];   // unused by the generated operand
   if (!make_map(&prm.tmB[0], X, n, tokens, ldx, BK, pz.bn)) return COMPACT_ERR_CUDA;
-  if (!make_map(&prm.tmB[1], W, m, n, ldw, 64, BK)) return COMPACT_ERR_CUDA;
+  py.b_blocked = m % 64 == 0;
+  if (py.b_blocked ? !make_map_blocked(&prm.tmB[1], W, m, n, ldw, BK, py.bn / 64) : !make_map(&prm.tmB[1], W, m, n, ldw, 64, BK))
+    return COMPACT_ERR_CUDA;
   if (!make_map(&prm.tmC[0], Z, zcols, tokens, ldz, 32, 64, false)) return COMPACT_ERR_CUDA;
   if (!make_map(&prm.tmC[1], Y, m, tokens, ldy, 64, 32)) return COMPACT_ERR_CUDA;
   return launch(li, prm);
@@ -1177,8 +1245,13 @@ inline compact_status_t backward(const LaunchInfo& li, int64_t tokens, int n, in
   } else {
     if (!make_map_f32_3d(&prm.tmC[0], Gc, m, r, 1, ldg, (int64_t)r * ldg)) return COMPACT_ERR_CUDA;
   }
-  if (!make_map(&prm.tmA[0], Z, zcols, tokens, ldz, 64, BK)) return COMPACT_ERR_CUDA;
-  if (!make_map(&prm.tmB[0], dY, m, tokens, lddy, 64, BK)) return COMPACT_ERR_CUDA;
+  pg.a_blocked = zcols % 64 == 0;
+  pg.b_blocked = m % 64 == 0;
+  if (pg.a_blocked ? !make_map_blocked(&prm.tmA[0], Z, zcols, tokens, ldz, BK, 2) : !make_map(&prm.tmA[0], Z, zcols, tokens, ldz, 64, BK))
+    return COMPACT_ERR_CUDA;
+  if (pg.b_blocked ? !make_map_blocked(&prm.tmB[0], dY, m, tokens, lddy, BK, pg.bn / 64)
+                   : !make_map(&prm.tmB[0], dY, m, tokens, lddy, 64, BK))
+    return COMPACT_ERR_CUDA;
   if (dX) {
     Problem& px = prm.prob[1];
     px.M = (int)tokens; px.N = n; px.K = m;
@@ -1224,7 +1297,9 @@ inline compact_status_t update(const LaunchInfo& li, const ProjectionParams& pp,
   pu.a_mode = GENERATED; pu.b_mode = TMA_MNMAJOR; pu.epi_mode = EPI_UPDATE_W;
   pu.scale = scale;
   finish_problem(pu, 1);
-  if (!make_map(&prm.tmB[0], Nbuf, m, r, m, 64, BK)) return COMPACT_ERR_CUDA;
+  pu.b_blocked = m % 64 == 0;
+  if (pu.b_blocked ? !make_map_blocked(&prm.tmB[0], Nbuf, m, r, m, BK, pu.bn / 64) : !make_map(&prm.tmB[0], Nbuf, m, r, m, 64, BK))
+    return COMPACT_ERR_CUDA;
   prm.tmA[0] = prm.tmB[0];
   if (!make_map(&prm.tmC[0], W, m, n, ldw, 64, 32)) return COMPACT_ERR_CUDA;
   return launch(li, prm);
