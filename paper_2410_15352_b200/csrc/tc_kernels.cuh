@@ -58,8 +58,9 @@ constexpr int STAGING_BUFS = 1;          // staged tiles per epilogue warp
 constexpr int QDEPTH = 4;                // work items the scheduler may run ahead
 constexpr int NUM_EPI_WARPS = 8;         // two sets of four (one per TMEM lane quarter); each set drains one accumulator slot
 constexpr int NUM_GEN_WARPS = 16;
-constexpr int NUM_LOADERS = 2;           // loader threads besides the stage owner: A tile 0, A tile 1
-constexpr int THREADS_BASE = 64 + 32 * NUM_EPI_WARPS + 32 * NUM_LOADERS;   // owner/scheduler, MMA, epilogue, loaders
+constexpr int LOADER_WARP = 2 + NUM_EPI_WARPS;      // loads the A tiles
+constexpr int MMA1_WARP = 3 + NUM_EPI_WARPS;        // second MMA issuer
+constexpr int THREADS_BASE = 32 * (4 + NUM_EPI_WARPS);   // owner/scheduler, two MMA issuers, epilogue, loader
 constexpr int THREADS_GEN = THREADS_BASE + 32 * NUM_GEN_WARPS;
 constexpr int NUM_BARRIERS = NUM_RING_BARS + 4 + 2 * QDEPTH + NUM_EPI_WARPS * STAGING_BUFS;
 constexpr int TAIL_BYTES = 8 * NUM_BARRIERS + 4 * QDEPTH + 16;
@@ -353,10 +354,10 @@ __device__ __forceinline__ TileCoord decode_tile(const Params& prm, int tile) {
 // --------------------------------------------------------------------------------------
 // The kernel.  Warp roles:
 //   0      item scheduler and stage owner: waits for a free stage, declares the bytes that will land
-//          on its full barrier, arrives, and loads the (lower half of the) B tile
-//   1      tcgen05.mma issuer (one thread), owner of TMEM
+//          on its full barrier, arrives, and loads the B tile
+//   1, 11  tcgen05.mma issuers (one elected lane each); warp 1 owns TMEM
 //   2..9   epilogue: two sets of four warps; with two accumulator slots each set drains one of them
-//   10,11  loaders: A tile 0, A tile 1 (each only issues TMA)
+//   10     loader of the A tiles (only issues TMA)
 //   12..27 generators of P (launches with a generated operand only)
 // --------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __grid_constant__ Params prm) {
@@ -391,16 +392,16 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
     for (int g = 0; g < 2; ++g)
       for (int s = 0; s < (g ? NS1 : NS0); ++s) {
         mbar_init(full_bar(g, s), 1 + (has_gen ? GEN_ARRIVALS : 0));   // the stage owner, and the generator warps
-        // in an item with a generated operand a stage is free once the MMAs of all cs CTAs have read
-        // it; in every other item the owner supplies the cs - 1 arrivals that will not come
-        mbar_init(empty_bar(g, s), cs);
+        // a stage is handed back by up to two MMA issuers in each of cs CTAs (items with a generated
+        // operand) or of this CTA; the owner supplies the arrivals that a given use will not get
+        mbar_init(empty_bar(g, s), 2 * cs);
       }
     for (int a = 0; a < 2; ++a) {
       mbar_init(tfull_bar(a), 1);
       mbar_init(tempty_bar(a), NUM_EPI_WARPS);
     }
     // consumers of the item queue: MMA thread, loaders, epilogue warps, generator warps
-    const int consumers = 1 + NUM_LOADERS + NUM_EPI_WARPS + (has_gen ? NUM_GEN_WARPS : 0);
+    const int consumers = 3 + NUM_EPI_WARPS + (has_gen ? NUM_GEN_WARPS : 0);
     for (int s = 0; s < QDEPTH; ++s) {
       mbar_init(qfull(s), 1);
       mbar_init(qempty(s), consumers);
@@ -444,7 +445,13 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
     return min(2, t.nsub - 2 * j);
   };
 
-  const int loader = (warp >= 2 + NUM_EPI_WARPS && warp < 2 + NUM_EPI_WARPS + NUM_LOADERS) ? warp - 2 - NUM_EPI_WARPS : -1;
+  // An item whose two accumulators sit in one TMEM slot each is issued by two warps, one accumulator
+  // each: a tcgen05.mma costs its issuing thread about as long as the tensor core needs for it, so a
+  // single issuer leaves the tensor core idle while it waits on barriers and commits.
+  auto item_is_split = [&](const Problem& p, const TileCoord& t) {
+    const int naccs = p.nsub * p.ncol;
+    return naccs == 2 && t.nsub * t.ncol == 2 && (naccs * p.bn + BN_MAX - 1) / BN_MAX == 2;
+  };
   if (warp == 0) {
     // ------------------------- scheduler + stage owner --------------------------
     // Like the MMA warp, these warps walk their loops whole (warp-uniform addresses and counters) and
@@ -488,6 +495,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const Problem& p = prm.prob[t.prob];
         const CUtensorMap* mapB = &prm.tmB[t.prob];
         const bool a_tma = p.a_mode < GENERATED, b_tma = p.b_mode < GENERATED;
+        const bool split = item_is_split(p, t);
         const int geo = p.geo, ns = geo ? NS1 : NS0;
         if (cur_geo >= 0 && geo != cur_geo && !(ok = __all_sync(0xffffffffu, drain(cur_geo, cur_geo ? r1 : r0)))) break;
         cur_geo = geo;
@@ -508,11 +516,14 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             if (prm.debug_flags & 2) tx = 0;
 #endif
             if (elect_one()) {
-              // Items with a generated operand hand every stage back with a commit from each CTA of the
+              // Items with a generated operand hand every stage back with commits from each CTA of the
               // cluster, so that no CTA writes its share of the next tile (or counts its bytes) into a
-              // stage that its neighbour has not finished with.  Other items hand stages back locally
-              // and the owner supplies the arrivals that will not come.
-              if (cs > 1 && a_tma && b_tma) mbar_arrive_n(empty_bar(geo, s), cs - 1);
+              // stage that its neighbour has not finished with.  Other items hand stages back locally.
+              // The owner supplies the arrivals that will not come.
+              // commits this use will get: from both issuers if they both read the stage, times cs for
+              // items with a generated operand (whose stages every CTA of the cluster hands back)
+              const int commits = (split && (p.ncol == 1 || j == 0) ? 2 : 1) * ((a_tma && b_tma) ? 1 : cs);
+              if (commits < 2 * cs) mbar_arrive_n(empty_bar(geo, s), 2 * cs - commits);
               const uint32_t fb = full_bar(geo, s);
               if (tx) mbar_expect_tx(fb, tx);
               // arrive for this thread, and for the generator warps when they have nothing to write here
@@ -535,9 +546,9 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         if (geo) r1 = r; else r0 = r;
       }
     }
-  } else if (loader >= 0) {
-    // ------------------------------ loaders --------------------------------------
-    // 0: A tile in slot 0, 1: A tile in slot 1.  They only issue TMA; the bytes were declared by the stage owner.
+  } else if (warp == LOADER_WARP) {
+    // ------------------------------ loader ---------------------------------------
+    // Issues the TMA copies of the A tiles; the bytes were declared by the stage owner.
     {
       Ring r0 = {0, 0u}, r1 = {0, 0u};
       int cur_geo = -1;
@@ -564,20 +575,23 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             const int s = r.s;
             const uint32_t eph = r.ph ^ 1u;
             ring_next(r, ns);
-            if (loader >= stage_num_a(p, t, j)) continue;
+            const int na = stage_num_a(p, t, j);
+            if (na <= 0) continue;
             if (!(ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(geo, s), eph, abort_flag, prm.status)))) break;
             if (elect_one()) {
               const uint32_t fb = full_bar(geo, s);
-              const int mi = p.ncol > 1 ? 0 : 2 * j + loader;
-              const int m0 = t.m0 + mi * BM;
-              const uint32_t dst = stage_addr(geo, s) + (loader == 0 ? STAGE_A0_OFF : STAGE_A1_OFF);
-              if (p.a_mode == TMA_KMAJOR) {
-                tma_load_2d(dst, mapA, fb, k0, m0);
-              } else if (p.a_blocked) {
-                tma_load_3d(dst, mapA, fb, 0, k0, m0 >> 6);
-              } else {
-                tma_load_2d(dst, mapA, fb, m0, k0);
-                tma_load_2d(dst + 8192, mapA, fb, m0 + 64, k0);
+              for (int l = 0; l < na; ++l) {
+                const int mi = p.ncol > 1 ? 0 : 2 * j + l;
+                const int m0 = t.m0 + mi * BM;
+                const uint32_t dst = stage_addr(geo, s) + (l == 0 ? STAGE_A0_OFF : STAGE_A1_OFF);
+                if (p.a_mode == TMA_KMAJOR) {
+                  tma_load_2d(dst, mapA, fb, k0, m0);
+                } else if (p.a_blocked) {
+                  tma_load_3d(dst, mapA, fb, 0, k0, m0 >> 6);
+                } else {
+                  tma_load_2d(dst, mapA, fb, m0, k0);
+                  tma_load_2d(dst + 8192, mapA, fb, m0 + 64, k0);
+                }
               }
             }
             __syncwarp();
@@ -586,11 +600,14 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         if (geo) r1 = r; else r0 = r;
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------ MMA issuer ---------------------------------
+  } else if (warp == 1 || warp == MMA1_WARP) {
+    // ------------------------------ MMA issuers --------------------------------
     // The whole warp walks the loops, so that addresses, descriptors and counters are warp-uniform
-    // values; one elected lane issues the MMAs and the commits.
+    // values; one elected lane issues the MMAs and the commits.  Issuer 0 (warp 1) owns TMEM.  In a
+    // split item issuer x computes accumulator x; any other item is issuer 0's alone, and issuer 1
+    // only keeps its counters in step.
     {
+      const int iss = warp == 1 ? 0 : 1;
       Ring r0 = {0, 0u}, r1 = {0, 0u};
       int acc = 0;
       uint32_t acc_phase = 0;
@@ -602,15 +619,19 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const TileCoord t = decode_tile(prm, tile);
         const Problem& p = prm.prob[t.prob];
         const bool a_mn = p.a_mode == TMA_MNMAJOR || p.a_mode == GENERATED_T;
-        const bool b_mn = p.b_mode != TMA_KMAJOR;          // generated B tiles are written MN-major
+        const bool b_mn = p.b_mode != TMA_KMAJOR;
         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
                                ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
         const int slots = (p.nsub * p.ncol * p.bn + BN_MAX - 1) / BN_MAX;   // accumulator slots this item occupies
+        const bool split = item_is_split(p, t);
+        const bool active = split || iss == 0;
         if (slots == 2 && acc == 1) {
           // a two-slot item starts at slot 0: pass slot 1 through unused
-          if (!(ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(1), acc_phase ^ 1, abort_flag, prm.status)))) break;
-          if (elect_one()) umma_commit(tfull_bar(1));
-          __syncwarp();
+          if (iss == 0) {
+            if (!(ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(1), acc_phase ^ 1, abort_flag, prm.status)))) break;
+            if (elect_one()) umma_commit(tfull_bar(1));
+            __syncwarp();
+          }
           acc = 0;
           acc_phase ^= 1;
         }
@@ -619,7 +640,9 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         long long mwait = 0, missue = 0;
 #endif
         for (int sl = 0; sl < slots && ok; ++sl) {
-          ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag, prm.status));
+          // a split item's issuer x waits for slot x only
+          if (active && (!split || sl == iss))
+            ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag, prm.status));
           if (++acc == 2) { acc = 0; acc_phase ^= 1; }
         }
         if (!ok) break;
@@ -634,6 +657,11 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const bool by_col = p.ncol > 1;
         const int geo = p.geo, ns = geo ? NS1 : NS0;
         Ring r = geo ? r1 : r0;
+        if (!active) {
+          ring_skip(r, ns, (t.k_end - t.k_begin) * nst);
+          if (geo) r1 = r; else r0 = r;
+          continue;
+        }
         // items with a generated operand walk the ring in step with the other CTAs of the cluster
         const bool gen_shared = cs > 1 && (p.a_mode >= GENERATED || p.b_mode >= GENERATED);
         // accumulator ai of the item sits in slot ai / sps at column (ai % sps) * bn (a slot is 256 columns)
@@ -655,12 +683,18 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
           umma_bf16(d, a_lo + 2 * a_step, DESC_HI, b_lo + 2 * b_step, DESC_HI, idesc, 1u);
           umma_bf16(d, a_lo + 3 * a_step, DESC_HI, b_lo + 3 * b_step, DESC_HI, idesc, 1u);
         };
+        auto commit_stage = [&](int s) {
+          if (gen_shared) umma_commit_mc(empty_bar(geo, s), cta_mask);
+          else umma_commit(empty_bar(geo, s));
+        };
         for (int ks = t.k_begin; ks < t.k_end && ok; ++ks) {
           const uint32_t first = ks > t.k_begin ? 1u : 0u;
           const int s0 = r.s;
           const uint32_t base0 = ring_lo + (uint32_t)s0 * stage_step;       // first stage: holds the shared operand
           for (int j = 0; j < nst; ++j, ring_next(r, ns)) {
             const int s = r.s;
+            // split by columns: issuer 0 needs the first stage only, issuer 1 both
+            if (split && by_col && iss == 0 && j == 1) continue;
 #ifdef COMPACT_PROFILE_GEN
             const long long w0c = clock64();
 #endif
@@ -668,6 +702,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
 #ifdef COMPACT_PROFILE_GEN
             mwait += clock64() - w0c;
 #endif
+            if (split && by_col && iss == 1 && j == 0) continue;
             tc_fence_after();
 #ifdef COMPACT_PROFILE_GEN
             const long long i0c = clock64();
@@ -675,21 +710,17 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             const uint32_t base = ring_lo + (uint32_t)s * stage_step;
             if (elect_one()) {
               if (by_col) {
-                issue4(j == 0 ? d0 : d1, (base0 + (STAGE_A0_OFF >> 4)) | a_flags, (base + (STAGE_B_OFF >> 4)) | b_flags, first);
+                if (!split || j == iss)
+                  issue4(j == 0 ? d0 : d1, (base0 + (STAGE_A0_OFF >> 4)) | a_flags, (base + (STAGE_B_OFF >> 4)) | b_flags, first);
               } else {
                 const uint32_t b_lo = (base0 + (STAGE_B_OFF >> 4)) | b_flags;
-                issue4(j == 0 ? d0 : d2, (base + (STAGE_A0_OFF >> 4)) | a_flags, b_lo, first);
-                if (2 * j + 1 < nsub) issue4(j == 0 ? d1 : d3, (base + (STAGE_A1_OFF >> 4)) | a_flags, b_lo, first);
+                if (!split || iss == 0) issue4(j == 0 ? d0 : d2, (base + (STAGE_A0_OFF >> 4)) | a_flags, b_lo, first);
+                if ((!split || iss == 1) && 2 * j + 1 < nsub)
+                  issue4(j == 0 ? d1 : d3, (base + (STAGE_A1_OFF >> 4)) | a_flags, b_lo, first);
               }
               // a stage that holds nothing shared goes back at once; the first stage of the k-step goes last
-              if (j > 0) {
-                if (gen_shared) umma_commit_mc(empty_bar(geo, s), cta_mask);
-                else umma_commit(empty_bar(geo, s));
-              }
-              if (j == nst - 1) {
-                if (gen_shared) umma_commit_mc(empty_bar(geo, s0), cta_mask);
-                else umma_commit(empty_bar(geo, s0));
-              }
+              if (j > 0) commit_stage(s);
+              if (j == nst - 1 || (split && by_col && iss == 0)) commit_stage(s0);
             }
             __syncwarp();
 #ifdef COMPACT_PROFILE_GEN
@@ -700,7 +731,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         if (!ok) break;
         if (geo) r1 = r; else r0 = r;
 #ifdef COMPACT_PROFILE_GEN
-        if (lane == 0) {
+        if (lane == 0 && iss == 0) {
           if (p.a_mode >= GENERATED || p.b_mode >= GENERATED) {
             atomicAdd(&g_prof[4], (unsigned long long)mwait);                 // waiting for full stages
             atomicAdd(&g_prof[5], (unsigned long long)missue);               // issuing MMAs and commits
@@ -714,8 +745,11 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
           }
         }
 #endif
-        if (elect_one())
-          for (int sl = 0; sl < slots; ++sl) umma_commit(tfull_bar((acc0 + sl) & 1));
+        if (elect_one()) {
+          if (split) umma_commit(tfull_bar((acc0 + iss) & 1));
+          else
+            for (int sl = 0; sl < slots; ++sl) umma_commit(tfull_bar((acc0 + sl) & 1));
+        }
         __syncwarp();
       }
     }
