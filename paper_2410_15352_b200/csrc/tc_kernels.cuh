@@ -613,8 +613,26 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       uint32_t acc_phase = 0;
       bool ok = true;
       const uint16_t cta_mask = (uint16_t)((1u << cs) - 1u);
+#ifdef COMPACT_PROFILE_GEN
+      const long long life0 = clock64();
+      long long qwait = 0, twait = 0, nitems = 0;
+#endif
       while (ok) {
+#ifdef COMPACT_PROFILE_GEN
+        const long long q0c = clock64();
+#endif
         const int tile = __shfl_sync(0xffffffffu, next_tile(true, lane == 0), 0);
+#ifdef COMPACT_PROFILE_GEN
+        qwait += clock64() - q0c;
+        if (tile < 0 && lane == 0 && iss == 0 && !has_gen) {
+          atomicAdd(&g_prof[4], (unsigned long long)(clock64() - life0));
+          atomicAdd(&g_prof[5], (unsigned long long)twait);
+          atomicAdd(&g_prof[6], (unsigned long long)qwait);
+          atomicAdd(&g_prof[7], (unsigned long long)nitems);
+        }
+        ++nitems;
+        const long long t0c = clock64();
+#endif
         if (tile < 0) break;
         const TileCoord t = decode_tile(prm, tile);
         const Problem& p = prm.prob[t.prob];
@@ -649,6 +667,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         tc_fence_after();
 #ifdef COMPACT_PROFILE_GEN
         const long long m1c = clock64();
+        twait += m1c - t0c;
 #endif
         const uint32_t d_base = tmem_base + acc0 * BN_MAX;
         // one UMMA consumes K = 16: 32 bytes along a K-major row, or two 8-row groups (2048 bytes) MN-major
