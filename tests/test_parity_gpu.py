@@ -25,7 +25,9 @@ def _built():
     cb.set_kernel_family(0)
 
 
-@pytest.fixture(params=[0, 1], ids=["auto", "simt"])
+# 0: tensor-core kernels with cluster-shared generation of P; 1: SIMT kernels; 2: tensor-core kernels in which every
+# CTA generates its own tiles of P
+@pytest.fixture(params=[0, 1, 2], ids=["auto", "simt", "nocluster"])
 def family(request):
     cb.set_kernel_family(request.param)
     yield request.param
@@ -91,6 +93,9 @@ SMALL = [
     (1, 64, 64, 8),              # a single token
     (129, 128, 136, 24),         # one row past a block, m not a multiple of 64
     (640, 320, 520, 320),        # r == n (full rank), three 128-column blocks of P
+    (1300, 192, 1544, 136),      # three 512-token blocks and four 512-column blocks of W (one ragged): a cluster's
+                                 # second CTA gets an item that is all padding in the forward
+    (2100, 448, 2056, 200),      # five token blocks, five column blocks: odd group counts on both sides
 ]
 
 
@@ -135,6 +140,27 @@ def test_z_token_indexing_bit_exact(family):
     _, Z1, _ = lay.forward(Xr, W)
     _, Z2, _ = lay.forward(Xr[perm].contiguous(), W)
     assert torch.equal(Z1[perm].view(torch.int16), Z2.view(torch.int16))
+
+
+def test_cluster_and_single_cta_generation_agree_bitwise():
+    # sharing generated tiles across a cluster changes who computes an entry of P, not its value, and leaves the
+    # accumulation order of every output alone
+    tokens, n, m, r = 1300, 320, 1096, 200
+    wl = wlm.Workload("clu", 99, "bf16", tokens, [wlm.LayerShape("l", n, m, r)], x_scale_inv_sqrt_n=True)
+    X, dY = wlm.draw_X(wl, 0, 0).cuda(), wlm.draw_dY(wl, 0, 0).cuda()
+    out = []
+    for fam in (0, 2):
+        cb.set_kernel_family(fam)
+        gpu, _, W0 = make_pair(wl, 0)
+        W = W0.cuda()
+        Y, Z, ep = gpu.forward(X, W)
+        dX, Gc = gpu.backward(dY, Z, W)
+        M, V = torch.zeros_like(Gc), torch.zeros_like(Gc)
+        gpu.adam_update(W, Gc, M, V, ep)
+        out.append((Y, Z, dX, Gc, W))
+    cb.set_kernel_family(0)
+    for a, b in zip(*out):
+        assert torch.equal(a.view(torch.int16) if a.dtype == torch.bfloat16 else a, b.view(torch.int16) if b.dtype == torch.bfloat16 else b)
 
 
 # ---- determinism, accumulation, empty input, epoch guard -----------------------------------
