@@ -441,6 +441,12 @@ void compact_debug_profile(unsigned long long* out) {
   cudaMemcpyToSymbol(tc::g_prof, z, sizeof(z));
 }
 #endif
+#ifdef COMPACT_PROFILE_GEN
+void compact_debug_trace(long long* out) {
+  cudaDeviceSynchronize();
+  cudaMemcpyFromSymbol(out, tc::g_trace, sizeof(long long) * 128);
+}
+#endif
 
 const char* compact_status_string(compact_status_t s) {
   switch (s) {

@@ -86,13 +86,30 @@ __device__ __forceinline__ float sqrt_approx(float x) {
   asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// Flush-to-zero forms: every argument here is a normal number or zero, and they spare the
+// instructions that rescale denormal arguments.
+__device__ __forceinline__ float lg2_approx(float x) {
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float sin_approx(float x) {
+  float y;
+  asm("sin.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float cos_approx(float x) {
+  float y;
+  asm("cos.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ void box_muller_fast(uint32_t xa, uint32_t xb, float neg2ln2_over_r, float& c, float& s) {
   const float u1 = __uint_as_float((xa >> 9) | 0x3F800000u) - 0.99999994f;
-  const float rad = sqrt_approx(fmaxf(__log2f(u1) * neg2ln2_over_r, 0.0f));
+  const float rad = sqrt_approx(fmaxf(lg2_approx(u1) * neg2ln2_over_r, 0.0f));
   const float th = (__uint_as_float(((xb >> 8) & 0x007FFFFFu) | 0x3F800000u) - 1.0f) * 3.14159265358979f;
   const float rs = __uint_as_float(__float_as_uint(rad) ^ (xb & 0x80000000u));
-  c = rs * __cosf(th);
-  s = rs * __sinf(th);
+  c = rs * cos_approx(th);
+  s = rs * sin_approx(th);
 }
 __device__ __forceinline__ float4 gaussian4_fast_scaled(uint4 x, float neg2ln2_over_r) {
   float4 g;

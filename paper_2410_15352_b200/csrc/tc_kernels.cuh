@@ -52,6 +52,7 @@ constexpr int NS0 = 3, STAGE0_BYTES = B_BYTES + 2 * A_BYTES;
 constexpr int NS1 = 4, STAGE1_BYTES = B_BYTES + A_BYTES;
 constexpr int RING_BYTES = NS0 * STAGE0_BYTES;
 static_assert(NS1 * STAGE1_BYTES <= RING_BYTES, "both geometries share the ring memory");
+static_assert(NS1 % 2 == 0, "two-stage k-steps of generated items must keep each stage's role");
 constexpr int NUM_RING_BARS = 2 * (NS0 + NS1);
 constexpr int STAGING_BYTES = 4096;      // one staged tile: 32 rows x 128 bytes
 constexpr int STAGING_BUFS = 1;          // staged tiles per epilogue warp
@@ -80,6 +81,17 @@ enum GenRing { GEN_NONE = 0, GEN_A = 1, GEN_B = 2 };
 constexpr unsigned int STATUS_TIMEOUT = 1u;
 #if defined(COMPACT_PROFILE) || defined(COMPACT_PROFILE_GEN)
 __device__ unsigned long long g_prof[8];
+#endif
+#ifdef COMPACT_PROFILE_GEN
+// event trace of CTA 0, first item, k-steps 16..23
+__device__ long long g_trace[8][16];
+#define TRACE(first_item, ks, ev)                                                              \
+  do {                                                                                         \
+    if (blockIdx.x == 0 && (first_item) && (ks) >= 16 && (ks) < 24 && (threadIdx.x & 31) == 0) \
+      g_trace[(ks) - 16][ev] = clock64();                                                      \
+  } while (0)
+#else
+#define TRACE(first_item, ks, ev) ((void)0)
 #endif
 #ifdef COMPACT_PROFILE
 #define PROF_T() clock64()
@@ -298,10 +310,23 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 
-// Eight consecutive entries P[i, j0 .. j0+7] (j0 a multiple of 8) as packed bf16.
-__device__ __forceinline__ uint4 projection8_bf16(const ProjectionParams& pp, int i, int j0) {
-  const float4 a = projection4<true>(pp, i, j0 >> 2);
-  const float4 b = projection4<true>(pp, i, (j0 >> 2) + 1);
+// Eight consecutive entries P[i, j0 .. j0+7] (j0 a multiple of 8) as packed bf16, in two steps so that a
+// generator thread can run the Philox rounds of its next tile (32x32->64 multiplies) between the Box-Muller
+// transforms of the current one (MUFU): the raw words, then the Gaussians.  Entries outside n x r are zero.
+__device__ __forceinline__ void projection8_words(const ProjectionParams& pp, int i, int j0, uint4& xa, uint4& xb) {
+  const uint32_t q = (uint32_t)(j0 >> 2);
+  xa = philox4x32_10_layer(q, (uint32_t)i, pp.epoch, pp.layer_hi, pp.layer_lo, pp.key);
+  xb = philox4x32_10_layer(q + 1, (uint32_t)i, pp.epoch, pp.layer_hi, pp.layer_lo, pp.key);
+}
+__device__ __forceinline__ uint4 projection8_from_words(const ProjectionParams& pp, const uint4& xa, const uint4& xb, int i,
+                                                        int j0) {
+  float4 a = gaussian4_fast_scaled(xa, pp.neg2ln2_over_r);
+  float4 b = gaussian4_fast_scaled(xb, pp.neg2ln2_over_r);
+  const int left = i < pp.n ? pp.r - j0 : 0;      // valid entries among the eight
+  if (left < 8) {
+    a.x = left > 0 ? a.x : 0.f; a.y = left > 1 ? a.y : 0.f; a.z = left > 2 ? a.z : 0.f; a.w = left > 3 ? a.w : 0.f;
+    b.x = left > 4 ? b.x : 0.f; b.y = left > 5 ? b.y : 0.f; b.z = left > 6 ? b.z : 0.f; b.w = left > 7 ? b.w : 0.f;
+  }
   return make_uint4(pack_bf16x2(a.x, a.y), pack_bf16x2(a.z, a.w), pack_bf16x2(b.x, b.y), pack_bf16x2(b.z, b.w));
 }
 
@@ -460,6 +485,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       Ring r0 = {0, 0u}, r1 = {0, 0u};     // position in each geometry's ring
       int cur_geo = -1;
       bool ok = true;
+      int first_tile = -2;
       int group = (int)(blockIdx.x / cs);  // static part: cluster c takes groups c, c + clusters, ...
       const int group_step = (int)(gridDim.x / cs);
       while (ok) {
@@ -491,6 +517,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         __syncwarp();
         if (++qs == QDEPTH) { qs = 0; qph ^= 1; }
         if (tile < 0) break;
+        if (first_tile == -2) first_tile = tile;
         const TileCoord t = decode_tile(prm, tile);
         const Problem& p = prm.prob[t.prob];
         const CUtensorMap* mapB = &prm.tmB[t.prob];
@@ -505,6 +532,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
           for (int j = 0; j < t.nst; ++j, ring_next(r, ns)) {
             const int s = r.s;
             if (!(ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(geo, s), r.ph ^ 1u, abort_flag, prm.status)))) break;
+            TRACE(tile == first_tile, ks, 4 + j);
             const bool hb = stage_has_b(p, j);
             const int na = stage_num_a(p, t, j);
             uint32_t tx = 0;
@@ -516,13 +544,13 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             if (prm.debug_flags & 2) tx = 0;
 #endif
             if (elect_one()) {
-              // Items with a generated operand hand every stage back with commits from each CTA of the
+              // A stage that holds a generated tile is handed back with commits from each CTA of the
               // cluster, so that no CTA writes its share of the next tile (or counts its bytes) into a
-              // stage that its neighbour has not finished with.  Other items hand stages back locally.
-              // The owner supplies the arrivals that will not come.
-              // commits this use will get: from both issuers if they both read the stage, times cs for
-              // items with a generated operand (whose stages every CTA of the cluster hands back)
-              const int commits = (split && (p.ncol == 1 || j == 0) ? 2 : 1) * ((a_tma && b_tma) ? 1 : cs);
+              // stage that its neighbour has not finished with.  This relies on a stage keeping its role
+              // while generated items run: their k-steps take one stage, or two of an even-sized ring.
+              // All other stages are handed back locally.  The owner supplies the arrivals that will not
+              // come: a use gets commits from both issuers if both read the stage, times cs if shared.
+              const int commits = (split && (p.ncol == 1 || j == 0) ? 2 : 1) * (gen_here ? cs : 1);
               if (commits < 2 * cs) mbar_arrive_n(empty_bar(geo, s), 2 * cs - commits);
               const uint32_t fb = full_bar(geo, s);
               if (tx) mbar_expect_tx(fb, tx);
@@ -721,6 +749,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
 #ifdef COMPACT_PROFILE_GEN
             mwait += clock64() - w0c;
 #endif
+            TRACE(nitems == 1, ks, iss == 0 ? 6 : 8 + j);
             if (split && by_col && iss == 1 && j == 0) continue;
             tc_fence_after();
 #ifdef COMPACT_PROFILE_GEN
@@ -738,10 +767,11 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
                   issue4(j == 0 ? d1 : d3, (base + (STAGE_A1_OFF >> 4)) | a_flags, b_lo, first);
               }
               // a stage that holds nothing shared goes back at once; the first stage of the k-step goes last
-              if (j > 0) commit_stage(s);
+              if (j > 0) umma_commit(empty_bar(geo, s));
               if (j == nst - 1 || (split && by_col && iss == 0)) commit_stage(s0);
             }
             __syncwarp();
+            TRACE(nitems == 1, ks, iss == 0 ? 7 : 10);
 #ifdef COMPACT_PROFILE_GEN
             missue += clock64() - i0c;
 #endif
@@ -826,6 +856,33 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
           for (int ci = (slots == 2 ? 0 : eset); ci < cpa && ok; ci += (slots == 2 ? 1 : 2)) {
             const int col = ncol0 + ci * cw;
             if (col >= p.N) break;
+            if (p.epi_mode == EPI_BF16) {
+              // convert the whole chunk first; the previous store's read of the staging tile hides behind it
+              uint32_t o[32];
+#pragma unroll
+              for (int h = 0; h < 2; ++h) {
+                uint32_t v[32];
+                tmem_ld32(tcol + ci * cw + 32 * h, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) o[16 * h + j] = pack_bf16x2(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+              }
+              if (lane == 0) tma_store_wait_read();
+              __syncwarp();
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                *reinterpret_cast<uint4*>(stg_gen + lane * 128 + ((j ^ sw) << 4)) = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+#if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
+              if (prm.debug_flags & 8) continue;
+#endif
+              fence_proxy_async_smem();
+              __syncwarp();
+              if (lane == 0) {
+                tma_store_2d(mapC, stg, col, row0);
+                tma_store_commit();
+              }
+              continue;
+            }
             if (lane == 0) tma_store_wait_read();          // the previous store has read the staging tile
             __syncwarp();
             if (p.epi_mode == EPI_F32) {
@@ -887,16 +944,6 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
                   w.w = pack_bf16x2(fmaf(sc, __uint_as_float(v[8 * j + 6]), bf16lo(w.w)), fmaf(sc, __uint_as_float(v[8 * j + 7]), bf16hi(w.w)));
                   *cell = w;
                 }
-              } else {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  uint4 o;
-                  o.x = pack_bf16x2(__uint_as_float(v[8 * j + 0]), __uint_as_float(v[8 * j + 1]));
-                  o.y = pack_bf16x2(__uint_as_float(v[8 * j + 2]), __uint_as_float(v[8 * j + 3]));
-                  o.z = pack_bf16x2(__uint_as_float(v[8 * j + 4]), __uint_as_float(v[8 * j + 5]));
-                  o.w = pack_bf16x2(__uint_as_float(v[8 * j + 6]), __uint_as_float(v[8 * j + 7]));
-                  *reinterpret_cast<uint4*>(stg_gen + lane * 128 + (((4 * h + j) ^ sw) << 4)) = o;
-                }
               }
             }
             if (!ok) break;
@@ -924,14 +971,11 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
     // ------------------------------ P generators --------------------------------
     // Write bf16 tiles of P straight into the swizzled operand layout the MMA reads: as the B tile
     // of the first stage of a k-step (forward) or as its A tile 0 (update).
-#ifdef CFG_GEN_SKIP1
-    // experiment: the four generator warps that share a scheduler with the MMA warp do no work
-    const int gw_ = warp - (THREADS_BASE >> 5), sc_ = gw_ & 3;
-    const int gtid = sc_ == 1 ? (1 << 20) : (((gw_ >> 2) * 3 + (sc_ == 0 ? 0 : sc_ - 1)) * 32 + lane);
-    constexpr int GSTRIDE = 32 * NUM_GEN_WARPS * 3 / 4;
-#else
     const int gtid = threadIdx.x - THREADS_BASE;
     constexpr int GSTRIDE = 32 * NUM_GEN_WARPS;
+    int first_tile = -2;
+#ifdef COMPACT_PROFILE_GEN
+    long long pg_wait = 0, pg_gen = 0, pg_arr = 0, pg_cnt = 0;
 #endif
     Ring r0 = {0, 0u}, r1 = {0, 0u};
     bool ok = true;
@@ -945,61 +989,116 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       const TileCoord t = decode_tile(prm, tile);
       const Problem& p = prm.prob[t.prob];
       const int klen = t.k_end - t.k_begin;
+      if (first_tile == -2) first_tile = tile;
       const bool gen_a = p.a_mode == GENERATED, gen_at = p.a_mode == GENERATED_T;
       const int geo = p.geo, ns = geo ? NS1 : NS0;
       Ring r = geo ? r1 : r0;
       // The generated problem is the first of its launch, so the generators never write into a ring
       // whose geometry has changed.  In other items the stage owner arrives for them.
       if (!gen_a && !gen_at) ring_skip(r, ns, klen * t.nst);
+      // A thread's tasks (eight consecutive entries of a row of P each) keep their place in the tile
+      // from k-step to k-step; only the row (transposed forward) or the column (update) of P moves on.
+      //   transposed forward: A[m = column j of P][k = row i of P], MN-major, two 64-column blocks of [64 k][128 B]
+      //   update:             A[m = row i of P][k = column j of P], K-major, [128 rows][128 B]
+      // Of a tile shared by a cluster this CTA writes the rows crank * (rows / cs) onward.
+      const int ntask = 2 >> csh;                       // tasks per thread and tile: 1024 / (512 cs)
+      const bool philox_first = ((warp >> 2) & 1) != 0;  // two of the four generator warps of each scheduler
+      const int ik = gen_at ? 1 : 0, jk = 1 - ik;       // which index of P advances with k
+      int t_i[2], t_j[2];
+      uint32_t t_off[2];
+      uint4 xa[2], xb[2];
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const int id = gtid + u * GSTRIDE;
+        if (gen_at) {
+          const int c = id & 15, kr = (int)crank * (BK >> csh) + (id >> 4);
+          t_i[u] = kr; t_j[u] = t.m0 + c * 8;
+          t_off[u] = STAGE_A0_OFF + (c >> 3) * 8192 + kr * 128 + (((c & 7) ^ (kr & 7)) << 4);
+        } else {
+          const int c = id & 7, rr = (int)crank * (BM >> csh) + (id >> 3);
+          t_i[u] = t.m0 + rr; t_j[u] = c * 8;
+          t_off[u] = STAGE_A0_OFF + rr * 128 + ((c ^ (rr & 7)) << 4);
+        }
+      }
+      if (gen_a || gen_at) {
+        const int k0 = t.k_begin * BK;
+#pragma unroll
+        for (int u = 0; u < 2; ++u)
+          if (u < ntask) projection8_words(prm.pp, t_i[u] + ik * k0, t_j[u] + jk * k0, xa[u], xb[u]);
+      }
       for (int ks = t.k_begin; ks < t.k_end && ok && (gen_a || gen_at); ++ks) {
         const int s = r.s;
         const uint32_t eph = r.ph ^ 1u;
-        ring_skip(r, ns, t.nst);
+        ring_next(r, ns);
+        if (t.nst > 1) ring_next(r, ns);            // a k-step takes one or two stages
         const uint32_t stage_off = (uint32_t)s * (geo ? STAGE1_BYTES : STAGE0_BYTES);
         const uint32_t full_off = full_bar(geo, s) - bars;
 #ifdef COMPACT_PROFILE_GEN
         const long long g0 = clock64();
 #endif
+#ifdef CFG_GEN_WAIT_LANE0
+        bool w = true;
+        if (lane == 0) w = mbar_wait(empty_bar(geo, s), eph, abort_flag, prm.status);
+        w = __all_sync(0xffffffffu, w);
+#else
         const bool w = mbar_wait(empty_bar(geo, s), eph, abort_flag, prm.status);
+#endif
 #ifdef COMPACT_PROFILE_GEN
         const long long g1 = clock64();
 #endif
+        if (warp == (THREADS_BASE >> 5)) TRACE(tile == first_tile, ks, 0);
         const int k0 = ks * BK;
-        if (w && gen_at) {
-          // A[m = column j of P][k = row i of P], MN-major: two 64-column blocks of [64 k][128 B]
-          const int kr0 = (int)crank * (BK >> csh);           // this CTA's rows of the tile
-          for (int id = gtid; id < (BK >> csh) * 16; id += GSTRIDE) {
-            const int c = id & 15, kr = kr0 + (id >> 4);
-            const uint4 val = projection8_bf16(prm.pp, k0 + kr, t.m0 + c * 8);
-            const uint32_t off = stage_off + STAGE_A0_OFF + (c >> 3) * 8192 + kr * 128 + (((c & 7) ^ (kr & 7)) << 4);
-            *reinterpret_cast<uint4*>(smem_gen + off) = val;
-            if (cs > 1) st_async_16(peer_base + off, val, peer_full + full_off);
-          }
-        }
-        if (w && gen_a) {
-          // A[m = row i of P][k = column j of P], K-major: [128 rows][128 B]
-          const int rr0 = (int)crank * (BM >> csh);           // this CTA's rows of the tile
-          for (int id = gtid; id < (BM >> csh) * 8; id += GSTRIDE) {
-            const int c = id & 7, rr = rr0 + (id >> 3);
-            const uint4 val = projection8_bf16(prm.pp, t.m0 + rr, k0 + c * 8);
-            const uint32_t off = stage_off + STAGE_A0_OFF + rr * 128 + ((c ^ (rr & 7)) << 4);
-            *reinterpret_cast<uint4*>(smem_gen + off) = val;
-            if (cs > 1) st_async_16(peer_base + off, val, peer_full + full_off);
+        int k1 = k0 + BK;
+        // Each pass turns this tile's words into Gaussians (Box-Muller: the MUFU pipe) and runs the Philox
+        // rounds of the next tile (the 32x32->64 multiply pipe; past the item's end the words are simply not
+        // used).  Half of the warps on every scheduler do the one first, half the other, so that the two pipes
+        // work at the same time instead of all warps queueing on one and then on the other.  The empty asm
+        // statements pin the order (and keep both parts on this side of the wait).
+        asm volatile("" : "+r"(k1));
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          if (u < ntask) {
+            uint4 val, nxa, nxb;
+            if (philox_first) {
+              projection8_words(prm.pp, t_i[u] + ik * k1, t_j[u] + jk * k1, nxa, nxb);
+              asm volatile("" : "+r"(xa[u].x) : "r"(nxa.x), "r"(nxb.x));
+              val = projection8_from_words(prm.pp, xa[u], xb[u], t_i[u] + ik * k0, t_j[u] + jk * k0);
+            } else {
+              asm volatile("" : "+r"(xa[u].x));
+              val = projection8_from_words(prm.pp, xa[u], xb[u], t_i[u] + ik * k0, t_j[u] + jk * k0);
+              asm volatile("" : "+r"(k1) : "r"(val.x), "r"(val.w));
+              projection8_words(prm.pp, t_i[u] + ik * k1, t_j[u] + jk * k1, nxa, nxb);
+            }
+            xa[u] = nxa; xb[u] = nxb;
+            if (w) {
+              const uint32_t off = stage_off + t_off[u];
+              *reinterpret_cast<uint4*>(smem_gen + off) = val;
+              if (cs > 1) st_async_16(peer_base + off, val, peer_full + full_off);
+            }
           }
         }
 #ifdef COMPACT_PROFILE_GEN
         const long long g2 = clock64();
 #endif
+        if (warp == (THREADS_BASE >> 5)) TRACE(tile == first_tile, ks, 1);
+        if (warp == (THREADS_BASE >> 5) + NUM_GEN_WARPS - 1) TRACE(tile == first_tile, ks, 3);
         fence_proxy_async_smem();
         ok = __all_sync(0xffffffffu, w);
         if (ok && lane == 0) mbar_arrive(full_bar(geo, s));
+        if (warp == (THREADS_BASE >> 5)) TRACE(tile == first_tile, ks, 2);
 #ifdef COMPACT_PROFILE_GEN
-        if (warp == (THREADS_BASE >> 5) && lane == 0) { atomicAdd(&g_prof[0], (unsigned long long)(g1 - g0)); atomicAdd(&g_prof[1], (unsigned long long)(g2 - g1)); atomicAdd(&g_prof[2], (unsigned long long)(clock64() - g2)); atomicAdd(&g_prof[3], 1ull); }
+        pg_wait += g1 - g0; pg_gen += g2 - g1; pg_arr += clock64() - g2; pg_cnt += 1;
 #endif
         // later stages of the k-step hold no generated data: the stage owner arrives for the generators there
       }
       if (geo) r1 = r; else r0 = r;
     }
+#ifdef COMPACT_PROFILE_GEN
+    if (warp == (THREADS_BASE >> 5) && lane == 0) {
+      atomicAdd(&g_prof[0], (unsigned long long)pg_wait); atomicAdd(&g_prof[1], (unsigned long long)pg_gen);
+      atomicAdd(&g_prof[2], (unsigned long long)pg_arr); atomicAdd(&g_prof[3], (unsigned long long)pg_cnt);
+    }
+#endif
   }
 
   tc_fence_before();
@@ -1194,7 +1293,8 @@ inline compact_status_t launch(const LaunchInfo& li, Params& prm) {
     }
     attr_set = true;
   }
-  const int cs = (prm.gen_ring != GEN_NONE && li.cluster > 1) ? li.cluster : 1;
+  // sharing generated tiles needs the four-stage ring, where a stage keeps its role (see the stage owner)
+  const int cs = (prm.gen_ring != GEN_NONE && li.cluster > 1 && prm.prob[0].geo == 1) ? 2 : 1;
   prm.cs = cs;
   if (cs > 1) {
     // the generated problem is problem 0; its items come in groups of cs neighbours
