@@ -673,11 +673,9 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const bool active = split || iss == 0;
         if (slots == 2 && acc == 1) {
           // a two-slot item starts at slot 0: pass slot 1 through unused
-          if (iss == 0) {
-            if (!(ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(1), acc_phase ^ 1, abort_flag, prm.status)))) break;
-            if (elect_one()) umma_commit(tfull_bar(1));
-            __syncwarp();
-          }
+          if (!(ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(1), acc_phase ^ 1, abort_flag, prm.status)))) break;
+          if (iss == 0 && elect_one()) umma_commit(tfull_bar(1));
+          __syncwarp();
           acc = 0;
           acc_phase ^= 1;
         }
@@ -686,8 +684,10 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         long long mwait = 0, missue = 0;
 #endif
         for (int sl = 0; sl < slots && ok; ++sl) {
-          // a split item's issuer x waits for slot x only
-          if (active && (!split || sl == iss))
+          // a split item's issuer x waits for slot x only; an issuer without work in the item waits all the
+          // same, so that it never runs more than a phase ahead of these barriers (a parity wait is only
+          // sound one phase ahead)
+          if (!split || sl == iss)
             ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(acc), acc_phase ^ 1, abort_flag, prm.status));
           if (++acc == 2) { acc = 0; acc_phase ^= 1; }
         }
