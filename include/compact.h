@@ -115,7 +115,10 @@ compact_status_t compact_linear_bwd(compact_layer_t* layer, int64_t tokens,
  * stored moments are the uncorrected running averages and the bias correction
  * uses the 1-based count of this update.  epoch_of_Gc must equal the layer's
  * current epoch (the one the forward reported).  lr = NaN uses the config's.
- * Increments the layer's step. */
+ * Increments the layer's step.  bf16 layers on the tensor-core path form the
+ * increment -eta * alpha * (P N) in fp32, round it to bf16 and add it to W with
+ * one more rounding (the add is done by the TMA unit at the L2, so W makes one
+ * trip instead of two); fp32 layers and the SIMT path round W once. */
 compact_status_t compact_adam_update(compact_layer_t* layer,
                                      void* W, int64_t ldw,
                                      const float* Gc, int64_t ldg,

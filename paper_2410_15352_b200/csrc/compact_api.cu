@@ -446,6 +446,11 @@ void compact_debug_trace(long long* out) {
   cudaDeviceSynchronize();
   cudaMemcpyFromSymbol(out, tc::g_trace, sizeof(long long) * 128);
 }
+void compact_debug_timeline(long long* out, unsigned int* n) {
+  cudaDeviceSynchronize();
+  cudaMemcpyFromSymbol(out, tc::g_tl, sizeof(long long) * 128);
+  cudaMemcpyFromSymbol(n, tc::g_tl_n, sizeof(unsigned int));
+}
 #endif
 
 const char* compact_status_string(compact_status_t s) {

@@ -85,6 +85,8 @@ __device__ unsigned long long g_prof[8];
 #ifdef COMPACT_PROFILE_GEN
 // event trace of CTA 0, first item, k-steps 16..23
 __device__ long long g_trace[8][16];
+__device__ long long g_tl[64][2];      // start and end (globaltimer) of the last 64 launches, by CTA 0
+__device__ unsigned int g_tl_n;
 #define TRACE(first_item, ks, ev)                                                              \
   do {                                                                                         \
     if (blockIdx.x == 0 && (first_item) && (ks) >= 16 && (ks) < 24 && (threadIdx.x & 31) == 0) \
@@ -202,6 +204,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src), "r"(x),
                "r"(y)
+               : "memory");
+}
+// global tile += shared tile, element-wise in the tensor map's type (bf16), done by the TMA unit at the L2
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map),
+               "r"(src), "r"(x), "r"(y)
                : "memory");
 }
 __device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int x, int y, int z) {
@@ -387,6 +395,12 @@ __device__ __forceinline__ TileCoord decode_tile(const Params& prm, int tile) {
 // --------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __grid_constant__ Params prm) {
   extern __shared__ uint8_t smem_raw[];
+#ifdef COMPACT_PROFILE_GEN
+  auto gtime = []() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return (long long)t; };
+  if (threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == 147)) g_trace[6][blockIdx.x == 0 ? 0 : 8] = gtime();
+  __shared__ unsigned int tl_slot;
+  if (threadIdx.x == 0 && blockIdx.x == 0) { tl_slot = atomicAdd(&g_tl_n, 1u) & 63u; g_tl[tl_slot][0] = gtime(); }
+#endif
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));   // generic pointer to the aligned base
   const uint32_t staging = smem_base + RING_BYTES;
@@ -444,6 +458,9 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
   __syncthreads();
   tc_fence_after();
   if (cs > 1) cluster_sync_all();          // every CTA's barriers exist before anything crosses CTAs
+#ifdef COMPACT_PROFILE_GEN
+  if (threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == 147)) g_trace[6][blockIdx.x == 0 ? 1 : 9] = gtime();
+#endif
   const uint32_t tmem_base = *tmem_slot;
 
   // Every consumer role reads the next item from the queue the scheduler fills.
@@ -658,6 +675,12 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
           atomicAdd(&g_prof[6], (unsigned long long)qwait);
           atomicAdd(&g_prof[7], (unsigned long long)nitems);
         }
+        if (tile < 0 && lane == 0 && iss == 0 && has_gen) {
+          atomicAdd((unsigned long long*)&g_trace[7][0], (unsigned long long)(clock64() - life0));
+          atomicAdd((unsigned long long*)&g_trace[7][1], (unsigned long long)twait);
+          atomicAdd((unsigned long long*)&g_trace[7][2], (unsigned long long)qwait);
+          atomicAdd((unsigned long long*)&g_trace[7][3], (unsigned long long)nitems);
+        }
         ++nitems;
         const long long t0c = clock64();
 #endif
@@ -813,8 +836,6 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
     const int eset = (warp - 2) >> 2;       // 0 or 1
     const uint32_t stg = staging + (warp - 2) * STAGING_BYTES;
     uint8_t* stg_gen = smem_gen + RING_BYTES + (warp - 2) * STAGING_BYTES;
-    const uint32_t my_wbar = wbar(warp - 2);
-    uint32_t wph = 0;
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
@@ -856,16 +877,24 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
           for (int ci = (slots == 2 ? 0 : eset); ci < cpa && ok; ci += (slots == 2 ? 1 : 2)) {
             const int col = ncol0 + ci * cw;
             if (col >= p.N) break;
-            if (p.epi_mode == EPI_BF16) {
-              // convert the whole chunk first; the previous store's read of the staging tile hides behind it
+            if (p.epi_mode == EPI_BF16 || p.epi_mode == EPI_UPDATE_W) {
+              // convert the whole chunk first; the previous store's read of the staging tile hides behind it.
+              // The update stages -(eta alpha) (P N) and lets the TMA unit add it to W (Algorithm 3 line 9).
               uint32_t o[32];
 #pragma unroll
               for (int h = 0; h < 2; ++h) {
                 uint32_t v[32];
                 tmem_ld32(tcol + ci * cw + 32 * h, v);
                 tmem_ld_wait();
+                if (p.epi_mode == EPI_UPDATE_W) {
+                  const float sc = -p.scale;
 #pragma unroll
-                for (int j = 0; j < 16; ++j) o[16 * h + j] = pack_bf16x2(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+                  for (int j = 0; j < 16; ++j)
+                    o[16 * h + j] = pack_bf16x2(sc * __uint_as_float(v[2 * j]), sc * __uint_as_float(v[2 * j + 1]));
+                } else {
+#pragma unroll
+                  for (int j = 0; j < 16; ++j) o[16 * h + j] = pack_bf16x2(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+                }
               }
               if (lane == 0) tma_store_wait_read();
               __syncwarp();
@@ -878,7 +907,8 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
               fence_proxy_async_smem();
               __syncwarp();
               if (lane == 0) {
-                tma_store_2d(mapC, stg, col, row0);
+                if (p.epi_mode == EPI_UPDATE_W) tma_reduce_add_2d(mapC, stg, col, row0);
+                else tma_store_2d(mapC, stg, col, row0);
                 tma_store_commit();
               }
               continue;
@@ -901,13 +931,6 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
               }
               continue;
             }
-            if (p.epi_mode == EPI_UPDATE_W) {
-              // bring the W tile in first: W <- W - (eta alpha) (P N), one rounding (Algorithm 3 line 9)
-              if (lane == 0) {
-                mbar_arrive_expect_tx(my_wbar, STAGING_BYTES);
-                tma_load_2d(stg, mapC, my_wbar, col, row0);
-              }
-            }
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
               uint32_t v[32];
@@ -928,22 +951,6 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
                 for (int z = 0; z < 32; ++z)
                   *reinterpret_cast<__nv_bfloat16*>(stg_gen + (32 * h + z) * 64 + lane * 2) =
                       __float2bfloat16_rn(__uint_as_float(v[z]));
-              } else if (p.epi_mode == EPI_UPDATE_W) {
-                if (h == 0) {
-                  if (!(ok = mbar_wait(my_wbar, wph, abort_flag, prm.status))) break;
-                  wph ^= 1;
-                }
-                const float sc = -p.scale;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  uint4* cell = reinterpret_cast<uint4*>(stg_gen + lane * 128 + (((4 * h + j) ^ sw) << 4));
-                  uint4 w = *cell;
-                  w.x = pack_bf16x2(fmaf(sc, __uint_as_float(v[8 * j + 0]), bf16lo(w.x)), fmaf(sc, __uint_as_float(v[8 * j + 1]), bf16hi(w.x)));
-                  w.y = pack_bf16x2(fmaf(sc, __uint_as_float(v[8 * j + 2]), bf16lo(w.y)), fmaf(sc, __uint_as_float(v[8 * j + 3]), bf16hi(w.y)));
-                  w.z = pack_bf16x2(fmaf(sc, __uint_as_float(v[8 * j + 4]), bf16lo(w.z)), fmaf(sc, __uint_as_float(v[8 * j + 5]), bf16hi(w.z)));
-                  w.w = pack_bf16x2(fmaf(sc, __uint_as_float(v[8 * j + 6]), bf16lo(w.w)), fmaf(sc, __uint_as_float(v[8 * j + 7]), bf16hi(w.w)));
-                  *cell = w;
-                }
               }
             }
             if (!ok) break;
@@ -1101,8 +1108,15 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
 #endif
   }
 
+#ifdef COMPACT_PROFILE_GEN
+  if (threadIdx.x == 32 && (blockIdx.x == 0 || blockIdx.x == 147)) g_trace[6][blockIdx.x == 0 ? 2 : 10] = gtime();
+#endif
   tc_fence_before();
   __syncthreads();
+#ifdef COMPACT_PROFILE_GEN
+  if (threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == 147)) g_trace[6][blockIdx.x == 0 ? 3 : 11] = gtime();
+  if (threadIdx.x == 0 && blockIdx.x == 0) g_tl[tl_slot][1] = gtime();
+#endif
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
