@@ -91,7 +91,9 @@ size_t compact_saved_bytes(const compact_layer_t* layer, int64_t tokens);
 
 /* Algorithm 1.  Y[tokens x m] = X W and Z[tokens x ldz] = X P, both rounded once
  * from fp32 accumulators.  Row t of Z belongs to row t of X.  *epoch_used
- * (host pointer, may be NULL) receives the epoch P was generated with. */
+ * (host pointer, may be NULL) receives the epoch P was generated with.
+ * Z may be NULL: then nothing is kept for the backward, which must be
+ * compact_linear_bwd_recompute (for layers under activation checkpointing). */
 compact_status_t compact_linear_fwd(compact_layer_t* layer, int64_t tokens,
                                     const void* X, int64_t ldx,
                                     const void* W, int64_t ldw,
@@ -110,6 +112,23 @@ compact_status_t compact_linear_bwd(compact_layer_t* layer, int64_t tokens,
                                     void* dX, int64_t lddx,
                                     float* Gc, int64_t ldg, int accumulate,
                                     void* workspace, size_t workspace_bytes, void* stream);
+
+/* Algorithm 2 without a stored z: recomputes Z = X P (the projection of epoch
+ * epoch_of_fwd, which must be the layer's current epoch) into the workspace and
+ * then does what compact_linear_bwd does.  This is the combination with
+ * activation checkpointing that the paper's Limitations section proposes
+ * ("recomputing the activation compression during the backward pass"): the
+ * checkpointed segment recomputes X anyway, so z need not be kept at all.
+ * Results are bitwise those of compact_linear_fwd + compact_linear_bwd.
+ * workspace: at least compact_recompute_workspace_bytes(layer, tokens). */
+size_t compact_recompute_workspace_bytes(const compact_layer_t* layer, int64_t tokens);
+compact_status_t compact_linear_bwd_recompute(compact_layer_t* layer, int64_t tokens,
+                                              const void* X, int64_t ldx, uint32_t epoch_of_fwd,
+                                              const void* dY, int64_t lddy,
+                                              const void* W, int64_t ldw,
+                                              void* dX, int64_t lddx,
+                                              float* Gc, int64_t ldg, int accumulate,
+                                              void* workspace, size_t workspace_bytes, void* stream);
 
 /* Algorithm 3 lines 1-10.  In place on W, M, V (M, V: r x m fp32, pitch ldg);
  * stored moments are the uncorrected running averages and the bias correction

@@ -152,6 +152,14 @@ def linear_bwd(dY: np.ndarray, Z: np.ndarray, W: np.ndarray, mode: str = "exact"
     return _store(dX, mode), Gc
 
 
+def linear_bwd_recompute(X: np.ndarray, dY: np.ndarray, W: np.ndarray, P: np.ndarray, mode: str = "exact"):
+    """Algorithm 2 when no z was kept (the combination with activation checkpointing proposed in the
+    Limitations section): z = x P is formed again from the recomputed x, as line 4 of Algorithm 1 does,
+    and then the two products of Algorithm 2 follow."""
+    Z = _store(np.asarray(X, dtype=np.float64) @ np.asarray(P, dtype=np.float64), mode)
+    return linear_bwd(dY, Z, W, mode)
+
+
 def adam_update(W, Gc, M, V, t: int, P, lr: float, beta1: float, beta2: float, eps: float,
                 alpha: float = 1.0, mode: str = "exact"):
     """Algorithm 3 lines 1-9 for the update whose 1-based count is t.
@@ -212,6 +220,9 @@ class CompActLayerOracle:
 
     def backward(self, dY, Z):
         return linear_bwd(dY, Z, self.W, self.mode)
+
+    def backward_recompute(self, X, dY):
+        return linear_bwd_recompute(X, dY, self.W, self.P(), self.mode)
 
     def update(self, Gc, lr: float | None = None) -> None:
         t = self.state.step + 1

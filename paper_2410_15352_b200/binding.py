@@ -25,7 +25,8 @@ F32, BF16 = 0, 1
 
 EXPORTS = [
     "compact_layer_create", "compact_layer_destroy", "compact_z_ld", "compact_workspace_bytes",
-    "compact_saved_bytes", "compact_linear_fwd", "compact_linear_bwd", "compact_adam_update", "compact_adam_update_noalloc",
+    "compact_saved_bytes", "compact_linear_fwd", "compact_linear_bwd", "compact_recompute_workspace_bytes",
+    "compact_linear_bwd_recompute", "compact_adam_update", "compact_adam_update_noalloc",
     "compact_refresh_projection", "compact_layer_get_state", "compact_layer_set_state",
     "compact_layer_status", "compact_debug_philox_u32", "compact_debug_projection",
     "compact_set_kernel_family", "compact_kernel_launch_count", "compact_status_string",
@@ -67,6 +68,10 @@ def lib() -> C.CDLL:
     L.compact_linear_fwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, i64, u32p, vp]
     L.compact_linear_bwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, i64, vp, i64, C.c_int, vp,
                                      C.c_size_t, vp]
+    L.compact_recompute_workspace_bytes.argtypes = [vp, i64]
+    L.compact_recompute_workspace_bytes.restype = C.c_size_t
+    L.compact_linear_bwd_recompute.argtypes = [vp, i64, vp, i64, C.c_uint32, vp, i64, vp, i64, vp, i64, vp, i64, C.c_int,
+                                               vp, C.c_size_t, vp]
     L.compact_adam_update.argtypes = [vp, vp, i64, vp, i64, vp, vp, C.c_uint32, C.c_float, vp, C.c_size_t, vp]
     L.compact_adam_update_noalloc.argtypes = [vp, vp, i64, vp, i64, vp, vp, C.c_uint32, C.c_float, vp]
     L.compact_refresh_projection.argtypes = [vp, C.c_int, u32p]
@@ -179,16 +184,18 @@ class CompactLinear:
 
     # -- Algorithm 1 ---------------------------------------------------------------
     def forward(self, X: torch.Tensor, W: torch.Tensor, Y: Optional[torch.Tensor] = None,
-                Z: Optional[torch.Tensor] = None, stream=None):
+                Z: Optional[torch.Tensor] = None, keep_z: bool = True, stream=None):
+        """keep_z=False: nothing is kept for the backward (returns Z=None); use backward_recompute."""
         tokens = X.shape[0]
         if Y is None:
             Y = torch.empty((tokens, self.m), dtype=self.dtype, device=X.device)
-        if Z is None:
+        if Z is None and keep_z:
             Z = torch.empty((tokens, self.ldz), dtype=self.dtype, device=X.device)
         ep = C.c_uint32()
         _check(lib().compact_linear_fwd(self._h, tokens, _ptr(X), X.stride(0) if tokens else self.n, _ptr(W),
                                         W.stride(0), _ptr(Y), Y.stride(0) if tokens else self.m, _ptr(Z),
-                                        Z.stride(0) if tokens else self.ldz, C.byref(ep), _stream(stream)),
+                                        (Z.stride(0) if tokens else self.ldz) if Z is not None else 0, C.byref(ep),
+                                        _stream(stream)),
                "compact_linear_fwd")
         return Y, Z, int(ep.value)
 
@@ -206,6 +213,28 @@ class CompactLinear:
                                         (dX.stride(0) if tokens else self.n) if dX is not None else 0, _ptr(Gc),
                                         Gc.stride(0), int(accumulate), _ptr(ws), ws.numel(), _stream(stream)),
                "compact_linear_bwd")
+        return dX, Gc
+
+    def backward_recompute(self, X: torch.Tensor, epoch_of_fwd: int, dY: torch.Tensor, W: torch.Tensor,
+                           Gc: Optional[torch.Tensor] = None, dX: Optional[torch.Tensor] = None, need_dX: bool = True,
+                           accumulate: bool = False, stream=None):
+        """Algorithm 2 for a forward that kept no Z: Z = X P is computed again into scratch."""
+        tokens = dY.shape[0]
+        if Gc is None:
+            Gc = torch.empty((self.r, self.m), dtype=torch.float32, device=dY.device)
+        if dX is None and need_dX:
+            dX = torch.empty((tokens, self.n), dtype=self.dtype, device=dY.device)
+        need = max(int(lib().compact_recompute_workspace_bytes(self._h, tokens)), 256)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+        ws = self._ws
+        _check(lib().compact_linear_bwd_recompute(self._h, tokens, _ptr(X), X.stride(0) if tokens else self.n,
+                                                  epoch_of_fwd, _ptr(dY), dY.stride(0) if tokens else self.m, _ptr(W),
+                                                  W.stride(0), _ptr(dX),
+                                                  (dX.stride(0) if tokens else self.n) if dX is not None else 0,
+                                                  _ptr(Gc), Gc.stride(0), int(accumulate), _ptr(ws), ws.numel(),
+                                                  _stream(stream)),
+               "compact_linear_bwd_recompute")
         return dX, Gc
 
     # -- Algorithm 3 ---------------------------------------------------------------

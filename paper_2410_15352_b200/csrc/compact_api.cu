@@ -106,7 +106,8 @@ compact_status_t fwd_simt(compact_layer_t* L, int64_t tokens, const T* X, int64_
                           T* Y, int64_t ldy, T* Z, int64_t ldz, cudaStream_t st) {
   constexpr bool kBf16 = sizeof(T) == 2;
   const int n = L->cfg.n, m = L->cfg.m, r = L->cfg.r;
-  simt_gemm((int)tokens, m, n, simt::RowMajor<T>{X, ldx}, simt::Transposed<T>{W, ldw}, simt::StoreAs<T>{Y, ldy}, st);
+  if (Y) simt_gemm((int)tokens, m, n, simt::RowMajor<T>{X, ldx}, simt::Transposed<T>{W, ldw}, simt::StoreAs<T>{Y, ldy}, st);
+  if (!Z) return launch_result();
   simt::GeneratedP<kBf16, true> gp{make_pp(L, L->epoch)};
   simt_gemm((int)tokens, r, n, simt::RowMajor<T>{X, ldx}, gp, simt::StoreAs<T>{Z, ldz}, st);
   const int zc = (int)compact_z_ld(L);
@@ -212,11 +213,11 @@ compact_status_t compact_linear_fwd(compact_layer_t* L, int64_t tokens, const vo
   if (!L || tokens < 0 || tokens > 0x7fffffff) return COMPACT_ERR_INVALID_ARG;
   if (epoch_used) *epoch_used = L->epoch;
   if (tokens == 0) return COMPACT_OK;
-  if (!X || !W || !Y || !Z) return COMPACT_ERR_INVALID_ARG;
+  if (!X || !W || !Y) return COMPACT_ERR_INVALID_ARG;
   const size_t es = elem_size(L->cfg.dtype);
-  if (!aligned16(X) || !aligned16(W) || !aligned16(Y) || !aligned16(Z)) return COMPACT_ERR_ALIGNMENT;
+  if (!aligned16(X) || !aligned16(W) || !aligned16(Y) || (Z && !aligned16(Z))) return COMPACT_ERR_ALIGNMENT;
   if (!pitch_ok(ldx, L->cfg.n, es) || !pitch_ok(ldw, L->cfg.m, es) || !pitch_ok(ldy, L->cfg.m, es) ||
-      !pitch_ok(ldz, compact_z_ld(L), es))
+      (Z && !pitch_ok(ldz, compact_z_ld(L), es)))
     return COMPACT_ERR_ALIGNMENT;
   compact_status_t s = check_device(L);
   if (s != COMPACT_OK) return s;
@@ -276,6 +277,49 @@ compact_status_t compact_linear_bwd(compact_layer_t* L, int64_t tokens, const vo
   }
   return bwd_simt<float>(L, tokens, (const float*)dY, lddy, (const float*)Z, ldz, (const float*)W, ldw, (float*)dX,
                          lddx, Gc, ldg, accumulate, st);
+}
+
+size_t compact_recompute_workspace_bytes(const compact_layer_t* layer, int64_t tokens) {
+  if (!layer || tokens < 0) return 0;
+  return (size_t)round_up((int64_t)compact_saved_bytes(layer, tokens), 256) + compact_workspace_bytes(layer, tokens);
+}
+
+compact_status_t compact_linear_bwd_recompute(compact_layer_t* L, int64_t tokens, const void* X, int64_t ldx,
+                                              uint32_t epoch_of_fwd, const void* dY, int64_t lddy, const void* W,
+                                              int64_t ldw, void* dX, int64_t lddx, float* Gc, int64_t ldg, int accumulate,
+                                              void* workspace, size_t workspace_bytes, void* stream) {
+  if (!L || tokens < 0 || tokens > 0x7fffffff) return COMPACT_ERR_INVALID_ARG;
+  if (epoch_of_fwd != L->epoch) return COMPACT_ERR_EPOCH_MISMATCH;
+  const int64_t ldz = compact_z_ld(L);
+  const size_t zbytes = (size_t)round_up((int64_t)compact_saved_bytes(L, tokens), 256);
+  if (tokens > 0) {
+    if (!X) return COMPACT_ERR_INVALID_ARG;
+    const size_t es = elem_size(L->cfg.dtype);
+    if (!aligned16(X) || !pitch_ok(ldx, L->cfg.n, es)) return COMPACT_ERR_ALIGNMENT;
+    if (!workspace || workspace_bytes < compact_recompute_workspace_bytes(L, tokens)) return COMPACT_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return COMPACT_ERR_ALIGNMENT;
+    compact_status_t s = check_device(L);
+    if (s != COMPACT_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    // Z = X P again, into the front of the workspace
+    if (L->cfg.dtype == COMPACT_BF16) {
+      typedef __nv_bfloat16 T;
+      s = COMPACT_ERR_SHAPE;
+      if (g_family.load() != 1) {
+        tc::LaunchInfo li{g_family.load() == 2 ? 1 : CFG_CS, st, status_word(L), sched_words(L), &g_launches};
+        s = tc::forward(li, make_pp(L, L->epoch), tokens, L->cfg.m, (const T*)X, ldx, nullptr, 0, nullptr, 0, (T*)workspace, ldz,
+                        (int)ldz);
+      }
+      if (s == COMPACT_ERR_SHAPE)
+        s = fwd_simt<T>(L, tokens, (const T*)X, ldx, nullptr, 0, nullptr, 0, (T*)workspace, ldz, st);
+    } else {
+      s = fwd_simt<float>(L, tokens, (const float*)X, ldx, nullptr, 0, nullptr, 0, (float*)workspace, ldz, st);
+    }
+    if (s != COMPACT_OK) return s;
+  }
+  return compact_linear_bwd(L, tokens, dY, lddy, workspace, ldz, W, ldw, dX, lddx, Gc, ldg, accumulate,
+                            tokens > 0 ? (char*)workspace + zbytes : workspace,
+                            tokens > 0 ? workspace_bytes - zbytes : workspace_bytes, stream);
 }
 
 compact_status_t compact_adam_update(compact_layer_t* L, void* W, int64_t ldw, const float* Gc, int64_t ldg, float* M,

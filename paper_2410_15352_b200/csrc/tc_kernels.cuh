@@ -1353,39 +1353,48 @@ inline compact_status_t launch(const LaunchInfo& li, Params& prm) {
 
 inline bool tc_shape_ok(int64_t tokens, int n, int m) { return tokens >= 1 && n % 8 == 0 && m % 8 == 0; }
 
-// Algorithm 1: problem 0 = Z = X P (generated B operand; longest items go first), problem 1 = Y = X W.
+// Algorithm 1: problem 0 = Z = X P (generated operand; longest items go first), problem 1 = Y = X W.
+// Either output may be absent (nullptr): Y alone is the forward of a layer that will recompute Z in its
+// backward, Z alone is that recomputation.
 inline compact_status_t forward(const LaunchInfo& li, const ProjectionParams& pp, int64_t tokens, int m,
                                 const __nv_bfloat16* X, int64_t ldx, const __nv_bfloat16* W, int64_t ldw,
                                 __nv_bfloat16* Y, int64_t ldy, __nv_bfloat16* Z, int64_t ldz, int zcols) {
   const int n = pp.n;
   if (!tc_shape_ok(tokens, n, m)) return COMPACT_ERR_SHAPE;
   if (!li.status || !li.sched) return COMPACT_ERR_CUDA;
+  if (!Y && !Z) return COMPACT_OK;
   Params prm;
   memset(&prm, 0, sizeof(prm));
   prm.pp = pp;
-  prm.num_problems = 2;
-  prm.gen_ring = GEN_A;
-  // Z is computed transposed, Z^T = P^T X^T: the generated tile of P (64 rows of P by 128 of its columns)
-  // is the A operand, and up to 512 tokens of X ride on the N side in two 256-wide accumulators, so the
-  // MMAs run at N = 256 and one generated tile feeds 512 tokens.
-  Problem& pz = prm.prob[0];
-  pz.M = zcols; pz.N = (int)tokens; pz.K = n;
-  pz.nsub = 1;
-  pz.ncol = tokens > BN_MAX ? 2 : 1;
-  pz.a_mode = GENERATED_T; pz.b_mode = TMA_KMAJOR; pz.epi_mode = EPI_BF16_T;
-  finish_problem(pz, 1);
-  Problem& py = prm.prob[1];
-  py.M = (int)tokens; py.N = m; py.K = n;
-  py.a_mode = TMA_KMAJOR; py.b_mode = TMA_MNMAJOR; py.epi_mode = EPI_BF16;
-  finish_problem(py, 1);
-  if (!make_map(&prm.tmA[1], X, n, tokens, ldx, BK, BM)) return COMPACT_ERR_CUDA;
-  prm.tmA[0] = prm.tmA[1];   // unused by the generated operand
-  if (!make_map(&prm.tmB[0], X, n, tokens, ldx, BK, pz.bn)) return COMPACT_ERR_CUDA;
-  py.b_blocked = m % 64 == 0;
-  if (py.b_blocked ? !make_map_blocked(&prm.tmB[1], W, m, n, ldw, BK, py.bn / 64) : !make_map(&prm.tmB[1], W, m, n, ldw, 64, BK))
-    return COMPACT_ERR_CUDA;
-  if (!make_map(&prm.tmC[0], Z, zcols, tokens, ldz, 32, 64, false)) return COMPACT_ERR_CUDA;
-  if (!make_map(&prm.tmC[1], Y, m, tokens, ldy, 64, 32)) return COMPACT_ERR_CUDA;
+  prm.num_problems = (Y && Z) ? 2 : 1;
+  prm.gen_ring = Z ? GEN_A : GEN_NONE;
+  const int iy = Z ? 1 : 0;       // where the Y problem sits
+  if (Z) {
+    // Z is computed transposed, Z^T = P^T X^T: the generated tile of P (64 rows of P by 128 of its columns)
+    // is the A operand, and up to 512 tokens of X ride on the N side in two 256-wide accumulators, so the
+    // MMAs run at N = 256 and one generated tile feeds 512 tokens.
+    Problem& pz = prm.prob[0];
+    pz.M = zcols; pz.N = (int)tokens; pz.K = n;
+    pz.nsub = 1;
+    pz.ncol = tokens > BN_MAX ? 2 : 1;
+    pz.a_mode = GENERATED_T; pz.b_mode = TMA_KMAJOR; pz.epi_mode = EPI_BF16_T;
+    finish_problem(pz, 1);
+    prm.tmA[0] = prm.tmA[iy];   // unused by the generated operand (set below when Y is present)
+    if (!make_map(&prm.tmB[0], X, n, tokens, ldx, BK, pz.bn)) return COMPACT_ERR_CUDA;
+    if (!make_map(&prm.tmC[0], Z, zcols, tokens, ldz, 32, 64, false)) return COMPACT_ERR_CUDA;
+  }
+  if (Y) {
+    Problem& py = prm.prob[iy];
+    py.M = (int)tokens; py.N = m; py.K = n;
+    py.a_mode = TMA_KMAJOR; py.b_mode = TMA_MNMAJOR; py.epi_mode = EPI_BF16;
+    finish_problem(py, 1);
+    if (!make_map(&prm.tmA[iy], X, n, tokens, ldx, BK, BM)) return COMPACT_ERR_CUDA;
+    py.b_blocked = m % 64 == 0;
+    if (py.b_blocked ? !make_map_blocked(&prm.tmB[iy], W, m, n, ldw, BK, py.bn / 64) : !make_map(&prm.tmB[iy], W, m, n, ldw, 64, BK))
+      return COMPACT_ERR_CUDA;
+    if (!make_map(&prm.tmC[iy], Y, m, tokens, ldy, 64, 32)) return COMPACT_ERR_CUDA;
+  }
+  if (Z) prm.tmA[0] = prm.tmB[0];   // any valid map: the loader never uses it for a generated operand
   return launch(li, prm);
 }
 

@@ -244,6 +244,29 @@ def test_dx_is_gradient_of_inner_product():
         assert dX[t, k] == pytest.approx(fd, rel=1e-7)
 
 
+def test_bwd_recompute_is_the_sketched_gradient_by_brute_force():
+    # without a stored z the compressed gradient is still P^T (X^T dY): element loops on a tiny case,
+    # and with r = n and an orthonormal P the full gradient comes back
+    rng = np.random.default_rng(8)
+    bl, n, m, r = 7, 6, 5, 3
+    X, W, dY = rng.standard_normal((bl, n)), rng.standard_normal((n, m)), rng.standard_normal((bl, m))
+    P = co.projection(11, 2, 1, n, r)
+    dX, Gc = co.linear_bwd_recompute(X, dY, W, P)
+    for j in range(r):
+        for c in range(m):
+            want = sum(P[i, j] * X[t, i] * dY[t, c] for t in range(bl) for i in range(n))
+            assert Gc[j, c] == pytest.approx(want, rel=1e-12, abs=1e-13)
+    for t in range(bl):
+        for i in range(n):
+            assert dX[t, i] == pytest.approx(sum(dY[t, c] * W[i, c] for c in range(m)), rel=1e-12, abs=1e-13)
+    Q, _ = np.linalg.qr(co.projection(4, 0, 0, n, n))
+    _, Gq = co.linear_bwd_recompute(X, dY, W, Q)
+    assert np.allclose(Q @ Gq, X.T @ dY, rtol=1e-12, atol=1e-12)
+    # bf16 storage: z is rounded where Algorithm 1 would have stored it
+    _, Gb = co.linear_bwd_recompute(X, dY, W, P, mode="bf16")
+    assert np.array_equal(Gb, co.linear_bwd(dY, co.round_bf16(X @ P), W, mode="bf16")[1])
+
+
 # --- Adam ----------------------------------------------------------------------------
 def test_adam_constant_gradient_closed_form():
     rng = np.random.default_rng(4)

@@ -214,6 +214,47 @@ def test_padded_pitches(family):
     assert torch.all(W._base[:, m:] == 7.0)
 
 
+def test_backward_recompute_matches_stored_z_bitwise_and_oracle(family):
+    # a forward that keeps no Z, then Algorithm 2 with Z recomputed from X
+    tokens, n, m, r = 1100, 320, 520, 72
+    wl = wlm.Workload("rec", 97, "bf16", tokens, [wlm.LayerShape("l", n, m, r)], x_scale_inv_sqrt_n=True)
+    gpu, ora, W0 = make_pair(wl, 0)
+    W = W0.cuda()
+    X, dY = wlm.draw_X(wl, 0, 0).cuda(), wlm.draw_dY(wl, 0, 0).cuda()
+    Y1, Z1, ep = gpu.forward(X, W)
+    dX1, G1 = gpu.backward(dY, Z1, W)
+    Y2, Z2, ep2 = gpu.forward(X, W, keep_z=False)
+    assert Z2 is None and ep2 == ep
+    assert torch.equal(Y1.view(torch.int16), Y2.view(torch.int16))
+    dX2, G2 = gpu.backward_recompute(X, ep, dY, W)
+    assert torch.equal(G1, G2) and torch.equal(dX1.view(torch.int16), dX2.view(torch.int16))
+    dXo, Gco = ora.backward_recompute(to64(X), to64(dY))
+    assert co.rel_frobenius(to64(G2), Gco) <= TOL["bf16"]
+    assert co.rel_frobenius(to64(dX2), dXo) <= TOL["bf16"]
+    # micro-batches accumulate as with a stored Z
+    Ga = torch.empty_like(G1)
+    h = 512
+    gpu.backward_recompute(X[:h], ep, dY[:h], W, Gc=Ga, need_dX=False)
+    gpu.backward_recompute(X[h:], ep, dY[h:], W, Gc=Ga, need_dX=False, accumulate=True)
+    assert co.rel_frobenius(to64(Ga), Gco) <= TOL["bf16"]
+    # the projection of another epoch is refused
+    with pytest.raises(cb.CompactError) as e:
+        gpu.backward_recompute(X, ep + 1, dY, W)
+    assert e.value.code == cb.ERR_EPOCH_MISMATCH
+
+
+def test_backward_recompute_fp32():
+    tokens, n, m, r = 96, 64, 40, 12
+    wl = wlm.Workload("rec32", 96, "f32", tokens, [wlm.LayerShape("l", n, m, r)])
+    gpu, ora, W0 = make_pair(wl, 0)
+    W = W0.cuda()
+    X, dY = wlm.draw_X(wl, 0, 0).cuda(), wlm.draw_dY(wl, 0, 0).cuda()
+    _, _, ep = gpu.forward(X, W, keep_z=False)
+    dX, Gc = gpu.backward_recompute(X, ep, dY, W)
+    dXo, Gco = ora.backward_recompute(to64(X), to64(dY))
+    assert co.rel_frobenius(to64(Gc), Gco) <= TOL["f32"] and co.rel_frobenius(to64(dX), dXo) <= TOL["f32"]
+
+
 def test_empty_batch_and_epoch_guard():
     lay = cb.CompactLinear(128, 512, 16, refresh_T=1)
     W = torch.zeros((128, 512), dtype=torch.bfloat16, device="cuda")
