@@ -3,10 +3,12 @@
 // with fp32 accumulators in TMEM -> tcgen05.ld -> swizzled staging -> TMA store)
 // whose operands come from TMA in either major-ness or from the in-kernel
 // Philox/Box-Muller generator of P.  It serves
-//   forward  : [Y | Z] = X [W | P]        (Algorithm 1; P tiles generated as the B operand)
+//   forward  : [Y | Z] = X [W | P]        (Algorithm 1; Z computed as Z^T = P^T X^T, P tiles generated as A)
 //   backward : dX = dY W^T and Gc = Z^T dY (Algorithm 2; Gc split over tokens)
 //   update   : W <- W - eta alpha P N      (Algorithm 3 lines 6-9; P tiles generated as A)
-// Work items are handed out dynamically (one atomic counter per launch), longest first.
+// Launches with a generated operand run as clusters of two CTAs that share every generated tile.
+// Work items are numbered longest first; those with a generated operand are dealt statically to the
+// clusters, the rest come from one atomic counter per launch.
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -67,16 +69,15 @@ constexpr int NUM_BARRIERS = NUM_RING_BARS + 4 + 2 * QDEPTH + NUM_EPI_WARPS * ST
 constexpr int TAIL_BYTES = 8 * NUM_BARRIERS + 4 * QDEPTH + 16;
 constexpr int SMEM_BYTES = 1024 + RING_BYTES + NUM_EPI_WARPS * STAGING_BUFS * STAGING_BYTES + ((TAIL_BYTES + 127) / 128) * 128;
 constexpr int NUM_SMS = 148;
-constexpr int MAX_SUB = 4;           // row blocks that share one generated B tile
 static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 
-// GENERATED: tiles of P with the tile's M (or N) index running over rows of P; as the A operand they are
-// written K-major.  GENERATED_T (A operand only): the M index runs over columns of P and the K index
-// over its rows, written MN-major -- the operand of Z^T = P^T X^T.
+// Generated operands are always the A operand.  GENERATED: the tile's M index runs over rows of P and its K
+// index over columns of P, written K-major (the update).  GENERATED_T: the M index runs over columns of P
+// and the K index over its rows, written MN-major -- the operand of Z^T = P^T X^T (the forward).
 enum OperandMode { TMA_KMAJOR = 0, TMA_MNMAJOR = 1, GENERATED = 2, GENERATED_T = 3 };
 // EPI_BF16_T stores the transpose of the accumulator (lanes become columns of the output).
 enum EpiMode { EPI_BF16 = 0, EPI_F32 = 1, EPI_UPDATE_W = 2, EPI_BF16_T = 3 };
-enum GenRing { GEN_NONE = 0, GEN_A = 1, GEN_B = 2 };
+enum GenRing { GEN_NONE = 0, GEN_A = 1 };
 
 constexpr unsigned int STATUS_TIMEOUT = 1u;
 #if defined(COMPACT_PROFILE) || defined(COMPACT_PROFILE_GEN)
@@ -318,16 +319,11 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 
-// Eight consecutive entries P[i, j0 .. j0+7] (j0 a multiple of 8) as packed bf16, in two steps so that a
-// generator thread can run the Philox rounds of its next tile (32x32->64 multiplies) between the Box-Muller
-// transforms of the current one (MUFU): the raw words, then the Gaussians.  Entries outside n x r are zero.
-__device__ __forceinline__ void projection8_words(const ProjectionParams& pp, int i, int j0, uint4& xa, uint4& xb) {
+// Eight consecutive entries P[i, j0 .. j0+7] (j0 a multiple of 8) as packed bf16; entries outside n x r are zero.
+__device__ __forceinline__ uint4 projection8_bf16(const ProjectionParams& pp, int i, int j0) {
   const uint32_t q = (uint32_t)(j0 >> 2);
-  xa = philox4x32_10_layer(q, (uint32_t)i, pp.epoch, pp.layer_hi, pp.layer_lo, pp.key);
-  xb = philox4x32_10_layer(q + 1, (uint32_t)i, pp.epoch, pp.layer_hi, pp.layer_lo, pp.key);
-}
-__device__ __forceinline__ uint4 projection8_from_words(const ProjectionParams& pp, const uint4& xa, const uint4& xb, int i,
-                                                        int j0) {
+  const uint4 xa = philox4x32_10_layer(q, (uint32_t)i, pp.epoch, pp.layer_hi, pp.layer_lo, pp.key);
+  const uint4 xb = philox4x32_10_layer(q + 1, (uint32_t)i, pp.epoch, pp.layer_hi, pp.layer_lo, pp.key);
   float4 a = gaussian4_fast_scaled(xa, pp.neg2ln2_over_r);
   float4 b = gaussian4_fast_scaled(xb, pp.neg2ln2_over_r);
   const int left = i < pp.n ? pp.r - j0 : 0;      // valid entries among the eight
@@ -538,7 +534,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const TileCoord t = decode_tile(prm, tile);
         const Problem& p = prm.prob[t.prob];
         const CUtensorMap* mapB = &prm.tmB[t.prob];
-        const bool a_tma = p.a_mode < GENERATED, b_tma = p.b_mode < GENERATED;
+        const bool a_tma = p.a_mode < GENERATED;
         const bool split = item_is_split(p, t);
         const int geo = p.geo, ns = geo ? NS1 : NS0;
         if (cur_geo >= 0 && geo != cur_geo && !(ok = __all_sync(0xffffffffu, drain(cur_geo, cur_geo ? r1 : r0)))) break;
@@ -555,7 +551,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             uint32_t tx = 0;
             bool gen_here = false;
             // of a generated tile, the shares of the other CTAs arrive as counted bytes
-            if (hb) { if (b_tma) tx += p.bn * BK * 2; else { gen_here = true; tx += (p.bn * BK * 2 / cs) * (cs - 1); } }
+            if (hb) tx += p.bn * BK * 2;
             if (na > 0) { if (a_tma) tx += na * A_BYTES; else { gen_here = true; tx += (A_BYTES / cs) * (cs - 1); } }
 #if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
             if (prm.debug_flags & 2) tx = 0;
@@ -573,7 +569,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
               if (tx) mbar_expect_tx(fb, tx);
               // arrive for this thread, and for the generator warps when they have nothing to write here
               mbar_arrive_n(fb, 1 + ((has_gen && !gen_here) ? GEN_ARRIVALS : 0));
-              if (hb && b_tma && tx) {
+              if (hb && tx) {
                 const uint32_t dst = stage_addr(geo, s) + STAGE_B_OFF;
                 const int n0 = t.n0 + (p.ncol > 1 ? j : 0) * p.bn;
                 if (p.b_mode == TMA_KMAJOR) {
@@ -733,7 +729,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
           continue;
         }
         // items with a generated operand walk the ring in step with the other CTAs of the cluster
-        const bool gen_shared = cs > 1 && (p.a_mode >= GENERATED || p.b_mode >= GENERATED);
+        const bool gen_shared = cs > 1 && p.a_mode >= GENERATED;
         // accumulator ai of the item sits in slot ai / sps at column (ai % sps) * bn (a slot is 256 columns)
         const int naccs = p.nsub * p.ncol;
         const int sps = BN_MAX / bn > naccs ? naccs : BN_MAX / bn;
@@ -804,7 +800,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         if (geo) r1 = r; else r0 = r;
 #ifdef COMPACT_PROFILE_GEN
         if (lane == 0 && iss == 0) {
-          if (p.a_mode >= GENERATED || p.b_mode >= GENERATED) {
+          if (p.a_mode >= GENERATED) {
             atomicAdd(&g_prof[4], (unsigned long long)mwait);                 // waiting for full stages
             atomicAdd(&g_prof[5], (unsigned long long)missue);               // issuing MMAs and commits
             atomicAdd(&g_prof[6], (unsigned long long)(clock64() - m1c));    // whole k loop
@@ -1009,11 +1005,9 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       //   update:             A[m = row i of P][k = column j of P], K-major, [128 rows][128 B]
       // Of a tile shared by a cluster this CTA writes the rows crank * (rows / cs) onward.
       const int ntask = 2 >> csh;                       // tasks per thread and tile: 1024 / (512 cs)
-      const bool philox_first = ((warp >> 2) & 1) != 0;  // two of the four generator warps of each scheduler
       const int ik = gen_at ? 1 : 0, jk = 1 - ik;       // which index of P advances with k
       int t_i[2], t_j[2];
       uint32_t t_off[2];
-      uint4 xa[2], xb[2];
 #pragma unroll
       for (int u = 0; u < 2; ++u) {
         const int id = gtid + u * GSTRIDE;
@@ -1027,12 +1021,6 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
           t_off[u] = STAGE_A0_OFF + rr * 128 + ((c ^ (rr & 7)) << 4);
         }
       }
-      if (gen_a || gen_at) {
-        const int k0 = t.k_begin * BK;
-#pragma unroll
-        for (int u = 0; u < 2; ++u)
-          if (u < ntask) projection8_words(prm.pp, t_i[u] + ik * k0, t_j[u] + jk * k0, xa[u], xb[u]);
-      }
       for (int ks = t.k_begin; ks < t.k_end && ok && (gen_a || gen_at); ++ks) {
         const int s = r.s;
         const uint32_t eph = r.ph ^ 1u;
@@ -1043,45 +1031,19 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
 #ifdef COMPACT_PROFILE_GEN
         const long long g0 = clock64();
 #endif
-#ifdef CFG_GEN_WAIT_LANE0
-        bool w = true;
-        if (lane == 0) w = mbar_wait(empty_bar(geo, s), eph, abort_flag, prm.status);
-        w = __all_sync(0xffffffffu, w);
-#else
         const bool w = mbar_wait(empty_bar(geo, s), eph, abort_flag, prm.status);
-#endif
 #ifdef COMPACT_PROFILE_GEN
         const long long g1 = clock64();
 #endif
         if (warp == (THREADS_BASE >> 5)) TRACE(tile == first_tile, ks, 0);
         const int k0 = ks * BK;
-        int k1 = k0 + BK;
-        // Each pass turns this tile's words into Gaussians (Box-Muller: the MUFU pipe) and runs the Philox
-        // rounds of the next tile (the 32x32->64 multiply pipe; past the item's end the words are simply not
-        // used).  Half of the warps on every scheduler do the one first, half the other, so that the two pipes
-        // work at the same time instead of all warps queueing on one and then on the other.  The empty asm
-        // statements pin the order (and keep both parts on this side of the wait).
-        asm volatile("" : "+r"(k1));
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
-          if (u < ntask) {
-            uint4 val, nxa, nxb;
-            if (philox_first) {
-              projection8_words(prm.pp, t_i[u] + ik * k1, t_j[u] + jk * k1, nxa, nxb);
-              asm volatile("" : "+r"(xa[u].x) : "r"(nxa.x), "r"(nxb.x));
-              val = projection8_from_words(prm.pp, xa[u], xb[u], t_i[u] + ik * k0, t_j[u] + jk * k0);
-            } else {
-              asm volatile("" : "+r"(xa[u].x));
-              val = projection8_from_words(prm.pp, xa[u], xb[u], t_i[u] + ik * k0, t_j[u] + jk * k0);
-              asm volatile("" : "+r"(k1) : "r"(val.x), "r"(val.w));
-              projection8_words(prm.pp, t_i[u] + ik * k1, t_j[u] + jk * k1, nxa, nxb);
-            }
-            xa[u] = nxa; xb[u] = nxb;
-            if (w) {
-              const uint32_t off = stage_off + t_off[u];
-              *reinterpret_cast<uint4*>(smem_gen + off) = val;
-              if (cs > 1) st_async_16(peer_base + off, val, peer_full + full_off);
-            }
+          if (u < ntask && w) {
+            const uint4 val = projection8_bf16(prm.pp, t_i[u] + ik * k0, t_j[u] + jk * k0);
+            const uint32_t off = stage_off + t_off[u];
+            *reinterpret_cast<uint4*>(smem_gen + off) = val;
+            if (cs > 1) st_async_16(peer_base + off, val, peer_full + full_off);
           }
         }
 #ifdef COMPACT_PROFILE_GEN
