@@ -116,16 +116,30 @@ struct Problem {
   int a_mode, b_mode, epi_mode;
   int geo;                // ring geometry its items use (0 or 1)
   int a_blocked, b_blocked;   // MN-major operand read through a map that brings a whole tile in one copy
+  int map_base;           // its tensor maps: C at map_base, A and B of K segment s at map_base + s
+  // the projection a generated operand is a tile of; the Philox key (the seed) is the launch's
+  uint32_t pp_layer_hi, pp_layer_lo, pp_epoch;
+  int pp_n, pp_r;
+  float pp_scale;         // -2 ln 2 / r
+  // K may run over up to three segments with operands of their own (dX of a group of layers that share
+  // their input is the sum over the layers of dY_g W_g^T): segment s covers k-steps seg_begin[s] .. seg_begin[s+1]
+  int nseg;
+  int seg_begin[4];
+  int group_begin;        // generated problems: number of cluster groups before this problem's
   int tile_begin;
   float scale;
 };
 
+constexpr int MAXP = 6;     // problems (and tensor-map triples) per launch
+constexpr int MAXG = 3;     // layers in a group that shares its input
+
 struct alignas(64) Params {
-  CUtensorMap tmA[2];
-  CUtensorMap tmB[2];
-  CUtensorMap tmC[2];     // output (and, for the update, input) tiles of the epilogue
-  Problem prob[2];
+  CUtensorMap tmA[MAXP];
+  CUtensorMap tmB[MAXP];
+  CUtensorMap tmC[MAXP];  // output tiles of the epilogue
+  Problem prob[MAXP];
   int num_problems;
+  int num_gen;            // problems with a generated operand: the first num_gen of the launch
   int total_tiles;
   int gen_ring;
   // Cluster-shared generation: the `cs` CTAs of a cluster take items that need the same tiles of P
@@ -136,7 +150,7 @@ struct alignas(64) Params {
   int gen_groups;         // groups of cs generated items; handed out statically, cluster by cluster
   int dyn_begin;          // first item handed out dynamically (0 when cs == 1)
   int debug_flags;        // profiling builds only: bit 0 = issue no MMAs (measures the load path alone)
-  ProjectionParams pp;
+  PhiloxKey key;          // round keys of the seed shared by the launch's generated problems
   unsigned int* status;
   unsigned int* sched;
 };
@@ -319,14 +333,16 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 
-// Eight consecutive entries P[i, j0 .. j0+7] (j0 a multiple of 8) as packed bf16; entries outside n x r are zero.
-__device__ __forceinline__ uint4 projection8_bf16(const ProjectionParams& pp, int i, int j0) {
+// Eight consecutive entries P[i, j0 .. j0+7] (j0 a multiple of 8) of a problem's projection as packed bf16;
+// entries outside n x r are zero.
+__device__ __forceinline__ uint4 projection8_bf16(const PhiloxKey& key, uint32_t layer_hi, uint32_t layer_lo, uint32_t epoch,
+                                                  int n, int r, float neg2ln2_over_r, int i, int j0) {
   const uint32_t q = (uint32_t)(j0 >> 2);
-  const uint4 xa = philox4x32_10_layer(q, (uint32_t)i, pp.epoch, pp.layer_hi, pp.layer_lo, pp.key);
-  const uint4 xb = philox4x32_10_layer(q + 1, (uint32_t)i, pp.epoch, pp.layer_hi, pp.layer_lo, pp.key);
-  float4 a = gaussian4_fast_scaled(xa, pp.neg2ln2_over_r);
-  float4 b = gaussian4_fast_scaled(xb, pp.neg2ln2_over_r);
-  const int left = i < pp.n ? pp.r - j0 : 0;      // valid entries among the eight
+  const uint4 xa = philox4x32_10_layer(q, (uint32_t)i, epoch, layer_hi, layer_lo, key);
+  const uint4 xb = philox4x32_10_layer(q + 1, (uint32_t)i, epoch, layer_hi, layer_lo, key);
+  float4 a = gaussian4_fast_scaled(xa, neg2ln2_over_r);
+  float4 b = gaussian4_fast_scaled(xb, neg2ln2_over_r);
+  const int left = i < n ? r - j0 : 0;      // valid entries among the eight
   if (left < 8) {
     a.x = left > 0 ? a.x : 0.f; a.y = left > 1 ? a.y : 0.f; a.z = left > 2 ? a.z : 0.f; a.w = left > 3 ? a.w : 0.f;
     b.x = left > 4 ? b.x : 0.f; b.y = left > 5 ? b.y : 0.f; b.z = left > 6 ? b.z : 0.f; b.w = left > 7 ? b.w : 0.f;
@@ -352,9 +368,19 @@ struct TileCoord {
   int prob, m0, n0, k_begin, k_end, split, nsub, ncol, nst;
 };
 
+// kGroup: the launch may hold more than two problems and problems whose K runs over several segments (a group
+// of layers that share their input).  The plain instantiation keeps the two-problem arithmetic and reads the
+// projection's scalars straight from the constant bank.
+template <bool kGroup>
 __device__ __forceinline__ TileCoord decode_tile(const Params& prm, int tile) {
   TileCoord t;
-  t.prob = (prm.num_problems > 1 && tile >= prm.prob[1].tile_begin) ? 1 : 0;
+  if (kGroup) {
+    t.prob = 0;
+    for (int i = 1; i < prm.num_problems; ++i)
+      if (tile >= prm.prob[i].tile_begin) t.prob = i;
+  } else {
+    t.prob = (prm.num_problems > 1 && tile >= prm.prob[1].tile_begin) ? 1 : 0;
+  }
   const Problem& p = prm.prob[t.prob];
   int local = tile - p.tile_begin;
   const int nb = local % p.tiles_n;
@@ -365,7 +391,7 @@ __device__ __forceinline__ TileCoord decode_tile(const Params& prm, int tile) {
   t.n0 = nb * p.bn * p.ncol;
   t.k_begin = t.split * p.ksteps_per_split;
   t.k_end = min(p.ksteps_total, t.k_begin + p.ksteps_per_split);
-  if (prm.cs > 1 && t.prob == 0) {
+  if (prm.cs > 1 && t.prob < prm.num_gen) {
     // items of a cluster walk the stage ring in step: all of them take the full shape, the rows and
     // columns past the edge load as zeros and are never stored
     t.nsub = p.nsub;
@@ -389,6 +415,7 @@ __device__ __forceinline__ TileCoord decode_tile(const Params& prm, int tile) {
 //   10     loader of the A tiles (only issues TMA)
 //   12..27 generators of P (launches with a generated operand only)
 // --------------------------------------------------------------------------------------
+template <bool kGroup>
 __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __grid_constant__ Params prm) {
   extern __shared__ uint8_t smem_raw[];
 #ifdef COMPACT_PROFILE_GEN
@@ -505,17 +532,22 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         if (!(ok = __all_sync(0xffffffffu, mbar_wait(qempty(qs), qph ^ 1, abort_flag, prm.status)))) break;
         int tile;
         if (cs > 1 && group < prm.gen_groups) {
-          const Problem& p0 = prm.prob[0];
+          int pi = 0;
+          if (kGroup)
+            for (int i = 1; i < prm.num_gen; ++i)
+              if (group >= prm.prob[i].group_begin) pi = i;
+          const Problem& p0 = prm.prob[pi];
+          const int g = group - p0.group_begin;
           int mb, nb;
           if (prm.share_n) {
             const int per_row = p0.tiles_n / cs;
-            mb = group / per_row;
-            nb = (group % per_row) * cs + (int)crank;
+            mb = g / per_row;
+            nb = (g % per_row) * cs + (int)crank;
           } else {
-            nb = group % p0.tiles_n;
-            mb = (group / p0.tiles_n) * cs + (int)crank;
+            nb = g % p0.tiles_n;
+            mb = (g / p0.tiles_n) * cs + (int)crank;
           }
-          tile = mb * p0.tiles_n + nb;
+          tile = p0.tile_begin + mb * p0.tiles_n + nb;
           group += group_step;
         } else {
           tile = 0;
@@ -531,9 +563,8 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         if (++qs == QDEPTH) { qs = 0; qph ^= 1; }
         if (tile < 0) break;
         if (first_tile == -2) first_tile = tile;
-        const TileCoord t = decode_tile(prm, tile);
+        const TileCoord t = decode_tile<kGroup>(prm, tile);
         const Problem& p = prm.prob[t.prob];
-        const CUtensorMap* mapB = &prm.tmB[t.prob];
         const bool a_tma = p.a_mode < GENERATED;
         const bool split = item_is_split(p, t);
         const int geo = p.geo, ns = geo ? NS1 : NS0;
@@ -541,7 +572,9 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         cur_geo = geo;
         Ring r = geo ? r1 : r0;
         for (int ks = t.k_begin; ks < t.k_end && ok; ++ks) {
-          const int k0 = ks * BK;
+          const int seg = (kGroup && p.nseg > 1) ? (ks >= p.seg_begin[1]) + (ks >= p.seg_begin[2]) : 0;
+          const int k0 = kGroup ? (ks - p.seg_begin[seg]) * BK : ks * BK;
+          const CUtensorMap* mapB = &prm.tmB[kGroup ? p.map_base + seg : t.prob];
           for (int j = 0; j < t.nst; ++j, ring_next(r, ns)) {
             const int s = r.s;
             if (!(ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(geo, s), r.ph ^ 1u, abort_flag, prm.status)))) break;
@@ -597,9 +630,8 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       while (ok) {
         const int tile = __shfl_sync(0xffffffffu, next_tile(true, lane == 0), 0);
         if (tile < 0) break;
-        const TileCoord t = decode_tile(prm, tile);
+        const TileCoord t = decode_tile<kGroup>(prm, tile);
         const Problem& p = prm.prob[t.prob];
-        const CUtensorMap* mapA = &prm.tmA[t.prob];
         const int geo = p.geo, ns = geo ? NS1 : NS0;
         if (cur_geo >= 0 && geo != cur_geo && !(ok = __all_sync(0xffffffffu, drain(cur_geo, cur_geo ? r1 : r0)))) break;
         cur_geo = geo;
@@ -611,7 +643,9 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const int klen = t.k_end - t.k_begin;
         if (!mine) ring_skip(r, ns, klen * t.nst);
         for (int ks = t.k_begin; ks < t.k_end && ok && mine; ++ks) {
-          const int k0 = ks * BK;
+          const int seg = (kGroup && p.nseg > 1) ? (ks >= p.seg_begin[1]) + (ks >= p.seg_begin[2]) : 0;
+          const int k0 = kGroup ? (ks - p.seg_begin[seg]) * BK : ks * BK;
+          const CUtensorMap* mapA = &prm.tmA[kGroup ? p.map_base + seg : t.prob];
           for (int j = 0; j < t.nst; ++j) {
             const int s = r.s;
             const uint32_t eph = r.ph ^ 1u;
@@ -681,7 +715,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const long long t0c = clock64();
 #endif
         if (tile < 0) break;
-        const TileCoord t = decode_tile(prm, tile);
+        const TileCoord t = decode_tile<kGroup>(prm, tile);
         const Problem& p = prm.prob[t.prob];
         const bool a_mn = p.a_mode == TMA_MNMAJOR || p.a_mode == GENERATED_T;
         const bool b_mn = p.b_mode != TMA_KMAJOR;
@@ -839,9 +873,9 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
     while (ok) {
       const int tile = next_tile(true, lane == 0);
       if (tile < 0) break;
-      const TileCoord t = decode_tile(prm, tile);
+      const TileCoord t = decode_tile<kGroup>(prm, tile);
       const Problem& p = prm.prob[t.prob];
-      const CUtensorMap* mapC = &prm.tmC[t.prob];
+      const CUtensorMap* mapC = &prm.tmC[kGroup ? p.map_base : t.prob];
       const int naccs = p.nsub * p.ncol;
       const int slots = (naccs * p.bn + BN_MAX - 1) / BN_MAX;
       const int sub_per_slot = BN_MAX / p.bn > naccs ? naccs : BN_MAX / p.bn;
@@ -989,7 +1023,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
     while (ok) {
       const int tile = next_tile(true, lane == 0);
       if (tile < 0) break;
-      const TileCoord t = decode_tile(prm, tile);
+      const TileCoord t = decode_tile<kGroup>(prm, tile);
       const Problem& p = prm.prob[t.prob];
       const int klen = t.k_end - t.k_begin;
       if (first_tile == -2) first_tile = tile;
@@ -1005,6 +1039,8 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       //   update:             A[m = row i of P][k = column j of P], K-major, [128 rows][128 B]
       // Of a tile shared by a cluster this CTA writes the rows crank * (rows / cs) onward.
       const int ntask = 2 >> csh;                       // tasks per thread and tile: 1024 / (512 cs)
+      // the plain instantiation's only generated problem is problem 0: constant-bank operands
+      const Problem& gp = kGroup ? p : prm.prob[0];
       const int ik = gen_at ? 1 : 0, jk = 1 - ik;       // which index of P advances with k
       int t_i[2], t_j[2];
       uint32_t t_off[2];
@@ -1040,7 +1076,8 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
           if (u < ntask && w) {
-            const uint4 val = projection8_bf16(prm.pp, t_i[u] + ik * k0, t_j[u] + jk * k0);
+            const uint4 val = projection8_bf16(prm.key, gp.pp_layer_hi, gp.pp_layer_lo, gp.pp_epoch, gp.pp_n, gp.pp_r,
+                                               gp.pp_scale, t_i[u] + ik * k0, t_j[u] + jk * k0);
             const uint32_t off = stage_off + t_off[u];
             *reinterpret_cast<uint4*>(smem_gen + off) = val;
             if (cs > 1) st_async_16(peer_base + off, val, peer_full + full_off);
@@ -1220,6 +1257,11 @@ inline int pick_bn(int N) { return N >= BN_MAX ? BN_MAX : (int)((N + 63) / 64 * 
 #define CFG_NSUB 2
 #endif
 
+inline void set_projection(Problem& p, const ProjectionParams& pp) {
+  p.pp_layer_hi = pp.layer_hi; p.pp_layer_lo = pp.layer_lo; p.pp_epoch = pp.epoch;
+  p.pp_n = pp.n; p.pp_r = pp.r; p.pp_scale = pp.neg2ln2_over_r;
+}
+
 inline void finish_problem(Problem& p, int splits_wanted) {
   if (p.bn == 0) p.bn = pick_bn(p.N);
   // two row blocks share each B tile: 256 x 256 items halve the shared-memory refill per flop and
@@ -1234,6 +1276,11 @@ inline void finish_problem(Problem& p, int splits_wanted) {
   if (s > p.ksteps_total) s = p.ksteps_total;
   p.ksteps_per_split = (p.ksteps_total + s - 1) / s;
   p.splits = (p.ksteps_total + p.ksteps_per_split - 1) / p.ksteps_per_split;
+  if (p.nseg <= 1) {
+    p.nseg = 1;
+    p.seg_begin[0] = 0;
+    p.seg_begin[1] = p.seg_begin[2] = p.seg_begin[3] = p.ksteps_total;
+  }
 }
 
 // Number of token splits of Gc = Z^T dY.  A split should be about as long as one dX item
@@ -1263,29 +1310,43 @@ inline size_t gc_workspace_bytes(int64_t tokens, int r, int m) {
 inline compact_status_t launch(const LaunchInfo& li, Params& prm) {
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(compact_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
+    if (cudaFuncSetAttribute(compact_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(compact_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
       cudaGetLastError();
       return COMPACT_ERR_CUDA;
     }
     attr_set = true;
   }
-  // sharing generated tiles needs the four-stage ring, where a stage keeps its role (see the stage owner)
-  const int cs = (prm.gen_ring != GEN_NONE && li.cluster > 1 && prm.prob[0].geo == 1) ? 2 : 1;
+  bool group = prm.num_problems > 2;
+  for (int i = 0; i < prm.num_problems; ++i) group = group || prm.prob[i].nseg > 1;
+  // The problems with a generated operand come first.  Sharing generated tiles needs the four-stage ring,
+  // where a stage keeps its role (see the stage owner).
+  prm.num_gen = 0;
+  bool gen_geo1 = true;
+  while (prm.num_gen < prm.num_problems && prm.prob[prm.num_gen].a_mode >= GENERATED) {
+    gen_geo1 = gen_geo1 && prm.prob[prm.num_gen].geo == 1;
+    ++prm.num_gen;
+  }
+  const int cs = (prm.num_gen > 0 && li.cluster > 1 && gen_geo1) ? 2 : 1;
   prm.cs = cs;
-  if (cs > 1) {
-    // the generated problem is problem 0; its items come in groups of cs neighbours
-    Problem& p0 = prm.prob[0];
-    prm.share_n = prm.gen_ring == GEN_A ? 1 : 0;
-    if (prm.share_n) p0.tiles_n = (p0.tiles_n + cs - 1) / cs * cs;
-    else p0.tiles_m = (p0.tiles_m + cs - 1) / cs * cs;
-    prm.gen_groups = p0.tiles_m * p0.tiles_n / cs;
-    prm.dyn_begin = p0.tiles_m * p0.tiles_n;
-  }
-  int t = 0;
+  prm.share_n = 1;      // the cs items of a group are neighbours along N (tokens in the forward, columns of W in the update)
+  prm.gen_groups = 0;
+  int t = 0, maps = 0;
   for (int i = 0; i < prm.num_problems; ++i) {
-    prm.prob[i].tile_begin = t;
-    t += prm.prob[i].tiles_m * prm.prob[i].tiles_n * prm.prob[i].splits;
+    Problem& p = prm.prob[i];
+    if (cs > 1 && i < prm.num_gen) {
+      // items with a generated operand come in groups of cs neighbours
+      p.tiles_n = (p.tiles_n + cs - 1) / cs * cs;
+      p.group_begin = prm.gen_groups;
+      prm.gen_groups += p.tiles_m * p.tiles_n / cs;
+    }
+    p.tile_begin = t;
+    t += p.tiles_m * p.tiles_n * p.splits;
+    if (i + 1 == prm.num_gen) prm.dyn_begin = cs > 1 ? t : 0;
+    p.map_base = maps;
+    maps += p.nseg;
   }
+  if (maps > MAXP) return COMPACT_ERR_INVALID_ARG;
   prm.total_tiles = t;
   prm.status = li.status;
   prm.sched = li.sched;
@@ -1307,7 +1368,8 @@ inline compact_status_t launch(const LaunchInfo& li, Params& prm) {
   attr.val.clusterDim.z = 1;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  const cudaError_t e = cudaLaunchKernelEx(&cfg, compact_gemm_kernel, prm);
+  const cudaError_t e = group ? cudaLaunchKernelEx(&cfg, compact_gemm_kernel<true>, prm)
+                              : cudaLaunchKernelEx(&cfg, compact_gemm_kernel<false>, prm);
   (*li.launches)++;
   if (e != cudaSuccess) { cudaGetLastError(); return COMPACT_ERR_CUDA; }
   return cudaGetLastError() == cudaSuccess ? COMPACT_OK : COMPACT_ERR_CUDA;
@@ -1327,7 +1389,7 @@ inline compact_status_t forward(const LaunchInfo& li, const ProjectionParams& pp
   if (!Y && !Z) return COMPACT_OK;
   Params prm;
   memset(&prm, 0, sizeof(prm));
-  prm.pp = pp;
+  prm.key = pp.key;
   prm.num_problems = (Y && Z) ? 2 : 1;
   prm.gen_ring = Z ? GEN_A : GEN_NONE;
   const int iy = Z ? 1 : 0;       // where the Y problem sits
@@ -1340,6 +1402,7 @@ inline compact_status_t forward(const LaunchInfo& li, const ProjectionParams& pp
     pz.nsub = 1;
     pz.ncol = tokens > BN_MAX ? 2 : 1;
     pz.a_mode = GENERATED_T; pz.b_mode = TMA_KMAJOR; pz.epi_mode = EPI_BF16_T;
+    set_projection(pz, pp);
     finish_problem(pz, 1);
     prm.tmA[0] = prm.tmA[iy];   // unused by the generated operand (set below when Y is present)
     if (!make_map(&prm.tmB[0], X, n, tokens, ldx, BK, pz.bn)) return COMPACT_ERR_CUDA;
@@ -1425,7 +1488,7 @@ inline compact_status_t update(const LaunchInfo& li, const ProjectionParams& pp,
   if (cudaGetLastError() != cudaSuccess) return COMPACT_ERR_CUDA;
   Params prm;
   memset(&prm, 0, sizeof(prm));
-  prm.pp = pp;
+  prm.key = pp.key;
   prm.num_problems = 1;
   prm.gen_ring = GEN_A;
   Problem& pu = prm.prob[0];
@@ -1433,6 +1496,7 @@ inline compact_status_t update(const LaunchInfo& li, const ProjectionParams& pp,
   pu.nsub = 1;
   pu.ncol = m > BN_MAX ? 2 : 1;     // the generator is the bound here: one generated tile of P feeds two column blocks
   pu.a_mode = GENERATED; pu.b_mode = TMA_MNMAJOR; pu.epi_mode = EPI_UPDATE_W;
+  set_projection(pu, pp);
   pu.scale = scale;
   finish_problem(pu, 1);
   pu.b_blocked = m % 64 == 0;
