@@ -130,6 +130,34 @@ compact_status_t compact_linear_bwd_recompute(compact_layer_t* layer, int64_t to
                                               float* Gc, int64_t ldg, int accumulate,
                                               void* workspace, size_t workspace_bytes, void* stream);
 
+/* Layers that share their input (q, k, v of an attention block; gate and up of an
+ * MLP): each has its own W and its own projection -- the paper's appendix on saved
+ * tensors lists x P_q, x P_k, x P_v (and x P_gate, x P_up) as separate compressed
+ * activations of the one input.  compact_group_fwd is Algorithm 1 for every layer of
+ * the group in one launch (X is read once); compact_group_bwd is Algorithm 2 for
+ * every layer with the input gradients summed, dX = sum_g dY_g W_g^T, accumulated in
+ * one place instead of G tensors added afterwards.  Y and Z are bitwise those of the
+ * single-layer calls; Gc may differ in summation order over tokens (still fixed, so
+ * reproducible); dX is the sum rounded once.
+ * Arrays have `count` entries, one per layer, in the same order.  All layers must
+ * have the same n and dtype.  bf16 layers with one seed and count <= 3 run fused;
+ * other groups run layer by layer with the same results up to the rounding of dX.
+ * workspace: at least compact_group_workspace_bytes(layers, count, tokens). */
+size_t compact_group_workspace_bytes(compact_layer_t* const* layers, int count, int64_t tokens);
+compact_status_t compact_group_fwd(compact_layer_t* const* layers, int count, int64_t tokens,
+                                   const void* X, int64_t ldx,
+                                   const void* const* W, const int64_t* ldw,
+                                   void* const* Y, const int64_t* ldy,
+                                   void* const* Z, const int64_t* ldz,
+                                   uint32_t* epochs_used, void* stream);
+compact_status_t compact_group_bwd(compact_layer_t* const* layers, int count, int64_t tokens,
+                                   const void* const* dY, const int64_t* lddy,
+                                   const void* const* Z, const int64_t* ldz,
+                                   const void* const* W, const int64_t* ldw,
+                                   void* dX, int64_t lddx,
+                                   float* const* Gc, const int64_t* ldg, int accumulate,
+                                   void* workspace, size_t workspace_bytes, void* stream);
+
 /* Algorithm 3 lines 1-10.  In place on W, M, V (M, V: r x m fp32, pitch ldg);
  * stored moments are the uncorrected running averages and the bias correction
  * uses the 1-based count of this update.  epoch_of_Gc must equal the layer's

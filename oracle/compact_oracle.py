@@ -160,6 +160,21 @@ def linear_bwd_recompute(X: np.ndarray, dY: np.ndarray, W: np.ndarray, P: np.nda
     return linear_bwd(dY, Z, W, mode)
 
 
+def group_fwd(X: np.ndarray, Ws, Ps, mode: str = "exact"):
+    """Algorithm 1 for layers that share their input x (q, k, v; gate, up): each layer g has its own W_g and its
+    own P_g, and keeps its own z_g = x P_g (appendix on saved tensors, Table 6)."""
+    outs = [linear_fwd(X, W, P, mode) for W, P in zip(Ws, Ps)]
+    return [o[0] for o in outs], [o[1] for o in outs]
+
+
+def group_bwd(dYs, Zs, Ws, mode: str = "exact"):
+    """Algorithm 2 for such a group: G_hat_g = z_g^T dL/do_g per layer, and the gradient with respect to the shared
+    input is the sum of the layers' contributions, dL/dx = sum_g dL/do_g W_g^T (stored once)."""
+    Gcs = [np.asarray(Z, dtype=np.float64).T @ np.asarray(dY, dtype=np.float64) for dY, Z in zip(dYs, Zs)]
+    dX = sum(np.asarray(dY, dtype=np.float64) @ np.asarray(W, dtype=np.float64).T for dY, W in zip(dYs, Ws))
+    return _store(dX, mode), Gcs
+
+
 def adam_update(W, Gc, M, V, t: int, P, lr: float, beta1: float, beta2: float, eps: float,
                 alpha: float = 1.0, mode: str = "exact"):
     """Algorithm 3 lines 1-9 for the update whose 1-based count is t.

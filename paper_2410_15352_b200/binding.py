@@ -26,7 +26,8 @@ F32, BF16 = 0, 1
 EXPORTS = [
     "compact_layer_create", "compact_layer_destroy", "compact_z_ld", "compact_workspace_bytes",
     "compact_saved_bytes", "compact_linear_fwd", "compact_linear_bwd", "compact_recompute_workspace_bytes",
-    "compact_linear_bwd_recompute", "compact_adam_update", "compact_adam_update_noalloc",
+    "compact_linear_bwd_recompute", "compact_group_workspace_bytes", "compact_group_fwd", "compact_group_bwd",
+    "compact_adam_update", "compact_adam_update_noalloc",
     "compact_refresh_projection", "compact_layer_get_state", "compact_layer_set_state",
     "compact_layer_status", "compact_debug_philox_u32", "compact_debug_projection",
     "compact_set_kernel_family", "compact_kernel_launch_count", "compact_status_string",
@@ -72,6 +73,11 @@ def lib() -> C.CDLL:
     L.compact_recompute_workspace_bytes.restype = C.c_size_t
     L.compact_linear_bwd_recompute.argtypes = [vp, i64, vp, i64, C.c_uint32, vp, i64, vp, i64, vp, i64, vp, i64, C.c_int,
                                                vp, C.c_size_t, vp]
+    pp, ip = C.POINTER(C.c_void_p), C.POINTER(C.c_int64)
+    L.compact_group_workspace_bytes.argtypes = [pp, C.c_int, i64]
+    L.compact_group_workspace_bytes.restype = C.c_size_t
+    L.compact_group_fwd.argtypes = [pp, C.c_int, i64, vp, i64, pp, ip, pp, ip, pp, ip, u32p, vp]
+    L.compact_group_bwd.argtypes = [pp, C.c_int, i64, pp, ip, pp, ip, pp, ip, vp, i64, pp, ip, C.c_int, vp, C.c_size_t, vp]
     L.compact_adam_update.argtypes = [vp, vp, i64, vp, i64, vp, vp, C.c_uint32, C.c_float, vp, C.c_size_t, vp]
     L.compact_adam_update_noalloc.argtypes = [vp, vp, i64, vp, i64, vp, vp, C.c_uint32, C.c_float, vp]
     L.compact_refresh_projection.argtypes = [vp, C.c_int, u32p]
@@ -265,3 +271,50 @@ class CompactLinear:
         _check(lib().compact_debug_projection(self._h, self.epoch if epoch is None else epoch, _ptr(P),
                                               _stream(stream)), "compact_debug_projection")
         return P
+
+
+# -- groups of layers that share their input (q, k, v; gate, up) ----------------------------------
+def _ptr_array(tensors):
+    return (C.c_void_p * len(tensors))(*[t.data_ptr() for t in tensors])
+
+
+def _ld_array(tensors):
+    return (C.c_int64 * len(tensors))(*[t.stride(0) for t in tensors])
+
+
+class CompactGroup:
+    """Layers with one input: Algorithm 1 and Algorithm 2 for all of them in one launch each."""
+
+    def __init__(self, layers):
+        self.layers = list(layers)
+        self._h = (C.c_void_p * len(self.layers))(*[l._h for l in self.layers])
+        self._ws = None
+
+    def forward(self, X: torch.Tensor, Ws, Ys=None, Zs=None, stream=None):
+        tokens = X.shape[0]
+        if Ys is None:
+            Ys = [torch.empty((tokens, l.m), dtype=l.dtype, device=X.device) for l in self.layers]
+        if Zs is None:
+            Zs = [torch.empty((tokens, l.ldz), dtype=l.dtype, device=X.device) for l in self.layers]
+        eps = (C.c_uint32 * len(self.layers))()
+        _check(lib().compact_group_fwd(self._h, len(self.layers), tokens, _ptr(X), X.stride(0), _ptr_array(Ws), _ld_array(Ws),
+                                       _ptr_array(Ys), _ld_array(Ys), _ptr_array(Zs), _ld_array(Zs), eps, _stream(stream)),
+               "compact_group_fwd")
+        return Ys, Zs, [int(e) for e in eps]
+
+    def backward(self, dYs, Zs, Ws, Gcs=None, dX=None, need_dX: bool = True, accumulate: bool = False, stream=None):
+        tokens = dYs[0].shape[0]
+        n = self.layers[0].n
+        if Gcs is None:
+            Gcs = [torch.empty((l.r, l.m), dtype=torch.float32, device=dYs[0].device) for l in self.layers]
+        if dX is None and need_dX:
+            dX = torch.empty((tokens, n), dtype=self.layers[0].dtype, device=dYs[0].device)
+        need = max(int(lib().compact_group_workspace_bytes(self._h, len(self.layers), tokens)), 256)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+        _check(lib().compact_group_bwd(self._h, len(self.layers), tokens, _ptr_array(dYs), _ld_array(dYs), _ptr_array(Zs),
+                                       _ld_array(Zs), _ptr_array(Ws), _ld_array(Ws), _ptr(dX), dX.stride(0) if dX is not None else 0,
+                                       _ptr_array(Gcs), _ld_array(Gcs), int(accumulate), _ptr(self._ws), self._ws.numel(),
+                                       _stream(stream)),
+               "compact_group_bwd")
+        return dX, Gcs

@@ -101,6 +101,23 @@ void simt_gemm(int M, int N, int K, AF a, BF b, EP ep, cudaStream_t st) {
 inline bool pitch_ok(int64_t ld, int64_t min_cols, size_t es) { return ld >= min_cols && (ld * (int64_t)es) % 16 == 0; }
 
 // ---- forward ---------------------------------------------------------------------------
+// dst[rows x cols] += src[rows x cols] (element type T, one rounding)
+template <typename T>
+__global__ void add_rows_kernel(T* dst, int64_t ldd, const T* src, int64_t lds, int64_t rows, int cols) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= rows * cols) return;
+  const int64_t r = idx / cols;
+  const int c = (int)(idx % cols);
+  dst[r * ldd + c] = simt::from_f32<T>(simt::to_f32(dst[r * ldd + c]) + simt::to_f32(src[r * lds + c]));
+}
+template <typename T>
+compact_status_t add_rows(T* dst, int64_t ldd, const T* src, int64_t lds, int64_t rows, int cols, cudaStream_t st) {
+  const int64_t cnt = rows * cols;
+  add_rows_kernel<T><<<(unsigned)((cnt + 255) / 256), 256, 0, st>>>(dst, ldd, src, lds, rows, cols);
+  g_launches++;
+  return launch_result();
+}
+
 template <typename T>
 compact_status_t fwd_simt(compact_layer_t* L, int64_t tokens, const T* X, int64_t ldx, const T* W, int64_t ldw,
                           T* Y, int64_t ldy, T* Z, int64_t ldz, cudaStream_t st) {
@@ -277,6 +294,130 @@ compact_status_t compact_linear_bwd(compact_layer_t* L, int64_t tokens, const vo
   }
   return bwd_simt<float>(L, tokens, (const float*)dY, lddy, (const float*)Z, ldz, (const float*)W, ldw, (float*)dX,
                          lddx, Gc, ldg, accumulate, st);
+}
+
+// ---- groups of layers that share their input ---------------------------------------------------
+namespace {
+// The fused launches take bf16 layers with one input width, one seed and at most three members;
+// anything else (and the SIMT family) runs layer by layer.
+bool group_fusable(compact_layer_t* const* Ls, int count) {
+  if (count < 1 || count > tc::MAXG || g_family.load() == 1) return false;
+  for (int g = 0; g < count; ++g) {
+    if (Ls[g]->cfg.dtype != COMPACT_BF16 || Ls[g]->cfg.n != Ls[0]->cfg.n || Ls[g]->cfg.seed != Ls[0]->cfg.seed) return false;
+    if (Ls[g]->cfg.n % 8 || Ls[g]->cfg.m % 8) return false;
+  }
+  return true;
+}
+}  // namespace
+
+size_t compact_group_workspace_bytes(compact_layer_t* const* layers, int count, int64_t tokens) {
+  if (!layers || count < 1 || tokens < 0) return 0;
+  size_t fused = 0, single = 0;
+  int r[tc::MAXG], m[tc::MAXG];
+  for (int g = 0; g < count; ++g) {
+    if (!layers[g]) return 0;
+    const size_t w = compact_workspace_bytes(layers[g], tokens);
+    single = w > single ? w : single;
+    if (g < tc::MAXG) { r[g] = layers[g]->cfg.r; m[g] = layers[g]->cfg.m; }
+  }
+  if (count <= tc::MAXG) fused = tc::group_gc_workspace_bytes(count, r, m, tokens);
+  // layer-by-layer fallback: one layer's workspace plus a dX-sized buffer for the partial input gradients
+  const size_t fallback = single + (size_t)round_up((int64_t)tokens * layers[0]->cfg.n * (int64_t)elem_size(layers[0]->cfg.dtype), 256);
+  const size_t need = fused > fallback ? fused : fallback;
+  return (size_t)round_up((int64_t)need, 256);
+}
+
+compact_status_t compact_group_fwd(compact_layer_t* const* layers, int count, int64_t tokens, const void* X, int64_t ldx,
+                                   const void* const* W, const int64_t* ldw, void* const* Y, const int64_t* ldy,
+                                   void* const* Z, const int64_t* ldz, uint32_t* epochs_used, void* stream) {
+  if (!layers || count < 1 || !W || !ldw || !Y || !ldy || !Z || !ldz) return COMPACT_ERR_INVALID_ARG;
+  for (int g = 0; g < count; ++g)
+    if (!layers[g] || layers[g]->cfg.n != layers[0]->cfg.n || layers[g]->cfg.dtype != layers[0]->cfg.dtype) return COMPACT_ERR_INVALID_ARG;
+  if (!group_fusable(layers, count) || tokens <= 0) {
+    for (int g = 0; g < count; ++g) {
+      compact_status_t s = compact_linear_fwd(layers[g], tokens, X, ldx, W[g], ldw[g], Y[g], ldy[g], Z[g], ldz[g],
+                                              epochs_used ? epochs_used + g : nullptr, stream);
+      if (s != COMPACT_OK) return s;
+    }
+    return COMPACT_OK;
+  }
+  typedef __nv_bfloat16 T;
+  if (tokens > 0x7fffffff || !X) return COMPACT_ERR_INVALID_ARG;
+  if (!aligned16(X) || !pitch_ok(ldx, layers[0]->cfg.n, 2)) return COMPACT_ERR_ALIGNMENT;
+  tc::GroupLayer gl[tc::MAXG];
+  memset(gl, 0, sizeof(gl));
+  for (int g = 0; g < count; ++g) {
+    compact_layer_t* L = layers[g];
+    if (epochs_used) epochs_used[g] = L->epoch;
+    if (!W[g] || !Y[g] || !Z[g]) return COMPACT_ERR_INVALID_ARG;
+    if (!aligned16(W[g]) || !aligned16(Y[g]) || !aligned16(Z[g])) return COMPACT_ERR_ALIGNMENT;
+    if (!pitch_ok(ldw[g], L->cfg.m, 2) || !pitch_ok(ldy[g], L->cfg.m, 2) || !pitch_ok(ldz[g], compact_z_ld(L), 2)) return COMPACT_ERR_ALIGNMENT;
+    gl[g].pp = make_pp(L, L->epoch);
+    gl[g].m = L->cfg.m; gl[g].r = L->cfg.r; gl[g].zcols = (int)compact_z_ld(L);
+    gl[g].W = (const T*)W[g]; gl[g].ldw = ldw[g];
+    gl[g].Y = (T*)Y[g]; gl[g].ldy = ldy[g];
+    gl[g].Z = (T*)Z[g]; gl[g].ldz = ldz[g];
+  }
+  compact_status_t s = check_device(layers[0]);
+  if (s != COMPACT_OK) return s;
+  tc::LaunchInfo li{g_family.load() == 2 ? 1 : CFG_CS, (cudaStream_t)stream, status_word(layers[0]), sched_words(layers[0]), &g_launches};
+  return tc::forward_group(li, count, gl, tokens, layers[0]->cfg.n, (const T*)X, ldx);
+}
+
+compact_status_t compact_group_bwd(compact_layer_t* const* layers, int count, int64_t tokens, const void* const* dY,
+                                   const int64_t* lddy, const void* const* Z, const int64_t* ldz, const void* const* W,
+                                   const int64_t* ldw, void* dX, int64_t lddx, float* const* Gc, const int64_t* ldg,
+                                   int accumulate, void* workspace, size_t workspace_bytes, void* stream) {
+  if (!layers || count < 1 || !dY || !lddy || !Z || !ldz || !W || !ldw || !Gc || !ldg) return COMPACT_ERR_INVALID_ARG;
+  for (int g = 0; g < count; ++g)
+    if (!layers[g] || layers[g]->cfg.n != layers[0]->cfg.n || layers[g]->cfg.dtype != layers[0]->cfg.dtype) return COMPACT_ERR_INVALID_ARG;
+  if (workspace_bytes < compact_group_workspace_bytes(layers, count, tokens) || !workspace) return COMPACT_ERR_WORKSPACE;
+  if (!aligned16(workspace)) return COMPACT_ERR_ALIGNMENT;
+  const int n = layers[0]->cfg.n;
+  if (!group_fusable(layers, count) || tokens <= 0) {
+    // layer by layer: the first layer writes dX, the others write their share into scratch and it is added
+    const size_t es = elem_size(layers[0]->cfg.dtype);
+    size_t single = 0;
+    for (int g = 0; g < count; ++g) {
+      const size_t w = compact_workspace_bytes(layers[g], tokens);
+      single = w > single ? w : single;
+    }
+    void* part = (char*)workspace + single;
+    for (int g = 0; g < count; ++g) {
+      void* dst = (dX && g > 0) ? part : dX;
+      compact_status_t s = compact_linear_bwd(layers[g], tokens, dY[g], lddy[g], Z[g], ldz[g], W[g], ldw[g], dst,
+                                              dst == dX ? lddx : n, Gc[g], ldg[g], accumulate, workspace, single, stream);
+      if (s != COMPACT_OK) return s;
+      if (dX && g > 0 && tokens > 0) {
+        s = es == 2 ? add_rows<__nv_bfloat16>((__nv_bfloat16*)dX, lddx, (const __nv_bfloat16*)part, n, tokens, n, (cudaStream_t)stream)
+                    : add_rows<float>((float*)dX, lddx, (const float*)part, n, tokens, n, (cudaStream_t)stream);
+        if (s != COMPACT_OK) return s;
+      }
+    }
+    return COMPACT_OK;
+  }
+  typedef __nv_bfloat16 T;
+  if (tokens > 0x7fffffff) return COMPACT_ERR_INVALID_ARG;
+  if (dX && (!aligned16(dX) || !pitch_ok(lddx, n, 2))) return COMPACT_ERR_ALIGNMENT;
+  tc::GroupLayer gl[tc::MAXG];
+  memset(gl, 0, sizeof(gl));
+  for (int g = 0; g < count; ++g) {
+    compact_layer_t* L = layers[g];
+    if (!dY[g] || !Z[g] || !W[g] || !Gc[g]) return COMPACT_ERR_INVALID_ARG;
+    if (!aligned16(dY[g]) || !aligned16(Z[g]) || !aligned16(W[g]) || !aligned16(Gc[g])) return COMPACT_ERR_ALIGNMENT;
+    if (!pitch_ok(lddy[g], L->cfg.m, 2) || !pitch_ok(ldz[g], compact_z_ld(L), 2) || !pitch_ok(ldw[g], L->cfg.m, 2) ||
+        !pitch_ok(ldg[g], L->cfg.m, 4))
+      return COMPACT_ERR_ALIGNMENT;
+    gl[g].m = L->cfg.m; gl[g].r = L->cfg.r; gl[g].zcols = (int)compact_z_ld(L);
+    gl[g].W = (const T*)W[g]; gl[g].ldw = ldw[g];
+    gl[g].Z = (T*)const_cast<void*>(Z[g]); gl[g].ldz = ldz[g];
+    gl[g].dY = (const T*)dY[g]; gl[g].lddy = lddy[g];
+    gl[g].Gc = Gc[g]; gl[g].ldg = ldg[g];
+  }
+  compact_status_t s = check_device(layers[0]);
+  if (s != COMPACT_OK) return s;
+  tc::LaunchInfo li{1, (cudaStream_t)stream, status_word(layers[0]), sched_words(layers[0]), &g_launches};
+  return tc::backward_group(li, count, gl, tokens, n, (T*)dX, lddx, accumulate, workspace, workspace_bytes);
 }
 
 size_t compact_recompute_workspace_bytes(const compact_layer_t* layer, int64_t tokens) {

@@ -1286,11 +1286,11 @@ inline void finish_problem(Problem& p, int splits_wanted) {
 // Number of token splits of Gc = Z^T dY.  A split should be about as long as one dX item
 // (m / 64 k-steps) so that the dynamic scheduler balances well, and there should be enough
 // items to occupy the SMs; at most 32.
-inline int plan_gc_splits(int64_t tokens, int r, int m) {
+inline int plan_gc_splits(int64_t tokens, int r, int m, int dx_ksteps = 0) {
   const int items = ((r + 2 * BM - 1) / (2 * BM)) * ((m + pick_bn(m) - 1) / pick_bn(m));
   const int ksteps = (int)((tokens + BK - 1) / BK);
   if (ksteps < 1) return 1;
-  const int dx_ksteps = (m + BK - 1) / BK;
+  if (dx_ksteps <= 0) dx_ksteps = (m + BK - 1) / BK;
   const int by_len = (ksteps + dx_ksteps - 1) / dx_ksteps;
   const int by_fill = (NUM_SMS + items - 1) / items;
   int s = by_len > by_fill ? by_len : by_fill;
@@ -1468,6 +1468,145 @@ inline compact_status_t backward(const LaunchInfo& li, int64_t tokens, int n, in
     const long long cnt = (long long)r * (m / 4);
     reduce_partials_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, li.stream>>>(
         (const float*)workspace, (long long)r * m, pg.splits, Gc, ldg, r, m, accumulate);
+    (*li.launches)++;
+    if (cudaGetLastError() != cudaSuccess) return COMPACT_ERR_CUDA;
+  }
+  return COMPACT_OK;
+}
+
+// --------------------------------------------------------------------------------------
+// Groups of layers that share their input (q, k, v; gate, up): each layer has its own W and its own P
+// (the paper's appendix on saved tensors lists x P_q, x P_k, x P_v as separate compressed activations).
+// One forward launch computes every Z_g = X P_g and Y_g = X W_g; one backward launch computes
+// dX = sum_g dY_g W_g^T in a single accumulator (K runs over the layers' segments) and every Gc_g.
+// --------------------------------------------------------------------------------------
+struct GroupLayer {
+  ProjectionParams pp;
+  int m, r, zcols;
+  const __nv_bfloat16* W; int64_t ldw;
+  __nv_bfloat16* Y; int64_t ldy;          // forward
+  __nv_bfloat16* Z; int64_t ldz;          // forward (output), backward (input)
+  const __nv_bfloat16* dY; int64_t lddy;  // backward
+  float* Gc; int64_t ldg;                 // backward
+};
+
+inline compact_status_t forward_group(const LaunchInfo& li, int G, const GroupLayer* L, int64_t tokens, int n,
+                                      const __nv_bfloat16* X, int64_t ldx) {
+  if (G < 1 || G > MAXG) return COMPACT_ERR_INVALID_ARG;
+  if (!li.status || !li.sched) return COMPACT_ERR_CUDA;
+  for (int g = 0; g < G; ++g)
+    if (!tc_shape_ok(tokens, n, L[g].m)) return COMPACT_ERR_SHAPE;
+  Params prm;
+  memset(&prm, 0, sizeof(prm));
+  prm.key = L[0].pp.key;
+  prm.num_problems = 2 * G;
+  prm.gen_ring = GEN_A;
+  for (int g = 0; g < G; ++g) {
+    Problem& pz = prm.prob[g];
+    pz.M = L[g].zcols; pz.N = (int)tokens; pz.K = n;
+    pz.nsub = 1;
+    pz.ncol = tokens > BN_MAX ? 2 : 1;
+    pz.a_mode = GENERATED_T; pz.b_mode = TMA_KMAJOR; pz.epi_mode = EPI_BF16_T;
+    set_projection(pz, L[g].pp);
+    finish_problem(pz, 1);
+    if (!make_map(&prm.tmB[g], X, n, tokens, ldx, BK, pz.bn)) return COMPACT_ERR_CUDA;
+    prm.tmA[g] = prm.tmB[g];   // unused by the generated operand
+    if (!make_map(&prm.tmC[g], L[g].Z, L[g].zcols, tokens, L[g].ldz, 32, 64, false)) return COMPACT_ERR_CUDA;
+    Problem& py = prm.prob[G + g];
+    py.M = (int)tokens; py.N = L[g].m; py.K = n;
+    py.a_mode = TMA_KMAJOR; py.b_mode = TMA_MNMAJOR; py.epi_mode = EPI_BF16;
+    finish_problem(py, 1);
+    if (!make_map(&prm.tmA[G + g], X, n, tokens, ldx, BK, BM)) return COMPACT_ERR_CUDA;
+    py.b_blocked = L[g].m % 64 == 0;
+    if (py.b_blocked ? !make_map_blocked(&prm.tmB[G + g], L[g].W, L[g].m, n, L[g].ldw, BK, py.bn / 64)
+                     : !make_map(&prm.tmB[G + g], L[g].W, L[g].m, n, L[g].ldw, 64, BK))
+      return COMPACT_ERR_CUDA;
+    if (!make_map(&prm.tmC[G + g], L[g].Y, L[g].m, tokens, L[g].ldy, 64, 32)) return COMPACT_ERR_CUDA;
+  }
+  return launch(li, prm);
+}
+
+// Workspace of the group backward: the layers' split-K partials, one after the other.
+inline size_t group_gc_workspace_bytes(int G, const int* r, const int* m, int64_t tokens) {
+  int dx_ksteps = 0;
+  for (int g = 0; g < G; ++g) dx_ksteps += (m[g] + BK - 1) / BK;
+  size_t total = 0;
+  for (int g = 0; g < G; ++g) total += (size_t)plan_gc_splits(tokens, r[g], m[g], dx_ksteps) * r[g] * m[g] * sizeof(float);
+  return total;
+}
+
+inline compact_status_t backward_group(const LaunchInfo& li, int G, const GroupLayer* L, int64_t tokens, int n,
+                                       __nv_bfloat16* dX, int64_t lddx, int accumulate, void* workspace,
+                                       size_t workspace_bytes) {
+  if (G < 1 || G > MAXG) return COMPACT_ERR_INVALID_ARG;
+  if (!li.status || !li.sched) return COMPACT_ERR_CUDA;
+  for (int g = 0; g < G; ++g)
+    if (!tc_shape_ok(tokens, n, L[g].m)) return COMPACT_ERR_SHAPE;
+  Params prm;
+  memset(&prm, 0, sizeof(prm));
+  prm.gen_ring = GEN_NONE;
+  int np = 0, slot = 0, dx_ksteps = 0;
+  for (int g = 0; g < G; ++g) dx_ksteps += (L[g].m + BK - 1) / BK;
+  if (dX) {
+    // dX = sum_g dY_g W_g^T: one problem whose K runs over the layers; its items are the longest, so it goes first
+    Problem& px = prm.prob[np++];
+    px.M = (int)tokens; px.N = n; px.K = dx_ksteps * BK;
+    px.a_mode = TMA_KMAJOR; px.b_mode = TMA_KMAJOR; px.epi_mode = EPI_BF16;
+    finish_problem(px, 1);
+    px.nseg = G;
+    int kb = 0;
+    for (int g = 0; g < 4; ++g) {
+      px.seg_begin[g] = kb;
+      if (g < G) kb += (L[g].m + BK - 1) / BK;
+    }
+    for (int g = 0; g < G; ++g) {
+      if (!make_map(&prm.tmA[slot + g], L[g].dY, L[g].m, tokens, L[g].lddy, BK, BM)) return COMPACT_ERR_CUDA;
+      if (!make_map(&prm.tmB[slot + g], L[g].W, L[g].m, n, L[g].ldw, BK, px.bn)) return COMPACT_ERR_CUDA;
+    }
+    if (!make_map(&prm.tmC[slot], dX, n, tokens, lddx, 64, 32)) return COMPACT_ERR_CUDA;
+    slot += G;
+  }
+  size_t ws_off = 0;
+  int splits[MAXG];
+  bool staged[MAXG];
+  size_t part_off[MAXG];
+  for (int g = 0; g < G; ++g) {
+    const int r = L[g].r, m = L[g].m;
+    splits[g] = plan_gc_splits(tokens, r, m, dx_ksteps);
+    staged[g] = splits[g] > 1 || accumulate;
+    part_off[g] = ws_off;
+    ws_off += (size_t)splits[g] * r * m * sizeof(float);
+    if (staged[g] && workspace_bytes < ws_off) return COMPACT_ERR_WORKSPACE;
+    Problem& pg = prm.prob[np++];
+    pg.M = r; pg.N = m; pg.K = (int)tokens;
+    pg.a_mode = TMA_MNMAJOR; pg.b_mode = TMA_MNMAJOR; pg.epi_mode = EPI_F32;
+    finish_problem(pg, splits[g]);
+    splits[g] = pg.splits;
+    float* part = (float*)((char*)workspace + part_off[g]);
+    if (staged[g]) {
+      if (!make_map_f32_3d(&prm.tmC[slot], part, m, r, pg.splits, m, (int64_t)r * m)) return COMPACT_ERR_CUDA;
+    } else {
+      if (!make_map_f32_3d(&prm.tmC[slot], L[g].Gc, m, r, 1, L[g].ldg, (int64_t)r * L[g].ldg)) return COMPACT_ERR_CUDA;
+    }
+    pg.a_blocked = L[g].zcols % 64 == 0;
+    pg.b_blocked = m % 64 == 0;
+    if (pg.a_blocked ? !make_map_blocked(&prm.tmA[slot], L[g].Z, L[g].zcols, tokens, L[g].ldz, BK, 2)
+                     : !make_map(&prm.tmA[slot], L[g].Z, L[g].zcols, tokens, L[g].ldz, 64, BK))
+      return COMPACT_ERR_CUDA;
+    if (pg.b_blocked ? !make_map_blocked(&prm.tmB[slot], L[g].dY, m, tokens, L[g].lddy, BK, pg.bn / 64)
+                     : !make_map(&prm.tmB[slot], L[g].dY, m, tokens, L[g].lddy, 64, BK))
+      return COMPACT_ERR_CUDA;
+    ++slot;
+  }
+  prm.num_problems = np;
+  compact_status_t s = launch(li, prm);
+  if (s != COMPACT_OK) return s;
+  for (int g = 0; g < G; ++g) {
+    if (!staged[g]) continue;
+    const int r = L[g].r, m = L[g].m;
+    const long long cnt = (long long)r * (m / 4);
+    reduce_partials_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, li.stream>>>(
+        (const float*)((char*)workspace + part_off[g]), (long long)r * m, splits[g], L[g].Gc, L[g].ldg, r, m, accumulate);
     (*li.launches)++;
     if (cudaGetLastError() != cudaSuccess) return COMPACT_ERR_CUDA;
   }

@@ -267,6 +267,36 @@ def test_bwd_recompute_is_the_sketched_gradient_by_brute_force():
     assert np.array_equal(Gb, co.linear_bwd(dY, co.round_bf16(X @ P), W, mode="bf16")[1])
 
 
+def test_group_backward_is_gradient_of_summed_inner_products():
+    # layers sharing x: d/dx sum_g <x W_g, dY_g> by finite differences, Gc_g by element loops
+    rng = np.random.default_rng(9)
+    bl, n = 5, 6
+    ms, rs = [4, 3, 4], [2, 3, 2]
+    X = rng.standard_normal((bl, n))
+    Ws = [rng.standard_normal((n, m)) for m in ms]
+    dYs = [rng.standard_normal((bl, m)) for m in ms]
+    Ps = [co.projection(21, g, 0, n, r) for g, r in enumerate(rs)]
+    Ys, Zs = co.group_fwd(X, Ws, Ps)
+    for g in range(3):
+        assert np.allclose(Ys[g], X @ Ws[g], rtol=1e-13) and np.allclose(Zs[g], X @ Ps[g], rtol=1e-13)
+    dX, Gcs = co.group_bwd(dYs, Zs, Ws)
+    f = lambda x: sum(np.sum((x @ W) * dY) for W, dY in zip(Ws, dYs))
+    h = 1e-6
+    for (t, k) in [(0, 0), (4, 5), (2, 3)]:
+        Xp = X.copy(); Xp[t, k] += h
+        Xm = X.copy(); Xm[t, k] -= h
+        assert dX[t, k] == pytest.approx((f(Xp) - f(Xm)) / (2 * h), rel=1e-7)
+    for g in range(3):
+        for j in range(rs[g]):
+            for c in range(ms[g]):
+                want = sum(Zs[g][t, j] * dYs[g][t, c] for t in range(bl))
+                assert Gcs[g][j, c] == pytest.approx(want, rel=1e-12, abs=1e-13)
+    # a group of one is the single layer
+    d1, g1 = co.group_bwd(dYs[:1], Zs[:1], Ws[:1])
+    d2, g2 = co.linear_bwd(dYs[0], Zs[0], Ws[0])
+    assert np.array_equal(d1, d2) and np.array_equal(g1[0], g2)
+
+
 # --- Adam ----------------------------------------------------------------------------
 def test_adam_constant_gradient_closed_form():
     rng = np.random.default_rng(4)

@@ -255,6 +255,43 @@ def test_backward_recompute_fp32():
     assert co.rel_frobenius(to64(Gc), Gco) <= TOL["f32"] and co.rel_frobenius(to64(dX), dXo) <= TOL["f32"]
 
 
+@pytest.mark.parametrize("tokens,n,shapes", [
+    (1100, 320, [(512, 72), (512, 72), (512, 72)]),       # q, k, v
+    (700, 256, [(1096, 40), (520, 136)]),                 # two layers of different width and rank, ragged
+    (300, 192, [(200, 24)]),                              # a group of one
+])
+def test_group_forward_backward(family, tokens, n, shapes):
+    wl = wlm.Workload("grp", 95, "bf16", tokens, [wlm.LayerShape(f"l{g}", n, m, r) for g, (m, r) in enumerate(shapes)],
+                      x_scale_inv_sqrt_n=True)
+    pairs = [make_pair(wl, g) for g in range(len(shapes))]
+    gpus, oras = [p[0] for p in pairs], [p[1] for p in pairs]
+    Ws = [p[2].cuda() for p in pairs]
+    X = wlm.draw_X(wl, 0, 0).cuda()
+    dYs = [wlm.draw_dY(wl, g, 0).cuda() for g in range(len(shapes))]
+    grp = cb.CompactGroup(gpus)
+    Ys, Zs, eps = grp.forward(X, Ws)
+    for g, lay in enumerate(gpus):
+        Y1, Z1, ep = lay.forward(X, Ws[g])
+        assert ep == eps[g]
+        assert torch.equal(Ys[g].view(torch.int16), Y1.view(torch.int16))
+        assert torch.equal(Zs[g].view(torch.int16), Z1.view(torch.int16))
+    dX, Gcs = grp.backward(dYs, Zs, Ws)
+    dXo, Gco = co.group_bwd([to64(d) for d in dYs], [to64(Zs[g][:, :shapes[g][1]]) for g in range(len(shapes))],
+                            [o.W for o in oras], mode="bf16")
+    assert co.rel_frobenius(to64(dX), dXo) <= TOL["bf16"]
+    for g in range(len(shapes)):
+        assert co.rel_frobenius(to64(Gcs[g]), Gco[g]) <= TOL["bf16"]
+    # run to run bitwise, and accumulation over two micro-batches
+    dX2, Gcs2 = grp.backward(dYs, Zs, Ws)
+    assert torch.equal(dX.view(torch.int16), dX2.view(torch.int16)) and all(torch.equal(a, b) for a, b in zip(Gcs, Gcs2))
+    h = 256
+    Ga = [torch.empty_like(G) for G in Gcs]
+    grp.backward([d[:h] for d in dYs], [z[:h] for z in Zs], Ws, Gcs=Ga, need_dX=False)
+    grp.backward([d[h:] for d in dYs], [z[h:] for z in Zs], Ws, Gcs=Ga, need_dX=False, accumulate=True)
+    for g in range(len(shapes)):
+        assert co.rel_frobenius(to64(Ga[g]), Gco[g]) <= TOL["bf16"]
+
+
 def test_empty_batch_and_epoch_guard():
     lay = cb.CompactLinear(128, 512, 16, refresh_T=1)
     W = torch.zeros((128, 512), dtype=torch.bfloat16, device="cuda")
