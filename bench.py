@@ -4,7 +4,7 @@
 One "step" is one pass of the whole hot path -- forward [Y|Z] = X[W|P], backward
 dX = dY W^T and Gc = Z^T dY, Adam update W <- W - lr*alpha*P N, refresh -- over
 every layer of the LLaMA-7B-shaped layer set (16384 tokens, hidden 4096) with
-synthetic inputs.  Prints ONE JSON line (see README for the keys).
+synthetic inputs.  Prints ONE JSON line.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c5|c4|c3|c2]
 
