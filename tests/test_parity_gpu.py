@@ -292,6 +292,32 @@ def test_group_forward_backward(family, tokens, n, shapes):
         assert co.rel_frobenius(to64(Ga[g]), Gco[g]) <= TOL["bf16"]
 
 
+@pytest.mark.parametrize("tokens,n,m,r", [(2304, 576, 1544, 200), (640, 128, 64, 24), (4100, 256, 520, 136)])
+def test_repeated_launches_bitwise_stable(tokens, n, m, r):
+    # the cluster hand-shakes, the two MMA issuers and the ring-geometry change are timing-dependent machinery:
+    # forty runs of each call must give the same bits and leave the status word clear
+    wl = wlm.Workload("rep", 94, "bf16", tokens, [wlm.LayerShape("l", n, m, r)], x_scale_inv_sqrt_n=True)
+    gpu, _, W0 = make_pair(wl, 0)
+    X, dY = wlm.draw_X(wl, 0, 0).cuda(), wlm.draw_dY(wl, 0, 0).cuda()
+    W = W0.cuda()
+    Y0, Z0, ep = gpu.forward(X, W)
+    dX0, G0 = gpu.backward(dY, Z0, W)
+    M0, V0 = torch.zeros_like(G0), torch.zeros_like(G0)
+    W1 = W.clone()
+    gpu.adam_update(W1, G0, M0, V0, ep)
+    st = gpu.state()
+    for _ in range(40):
+        Y, Z, _ = gpu.forward(X, W)
+        dX, G = gpu.backward(dY, Z, W)
+        assert torch.equal(Y.view(torch.int16), Y0.view(torch.int16)) and torch.equal(Z.view(torch.int16), Z0.view(torch.int16))
+        assert torch.equal(G, G0) and torch.equal(dX.view(torch.int16), dX0.view(torch.int16))
+        gpu.set_state(st.seed, st.layer_id, st.epoch, 0)       # same step count: same bias correction
+        Wk, Mk, Vk = W.clone(), torch.zeros_like(G0), torch.zeros_like(G0)
+        gpu.adam_update(Wk, G0, Mk, Vk, ep)
+        assert torch.equal(Wk.view(torch.int16), W1.view(torch.int16)) and torch.equal(Mk, M0) and torch.equal(Vk, V0)
+    assert gpu.status() == cb.OK
+
+
 def test_empty_batch_and_epoch_guard():
     lay = cb.CompactLinear(128, 512, 16, refresh_T=1)
     W = torch.zeros((128, 512), dtype=torch.bfloat16, device="cuda")
