@@ -346,10 +346,10 @@ def run_ours(args):
     upd_gbs = upd_bytes / (upd_ms * 1e-3) / 1e9
     gemm_launches = 2 * len(wl.layers)
     # DRAM traffic from the committed ncu capture of the C5 q_proj launches
-    # (profiles/compact_gemm_kernel_c5_qproj_full.md): forward 615.8 MB, backward 624.7 MB for
+    # (profiles/compact_gemm_kernel_c5_qproj_full.md): forward 578.9 MB, backward 629.6 MB for
     # 1236.95 algorithmic GFLOP; update 37.9 MB for 109.1 MB of algorithmic bytes (W stays in L2
     # at that size).  Scaled to this workload's launches in proportion to the algorithmic work.
-    traffic_gemm = (615.8e6 + 624.7e6) / 1236.95e9 * gemm_flops / gemm_launches
+    traffic_gemm = (578.9e6 + 629.6e6) / 1236.95e9 * gemm_flops / gemm_launches
     traffic_upd = None
     roofline = {"kernel": "compact_gemm_kernel (forward and backward launches)", "bound": "tensor",
                 "achieved": gemm_tflops, "peak": tens_peak, "unit": "TFLOP/s", "frac": gemm_tflops / tens_peak,
