@@ -1308,14 +1308,17 @@ inline size_t gc_workspace_bytes(int64_t tokens, int r, int m) {
 }
 
 inline compact_status_t launch(const LaunchInfo& li, Params& prm) {
-  static bool attr_set = false;
-  if (!attr_set) {
+  // the opt-in to large dynamic shared memory is a per-device attribute of the kernel
+  static std::atomic<bool> attr_set[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return COMPACT_ERR_CUDA; }
+  if (!attr_set[dev].load(std::memory_order_acquire)) {
     if (cudaFuncSetAttribute(compact_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
         cudaFuncSetAttribute(compact_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
       cudaGetLastError();
       return COMPACT_ERR_CUDA;
     }
-    attr_set = true;
+    attr_set[dev].store(true, std::memory_order_release);
   }
   bool group = prm.num_problems > 2;
   for (int i = 0; i < prm.num_problems; ++i) group = group || prm.prob[i].nseg > 1;
