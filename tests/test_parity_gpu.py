@@ -318,6 +318,36 @@ def test_repeated_launches_bitwise_stable(tokens, n, m, r):
     assert gpu.status() == cb.OK
 
 
+def test_group_of_four_runs_layer_by_layer_and_empty_group_call():
+    # more than three layers (or mixed seeds, fp32, the SIMT family) take the layer-by-layer route with the same results
+    tokens, n = 260, 128
+    shapes = [(72, 16), (136, 24), (64, 8), (200, 40)]
+    wl = wlm.Workload("grp4", 93, "bf16", tokens, [wlm.LayerShape(f"l{g}", n, m, r) for g, (m, r) in enumerate(shapes)],
+                      x_scale_inv_sqrt_n=True)
+    pairs = [make_pair(wl, g) for g in range(4)]
+    gpus, oras = [p[0] for p in pairs], [p[1] for p in pairs]
+    Ws = [p[2].cuda() for p in pairs]
+    X = wlm.draw_X(wl, 0, 0).cuda()
+    dYs = [wlm.draw_dY(wl, g, 0).cuda() for g in range(4)]
+    grp = cb.CompactGroup(gpus)
+    Ys, Zs, _ = grp.forward(X, Ws)
+    for g, lay in enumerate(gpus):
+        Y1, Z1, _ = lay.forward(X, Ws[g])
+        assert torch.equal(Ys[g].view(torch.int16), Y1.view(torch.int16)) and torch.equal(Zs[g].view(torch.int16), Z1.view(torch.int16))
+    dX, Gcs = grp.backward(dYs, Zs, Ws)
+    dXo, Gco = co.group_bwd([to64(d) for d in dYs], [to64(Zs[g][:, :shapes[g][1]]) for g in range(4)], [o.W for o in oras], mode="bf16")
+    assert co.rel_frobenius(to64(dX), dXo) <= TOL["bf16"]
+    for g in range(4):
+        assert co.rel_frobenius(to64(Gcs[g]), Gco[g]) <= TOL["bf16"]
+    # no tokens: outputs of zero rows, Gc zeroed
+    E = torch.empty((0, n), dtype=torch.bfloat16, device="cuda")
+    Ye, Ze, _ = grp.forward(E, Ws)
+    assert all(y.shape[0] == 0 for y in Ye)
+    Gz = [torch.full((r, m), 3.0, device="cuda") for (m, r) in shapes]
+    grp.backward([torch.empty((0, m), dtype=torch.bfloat16, device="cuda") for (m, r) in shapes], Ze, Ws, Gcs=Gz, need_dX=False)
+    assert not any(g.any() for g in Gz)
+
+
 def test_empty_batch_and_epoch_guard():
     lay = cb.CompactLinear(128, 512, 16, refresh_T=1)
     W = torch.zeros((128, 512), dtype=torch.bfloat16, device="cuda")
