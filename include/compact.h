@@ -49,7 +49,8 @@ typedef enum {
   COMPACT_ERR_UNSUPPORTED_ARCH = 7,
   COMPACT_ERR_CUDA = 8,
   COMPACT_ERR_DEVICE_TIMEOUT = 9,
-  COMPACT_ERR_SCRATCH_LIMIT = 10
+  COMPACT_ERR_SCRATCH_LIMIT = 10,
+  COMPACT_ERR_TOO_MANY_LAYERS = 11
 } compact_status_t;
 
 typedef enum { COMPACT_F32 = 0, COMPACT_BF16 = 1 } compact_dtype_t;
@@ -190,11 +191,16 @@ compact_status_t compact_adam_update(compact_layer_t* layer,
  * that allocates.  Layers with r * m * 4 bytes > COMPACT_NOALLOC_SCRATCH_BYTES are
  * rejected with COMPACT_ERR_SCRATCH_LIMIT before anything is launched.
  *
- * The first call on each device looks up the array's device address (one runtime query,
- * no allocation); make that first call outside any stream capture.  All calls on a device
- * share the one array, and it keeps whatever the previous call left in it (each call
- * overwrites the r x m entries it reads, so nothing needs clearing).  Two calls whose
- * kernels can overlap on the GPU -- different streams, different layers -- race on it:
+ * The array comes into existence when the CUDA runtime loads this library's device code on
+ * a GPU, which (with lazy loading) is the first library call that launches a kernel or asks
+ * for a symbol's address there -- possibly this one.  A process that hands all of HBM to its
+ * own pool must therefore make one library call on each device (any launch, or a first call
+ * of this function) BEFORE it gives the memory away, or that first call fails with
+ * COMPACT_ERR_CUDA.  That first call also looks up the array's device address (a runtime
+ * query); make it outside any stream capture.  Later calls allocate nothing and query nothing.
+ * All calls on a device share the one array, and it keeps whatever the previous call left in
+ * it (each call overwrites the r x m entries it reads, so nothing needs clearing).  Two calls
+ * whose kernels can overlap on the GPU -- different streams, different layers -- race on it:
  * keep them ordered on one stream or synchronise between them. */
 #define COMPACT_NOALLOC_SCRATCH_BYTES (32u << 20)
 compact_status_t compact_adam_update_noalloc(compact_layer_t* layer,
@@ -221,11 +227,15 @@ compact_status_t compact_layer_status(compact_layer_t* layer);
 
 /* Test hooks that make the in-kernel generator observable.
  * compact_debug_philox_u32: out_dev[n x 4*ceil(r/4)] receives the raw Philox
- * words behind P (Algorithm 1 lines 1-2).
+ * words behind P (Algorithm 1 lines 1-2), from the generic ten-round function.
+ * compact_debug_philox_layer_u32: the same words from the form the GEMM kernels'
+ * generators call (first round partly precomputed on the host per layer).
  * compact_debug_projection: P_dev[n x r] (layer dtype, pitch r) receives P at
  * `epoch`, produced by the same device function the GEMM kernels call. */
 compact_status_t compact_debug_philox_u32(uint64_t seed, uint32_t layer_id, uint32_t epoch,
                                           int32_t n, int32_t r, uint32_t* out_dev, void* stream);
+compact_status_t compact_debug_philox_layer_u32(uint64_t seed, uint32_t layer_id, uint32_t epoch,
+                                                int32_t n, int32_t r, uint32_t* out_dev, void* stream);
 compact_status_t compact_debug_projection(const compact_layer_t* layer, uint32_t epoch,
                                           void* P_dev, void* stream);
 

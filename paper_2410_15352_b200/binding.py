@@ -20,6 +20,7 @@ OK = 0
 ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGNMENT, ERR_DTYPE, ERR_EPOCH_MISMATCH, ERR_WORKSPACE, \
     ERR_UNSUPPORTED_ARCH, ERR_CUDA, ERR_DEVICE_TIMEOUT = range(1, 10)
 ERR_SCRATCH_LIMIT = 10
+ERR_TOO_MANY_LAYERS = 11
 NOALLOC_SCRATCH_BYTES = 32 << 20
 F32, BF16 = 0, 1
 
@@ -29,7 +30,7 @@ EXPORTS = [
     "compact_linear_bwd_recompute", "compact_group_workspace_bytes", "compact_group_fwd", "compact_group_bwd",
     "compact_adam_update", "compact_adam_update_noalloc",
     "compact_refresh_projection", "compact_layer_get_state", "compact_layer_set_state",
-    "compact_layer_status", "compact_debug_philox_u32", "compact_debug_projection",
+    "compact_layer_status", "compact_debug_philox_u32", "compact_debug_philox_layer_u32", "compact_debug_projection",
     "compact_set_kernel_family", "compact_kernel_launch_count", "compact_status_string",
 ]
 
@@ -85,6 +86,7 @@ def lib() -> C.CDLL:
     L.compact_layer_set_state.argtypes = [vp, C.POINTER(LayerState)]
     L.compact_layer_status.argtypes = [vp]
     L.compact_debug_philox_u32.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_int32, C.c_int32, vp, vp]
+    L.compact_debug_philox_layer_u32.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_int32, C.c_int32, vp, vp]
     L.compact_debug_projection.argtypes = [vp, C.c_uint32, vp, vp]
     L.compact_set_kernel_family.argtypes = [C.c_int]
     L.compact_kernel_launch_count.restype = C.c_uint64
@@ -126,9 +128,11 @@ def kernel_launch_count() -> int:
     return int(lib().compact_kernel_launch_count())
 
 
-def debug_philox_u32(seed: int, layer_id: int, epoch: int, n: int, r: int, stream=None) -> torch.Tensor:
+def debug_philox_u32(seed: int, layer_id: int, epoch: int, n: int, r: int, stream=None, layer_form: bool = False) -> torch.Tensor:
+    """Raw Philox words behind P; layer_form=True takes them from the function the GEMM kernels' generators call."""
     out = torch.empty((n, 4 * ((r + 3) // 4)), dtype=torch.int32, device="cuda")
-    _check(lib().compact_debug_philox_u32(seed, layer_id, epoch, n, r, _ptr(out), _stream(stream)), "debug_philox_u32")
+    fn = lib().compact_debug_philox_layer_u32 if layer_form else lib().compact_debug_philox_u32
+    _check(fn(seed, layer_id, epoch, n, r, _ptr(out), _stream(stream)), "debug_philox_u32")
     return out
 
 

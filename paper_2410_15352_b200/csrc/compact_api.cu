@@ -6,7 +6,9 @@
 #include <string.h>
 
 #include <atomic>
+#include <mutex>
 #include <new>
+#include <vector>
 
 #include "../../include/compact.h"
 #include "philox.cuh"
@@ -31,19 +33,60 @@ std::atomic<uint64_t> g_launches{0};
 #define CFG_CS 2   // CTAs of a cluster that share each generated tile of P
 #endif
 std::atomic<int> g_family{0};
-std::atomic<int> g_next_slot{0};
 
-constexpr int kStatusSlots = 256;
+// One status word per live layer: kernels OR error bits into it, compact_layer_status reads and clears it.
+// Slots come from a free list and go back on destroy; when none is left, compact_layer_create fails.
+constexpr int kStatusSlots = 4096;
 __device__ unsigned int g_status_words[kStatusSlots];
-// Two words per layer slot for the dynamic item scheduler of the tensor-core kernel
-// (next item, finished CTAs).  Zero at load; each launch leaves them zero again.
-__device__ unsigned int g_sched_words[kStatusSlots][2];
+// Two words per tensor-core launch for its dynamic item scheduler (next item, finished CTAs), taken from a
+// ring by launch sequence number, so that launches that overlap on the GPU (other layers, other streams)
+// never share them.  Zero at load; the last CTA of a launch leaves its pair zero again.  The ring is far
+// longer than the number of launches that can be in flight at once.
+constexpr int kSchedRing = 4096;
+__device__ unsigned int g_sched_words[kSchedRing][2];
+std::atomic<uint64_t> g_sched_seq{0};
+
+std::mutex g_slot_mutex;
+std::vector<int> g_free_slots;
+int g_slots_handed_out = 0;
+
+int take_status_slot() {
+  std::lock_guard<std::mutex> lock(g_slot_mutex);
+  if (!g_free_slots.empty()) {
+    const int s = g_free_slots.back();
+    g_free_slots.pop_back();
+    return s;
+  }
+  if (g_slots_handed_out < kStatusSlots) return g_slots_handed_out++;
+  return -1;
+}
+void give_back_status_slot(int s) {
+  std::lock_guard<std::mutex> lock(g_slot_mutex);
+  g_free_slots.push_back(s);
+}
+
+// Device addresses of the two arrays, asked once per device (with that device current).
+constexpr int kMaxDevices = 64;
+std::atomic<unsigned int*> g_status_base[kMaxDevices];
+std::atomic<unsigned int*> g_sched_base[kMaxDevices];
+
+template <class Sym>
+unsigned int* symbol_base(std::atomic<unsigned int*>* cache, const Sym& sym) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return nullptr; }
+  unsigned int* p = cache[dev].load(std::memory_order_acquire);
+  if (!p) {
+    if (cudaGetSymbolAddress((void**)&p, sym) != cudaSuccess || !p) { cudaGetLastError(); return nullptr; }
+    cache[dev].store(p, std::memory_order_release);
+  }
+  return p;
+}
 
 inline size_t elem_size(int dtype) { return dtype == COMPACT_BF16 ? 2 : 4; }
 inline int64_t round_up(int64_t a, int64_t b) { return (a + b - 1) / b * b; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-compact_status_t check_device(compact_layer_t* L) {
+compact_status_t check_device(compact_layer_t* L, void* stream) {
   if (L->device_checked == 1) return COMPACT_OK;
   if (L->device_checked == -1) return COMPACT_ERR_UNSUPPORTED_ARCH;
   int dev = 0;
@@ -54,20 +97,25 @@ compact_status_t check_device(compact_layer_t* L) {
     return COMPACT_ERR_CUDA;
   }
   if (major != 10) { L->device_checked = -1; return COMPACT_ERR_UNSUPPORTED_ARCH; }
+  // the slot may have belonged to a layer that was destroyed without its status having been read
+  unsigned int* w = symbol_base(g_status_base, g_status_words);
+  if (!w || cudaMemsetAsync(w + L->status_slot, 0, sizeof(unsigned int), (cudaStream_t)stream) != cudaSuccess) {
+    cudaGetLastError();
+    return COMPACT_ERR_CUDA;
+  }
   L->device_checked = 1;
   return COMPACT_OK;
 }
 
 unsigned int* status_word(const compact_layer_t* L) {
-  unsigned int* base = nullptr;
-  if (cudaGetSymbolAddress((void**)&base, g_status_words) != cudaSuccess) { cudaGetLastError(); return nullptr; }
-  return base + L->status_slot;
+  unsigned int* base = symbol_base(g_status_base, g_status_words);
+  return base ? base + L->status_slot : nullptr;
 }
 
-unsigned int* sched_words(const compact_layer_t* L) {
-  unsigned int* base = nullptr;
-  if (cudaGetSymbolAddress((void**)&base, g_sched_words) != cudaSuccess) { cudaGetLastError(); return nullptr; }
-  return base + 2 * L->status_slot;
+// The scheduler words of the next tensor-core launch.
+unsigned int* sched_words(const compact_layer_t*) {
+  unsigned int* base = symbol_base(g_sched_base, g_sched_words);
+  return base ? base + 2 * (g_sched_seq.fetch_add(1) % kSchedRing) : nullptr;
 }
 
 ProjectionParams make_pp(const compact_layer_t* L, uint32_t epoch) {
@@ -195,7 +243,8 @@ compact_status_t compact_layer_create(const compact_layer_config_t* cfg, compact
   L->epoch = 0;
   L->step = 0;
   L->last_refresh_step = 0;
-  L->status_slot = g_next_slot.fetch_add(1) % kStatusSlots;
+  L->status_slot = take_status_slot();
+  if (L->status_slot < 0) { delete L; return COMPACT_ERR_TOO_MANY_LAYERS; }
   L->device_checked = 0;
   *out = L;
   return COMPACT_OK;
@@ -203,6 +252,7 @@ compact_status_t compact_layer_create(const compact_layer_config_t* cfg, compact
 
 compact_status_t compact_layer_destroy(compact_layer_t* layer) {
   if (!layer) return COMPACT_ERR_INVALID_ARG;
+  give_back_status_slot(layer->status_slot);
   delete layer;
   return COMPACT_OK;
 }
@@ -236,7 +286,7 @@ compact_status_t compact_linear_fwd(compact_layer_t* L, int64_t tokens, const vo
   if (!pitch_ok(ldx, L->cfg.n, es) || !pitch_ok(ldw, L->cfg.m, es) || !pitch_ok(ldy, L->cfg.m, es) ||
       (Z && !pitch_ok(ldz, compact_z_ld(L), es)))
     return COMPACT_ERR_ALIGNMENT;
-  compact_status_t s = check_device(L);
+  compact_status_t s = check_device(L, stream);
   if (s != COMPACT_OK) return s;
   cudaStream_t st = (cudaStream_t)stream;
   if (L->cfg.dtype == COMPACT_BF16) {
@@ -260,7 +310,7 @@ compact_status_t compact_linear_bwd(compact_layer_t* L, int64_t tokens, const vo
   if (!Gc) return COMPACT_ERR_INVALID_ARG;
   const size_t es = elem_size(L->cfg.dtype);
   if (!aligned16(Gc) || !pitch_ok(ldg, L->cfg.m, 4)) return COMPACT_ERR_ALIGNMENT;
-  compact_status_t s = check_device(L);
+  compact_status_t s = check_device(L, stream);
   cudaStream_t st = (cudaStream_t)stream;
   if (tokens == 0) {
     // An empty micro-batch contributes nothing: Gc is zeroed unless accumulating.
@@ -358,7 +408,7 @@ compact_status_t compact_group_fwd(compact_layer_t* const* layers, int count, in
     gl[g].Y = (T*)Y[g]; gl[g].ldy = ldy[g];
     gl[g].Z = (T*)Z[g]; gl[g].ldz = ldz[g];
   }
-  compact_status_t s = check_device(layers[0]);
+  compact_status_t s = check_device(layers[0], stream);
   if (s != COMPACT_OK) return s;
   tc::LaunchInfo li{g_family.load() == 2 ? 1 : CFG_CS, (cudaStream_t)stream, status_word(layers[0]), sched_words(layers[0]), &g_launches};
   return tc::forward_group(li, count, gl, tokens, layers[0]->cfg.n, (const T*)X, ldx);
@@ -414,7 +464,7 @@ compact_status_t compact_group_bwd(compact_layer_t* const* layers, int count, in
     gl[g].dY = (const T*)dY[g]; gl[g].lddy = lddy[g];
     gl[g].Gc = Gc[g]; gl[g].ldg = ldg[g];
   }
-  compact_status_t s = check_device(layers[0]);
+  compact_status_t s = check_device(layers[0], stream);
   if (s != COMPACT_OK) return s;
   tc::LaunchInfo li{1, (cudaStream_t)stream, status_word(layers[0]), sched_words(layers[0]), &g_launches};
   return tc::backward_group(li, count, gl, tokens, n, (T*)dX, lddx, accumulate, workspace, workspace_bytes);
@@ -439,7 +489,7 @@ compact_status_t compact_linear_bwd_recompute(compact_layer_t* L, int64_t tokens
     if (!aligned16(X) || !pitch_ok(ldx, L->cfg.n, es)) return COMPACT_ERR_ALIGNMENT;
     if (!workspace || workspace_bytes < compact_recompute_workspace_bytes(L, tokens)) return COMPACT_ERR_WORKSPACE;
     if (!aligned16(workspace)) return COMPACT_ERR_ALIGNMENT;
-    compact_status_t s = check_device(L);
+    compact_status_t s = check_device(L, stream);
     if (s != COMPACT_OK) return s;
     cudaStream_t st = (cudaStream_t)stream;
     // Z = X P again, into the front of the workspace
@@ -473,7 +523,7 @@ compact_status_t compact_adam_update(compact_layer_t* L, void* W, int64_t ldw, c
   if (!pitch_ok(ldw, L->cfg.m, es) || !pitch_ok(ldg, L->cfg.m, 4)) return COMPACT_ERR_ALIGNMENT;
   if (!workspace || workspace_bytes < compact_workspace_bytes(L, 0)) return COMPACT_ERR_WORKSPACE;
   if (!aligned16(workspace)) return COMPACT_ERR_ALIGNMENT;
-  compact_status_t s = check_device(L);
+  compact_status_t s = check_device(L, stream);
   if (s != COMPACT_OK) return s;
   if (isnan(lr)) lr = L->cfg.lr;
   cudaStream_t st = (cudaStream_t)stream;
@@ -501,7 +551,6 @@ compact_status_t compact_adam_update(compact_layer_t* L, void* W, int64_t ldw, c
 static __device__ __align__(256) unsigned char g_noalloc_scratch[COMPACT_NOALLOC_SCRATCH_BYTES];
 
 namespace {
-constexpr int kMaxDevices = 64;
 std::atomic<void*> g_noalloc_ptr[kMaxDevices];
 
 // Device address of the scratch array on the current device (looked up on first use).
@@ -524,7 +573,7 @@ compact_status_t compact_adam_update_noalloc(compact_layer_t* L, void* W, int64_
   if (!L) return COMPACT_ERR_INVALID_ARG;
   // the update needs r x m scratch entries (fp32 in the plain kernels, bf16 in the tensor-core ones)
   if (compact_workspace_bytes(L, 0) > (size_t)COMPACT_NOALLOC_SCRATCH_BYTES) return COMPACT_ERR_SCRATCH_LIMIT;
-  compact_status_t s = check_device(L);
+  compact_status_t s = check_device(L, stream);
   if (s != COMPACT_OK) return s;
   void* scratch = nullptr;
   s = noalloc_scratch(&scratch);
@@ -569,8 +618,8 @@ compact_status_t compact_layer_set_state(compact_layer_t* L, const compact_layer
 
 compact_status_t compact_layer_status(compact_layer_t* L) {
   if (!L) return COMPACT_ERR_INVALID_ARG;
-  compact_status_t s = check_device(L);
-  if (s != COMPACT_OK) return s;
+  if (L->device_checked == 0) return COMPACT_OK;      // nothing has been launched for this layer yet
+  if (L->device_checked < 0) return COMPACT_ERR_UNSUPPORTED_ARCH;
   unsigned int* w = status_word(L);
   if (!w) return COMPACT_ERR_CUDA;
   unsigned int v = 0;
@@ -596,6 +645,19 @@ compact_status_t compact_debug_philox_u32(uint64_t seed, uint32_t layer_id, uint
   return launch_result();
 }
 
+compact_status_t compact_debug_philox_layer_u32(uint64_t seed, uint32_t layer_id, uint32_t epoch, int32_t n, int32_t r,
+                                                uint32_t* out_dev, void* stream) {
+  if (n < 1 || r < 1 || !out_dev) return COMPACT_ERR_INVALID_ARG;
+  if (!aligned16(out_dev)) return COMPACT_ERR_ALIGNMENT;
+  const int groups = (r + 3) / 4;
+  const int64_t cnt = (int64_t)n * groups;
+  const uint64_t pl = (uint64_t)0xCD9E8D57u * (uint64_t)layer_id;
+  debug_philox_layer_words_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
+      make_philox_key(seed), (uint32_t)(pl >> 32), (uint32_t)pl, epoch, n, groups, out_dev);
+  g_launches++;
+  return launch_result();
+}
+
 compact_status_t compact_debug_projection(const compact_layer_t* L, uint32_t epoch, void* P_dev, void* stream) {
   if (!L || !P_dev) return COMPACT_ERR_INVALID_ARG;
   const ProjectionParams pp = make_pp(L, epoch);
@@ -616,28 +678,6 @@ int compact_set_kernel_family(int family) {
 
 uint64_t compact_kernel_launch_count(void) { return g_launches.load(); }
 
-#if defined(COMPACT_PROFILE) || defined(COMPACT_PROFILE_GEN)
-// Profiling build only: cumulative clocks of the MMA-issuing threads
-// [wait accumulator, wait B, wait A, issue, total]; reading clears them.
-void compact_debug_profile(unsigned long long* out) {
-  cudaDeviceSynchronize();
-  cudaMemcpyFromSymbol(out, tc::g_prof, sizeof(unsigned long long) * 8);
-  unsigned long long z[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-  cudaMemcpyToSymbol(tc::g_prof, z, sizeof(z));
-}
-#endif
-#ifdef COMPACT_PROFILE_GEN
-void compact_debug_trace(long long* out) {
-  cudaDeviceSynchronize();
-  cudaMemcpyFromSymbol(out, tc::g_trace, sizeof(long long) * 128);
-}
-void compact_debug_timeline(long long* out, unsigned int* n) {
-  cudaDeviceSynchronize();
-  cudaMemcpyFromSymbol(out, tc::g_tl, sizeof(long long) * 128);
-  cudaMemcpyFromSymbol(n, tc::g_tl_n, sizeof(unsigned int));
-}
-#endif
-
 const char* compact_status_string(compact_status_t s) {
   switch (s) {
     case COMPACT_OK: return "ok";
@@ -650,6 +690,7 @@ const char* compact_status_string(compact_status_t s) {
     case COMPACT_ERR_UNSUPPORTED_ARCH: return "device is not compute capability 10.x";
     case COMPACT_ERR_CUDA: return "CUDA runtime error";
     case COMPACT_ERR_DEVICE_TIMEOUT: return "a kernel gave up on a bounded wait";
+    case COMPACT_ERR_TOO_MANY_LAYERS: return "too many live layers (4096 status slots); destroy some first";
     case COMPACT_ERR_SCRATCH_LIMIT: return "layer needs more scratch than the allocation-free entry point carries (r*m*4 > 32 MiB)";
   }
   return "unknown status";

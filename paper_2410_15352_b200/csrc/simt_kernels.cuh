@@ -151,6 +151,17 @@ __global__ void debug_philox_words_kernel(PhiloxKey key, uint32_t layer_id, uint
   reinterpret_cast<uint4*>(out)[idx] = x;
 }
 
+// The same words through the form the GEMM kernels' generators call: the first round's product with the
+// layer word comes precomputed from the host.
+__global__ void debug_philox_layer_words_kernel(PhiloxKey key, uint32_t layer_hi, uint32_t layer_lo, uint32_t epoch, int n,
+                                                int groups, uint32_t* out) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)n * groups) return;
+  const int i = (int)(idx / groups), q = (int)(idx % groups);
+  const uint4 x = philox4x32_10_layer((uint32_t)q, (uint32_t)i, epoch, layer_hi, layer_lo, key);
+  reinterpret_cast<uint4*>(out)[idx] = x;
+}
+
 template <typename T>
 __global__ void debug_projection_kernel(ProjectionParams pp, T* P) {
   const int groups = (pp.r + 3) / 4;

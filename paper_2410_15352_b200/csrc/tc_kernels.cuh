@@ -80,29 +80,6 @@ enum EpiMode { EPI_BF16 = 0, EPI_F32 = 1, EPI_UPDATE_W = 2, EPI_BF16_T = 3 };
 enum GenRing { GEN_NONE = 0, GEN_A = 1 };
 
 constexpr unsigned int STATUS_TIMEOUT = 1u;
-#if defined(COMPACT_PROFILE) || defined(COMPACT_PROFILE_GEN)
-__device__ unsigned long long g_prof[8];
-#endif
-#ifdef COMPACT_PROFILE_GEN
-// event trace of CTA 0, first item, k-steps 16..23
-__device__ long long g_trace[8][16];
-__device__ long long g_tl[64][2];      // start and end (globaltimer) of the last 64 launches, by CTA 0
-__device__ unsigned int g_tl_n;
-#define TRACE(first_item, ks, ev)                                                              \
-  do {                                                                                         \
-    if (blockIdx.x == 0 && (first_item) && (ks) >= 16 && (ks) < 24 && (threadIdx.x & 31) == 0) \
-      g_trace[(ks) - 16][ev] = clock64();                                                      \
-  } while (0)
-#else
-#define TRACE(first_item, ks, ev) ((void)0)
-#endif
-#ifdef COMPACT_PROFILE
-#define PROF_T() clock64()
-#define PROF_ADD(i, t0) prof[i] += clock64() - (t0)
-#else
-#define PROF_T() 0
-#define PROF_ADD(i, t0) ((void)(t0))
-#endif
 
 // One GEMM inside a launch.  An item is nsub row blocks (sharing each B tile) by ncol column
 // blocks of bn columns (sharing each A tile; ncol > 1 only with nsub == 1); its accumulators sit
@@ -149,7 +126,6 @@ struct alignas(64) Params {
   int share_n;            // 0: the cs items of a group are neighbours along M, 1: along N
   int gen_groups;         // groups of cs generated items; handed out statically, cluster by cluster
   int dyn_begin;          // first item handed out dynamically (0 when cs == 1)
-  int debug_flags;        // profiling builds only: bit 0 = issue no MMAs (measures the load path alone)
   PhiloxKey key;          // round keys of the seed shared by the launch's generated problems
   unsigned int* status;
   unsigned int* sched;
@@ -418,12 +394,6 @@ __device__ __forceinline__ TileCoord decode_tile(const Params& prm, int tile) {
 template <bool kGroup>
 __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __grid_constant__ Params prm) {
   extern __shared__ uint8_t smem_raw[];
-#ifdef COMPACT_PROFILE_GEN
-  auto gtime = []() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return (long long)t; };
-  if (threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == 147)) g_trace[6][blockIdx.x == 0 ? 0 : 8] = gtime();
-  __shared__ unsigned int tl_slot;
-  if (threadIdx.x == 0 && blockIdx.x == 0) { tl_slot = atomicAdd(&g_tl_n, 1u) & 63u; g_tl[tl_slot][0] = gtime(); }
-#endif
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));   // generic pointer to the aligned base
   const uint32_t staging = smem_base + RING_BYTES;
@@ -481,9 +451,6 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
   __syncthreads();
   tc_fence_after();
   if (cs > 1) cluster_sync_all();          // every CTA's barriers exist before anything crosses CTAs
-#ifdef COMPACT_PROFILE_GEN
-  if (threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == 147)) g_trace[6][blockIdx.x == 0 ? 1 : 9] = gtime();
-#endif
   const uint32_t tmem_base = *tmem_slot;
 
   // Every consumer role reads the next item from the queue the scheduler fills.
@@ -525,7 +492,6 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       Ring r0 = {0, 0u}, r1 = {0, 0u};     // position in each geometry's ring
       int cur_geo = -1;
       bool ok = true;
-      int first_tile = -2;
       int group = (int)(blockIdx.x / cs);  // static part: cluster c takes groups c, c + clusters, ...
       const int group_step = (int)(gridDim.x / cs);
       while (ok) {
@@ -562,7 +528,6 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         __syncwarp();
         if (++qs == QDEPTH) { qs = 0; qph ^= 1; }
         if (tile < 0) break;
-        if (first_tile == -2) first_tile = tile;
         const TileCoord t = decode_tile<kGroup>(prm, tile);
         const Problem& p = prm.prob[t.prob];
         const bool a_tma = p.a_mode < GENERATED;
@@ -578,7 +543,6 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
           for (int j = 0; j < t.nst; ++j, ring_next(r, ns)) {
             const int s = r.s;
             if (!(ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(geo, s), r.ph ^ 1u, abort_flag, prm.status)))) break;
-            TRACE(tile == first_tile, ks, 4 + j);
             const bool hb = stage_has_b(p, j);
             const int na = stage_num_a(p, t, j);
             uint32_t tx = 0;
@@ -586,9 +550,6 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             // of a generated tile, the shares of the other CTAs arrive as counted bytes
             if (hb) tx += p.bn * BK * 2;
             if (na > 0) { if (a_tma) tx += na * A_BYTES; else { gen_here = true; tx += (A_BYTES / cs) * (cs - 1); } }
-#if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
-            if (prm.debug_flags & 2) tx = 0;
-#endif
             if (elect_one()) {
               // A stage that holds a generated tile is handed back with commits from each CTA of the
               // cluster, so that no CTA writes its share of the next tile (or counts its bytes) into a
@@ -637,9 +598,6 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         cur_geo = geo;
         Ring r = geo ? r1 : r0;
         bool mine = p.a_mode < GENERATED;
-#if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
-        if (prm.debug_flags & 2) mine = false;
-#endif
         const int klen = t.k_end - t.k_begin;
         if (!mine) ring_skip(r, ns, klen * t.nst);
         for (int ks = t.k_begin; ks < t.k_end && ok && mine; ++ks) {
@@ -688,32 +646,8 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       uint32_t acc_phase = 0;
       bool ok = true;
       const uint16_t cta_mask = (uint16_t)((1u << cs) - 1u);
-#ifdef COMPACT_PROFILE_GEN
-      const long long life0 = clock64();
-      long long qwait = 0, twait = 0, nitems = 0;
-#endif
       while (ok) {
-#ifdef COMPACT_PROFILE_GEN
-        const long long q0c = clock64();
-#endif
         const int tile = __shfl_sync(0xffffffffu, next_tile(true, lane == 0), 0);
-#ifdef COMPACT_PROFILE_GEN
-        qwait += clock64() - q0c;
-        if (tile < 0 && lane == 0 && iss == 0 && !has_gen) {
-          atomicAdd(&g_prof[4], (unsigned long long)(clock64() - life0));
-          atomicAdd(&g_prof[5], (unsigned long long)twait);
-          atomicAdd(&g_prof[6], (unsigned long long)qwait);
-          atomicAdd(&g_prof[7], (unsigned long long)nitems);
-        }
-        if (tile < 0 && lane == 0 && iss == 0 && has_gen) {
-          atomicAdd((unsigned long long*)&g_trace[7][0], (unsigned long long)(clock64() - life0));
-          atomicAdd((unsigned long long*)&g_trace[7][1], (unsigned long long)twait);
-          atomicAdd((unsigned long long*)&g_trace[7][2], (unsigned long long)qwait);
-          atomicAdd((unsigned long long*)&g_trace[7][3], (unsigned long long)nitems);
-        }
-        ++nitems;
-        const long long t0c = clock64();
-#endif
         if (tile < 0) break;
         const TileCoord t = decode_tile<kGroup>(prm, tile);
         const Problem& p = prm.prob[t.prob];
@@ -733,9 +667,6 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
           acc_phase ^= 1;
         }
         const int acc0 = acc;
-#ifdef COMPACT_PROFILE_GEN
-        long long mwait = 0, missue = 0;
-#endif
         for (int sl = 0; sl < slots && ok; ++sl) {
           // a split item's issuer x waits for slot x only; an issuer without work in the item waits all the
           // same, so that it never runs more than a phase ahead of these barriers (a parity wait is only
@@ -746,10 +677,6 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         }
         if (!ok) break;
         tc_fence_after();
-#ifdef COMPACT_PROFILE_GEN
-        const long long m1c = clock64();
-        twait += m1c - t0c;
-#endif
         const uint32_t d_base = tmem_base + acc0 * BN_MAX;
         // one UMMA consumes K = 16: 32 bytes along a K-major row, or two 8-row groups (2048 bytes) MN-major
         const uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4), b_step = b_mn ? (2048u >> 4) : (32u >> 4);
@@ -775,9 +702,6 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const uint32_t stage_step = (uint32_t)(geo ? STAGE1_BYTES : STAGE0_BYTES) >> 4;
         const uint32_t ring_lo = (smem_base >> 4) & 0x3FFFu;
         auto issue4 = [&](uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t first) {
-#if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
-          if (prm.debug_flags & 1) return;
-#endif
           umma_bf16(d, a_lo, DESC_HI, b_lo, DESC_HI, idesc, first);
           umma_bf16(d, a_lo + a_step, DESC_HI, b_lo + b_step, DESC_HI, idesc, 1u);
           umma_bf16(d, a_lo + 2 * a_step, DESC_HI, b_lo + 2 * b_step, DESC_HI, idesc, 1u);
@@ -795,19 +719,9 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             const int s = r.s;
             // split by columns: issuer 0 needs the first stage only, issuer 1 both
             if (split && by_col && iss == 0 && j == 1) continue;
-#ifdef COMPACT_PROFILE_GEN
-            const long long w0c = clock64();
-#endif
             if (!(ok = __all_sync(0xffffffffu, mbar_wait(full_bar(geo, s), r.ph, abort_flag, prm.status)))) break;
-#ifdef COMPACT_PROFILE_GEN
-            mwait += clock64() - w0c;
-#endif
-            TRACE(nitems == 1, ks, iss == 0 ? 6 : 8 + j);
             if (split && by_col && iss == 1 && j == 0) continue;
             tc_fence_after();
-#ifdef COMPACT_PROFILE_GEN
-            const long long i0c = clock64();
-#endif
             const uint32_t base = ring_lo + (uint32_t)s * stage_step;
             if (elect_one()) {
               if (by_col) {
@@ -824,29 +738,10 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
               if (j == nst - 1 || (split && by_col && iss == 0)) commit_stage(s0);
             }
             __syncwarp();
-            TRACE(nitems == 1, ks, iss == 0 ? 7 : 10);
-#ifdef COMPACT_PROFILE_GEN
-            missue += clock64() - i0c;
-#endif
           }
         }
         if (!ok) break;
         if (geo) r1 = r; else r0 = r;
-#ifdef COMPACT_PROFILE_GEN
-        if (lane == 0 && iss == 0) {
-          if (p.a_mode >= GENERATED) {
-            atomicAdd(&g_prof[4], (unsigned long long)mwait);                 // waiting for full stages
-            atomicAdd(&g_prof[5], (unsigned long long)missue);               // issuing MMAs and commits
-            atomicAdd(&g_prof[6], (unsigned long long)(clock64() - m1c));    // whole k loop
-            atomicAdd(&g_prof[7], (unsigned long long)(t.k_end - t.k_begin));
-          } else if (!has_gen) {
-            atomicAdd(&g_prof[0], (unsigned long long)mwait);
-            atomicAdd(&g_prof[1], (unsigned long long)missue);
-            atomicAdd(&g_prof[2], (unsigned long long)(clock64() - m1c));
-            atomicAdd(&g_prof[3], (unsigned long long)(t.k_end - t.k_begin));
-          }
-        }
-#endif
         if (elect_one()) {
           if (split) umma_commit(tfull_bar((acc0 + iss) & 1));
           else
@@ -893,9 +788,6 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         if (!(ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, prm.status))) break;
         tc_fence_after();
         bool mine_slot = slots == 2 ? (sl == eset) : true;
-#if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
-        if (prm.debug_flags & 4) mine_slot = false;       // write nothing: hand the accumulators straight back
-#endif
         for (int su = 0; su < sub_per_slot && ok && mine_slot; ++su) {
           const int ai = sl * sub_per_slot + su;            // accumulator of the item: a row block or a column block
           const int mi = p.ncol > 1 ? 0 : ai, cb = p.ncol > 1 ? ai : 0;
@@ -931,9 +823,6 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
 #pragma unroll
               for (int j = 0; j < 8; ++j)
                 *reinterpret_cast<uint4*>(stg_gen + lane * 128 + ((j ^ sw) << 4)) = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
-#if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
-              if (prm.debug_flags & 8) continue;
-#endif
               fence_proxy_async_smem();
               __syncwarp();
               if (lane == 0) {
@@ -964,12 +853,6 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
               uint32_t v[32];
-#if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
-              if (prm.debug_flags & 16) {
-#pragma unroll
-                for (int z = 0; z < 32; ++z) v[z] = 0;
-              } else
-#endif
               {
                 tmem_ld32(tcol + ci * cw + 32 * h, v);
                 tmem_ld_wait();
@@ -984,9 +867,6 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
               }
             }
             if (!ok) break;
-#if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
-            if (prm.debug_flags & 8) continue;
-#endif
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) {
@@ -1010,10 +890,6 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
     // of the first stage of a k-step (forward) or as its A tile 0 (update).
     const int gtid = threadIdx.x - THREADS_BASE;
     constexpr int GSTRIDE = 32 * NUM_GEN_WARPS;
-    int first_tile = -2;
-#ifdef COMPACT_PROFILE_GEN
-    long long pg_wait = 0, pg_gen = 0, pg_arr = 0, pg_cnt = 0;
-#endif
     Ring r0 = {0, 0u}, r1 = {0, 0u};
     bool ok = true;
     const int csh = cs - 1;                                 // log2(cs), cs is 1 or 2
@@ -1026,7 +902,6 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       const TileCoord t = decode_tile<kGroup>(prm, tile);
       const Problem& p = prm.prob[t.prob];
       const int klen = t.k_end - t.k_begin;
-      if (first_tile == -2) first_tile = tile;
       const bool gen_a = p.a_mode == GENERATED, gen_at = p.a_mode == GENERATED_T;
       const int geo = p.geo, ns = geo ? NS1 : NS0;
       Ring r = geo ? r1 : r0;
@@ -1064,14 +939,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         if (t.nst > 1) ring_next(r, ns);            // a k-step takes one or two stages
         const uint32_t stage_off = (uint32_t)s * (geo ? STAGE1_BYTES : STAGE0_BYTES);
         const uint32_t full_off = full_bar(geo, s) - bars;
-#ifdef COMPACT_PROFILE_GEN
-        const long long g0 = clock64();
-#endif
         const bool w = mbar_wait(empty_bar(geo, s), eph, abort_flag, prm.status);
-#ifdef COMPACT_PROFILE_GEN
-        const long long g1 = clock64();
-#endif
-        if (warp == (THREADS_BASE >> 5)) TRACE(tile == first_tile, ks, 0);
         const int k0 = ks * BK;
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
@@ -1083,39 +951,17 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             if (cs > 1) st_async_16(peer_base + off, val, peer_full + full_off);
           }
         }
-#ifdef COMPACT_PROFILE_GEN
-        const long long g2 = clock64();
-#endif
-        if (warp == (THREADS_BASE >> 5)) TRACE(tile == first_tile, ks, 1);
-        if (warp == (THREADS_BASE >> 5) + NUM_GEN_WARPS - 1) TRACE(tile == first_tile, ks, 3);
         fence_proxy_async_smem();
         ok = __all_sync(0xffffffffu, w);
         if (ok && lane == 0) mbar_arrive(full_bar(geo, s));
-        if (warp == (THREADS_BASE >> 5)) TRACE(tile == first_tile, ks, 2);
-#ifdef COMPACT_PROFILE_GEN
-        pg_wait += g1 - g0; pg_gen += g2 - g1; pg_arr += clock64() - g2; pg_cnt += 1;
-#endif
         // later stages of the k-step hold no generated data: the stage owner arrives for the generators there
       }
       if (geo) r1 = r; else r0 = r;
     }
-#ifdef COMPACT_PROFILE_GEN
-    if (warp == (THREADS_BASE >> 5) && lane == 0) {
-      atomicAdd(&g_prof[0], (unsigned long long)pg_wait); atomicAdd(&g_prof[1], (unsigned long long)pg_gen);
-      atomicAdd(&g_prof[2], (unsigned long long)pg_arr); atomicAdd(&g_prof[3], (unsigned long long)pg_cnt);
-    }
-#endif
   }
 
-#ifdef COMPACT_PROFILE_GEN
-  if (threadIdx.x == 32 && (blockIdx.x == 0 || blockIdx.x == 147)) g_trace[6][blockIdx.x == 0 ? 2 : 10] = gtime();
-#endif
   tc_fence_before();
   __syncthreads();
-#ifdef COMPACT_PROFILE_GEN
-  if (threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == 147)) g_trace[6][blockIdx.x == 0 ? 3 : 11] = gtime();
-  if (threadIdx.x == 0 && blockIdx.x == 0) g_tl[tl_slot][1] = gtime();
-#endif
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, 512);
@@ -1189,18 +1035,16 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 inline EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
+  // initialised exactly once, also when several threads make their first launch together
+  static const EncodeTiledFn fn = []() -> EncodeTiledFn {
     void* p = nullptr;
     cudaDriverEntryPointQueryResult q;
     if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &p, 12000, cudaEnableDefault, &q) == cudaSuccess &&
         q == cudaDriverEntryPointSuccess)
-      fn = (EncodeTiledFn)p;
-    else
-      cudaGetLastError();
-  }
+      return (EncodeTiledFn)p;
+    cudaGetLastError();
+    return nullptr;
+  }();
   return fn;
 }
 
@@ -1353,9 +1197,6 @@ inline compact_status_t launch(const LaunchInfo& li, Params& prm) {
   prm.total_tiles = t;
   prm.status = li.status;
   prm.sched = li.sched;
-#if defined(COMPACT_PROFILE) || defined(COMPACT_DEBUG_FLAGS)
-  prm.debug_flags = (getenv("COMPACT_SKIP_MMA") ? 1 : 0) | (getenv("COMPACT_SKIP_LOADS") ? 2 : 0) | (getenv("COMPACT_SKIP_EPI") ? 4 : 0) | (getenv("COMPACT_SKIP_STORE") ? 8 : 0) | (getenv("COMPACT_SKIP_TMEMLD") ? 16 : 0);
-#endif
   const int grid = t < NUM_SMS ? (t + cs - 1) / cs * cs : NUM_SMS / cs * cs;
   const int threads = prm.gen_ring != GEN_NONE ? THREADS_GEN : THREADS_BASE;
   cudaLaunchConfig_t cfg;

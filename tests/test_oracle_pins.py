@@ -407,3 +407,38 @@ def test_saved_activation_accounting():
     comp = 3 * co.saved_elements(bl, n // 4) + 2 * co.saved_elements(bl, n // 4) + co.saved_elements(bl, m // 4)
     assert comp / dense == pytest.approx(1964 / 4784)
     assert 7.0 * comp / dense == pytest.approx(2.87, abs=0.005)   # Table 3 activation row at r = n/4
+
+
+# --- The yardstick itself: relative Frobenius error, whole tensors and tiles -------------
+def test_rel_frobenius_hand_values():
+    b = np.array([[3.0, 0.0], [0.0, 4.0]])                      # ||b|| = 5
+    a = b + np.array([[0.0, 0.3], [0.4, 0.0]])                  # ||a - b|| = 0.5
+    assert co.rel_frobenius(a, b) == pytest.approx(0.1, rel=1e-12)
+    assert co.rel_frobenius(b, b) == 0.0
+    assert co.rel_frobenius(2 * b, b) == pytest.approx(1.0)     # not symmetric: measured against the second argument
+    assert co.rel_frobenius(b, 2 * b) == pytest.approx(0.5)
+    # zero oracle tensor: the absolute norm of the difference
+    assert co.rel_frobenius(np.array([3.0, 4.0]), np.zeros(2)) == pytest.approx(5.0)
+    assert co.rel_frobenius(np.zeros((2, 3)), np.zeros((2, 3))) == 0.0
+    # a 1-D sum written out
+    x, y = np.array([1.0, 2.0, 2.0]), np.array([2.0, 2.0, 1.0])
+    assert co.rel_frobenius(x, y) == pytest.approx(math.sqrt(2.0) / 3.0)
+
+
+def test_tile_metric_hand_values():
+    from tests._harness import tile_sq_norms, worst_tile
+    a = np.arange(12, dtype=np.float64).reshape(3, 4)            # tiles of 2 x 3: ragged on both edges
+    want = np.array([[0 + 1 + 4 + 16 + 25 + 36, 9 + 49], [64 + 81 + 100, 121]], dtype=np.float64)
+    assert np.array_equal(tile_sq_norms(a, 2, 3), want)
+    b = np.ones((4, 4))
+    e = np.zeros((4, 4))
+    e[3, 3] = 0.2                                                # one wrong entry in the last 2 x 2 tile
+    assert worst_tile(b + e, b, (2, 2)) == pytest.approx(0.1)    # 0.2 / ||ones(2,2)||
+    assert co.rel_frobenius(b + e, b) == pytest.approx(0.05)     # the whole-tensor figure blurs it
+    assert worst_tile(b, b, (2, 2)) == 0.0
+    # a wrong tile of a large tensor passes the whole-tensor bound and fails the tile bound
+    rng = np.random.default_rng(0)
+    big = rng.standard_normal((1024, 512))
+    bad = big.copy()
+    bad[128:256, 64:128] = 0.0
+    assert co.rel_frobenius(bad, big) < 0.2 and worst_tile(bad, big, (128, 64)) == pytest.approx(1.0)

@@ -12,7 +12,7 @@ from oracle import compact_oracle as co
 from paper_2410_15352_b200 import binding as cb
 from paper_2410_15352_b200 import workloads as wlm
 from paper_2410_15352_b200.build import build_library
-from tests._harness import TOL, f32, make_pair, run_layer_trajectory, to64
+from tests._harness import TILE, TOL, assert_parity, f32, make_pair, run_layer_trajectory, to64, worst_tile
 
 pytestmark = pytest.mark.gpu
 
@@ -39,14 +39,17 @@ def family(request):
     (0, 0, 0, 128, 16), ((5 << 32) | 0xDEADBEEF, 6, 3, 300, 342), (2 ** 64 - 1, 0xFFFFFFFF, 0xFFFFFFFF, 64, 7),
     (1, 2, 1, 1376, 344)])
 def test_philox_words_bit_exact(seed, layer, epoch, n, r):
-    got = cb.debug_philox_u32(seed, layer, epoch, n, r).cpu().numpy().view(np.uint32)
     want = co.projection_words(seed, layer, epoch, n, r)
-    assert got.shape == want.shape and np.array_equal(got, want)
+    # both device forms of the function: the generic ten rounds, and the one the GEMM kernels' generators call
+    for layer_form in (False, True):
+        got = cb.debug_philox_u32(seed, layer, epoch, n, r, layer_form=layer_form).cpu().numpy().view(np.uint32)
+        assert got.shape == want.shape and np.array_equal(got, want), layer_form
 
 
 def test_philox_known_answer_on_device():
-    got = cb.debug_philox_u32(0, 0, 0, 1, 4).cpu().numpy().view(np.uint32)[0]
-    assert [int(x) for x in got] == [0x6627E8D5, 0xE169C58D, 0xBC57AC4C, 0x9B00DBD8]
+    for layer_form in (False, True):
+        got = cb.debug_philox_u32(0, 0, 0, 1, 4, layer_form=layer_form).cpu().numpy().view(np.uint32)[0]
+        assert [int(x) for x in got] == [0x6627E8D5, 0xE169C58D, 0xBC57AC4C, 0x9B00DBD8]
 
 
 def test_projection_fp32_entries():
@@ -75,11 +78,9 @@ def test_projection_bf16_entries():
 # ---- config 1: fp32, full trajectory with refresh -------------------------------------
 def test_config1_fp32_trajectory():
     wl = wlm.config1()
-    errs, epochs, dW = run_layer_trajectory(wl, 0, wl.steps)
+    errs, epochs, dW, dW_tile = run_layer_trajectory(wl, 0, wl.steps)
     assert epochs == [0, 0, 1]
-    for k, v in errs.items():
-        assert v <= TOL["f32"], (k, v)
-    assert dW <= 1e-4
+    assert_parity(errs, dW, dW_tile, "f32")
 
 
 # ---- small bf16 shapes spanning tiles and ragged tails, both kernel families ------------
@@ -103,19 +104,44 @@ SMALL = [
 def test_small_bf16_trajectory(family, tokens, n, m, r):
     wl = wlm.Workload("small", 90, "bf16", tokens, [wlm.LayerShape("l", n, m, r)], steps=3, refresh_T=2,
                       x_scale_inv_sqrt_n=True)
-    errs, epochs, dW = run_layer_trajectory(wl, 0, 3)
+    errs, epochs, dW, dW_tile = run_layer_trajectory(wl, 0, 3)
     assert epochs == [0, 0, 1]
-    for k, v in errs.items():
-        assert v <= TOL["bf16"], (k, v)
+    assert_parity(errs, dW, dW_tile, "bf16")
 
 
 @pytest.mark.parametrize("tokens,n,m,r", [(96, 64, 40, 12), (257, 132, 260, 33)])
 def test_small_fp32_ragged(tokens, n, m, r):
     wl = wlm.Workload("small32", 91, "f32", tokens, [wlm.LayerShape("l", n, m, r)], steps=2, refresh_T=1)
-    errs, epochs, _ = run_layer_trajectory(wl, 0, 2)
+    errs, epochs, dW, dW_tile = run_layer_trajectory(wl, 0, 2)
     assert epochs == [0, 1]
-    for k, v in errs.items():
-        assert v <= TOL["f32"], (k, v)
+    assert_parity(errs, dW, dW_tile, "f32")
+
+
+# ---- the scale alpha and a per-call learning rate (Algorithm 3 line 8; Section 3.2's optional constant) ------
+@pytest.mark.parametrize("dtype,tokens,n,m,r", [("bf16", 700, 320, 1096, 72), ("f32", 200, 96, 136, 20)])
+def test_alpha_and_per_call_learning_rate(family, dtype, tokens, n, m, r):
+    if dtype == "f32" and family != 0:
+        pytest.skip("fp32 layers have one kernel family")
+    # alpha = 0.25 as in the paper's pre-training runs, and a learning rate per call that differs from the
+    # layer configuration's (which a schedule outside the layer would do)
+    wl = wlm.Workload("alpha", 89, dtype, tokens, [wlm.LayerShape("l", n, m, r)], steps=4, refresh_T=3, lr=1e-3,
+                      alpha=0.25, x_scale_inv_sqrt_n=True)
+    errs, epochs, dW, dW_tile = run_layer_trajectory(wl, 0, 4, lr_call=7e-3)
+    assert epochs == [0, 0, 0, 1]
+    assert_parity(errs, dW, dW_tile, dtype)
+    # the per-call rate is what scales the step: with the same Gc the first update moves W seven times as far
+    # as one made with the configuration's rate
+    gpu, _, W0 = make_pair(wl, 0)
+    X, dY = wlm.draw_X(wl, 0, 0).cuda(), wlm.draw_dY(wl, 0, 0).cuda()
+    Wa, Wb = W0.cuda(), W0.cuda()
+    _, Z, ep = gpu.forward(X, Wa)
+    _, Gc = gpu.backward(dY, Z, Wa, need_dX=False)
+    gpu.adam_update(Wa, Gc, torch.zeros_like(Gc), torch.zeros_like(Gc), ep, lr=7e-3)
+    st = gpu.state()
+    gpu.set_state(st.seed, st.layer_id, st.epoch, 0)
+    gpu.adam_update(Wb, Gc, torch.zeros_like(Gc), torch.zeros_like(Gc), ep)
+    da, db = to64(Wa) - to64(W0), to64(Wb) - to64(W0)
+    assert abs(np.linalg.norm(da) / np.linalg.norm(db) - 7.0) < (0.35 if dtype == "bf16" else 1e-3)
 
 
 # ---- Z token indexing: bit-exact ----------------------------------------------------------
@@ -392,3 +418,37 @@ def test_checkpoint_resume_bitwise():
     run(c, Wc, Mc, Vc, 2, 5)
     assert torch.equal(Wa.view(torch.int16), Wc.view(torch.int16)) and torch.equal(Ma, Mc) and torch.equal(Va, Vc)
     assert a.epoch == c.epoch == 2
+
+
+def test_many_layers_on_two_streams_match_one_stream():
+    # Launches that overlap on the GPU -- other layers, other streams -- have scheduler words of their own,
+    # and every live layer a status word of its own: 300 layers stepped alternately on two streams give
+    # the bits of the same calls made one after the other on one stream.
+    tokens, n, m, r = 700, 192, 328, 40
+    wl = wlm.Workload("many", 88, "bf16", tokens, [wlm.LayerShape("l", n, m, r)], x_scale_inv_sqrt_n=True)
+    X, dY = wlm.draw_X(wl, 0, 0).cuda(), wlm.draw_dY(wl, 0, 0).cuda()
+    W = wlm.draw_W(wl, 0).cuda()
+    layers = [cb.CompactLinear(n, m, r, seed=7, layer_id=i % 5) for i in range(300)]
+    ref = {}
+    for i in range(5):
+        Y, Z, _ = layers[i].forward(X, W)
+        dX, Gc = layers[i].backward(dY, Z, W)
+        ref[i] = (Y, Z, dX, Gc)
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    outs = []
+    for i, lay in enumerate(layers):
+        st = streams[i % 2]
+        with torch.cuda.stream(st):
+            ws = torch.empty(max(lay.workspace_bytes(tokens), 256), dtype=torch.uint8, device="cuda")
+            lay._ws = ws                                  # a workspace per layer: the two streams share none
+            Y, Z, _ = lay.forward(X, W, stream=st)
+            dX, Gc = lay.backward(dY, Z, W, stream=st)
+        outs.append((Y, Z, dX, Gc))
+    torch.cuda.synchronize()
+    for i, (Y, Z, dX, Gc) in enumerate(outs):
+        Yr, Zr, dXr, Gcr = ref[i % 5]
+        assert torch.equal(Y.view(torch.int16), Yr.view(torch.int16)) and torch.equal(Z.view(torch.int16), Zr.view(torch.int16)), i
+        assert torch.equal(dX.view(torch.int16), dXr.view(torch.int16)) and torch.equal(Gc, Gcr), i
+    assert all(lay.status() == cb.OK for lay in layers[:8])
+    assert len({lay._h.value for lay in layers}) == 300

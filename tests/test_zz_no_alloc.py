@@ -45,8 +45,14 @@ def test_noalloc_update_matches_regular_update_twice(dtype, tokens, n, m, r):
         _, Z, ep = a.forward(X, Wa)
         _, Gc = a.backward(dY, Z, Wa, need_dX=False)
         a.adam_update(Wa, Gc, Ma, Va, ep)                       # regular entry point, caller's workspace
+        torch.cuda.synchronize()
+        free0, held0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
         b.adam_update_noalloc(Wb, Gc, Mb, Vb, ep)               # same step from the built-in scratch
         torch.cuda.synchronize()
+        if step == 1:
+            # once the library's device code is resident (the first call saw to that), a call leaves the
+            # device's free memory and torch's pool exactly as it found them
+            assert torch.cuda.mem_get_info()[0] == free0 and torch.cuda.memory_allocated() == held0
         for name, x, y in (("W", Wa, Wb), ("M", Ma, Mb), ("V", Va, Vb)):
             assert co.rel_frobenius(to64(y), to64(x)) <= TOL[dtype], (step, name)
             assert torch.equal(x, y), (step, name)              # same kernels, same inputs: identical bits
