@@ -14,6 +14,7 @@
 #include "philox.cuh"
 #include "simt_kernels.cuh"
 #include "tc_kernels.cuh"
+#include "update_kernel.cuh"
 
 using namespace compact;
 
@@ -38,12 +39,12 @@ std::atomic<int> g_family{0};
 // Slots come from a free list and go back on destroy; when none is left, compact_layer_create fails.
 constexpr int kStatusSlots = 4096;
 __device__ unsigned int g_status_words[kStatusSlots];
-// Two words per tensor-core launch for its dynamic item scheduler (next item, finished CTAs), taken from a
+// Four words per tensor-core launch for its dynamic schedulers (next item, finished CTAs, ...), taken from a
 // ring by launch sequence number, so that launches that overlap on the GPU (other layers, other streams)
-// never share them.  Zero at load; the last CTA of a launch leaves its pair zero again.  The ring is far
+// never share them.  Zero at load; the last CTA of a launch leaves them zero again.  The ring is far
 // longer than the number of launches that can be in flight at once.
 constexpr int kSchedRing = 4096;
-__device__ unsigned int g_sched_words[kSchedRing][2];
+__device__ unsigned int g_sched_words[kSchedRing][4];
 std::atomic<uint64_t> g_sched_seq{0};
 
 std::mutex g_slot_mutex;
@@ -115,7 +116,7 @@ unsigned int* status_word(const compact_layer_t* L) {
 // The scheduler words of the next tensor-core launch.
 unsigned int* sched_words(const compact_layer_t*) {
   unsigned int* base = symbol_base(g_sched_base, g_sched_words);
-  return base ? base + 2 * (g_sched_seq.fetch_add(1) % kSchedRing) : nullptr;
+  return base ? base + 4 * (g_sched_seq.fetch_add(1) % kSchedRing) : nullptr;
 }
 
 ProjectionParams make_pp(const compact_layer_t* L, uint32_t epoch) {
@@ -532,8 +533,14 @@ compact_status_t compact_adam_update(compact_layer_t* L, void* W, int64_t ldw, c
     s = COMPACT_ERR_SHAPE;
     if (g_family.load() != 1) {
       tc::LaunchInfo li{g_family.load() == 2 ? 1 : CFG_CS, st, status_word(L), sched_words(L), &g_launches};
-      s = tc::update(li, make_pp(L, L->epoch), adam_scalars(L, L->step + 1), L->cfg.n, L->cfg.m, L->cfg.r, (T*)W, ldw,
-                     Gc, ldg, M, V, lr * L->cfg.alpha, workspace, workspace_bytes);
+      // one launch (Adam, resident panel of P, sweep over W) where the rank fits the panel; otherwise the Adam
+      // kernel followed by the streaming GEMM
+      if (g_family.load() == 0 && upd::fused_update_ok(L->cfg.n, L->cfg.m, L->cfg.r))
+        s = upd::fused_update(li, make_pp(L, L->epoch), adam_scalars(L, L->step + 1), L->cfg.n, L->cfg.m, L->cfg.r, (T*)W, ldw,
+                              Gc, ldg, M, V, lr * L->cfg.alpha, workspace, workspace_bytes);
+      else
+        s = tc::update(li, make_pp(L, L->epoch), adam_scalars(L, L->step + 1), L->cfg.n, L->cfg.m, L->cfg.r, (T*)W, ldw,
+                       Gc, ldg, M, V, lr * L->cfg.alpha, workspace, workspace_bytes);
     }
     if (s == COMPACT_ERR_SHAPE) s = update_simt<T>(L, (T*)W, ldw, Gc, ldg, M, V, lr, (float*)workspace, st);
   } else {

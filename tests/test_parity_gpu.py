@@ -452,3 +452,31 @@ def test_many_layers_on_two_streams_match_one_stream():
         assert torch.equal(dX.view(torch.int16), dXr.view(torch.int16)) and torch.equal(Gc, Gcr), i
     assert all(lay.status() == cb.OK for lay in layers[:8])
     assert len({lay._h.value for lay in layers}) == 300
+
+
+@pytest.mark.parametrize("n,m,r", [
+    (4096, 4096, 512),        # the LLaMA-7B attention shape: 64 jobs, two column ranges per row panel
+    (1000, 1344, 200),        # ragged last row panel, a ragged last column block, rank short of a k-tile
+    (9736, 128, 24),          # more row panels than clusters: a cluster generates a second panel
+    (128, 64, 8),             # one panel, one block: the neighbour CTA has no block of its own
+    (640, 2752, 512),         # full panel, eleven column blocks over several ranges
+])
+def test_one_launch_update_equals_two_kernel_update_bitwise(n, m, r):
+    # The update that keeps a panel of P resident (one launch: Adam, barrier, sweep) and the update made of the
+    # Adam kernel followed by the streaming GEMM produce N, the products and the roundings in the same order.
+    g = torch.Generator().manual_seed(n + m + r)
+    Gc = (torch.randn((r, m), generator=g) * 1e-3).cuda()
+    W0 = (torch.randn((n, m), generator=g) * 0.02).to(torch.bfloat16).cuda()
+    out = []
+    for fam in (0, 2):
+        cb.set_kernel_family(fam)
+        lay = cb.CompactLinear(n, m, r, seed=11, layer_id=3, lr=2e-3, alpha=0.5)
+        W, M, V = W0.clone(), torch.full((r, m), 1e-4, device="cuda"), torch.full((r, m), 1e-7, device="cuda")
+        for _ in range(2):
+            lay.adam_update(W, Gc, M, V, 0)
+        assert lay.status() == cb.OK
+        out.append((W, M, V))
+    cb.set_kernel_family(0)
+    assert torch.equal(out[0][0].view(torch.int16), out[1][0].view(torch.int16))
+    assert torch.equal(out[0][1], out[1][1]) and torch.equal(out[0][2], out[1][2])
+    assert not torch.equal(out[0][0].view(torch.int16), W0.view(torch.int16))
