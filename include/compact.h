@@ -14,7 +14,8 @@
  *   - Matrices are row-major with an explicit leading dimension in ELEMENTS.
  *     W is n x m as in the paper's Section 3.1 (not [out, in]).
  *   - All tensor pointers are DEVICE pointers owned by the caller.  The library
- *     allocates no tensor memory and keeps no pointer after a call returns.
+ *     allocates no tensor memory and dereferences no pointer after a call returns
+ *     (it remembers encoded TMA descriptors by pointer, shape and pitch: values only).
  *   - Element type of X, W, Y, dY, dX, Z is the layer's dtype; Gc, M, V are
  *     always fp32.
  *   - `stream` is a cudaStream_t passed as void*.  Compute calls are asynchronous
@@ -23,7 +24,9 @@
  *     the element size a multiple of 16 bytes.
  *   - Every function returns a compact_status_t; nothing throws or aborts.
  *     Argument checks happen on the host before any launch.
- *   - A layer handle must not be used from two threads at once.
+ *   - A layer handle must not be used from two threads at once.  Calls on one layer
+ *     may go to different streams; workspaces and outputs of calls that can overlap
+ *     on the GPU must then be distinct.
  *   - Only compute capability 10.x devices are supported; there is no fallback.
  */
 #ifndef COMPACT_H_
@@ -224,6 +227,13 @@ compact_status_t compact_layer_set_state(compact_layer_t* layer, const compact_l
  * Returns DEVICE_TIMEOUT if a kernel gave up on a bounded wait since the last
  * call, OK otherwise. */
 compact_status_t compact_layer_status(compact_layer_t* layer);
+
+/* Test hook for the bounded waits (the paper has no counterpart): launches one small
+ * CTA that waits, with a limit of a few thousand polls, on a barrier nothing arrives
+ * at.  The wait gives up, sets the layer's status word and the kernel returns, exactly
+ * as every wait inside the GEMM kernels would; compact_layer_status then reports
+ * COMPACT_ERR_DEVICE_TIMEOUT once, and the context stays usable. */
+compact_status_t compact_debug_wait_that_runs_out(compact_layer_t* layer, void* stream);
 
 /* Test hooks that make the in-kernel generator observable.
  * compact_debug_philox_u32: out_dev[n x 4*ceil(r/4)] receives the raw Philox

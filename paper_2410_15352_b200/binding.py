@@ -30,7 +30,7 @@ EXPORTS = [
     "compact_linear_bwd_recompute", "compact_group_workspace_bytes", "compact_group_fwd", "compact_group_bwd",
     "compact_adam_update", "compact_adam_update_noalloc",
     "compact_refresh_projection", "compact_layer_get_state", "compact_layer_set_state",
-    "compact_layer_status", "compact_debug_philox_u32", "compact_debug_philox_layer_u32", "compact_debug_projection",
+    "compact_layer_status", "compact_debug_wait_that_runs_out", "compact_debug_philox_u32", "compact_debug_philox_layer_u32", "compact_debug_projection",
     "compact_set_kernel_family", "compact_kernel_launch_count", "compact_status_string",
 ]
 
@@ -85,6 +85,7 @@ def lib() -> C.CDLL:
     L.compact_layer_get_state.argtypes = [vp, C.POINTER(LayerState)]
     L.compact_layer_set_state.argtypes = [vp, C.POINTER(LayerState)]
     L.compact_layer_status.argtypes = [vp]
+    L.compact_debug_wait_that_runs_out.argtypes = [vp, vp]
     L.compact_debug_philox_u32.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_int32, C.c_int32, vp, vp]
     L.compact_debug_philox_layer_u32.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_int32, C.c_int32, vp, vp]
     L.compact_debug_projection.argtypes = [vp, C.c_uint32, vp, vp]
@@ -185,6 +186,10 @@ class CompactLinear:
 
     def status(self) -> int:
         return int(lib().compact_layer_status(self._h))
+
+    def debug_wait_that_runs_out(self, stream=None) -> None:
+        """Launches the test kernel whose bounded wait gives up (sets this layer's status word)."""
+        _check(lib().compact_debug_wait_that_runs_out(self._h, _stream(stream)), "compact_debug_wait_that_runs_out")
 
     def workspace(self, tokens: int) -> torch.Tensor:
         need = max(self.workspace_bytes(tokens), 256)

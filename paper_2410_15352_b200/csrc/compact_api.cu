@@ -640,6 +640,17 @@ compact_status_t compact_layer_status(compact_layer_t* L) {
   return COMPACT_OK;
 }
 
+compact_status_t compact_debug_wait_that_runs_out(compact_layer_t* L, void* stream) {
+  if (!L) return COMPACT_ERR_INVALID_ARG;
+  compact_status_t s = check_device(L, stream);
+  if (s != COMPACT_OK) return s;
+  unsigned int* w = status_word(L);
+  if (!w) return COMPACT_ERR_CUDA;
+  tc::wait_that_runs_out_kernel<<<1, 64, 0, (cudaStream_t)stream>>>(w, 4096u);
+  g_launches++;
+  return launch_result();
+}
+
 compact_status_t compact_debug_philox_u32(uint64_t seed, uint32_t layer_id, uint32_t epoch, int32_t n, int32_t r,
                                           uint32_t* out_dev, void* stream) {
   if (n < 1 || r < 1 || !out_dev) return COMPACT_ERR_INVALID_ARG;

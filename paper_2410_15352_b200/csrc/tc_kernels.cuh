@@ -15,8 +15,10 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <stdlib.h>
+#include <string.h>
 
 #include <atomic>
+#include <unordered_map>
 
 #include "../../include/compact.h"
 #include "philox.cuh"
@@ -163,9 +165,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait: gives up after about a second, records it, and lets the CTA drain.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned int* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned int* status,
+                                          uint32_t limit = 8000000u) {
   if (mbar_try_wait(bar, parity)) return true;
-  for (uint32_t it = 0; it < 8000000u; ++it) {
+  for (uint32_t it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if (it > 128) {
       __nanosleep(100);
@@ -328,6 +331,21 @@ __device__ __forceinline__ uint4 projection8_bf16(const PhiloxKey& key, uint32_t
     b.x = left > 4 ? b.x : 0.f; b.y = left > 5 ? b.y : 0.f; b.z = left > 6 ? b.z : 0.f; b.w = left > 7 ? b.w : 0.f;
   }
   return make_uint4(pack_bf16x2(a.x, a.y), pack_bf16x2(a.z, a.w), pack_bf16x2(b.x, b.y), pack_bf16x2(b.z, b.w));
+}
+
+// Test hook: one CTA waits, with a small limit, on a barrier that nothing will ever arrive at.  The wait gives
+// up, records it in the status word and the kernel returns: the path every bounded wait of the kernels takes
+// when its signal never comes.
+__global__ void wait_that_runs_out_kernel(unsigned int* status, uint32_t limit) {
+  __shared__ __align__(8) unsigned long long bar_mem;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(smem_u32(&bar_mem), 1);
+    fence_barrier_init();
+  }
+  __syncthreads();
+  mbar_wait(smem_u32(&bar_mem), 0u, &abort_flag, status, limit);
 }
 
 // Position in a stage ring: the next stage and the parity of the round it is in.
@@ -1052,19 +1070,57 @@ inline EncodeTiledFn encode_fn() {
   return fn;
 }
 
+// Tensor maps are pure functions of (pointer, extents, pitches, box, element type, swizzle): a layer that is
+// called step after step on the same buffers asks for the same few maps again and again, so each thread keeps
+// the ones it has encoded.
+struct MapKey {
+  uint64_t v[8];
+  bool operator==(const MapKey& o) const { return memcmp(v, o.v, sizeof(v)) == 0; }
+};
+struct MapKeyHash {
+  size_t operator()(const MapKey& k) const {
+    uint64_t h = 0x9E3779B97F4A7C15ull;
+    for (int i = 0; i < 8; ++i) h = (h ^ k.v[i]) * 0xFF51AFD7ED558CCDull + (h >> 29);
+    return (size_t)h;
+  }
+};
+
+inline bool encode_cached(CUtensorMap* map, CUtensorMapDataType type, uint32_t rank, const void* base, const cuuint64_t* dims,
+                          const cuuint64_t* strides, const cuuint32_t* box, CUtensorMapSwizzle swizzle) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  MapKey key;
+  memset(&key, 0, sizeof(key));
+  key.v[0] = (uint64_t)(uintptr_t)base;
+  key.v[1] = (uint64_t)type | ((uint64_t)rank << 8) | ((uint64_t)swizzle << 16);
+  for (uint32_t i = 0; i < rank; ++i) {
+    key.v[2 + i] = dims[i];
+    key.v[7] = key.v[7] * 1031u + box[i];
+  }
+  for (uint32_t i = 0; i + 1 < rank; ++i) key.v[5 + i] = strides[i];
+  thread_local std::unordered_map<MapKey, CUtensorMap, MapKeyHash> cache;
+  auto it = cache.find(key);
+  if (it != cache.end()) {
+    *map = it->second;
+    return true;
+  }
+  cuuint32_t estr[3] = {1, 1, 1};
+  if (fn(map, type, rank, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle,
+         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return false;
+  if (cache.size() >= 8192) cache.clear();
+  cache.emplace(key, *map);
+  return true;
+}
+
 // 2-D bf16 map over a row-major matrix: `inner` contiguous elements per row, `rows` rows, pitch in elements.
 inline bool make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t rows, int64_t pitch, int box_inner,
                      int box_rows, bool swizzle = true) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)pitch * 2};
   cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
-            CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_cached(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box,
+                       swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE);
 }
 
 // MN-major operand tiles: the matrix (rows x cols, cols a multiple of 64) seen as [cols / 64][rows][64], so
@@ -1072,30 +1128,20 @@ inline bool make_map(CUtensorMap* map, const void* base, int64_t inner, int64_t 
 // pieces -- the layout the MMA descriptor of an MN-major operand walks.
 inline bool make_map_blocked(CUtensorMap* map, const void* base, int64_t cols, int64_t rows, int64_t pitch, int box_rows,
                              int blocks) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
   cuuint64_t dims[3] = {64, (cuuint64_t)rows, (cuuint64_t)(cols / 64)};
   cuuint64_t strides[2] = {(cuuint64_t)pitch * 2, 128};
   cuuint32_t box[3] = {64, (cuuint32_t)box_rows, (cuuint32_t)blocks};
-  cuuint32_t estr[3] = {1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_cached(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
 // 3-D fp32 map over `planes` row-major matrices of rows x inner (pitch and plane stride in elements);
 // boxes are 32 columns x 32 rows of one plane.
 inline bool make_map_f32_3d(CUtensorMap* map, const void* base, int64_t inner, int64_t rows, int64_t planes, int64_t pitch,
                             int64_t plane_stride) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
   cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)rows, (cuuint64_t)planes};
   cuuint64_t strides[2] = {(cuuint64_t)pitch * 4, (cuuint64_t)plane_stride * 4};
   cuuint32_t box[3] = {32, 32, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_cached(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
 // Tile width: up to 256 columns, in whole 64-column blocks.

@@ -480,3 +480,23 @@ def test_one_launch_update_equals_two_kernel_update_bitwise(n, m, r):
     assert torch.equal(out[0][0].view(torch.int16), out[1][0].view(torch.int16))
     assert torch.equal(out[0][1], out[1][1]) and torch.equal(out[0][2], out[1][2])
     assert not torch.equal(out[0][0].view(torch.int16), W0.view(torch.int16))
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_context_survives():
+    # every mbarrier wait in the kernels is bounded; here one is made to run out (a barrier nothing arrives at,
+    # a limit of a few thousand polls): the kernel returns, the status word says so once, and work goes on
+    tokens, n, m, r = 300, 128, 192, 24
+    wl = wlm.Workload("tmo", 87, "bf16", tokens, [wlm.LayerShape("l", n, m, r)], x_scale_inv_sqrt_n=True)
+    gpu, ora, W0 = make_pair(wl, 0)
+    other = cb.CompactLinear(n, m, r, seed=1, layer_id=9)
+    X, W = wlm.draw_X(wl, 0, 0).cuda(), W0.cuda()
+    Y0, Z0, _ = gpu.forward(X, W)
+    assert gpu.status() == cb.OK
+    gpu.debug_wait_that_runs_out()
+    assert other.status() == cb.OK                       # another layer's status word is its own
+    assert gpu.status() == cb.ERR_DEVICE_TIMEOUT
+    assert gpu.status() == cb.OK                         # reading cleared it
+    Y1, Z1, _ = gpu.forward(X, W)                        # the context is intact
+    assert torch.equal(Y0.view(torch.int16), Y1.view(torch.int16)) and torch.equal(Z0.view(torch.int16), Z1.view(torch.int16))
+    Yo, Zo = ora.forward(to64(X))
+    assert co.rel_frobenius(to64(Y1), Yo) <= TOL["bf16"] and gpu.status() == cb.OK
