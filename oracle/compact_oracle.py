@@ -24,6 +24,15 @@ Readings of the paper taken here (the paper is silent or inconsistent):
   * The generator behind "set_random_seed(s); P <- N(0,1/r)" is Philox4x32-10
     keyed by the 64-bit seed with counter (j>>2, i, layer, epoch), followed by
     Box-Muller; the seed bump "s <- s+1" is the epoch word.
+  * The sparse Johnson-Lindenstrauss projection of the ablation study is the
+    construction the paper cites there (Dasgupta, Kumar, Sarlos: each input
+    coordinate is hashed s times into the r output coordinates with random
+    signs, scaled by 1/sqrt(s); terms that collide add).  Here term t of row i
+    of P is word t&3 of the Philox call with counter
+    (0x80000000 | t>>2, i, layer, epoch): sign = bit 31, column =
+    ((word & 0x7fffffff) * r) >> 31.  Its entries are multiples of 1/sqrt(s)
+    and are not rounded in bf16 mode (the device keeps the integer counts in
+    its tiles and scales the accumulated sums).
 """
 from __future__ import annotations
 
@@ -100,8 +109,41 @@ def box_muller_from_words(words: np.ndarray) -> np.ndarray:
     return out.reshape(shp)
 
 
-def projection(seed: int, layer_id: int, epoch: int, n: int, r: int, mode: str = "exact") -> np.ndarray:
-    """P (n x r), entries N(0, 1/r): Algorithm 1 lines 1-2, Algorithm 3 lines 6-7."""
+def sparse_jl_terms(seed: int, layer_id: int, epoch: int, n: int, r: int, s: int):
+    """The s hashed terms of every row of a sparse JL projection (Ablation Study, "Sparse
+    Johnson-Lindenstrauss (JL) Projection Matrices"): integer arrays (cols, signs) of shape (n, s)
+    with cols in [0, r) and signs in {+1, -1}.  Term t of row i comes from word t & 3 of the
+    Philox call with counter (0x80000000 | t >> 2, i, layer_id, epoch)."""
+    calls = (s + 3) // 4
+    i = np.arange(n, dtype=np.uint64)[:, None]
+    q = np.arange(calls, dtype=np.uint64)[None, :]
+    ctr = np.empty((n, calls, 4), dtype=np.uint64)
+    ctr[..., 0] = np.uint64(0x80000000) | q
+    ctr[..., 1] = i
+    ctr[..., 2] = np.uint64(layer_id & 0xFFFFFFFF)
+    ctr[..., 3] = np.uint64(epoch & 0xFFFFFFFF)
+    key = np.array([seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF], dtype=np.uint64)
+    words = philox4x32_10(ctr, key).reshape(n, calls * 4)[:, :s].astype(np.uint64)
+    cols = ((words & np.uint64(0x7FFFFFFF)) * np.uint64(r)) >> np.uint64(31)
+    signs = 1 - 2 * (words >> np.uint64(31)).astype(np.int64)
+    return cols.astype(np.int64), signs
+
+
+def projection_sparse_jl(seed: int, layer_id: int, epoch: int, n: int, r: int, s: int) -> np.ndarray:
+    """P (n x r) with P[i, j] = (1/sqrt(s)) * sum over the terms of row i that hash to column j of their signs."""
+    cols, signs = sparse_jl_terms(seed, layer_id, epoch, n, r, s)
+    K = np.zeros((n, r), dtype=np.float64)
+    for i in range(n):
+        for t in range(s):
+            K[i, cols[i, t]] += signs[i, t]
+    return K / math.sqrt(s)
+
+
+def projection(seed: int, layer_id: int, epoch: int, n: int, r: int, mode: str = "exact", sparse_s: int = 0) -> np.ndarray:
+    """P (n x r): Algorithm 1 lines 1-2, Algorithm 3 lines 6-7.  sparse_s == 0: entries N(0, 1/r);
+    sparse_s > 0: the sparse JL projection with sparse_s terms per row."""
+    if sparse_s > 0:
+        return projection_sparse_jl(seed, layer_id, epoch, n, r, sparse_s)
     g = box_muller_from_words(projection_words(seed, layer_id, epoch, n, r))[:, :r]
     P = g / math.sqrt(r)
     return round_bf16(P) if mode == "bf16" else P
@@ -214,7 +256,7 @@ class CompActLayerOracle:
 
     def __init__(self, W0, n: int, m: int, r: int, seed: int, layer_id: int, refresh_T: int,
                  lr: float, beta1: float, beta2: float, eps: float, alpha: float = 1.0,
-                 mode: str = "exact", P_override=None):
+                 mode: str = "exact", P_override=None, sparse_s: int = 0):
         self.n, self.m, self.r = n, m, r
         self.W = np.array(W0, dtype=np.float64)
         self.M = np.zeros((r, m))
@@ -223,12 +265,13 @@ class CompActLayerOracle:
         self.lr, self.beta1, self.beta2, self.eps, self.alpha = lr, beta1, beta2, eps, alpha
         self.mode = mode
         self.P_override = P_override      # explicit P for algebraic pins (orthonormal, identity)
+        self.sparse_s = sparse_s          # > 0: sparse JL projection with this many terms per row
 
     def P(self, epoch: int | None = None) -> np.ndarray:
         if self.P_override is not None:
             return np.asarray(self.P_override, dtype=np.float64)
         ep = self.state.epoch if epoch is None else epoch
-        return projection(self.state.seed, self.state.layer_id, ep, self.n, self.r, self.mode)
+        return projection(self.state.seed, self.state.layer_id, ep, self.n, self.r, self.mode, self.sparse_s)
 
     def forward(self, X):
         return linear_fwd(X, self.W, self.P(), self.mode)

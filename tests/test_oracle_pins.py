@@ -442,3 +442,87 @@ def test_tile_metric_hand_values():
     bad = big.copy()
     bad[128:256, 64:128] = 0.0
     assert co.rel_frobenius(bad, big) < 0.2 and worst_tile(bad, big, (128, 64)) == pytest.approx(1.0)
+
+
+# --- Sparse Johnson-Lindenstrauss projection (Ablation Study) ------------------------------------
+def test_sparse_jl_terms_counter_layout_and_hash():
+    seed, layer, epoch, n, r, s = (7 << 32) | 99, 3, 2, 5, 37, 6
+    cols, signs = co.sparse_jl_terms(seed, layer, epoch, n, r, s)
+    assert cols.shape == signs.shape == (n, s)
+    key = [seed & 0xFFFFFFFF, seed >> 32]
+    for i in range(n):
+        for t in range(s):
+            w = int(co.philox4x32_10([0x80000000 | (t >> 2), i, layer, epoch], key)[t & 3])   # pinned by the KATs
+            assert cols[i, t] == ((w & 0x7FFFFFFF) * r) >> 31 and signs[i, t] == (-1 if w >> 31 else 1)
+    assert cols.min() >= 0 and cols.max() < r
+    # the stream is its own: word 0 of the counter has its top bit set, so no call coincides with one behind the
+    # Gaussian projection of the same layer (whose word 0 is a column group below 2^30)
+    g = co.projection_words(seed, layer, epoch, n, 8)
+    first = np.array([int(co.philox4x32_10([0x80000000, i, layer, epoch], key)[0]) for i in range(n)])
+    assert not np.any(first == g[:, 0])
+
+
+def test_sparse_jl_projection_structure():
+    n, r, s = 300, 64, 8
+    P = co.projection_sparse_jl(5, 1, 0, n, r, s)
+    K = P * math.sqrt(s)
+    assert np.array_equal(K, np.rint(K))                                   # integer counts times 1/sqrt(s)
+    per_row = np.abs(K).sum(axis=1)
+    assert np.all(per_row <= s) and np.all((s - per_row) % 2 == 0)          # terms that cancel go in pairs
+    cols, signs = co.sparse_jl_terms(5, 1, 0, n, r, s)
+    distinct = np.array([len(set(c)) == s for c in cols])
+    assert distinct.any() and np.all(np.count_nonzero(K[distinct], axis=1) == s)   # no collision: exactly s entries of +-1
+    assert np.all(np.abs(K[distinct]).max(axis=1) == 1)
+    # a hand-built row: terms (col 2, +), (col 2, +), (col 0, -) give counts [-1, 0, 2]
+    Kh = np.zeros(3)
+    for c, sg in ((2, 1), (2, 1), (0, -1)):
+        Kh[c] += sg
+    assert list(Kh) == [-1.0, 0.0, 2.0]
+    # other epoch, layer or seed: another matrix; through the generic entry point: the same one
+    assert not np.array_equal(P, co.projection_sparse_jl(5, 1, 1, n, r, s))
+    assert not np.array_equal(P, co.projection_sparse_jl(5, 2, 0, n, r, s))
+    assert np.array_equal(P, co.projection(5, 1, 0, n, r, mode="bf16", sparse_s=s))
+
+
+def test_sparse_jl_scale_gives_identity_and_uniform_columns():
+    n, r, s, S = 6, 16, 4, 6000
+    acc = np.zeros((n, n))
+    for seed in range(S):
+        P = co.projection_sparse_jl(seed, 0, 0, n, r, s)
+        acc += P @ P.T
+    acc /= S
+    # diagonal: (1/s) * sum_j (count_j)^2 has mean 1; off-diagonal: mean 0, variance 1/r
+    assert np.all(np.abs(np.diag(acc) - 1.0) < 5 * math.sqrt(2.0 / (r * S)) + 5e-3)
+    off = acc - np.diag(np.diag(acc))
+    assert np.all(np.abs(off) < 5 * math.sqrt(1.0 / (r * S)))
+    cols, signs = co.sparse_jl_terms(1, 0, 0, 20000, 50, 8)
+    counts = np.bincount(cols.ravel(), minlength=50)
+    assert stats.chisquare(counts).pvalue > 1e-4
+    assert abs(signs.mean()) < 5 / math.sqrt(signs.size)
+
+
+def test_sparse_jl_layer_steps_like_the_dense_one():
+    # the layer with a sparse projection is Algorithms 1-3 with that P: compare with element loops
+    rng = np.random.default_rng(21)
+    bl, n, m, r, s = 5, 7, 4, 3, 2
+    lay = co.CompActLayerOracle(rng.standard_normal((n, m)), n, m, r, 9, 2, 0, 1e-2, 0.9, 0.999, 1e-8, sparse_s=s)
+    P = co.projection_sparse_jl(9, 2, 0, n, r, s)
+    assert np.array_equal(lay.P(), P)
+    X, dY = rng.standard_normal((bl, n)), rng.standard_normal((bl, m))
+    Y, Z = lay.forward(X)
+    Zl = np.zeros((bl, r))
+    cols, signs = co.sparse_jl_terms(9, 2, 0, n, r, s)
+    for t in range(bl):
+        for i in range(n):
+            for k in range(s):
+                Zl[t, cols[i, k]] += signs[i, k] * X[t, i] / math.sqrt(s)       # the signed gather the construction describes
+    assert np.allclose(Z, Zl, rtol=0, atol=1e-12)
+    W0 = lay.W.copy()
+    _, Gc = lay.backward(dY, Z)
+    lay.update(Gc)
+    N = (0.1 * Gc / 0.1) / (np.sqrt(0.001 * Gc * Gc / 0.001) + 1e-8)
+    Wl = W0.copy()
+    for i in range(n):
+        for k in range(s):
+            Wl[i] -= 1e-2 * signs[i, k] * N[cols[i, k]] / math.sqrt(s)          # the signed scatter of rows of N
+    assert np.allclose(lay.W, Wl, rtol=0, atol=1e-12)
