@@ -67,6 +67,9 @@ typedef struct {
   uint32_t layer_id;
   uint32_t refresh_T;
   float lr, beta1, beta2, eps, alpha;
+  int32_t sparse_s;   /* 0: Gaussian projection (Section 3.3).  s > 0: the sparse Johnson-Lindenstrauss
+                       * projection of the ablation study, s terms of +-1/sqrt(s) per row of P, at
+                       * Philox-hashed columns; terms that hit the same column add.  At most 64. */
 } compact_layer_config_t;
 
 typedef struct {
@@ -246,6 +249,10 @@ compact_status_t compact_debug_philox_u32(uint64_t seed, uint32_t layer_id, uint
                                           int32_t n, int32_t r, uint32_t* out_dev, void* stream);
 compact_status_t compact_debug_philox_layer_u32(uint64_t seed, uint32_t layer_id, uint32_t epoch,
                                                 int32_t n, int32_t r, uint32_t* out_dev, void* stream);
+/* compact_debug_sparse_terms: for a layer with sparse_s > 0, out_dev[n x sparse_s] receives
+ * the hashed terms of every row of P at `epoch`: column in the low 31 bits, sign in bit 31. */
+compact_status_t compact_debug_sparse_terms(const compact_layer_t* layer, uint32_t epoch,
+                                            uint32_t* out_dev, void* stream);
 compact_status_t compact_debug_projection(const compact_layer_t* layer, uint32_t epoch,
                                           void* P_dev, void* stream);
 

@@ -30,7 +30,7 @@ EXPORTS = [
     "compact_linear_bwd_recompute", "compact_group_workspace_bytes", "compact_group_fwd", "compact_group_bwd",
     "compact_adam_update", "compact_adam_update_noalloc",
     "compact_refresh_projection", "compact_layer_get_state", "compact_layer_set_state",
-    "compact_layer_status", "compact_debug_wait_that_runs_out", "compact_debug_philox_u32", "compact_debug_philox_layer_u32", "compact_debug_projection",
+    "compact_layer_status", "compact_debug_wait_that_runs_out", "compact_debug_philox_u32", "compact_debug_philox_layer_u32", "compact_debug_sparse_terms", "compact_debug_projection",
     "compact_set_kernel_family", "compact_kernel_launch_count", "compact_status_string",
 ]
 
@@ -39,7 +39,7 @@ class LayerConfig(C.Structure):
     _fields_ = [("n", C.c_int32), ("m", C.c_int32), ("r", C.c_int32), ("dtype", C.c_int32),
                 ("seed", C.c_uint64), ("layer_id", C.c_uint32), ("refresh_T", C.c_uint32),
                 ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
-                ("alpha", C.c_float)]
+                ("alpha", C.c_float), ("sparse_s", C.c_int32)]
 
 
 class LayerState(C.Structure):
@@ -88,6 +88,7 @@ def lib() -> C.CDLL:
     L.compact_debug_wait_that_runs_out.argtypes = [vp, vp]
     L.compact_debug_philox_u32.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_int32, C.c_int32, vp, vp]
     L.compact_debug_philox_layer_u32.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_int32, C.c_int32, vp, vp]
+    L.compact_debug_sparse_terms.argtypes = [vp, C.c_uint32, vp, vp]
     L.compact_debug_projection.argtypes = [vp, C.c_uint32, vp, vp]
     L.compact_set_kernel_family.argtypes = [C.c_int]
     L.compact_kernel_launch_count.restype = C.c_uint64
@@ -142,13 +143,15 @@ class CompactLinear:
 
     def __init__(self, n: int, m: int, r: int, dtype: torch.dtype = torch.bfloat16, seed: int = 0,
                  layer_id: int = 0, refresh_T: int = 0, lr: float = 1e-3, beta1: float = 0.9,
-                 beta2: float = 0.999, eps: float = 1e-8, alpha: float = 1.0):
+                 beta2: float = 0.999, eps: float = 1e-8, alpha: float = 1.0, sparse_s: int = 0):
+        """sparse_s > 0 selects the sparse Johnson-Lindenstrauss projection with that many terms per row of P."""
         self.n, self.m, self.r = n, m, r
+        self.sparse_s = sparse_s
         self.dtype = dtype
         code = {torch.float32: F32, torch.bfloat16: BF16}.get(dtype)
         if code is None:
             raise CompactError(ERR_DTYPE, "CompactLinear")
-        self.cfg = LayerConfig(n, m, r, code, seed, layer_id, refresh_T, lr, beta1, beta2, eps, alpha)
+        self.cfg = LayerConfig(n, m, r, code, seed, layer_id, refresh_T, lr, beta1, beta2, eps, alpha, sparse_s)
         self._h = C.c_void_p()
         _check(lib().compact_layer_create(C.byref(self.cfg), C.byref(self._h)), "compact_layer_create")
         self.ldz = int(lib().compact_z_ld(self._h))
@@ -274,6 +277,13 @@ class CompactLinear:
         ep = C.c_uint32()
         _check(lib().compact_refresh_projection(self._h, int(force), C.byref(ep)), "compact_refresh_projection")
         return int(ep.value)
+
+    def debug_sparse_terms(self, epoch: Optional[int] = None, stream=None) -> torch.Tensor:
+        """(n, sparse_s) int32: column in the low 31 bits, sign in bit 31, of every hashed term of P."""
+        out = torch.empty((self.n, self.sparse_s), dtype=torch.int32, device="cuda")
+        _check(lib().compact_debug_sparse_terms(self._h, self.epoch if epoch is None else epoch, _ptr(out),
+                                                _stream(stream)), "compact_debug_sparse_terms")
+        return out
 
     def debug_projection(self, epoch: Optional[int] = None, stream=None) -> torch.Tensor:
         P = torch.empty((self.n, self.r), dtype=self.dtype, device="cuda")

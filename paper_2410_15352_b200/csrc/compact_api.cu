@@ -133,6 +133,8 @@ ProjectionParams make_pp(const compact_layer_t* L, uint32_t epoch) {
   pp.r = L->cfg.r;
   pp.inv_sqrt_r = (float)(1.0 / sqrt((double)L->cfg.r));
   pp.neg2ln2_over_r = (float)(-2.0 * 0.6931471805599453 / (double)L->cfg.r);
+  pp.sparse_s = L->cfg.sparse_s;
+  pp.inv_sqrt_s = L->cfg.sparse_s > 0 ? (float)(1.0 / sqrt((double)L->cfg.sparse_s)) : 1.0f;
   return pp;
 }
 
@@ -238,6 +240,7 @@ compact_status_t compact_layer_create(const compact_layer_config_t* cfg, compact
   if (cfg->n % mult || cfg->m % mult) return COMPACT_ERR_SHAPE;
   if (!(cfg->beta1 >= 0.f && cfg->beta1 < 1.f) || !(cfg->beta2 >= 0.f && cfg->beta2 < 1.f)) return COMPACT_ERR_INVALID_ARG;
   if (!(cfg->eps >= 0.f) || isnan(cfg->lr) || isnan(cfg->alpha)) return COMPACT_ERR_INVALID_ARG;
+  if (cfg->sparse_s < 0 || cfg->sparse_s > 64) return COMPACT_ERR_INVALID_ARG;
   compact_layer_t* L = new (std::nothrow) compact_layer_t;
   if (!L) return COMPACT_ERR_INVALID_ARG;
   L->cfg = *cfg;
@@ -535,12 +538,15 @@ compact_status_t compact_adam_update(compact_layer_t* L, void* W, int64_t ldw, c
       tc::LaunchInfo li{g_family.load() == 2 ? 1 : CFG_CS, st, status_word(L), sched_words(L), &g_launches};
       // one launch (Adam, resident panel of P, sweep over W) where the rank fits the panel; otherwise the Adam
       // kernel followed by the streaming GEMM
+      // (the tiles of a sparse projection hold integer counts: its 1/sqrt(s) rides on the step size)
+      const ProjectionParams pp = make_pp(L, L->epoch);
+      const float step_scale = lr * L->cfg.alpha * pp.inv_sqrt_s;
       if (g_family.load() == 0 && upd::fused_update_ok(L->cfg.n, L->cfg.m, L->cfg.r))
-        s = upd::fused_update(li, make_pp(L, L->epoch), adam_scalars(L, L->step + 1), L->cfg.n, L->cfg.m, L->cfg.r, (T*)W, ldw,
-                              Gc, ldg, M, V, lr * L->cfg.alpha, workspace, workspace_bytes);
+        s = upd::fused_update(li, pp, adam_scalars(L, L->step + 1), L->cfg.n, L->cfg.m, L->cfg.r, (T*)W, ldw,
+                              Gc, ldg, M, V, step_scale, workspace, workspace_bytes);
       else
-        s = tc::update(li, make_pp(L, L->epoch), adam_scalars(L, L->step + 1), L->cfg.n, L->cfg.m, L->cfg.r, (T*)W, ldw,
-                       Gc, ldg, M, V, lr * L->cfg.alpha, workspace, workspace_bytes);
+        s = tc::update(li, pp, adam_scalars(L, L->step + 1), L->cfg.n, L->cfg.m, L->cfg.r, (T*)W, ldw,
+                       Gc, ldg, M, V, step_scale, workspace, workspace_bytes);
     }
     if (s == COMPACT_ERR_SHAPE) s = update_simt<T>(L, (T*)W, ldw, Gc, ldg, M, V, lr, (float*)workspace, st);
   } else {
@@ -672,6 +678,15 @@ compact_status_t compact_debug_philox_layer_u32(uint64_t seed, uint32_t layer_id
   const uint64_t pl = (uint64_t)0xCD9E8D57u * (uint64_t)layer_id;
   debug_philox_layer_words_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
       make_philox_key(seed), (uint32_t)(pl >> 32), (uint32_t)pl, epoch, n, groups, out_dev);
+  g_launches++;
+  return launch_result();
+}
+
+compact_status_t compact_debug_sparse_terms(const compact_layer_t* L, uint32_t epoch, uint32_t* out_dev, void* stream) {
+  if (!L || !out_dev || L->cfg.sparse_s <= 0) return COMPACT_ERR_INVALID_ARG;
+  const ProjectionParams pp = make_pp(L, epoch);
+  const int64_t cnt = (int64_t)pp.n * pp.sparse_s;
+  debug_sparse_terms_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, (cudaStream_t)stream>>>(pp, out_dev);
   g_launches++;
   return launch_result();
 }

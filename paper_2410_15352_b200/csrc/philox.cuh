@@ -127,7 +127,34 @@ struct ProjectionParams {
   int32_t r;
   float inv_sqrt_r;
   float neg2ln2_over_r;
+  int32_t sparse_s;              // > 0: sparse Johnson-Lindenstrauss projection with this many terms per row
+  float inv_sqrt_s;
 };
+
+// Sparse Johnson-Lindenstrauss projection (the paper's ablation study; the construction it cites hashes every
+// input coordinate s times into the r outputs with random signs, scaled by 1/sqrt(s); colliding terms add).
+// Terms 4q .. 4q+3 of row i are the words of the Philox call with counter (0x80000000 | q, i, layer_id, epoch):
+// the top bit of a word is the sign, its low 31 bits pick the column as ((word & 0x7fffffff) * r) >> 31.
+__device__ __forceinline__ uint4 sparse_words4(uint32_t q, uint32_t i, uint32_t epoch, uint32_t layer_hi, uint32_t layer_lo,
+                                               const PhiloxKey& key) {
+  return philox4x32_10_layer(0x80000000u | q, i, epoch, layer_hi, layer_lo, key);
+}
+__device__ __forceinline__ int sparse_col(uint32_t word, int r) { return (int)__umulhi(word << 1, (uint32_t)r); }
+__device__ __forceinline__ float sparse_sign(uint32_t word) { return (word >> 31) ? -1.0f : 1.0f; }
+
+// Entry (i, j) of the sparse projection as its integer count (the sum of the signs of the terms of row i that
+// hash to column j); the caller scales by 1/sqrt(s).
+__device__ __forceinline__ float sparse_count(const ProjectionParams& pp, int i, int j) {
+  float k = 0.f;
+  for (int q = 0; 4 * q < pp.sparse_s; ++q) {
+    const uint4 x = sparse_words4((uint32_t)q, (uint32_t)i, pp.epoch, pp.layer_hi, pp.layer_lo, pp.key);
+    const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+    for (int l = 0; l < 4; ++l)
+      if (4 * q + l < pp.sparse_s && sparse_col(w[l], pp.r) == j) k += sparse_sign(w[l]);
+  }
+  return k;
+}
 
 // P[i, 4q .. 4q+3] in fp32; columns >= r are zero, rows >= n are zero.
 // kFast selects the approximate Box-Muller (bf16 layers); fp32 layers use the accurate one.
@@ -152,6 +179,7 @@ __device__ __forceinline__ float4 projection4(const ProjectionParams& pp, int i,
 
 template <bool kFast>
 __device__ __forceinline__ float projection1(const ProjectionParams& pp, int i, int j) {
+  if (pp.sparse_s > 0) return (i < pp.n && j < pp.r) ? sparse_count(pp, i, j) * pp.inv_sqrt_s : 0.f;
   const float4 g = projection4<kFast>(pp, i, j >> 2);
   const int l = j & 3;
   return l == 0 ? g.x : (l == 1 ? g.y : (l == 2 ? g.z : g.w));

@@ -36,7 +36,8 @@ template <bool kRoundBf16, bool kAsB> struct GeneratedP {
   __device__ __forceinline__ float operator()(int a, int b) const {
     const int i = kAsB ? b : a, j = kAsB ? a : b;
     float v = projection1<kRoundBf16>(pp, i, j);
-    if (kRoundBf16) v = __bfloat162float(__float2bfloat16_rn(v));
+    // Gaussian entries are stored as bf16 in bf16 layers; the sparse projection's multiples of 1/sqrt(s) are not rounded
+    if (kRoundBf16 && pp.sparse_s == 0) v = __bfloat162float(__float2bfloat16_rn(v));
     return v;
   }
 };
@@ -162,14 +163,29 @@ __global__ void debug_philox_layer_words_kernel(PhiloxKey key, uint32_t layer_hi
   reinterpret_cast<uint4*>(out)[idx] = x;
 }
 
+// The terms of the sparse projection: out[i * s + t] = column | sign bit << 31.
+__global__ void debug_sparse_terms_kernel(ProjectionParams pp, uint32_t* out) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)pp.n * pp.sparse_s) return;
+  const int i = (int)(idx / pp.sparse_s), t = (int)(idx % pp.sparse_s);
+  const uint4 x = sparse_words4((uint32_t)(t >> 2), (uint32_t)i, pp.epoch, pp.layer_hi, pp.layer_lo, pp.key);
+  const uint32_t w = (t & 3) == 0 ? x.x : ((t & 3) == 1 ? x.y : ((t & 3) == 2 ? x.z : x.w));
+  out[idx] = (uint32_t)sparse_col(w, pp.r) | (w & 0x80000000u);
+}
+
 template <typename T>
 __global__ void debug_projection_kernel(ProjectionParams pp, T* P) {
   const int groups = (pp.r + 3) / 4;
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (int64_t)pp.n * groups) return;
   const int i = (int)(idx / groups), q = (int)(idx % groups);
-  const float4 g = projection4<sizeof(T) == 2>(pp, i, q);
-  const float v[4] = {g.x, g.y, g.z, g.w};
+  float v[4];
+  if (pp.sparse_s > 0) {
+    for (int l = 0; l < 4; ++l) v[l] = projection1<sizeof(T) == 2>(pp, i, 4 * q + l);
+  } else {
+    const float4 g = projection4<sizeof(T) == 2>(pp, i, q);
+    v[0] = g.x; v[1] = g.y; v[2] = g.z; v[3] = g.w;
+  }
   for (int l = 0; l < 4; ++l)
     if (4 * q + l < pp.r) P[(int64_t)i * pp.r + 4 * q + l] = simt::from_f32<T>(v[l]);
 }

@@ -99,6 +99,7 @@ struct Problem {
   // the projection a generated operand is a tile of; the Philox key (the seed) is the launch's
   uint32_t pp_layer_hi, pp_layer_lo, pp_epoch;
   int pp_n, pp_r;
+  int pp_sparse_s;        // > 0: the generated operand is the sparse projection, as integer counts (scaled in the epilogue)
   float pp_scale;         // -2 ln 2 / r
   // K may run over up to three segments with operands of their own (dX of a group of layers that share
   // their input is the sum over the layers of dY_g W_g^T): segment s covers k-steps seg_begin[s] .. seg_begin[s+1]
@@ -272,6 +273,11 @@ __device__ __forceinline__ void st_async_16(uint32_t raddr, uint4 v, uint32_t rb
   asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(raddr),
                "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"(rbar)
                : "memory");
+}
+
+// Barrier among `threads` threads of the CTA (a multiple of 32), by number; 0 is __syncthreads'.
+__device__ __forceinline__ void named_barrier(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
 // True in exactly one lane of a converged warp.
@@ -571,7 +577,8 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
             bool gen_here = false;
             // of a generated tile, the shares of the other CTAs arrive as counted bytes
             if (hb) tx += p.bn * BK * 2;
-            if (na > 0) { if (a_tma) tx += na * A_BYTES; else { gen_here = true; tx += (A_BYTES / cs) * (cs - 1); } }
+            // (a tile of the sparse projection is cheap: every CTA writes all of it itself)
+            if (na > 0) { if (a_tma) tx += na * A_BYTES; else { gen_here = true; if (p.pp_sparse_s == 0) tx += (A_BYTES / cs) * (cs - 1); } }
             if (elect_one()) {
               // A stage that holds a generated tile is handed back with commits from each CTA of the
               // cluster, so that no CTA writes its share of the next tile (or counts its bytes) into a
@@ -885,7 +892,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
 #pragma unroll
                 for (int z = 0; z < 32; ++z)
                   *reinterpret_cast<__nv_bfloat16*>(stg_gen + (32 * h + z) * 64 + lane * 2) =
-                      __float2bfloat16_rn(__uint_as_float(v[z]));
+                      __float2bfloat16_rn(__uint_as_float(v[z]) * p.scale);     // 1, or 1/sqrt(s) of the sparse projection
               }
             }
             if (!ok) break;
@@ -963,9 +970,40 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         const uint32_t full_off = full_bar(geo, s) - bars;
         const bool w = mbar_wait(empty_bar(geo, s), eph, abort_flag, prm.status);
         const int k0 = ks * BK;
+        if (gp.pp_sparse_s > 0) {
+          // Sparse projection: the tile holds the integer counts.  All generator threads clear it, then one
+          // thread per row of P adds the signs of that row's terms that fall into the tile's columns (a row
+          // has one writer, so colliding terms add without a race).  Every CTA writes the whole tile.
+          uint8_t* tile = smem_gen + stage_off + STAGE_A0_OFF;
+          if (w) {
+            reinterpret_cast<uint4*>(tile)[gtid] = make_uint4(0u, 0u, 0u, 0u);
+            reinterpret_cast<uint4*>(tile)[gtid + GSTRIDE] = make_uint4(0u, 0u, 0u, 0u);
+          }
+          named_barrier(2, GSTRIDE);
+          const int nrows = gen_at ? BK : BM;
+          const int i = gen_at ? k0 + gtid : t.m0 + gtid;              // the row of P this thread owns
+          const int c_first = gen_at ? t.m0 : k0, c_count = gen_at ? BM : BK;
+          if (w && gtid < nrows && i < gp.pp_n) {
+            for (int q = 0; 4 * q < gp.pp_sparse_s; ++q) {
+              const uint4 x = sparse_words4((uint32_t)q, (uint32_t)i, gp.pp_epoch, gp.pp_layer_hi, gp.pp_layer_lo, prm.key);
+              const uint32_t wd[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+              for (int l = 0; l < 4; ++l) {
+                const int c = sparse_col(wd[l], gp.pp_r) - c_first;
+                if (4 * q + l < gp.pp_sparse_s && c >= 0 && c < c_count) {
+                  const int rr = gtid;
+                  const uint32_t off = gen_at ? (uint32_t)((c >> 6) * 8192 + rr * 128 + ((((c >> 3) & 7) ^ (rr & 7)) << 4) + (c & 7) * 2)
+                                              : (uint32_t)(rr * 128 + (((c >> 3) ^ (rr & 7)) << 4) + (c & 7) * 2);
+                  __nv_bfloat16* e = reinterpret_cast<__nv_bfloat16*>(tile + off);
+                  *e = __float2bfloat16_rn(__bfloat162float(*e) + sparse_sign(wd[l]));
+                }
+              }
+            }
+          }
+        }
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
-          if (u < ntask && w) {
+          if (u < ntask && w && gp.pp_sparse_s == 0) {
             const uint4 val = projection8_bf16(prm.key, gp.pp_layer_hi, gp.pp_layer_lo, gp.pp_epoch, gp.pp_n, gp.pp_r,
                                                gp.pp_scale, t_i[u] + ik * k0, t_j[u] + jk * k0);
             const uint32_t off = stage_off + t_off[u];
@@ -1154,6 +1192,7 @@ inline int pick_bn(int N) { return N >= BN_MAX ? BN_MAX : (int)((N + 63) / 64 * 
 inline void set_projection(Problem& p, const ProjectionParams& pp) {
   p.pp_layer_hi = pp.layer_hi; p.pp_layer_lo = pp.layer_lo; p.pp_epoch = pp.epoch;
   p.pp_n = pp.n; p.pp_r = pp.r; p.pp_scale = pp.neg2ln2_over_r;
+  p.pp_sparse_s = pp.sparse_s;
 }
 
 inline void finish_problem(Problem& p, int splits_wanted) {
@@ -1297,6 +1336,7 @@ inline compact_status_t forward(const LaunchInfo& li, const ProjectionParams& pp
     pz.ncol = tokens > BN_MAX ? 2 : 1;
     pz.a_mode = GENERATED_T; pz.b_mode = TMA_KMAJOR; pz.epi_mode = EPI_BF16_T;
     set_projection(pz, pp);
+    pz.scale = pp.inv_sqrt_s;
     finish_problem(pz, 1);
     prm.tmA[0] = prm.tmA[iy];   // unused by the generated operand (set below when Y is present)
     if (!make_map(&prm.tmB[0], X, n, tokens, ldx, BK, pz.bn)) return COMPACT_ERR_CUDA;
@@ -1402,6 +1442,7 @@ inline compact_status_t forward_group(const LaunchInfo& li, int G, const GroupLa
     pz.ncol = tokens > BN_MAX ? 2 : 1;
     pz.a_mode = GENERATED_T; pz.b_mode = TMA_KMAJOR; pz.epi_mode = EPI_BF16_T;
     set_projection(pz, L[g].pp);
+    pz.scale = L[g].pp.inv_sqrt_s;
     finish_problem(pz, 1);
     if (!make_map(&prm.tmB[g], X, n, tokens, ldx, BK, pz.bn)) return COMPACT_ERR_CUDA;
     prm.tmA[g] = prm.tmB[g];   // unused by the generated operand

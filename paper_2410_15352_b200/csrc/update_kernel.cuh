@@ -53,6 +53,7 @@ struct alignas(64) UpdParams {
   PhiloxKey key;
   uint32_t layer_hi, layer_lo, epoch;
   float pp_scale;           // -2 ln 2 / r
+  int sparse_s;             // > 0: sparse projection (the panel holds integer counts; 1/sqrt(s) is part of `scale`)
   unsigned int* status;
   unsigned int* sched;      // three words, zero between launches: CTAs done with phase 1, CTAs finished, next run of phase 1
 };
@@ -62,9 +63,6 @@ __device__ __forceinline__ unsigned int ld_acquire_gpu(const unsigned int* p) {
   unsigned int v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
-}
-__device__ __forceinline__ void named_barrier(int id, int threads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
 // Warp roles:
@@ -377,6 +375,35 @@ __global__ void __launch_bounds__(U_THREADS, 1) compact_update_kernel(const __gr
         free_phase ^= 1u;
         if (!ok) break;
       }
+      if (prm.sparse_s > 0) {
+        // Sparse projection: every CTA builds the whole panel itself.  All threads clear it, then one thread per
+        // row adds the signs of the row's terms at their columns (one writer per row: colliding terms add).
+        if (gtid == 0)
+          for (int kt = 0; kt < prm.ktiles; ++kt) mbar_arrive(pfull_bar(kt));
+        for (int x = gtid; x < prm.ktiles * (A_BYTES / 16); x += 32 * U_GEN_WARPS)
+          reinterpret_cast<uint4*>(smem_gen)[x] = make_uint4(0u, 0u, 0u, 0u);
+        named_barrier(2, 32 * U_GEN_WARPS);
+        const int row = panel * BM + gtid;
+        if (gtid < BM && row < prm.n) {
+          for (int q = 0; 4 * q < prm.sparse_s; ++q) {
+            const uint4 x = sparse_words4((uint32_t)q, (uint32_t)row, prm.epoch, prm.layer_hi, prm.layer_lo, prm.key);
+            const uint32_t wd[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int l = 0; l < 4; ++l) {
+              if (4 * q + l >= prm.sparse_s) continue;
+              const int col = sparse_col(wd[l], prm.r), kt = col >> 6, cc = col & 63;
+              __nv_bfloat16* e = reinterpret_cast<__nv_bfloat16*>(smem_gen + kt * A_BYTES + gtid * 128 + (((cc >> 3) ^ (gtid & 7)) << 4) + (cc & 7) * 2);
+              *e = __float2bfloat16_rn(__bfloat162float(*e) + sparse_sign(wd[l]));
+            }
+          }
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0)
+          for (int kt = 0; kt < prm.ktiles; ++kt) mbar_arrive(pfull_bar(kt));
+        if (first_job) adam_slice();
+        continue;
+      }
       // the neighbour's half of every tile arrives as counted bytes
       if (gtid == 0)
         for (int kt = 0; kt < prm.ktiles; ++kt) mbar_arrive_expect_tx(pfull_bar(kt), A_BYTES / 2);
@@ -455,6 +482,7 @@ inline compact_status_t fused_update(const LaunchInfo& li, const ProjectionParam
   prm.key = pp.key;
   prm.layer_hi = pp.layer_hi; prm.layer_lo = pp.layer_lo; prm.epoch = pp.epoch;
   prm.pp_scale = pp.neg2ln2_over_r;
+  prm.sparse_s = pp.sparse_s;
   prm.status = li.status;
   prm.sched = li.sched;
   if (!make_map_blocked(&prm.tmN, workspace, m, r, ldn, U_SK, U_BN / 64)) return COMPACT_ERR_CUDA;

@@ -47,6 +47,7 @@ class Workload:
     seed: int = 0
     x_scale_inv_sqrt_n: bool = False
     dy_std: float | None = None   # None: 1/sqrt(n)
+    sparse_s: int = 0             # > 0: the layers use the sparse JL projection with this many terms per row
 
     def with_tokens(self, tokens: int) -> "Workload":
         return Workload(**{**self.__dict__, "tokens": tokens})

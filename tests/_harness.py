@@ -69,10 +69,10 @@ def make_pair(wl: wlm.Workload, li: int):
     dt = wlm.torch_dtype(wl.dtype)
     W0 = wlm.draw_W(wl, li)
     gpu = cb.CompactLinear(L.n, L.m, L.r, dtype=dt, seed=wl.seed, layer_id=li, refresh_T=wl.refresh_T,
-                           lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps, alpha=wl.alpha)
+                           lr=wl.lr, beta1=wl.beta1, beta2=wl.beta2, eps=wl.eps, alpha=wl.alpha, sparse_s=wl.sparse_s)
     ora = co.CompActLayerOracle(to64(W0), L.n, L.m, L.r, seed=wl.seed, layer_id=li, refresh_T=wl.refresh_T,
                                 lr=f32(wl.lr), beta1=f32(wl.beta1), beta2=f32(wl.beta2), eps=f32(wl.eps),
-                                alpha=f32(wl.alpha), mode="exact" if wl.dtype == "f32" else "bf16")
+                                alpha=f32(wl.alpha), mode="exact" if wl.dtype == "f32" else "bf16", sparse_s=wl.sparse_s)
     return gpu, ora, W0
 
 
