@@ -493,23 +493,17 @@ inline compact_status_t fused_update(const LaunchInfo& li, const ProjectionParam
   cfg.blockDim = dim3((unsigned)U_THREADS, 1, 1);
   cfg.dynamicSmemBytes = U_SMEM_BYTES;
   cfg.stream = li.stream;
-  cudaLaunchAttribute attr[2];
+  // The grid is one CTA per SM at most, so all of it is resident at once; the wait at the phase barrier is bounded
+  // like every other wait.  (A cooperative launch would state that requirement to the driver; it is left out
+  // because the profiler could not launch the kernel with it.)
+  cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
-  // phase 2 of every CTA waits for phase 1 of all: the grid must be resident as a whole
-  attr[1].id = cudaLaunchAttributeCooperative;
-  attr[1].val.cooperative = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 2;
-  cudaError_t e = cudaLaunchKernelEx(&cfg, compact_update_kernel, prm);
-  if (e != cudaSuccess) {
-    // a driver that does not combine the two attributes: the grid is one CTA per SM and every wait is bounded
-    cudaGetLastError();
-    cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, compact_update_kernel, prm);
-  }
+  cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, compact_update_kernel, prm);
   (*li.launches)++;
   if (e != cudaSuccess) { cudaGetLastError(); return COMPACT_ERR_CUDA; }
   return cudaGetLastError() == cudaSuccess ? COMPACT_OK : COMPACT_ERR_CUDA;
