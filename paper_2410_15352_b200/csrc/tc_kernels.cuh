@@ -942,7 +942,12 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       //   transposed forward: A[m = column j of P][k = row i of P], MN-major, two 64-column blocks of [64 k][128 B]
       //   update:             A[m = row i of P][k = column j of P], K-major, [128 rows][128 B]
       // Of a tile shared by a cluster this CTA writes the rows crank * (rows / cs) onward.
-      const int ntask = 2 >> csh;                       // tasks per thread and tile: 1024 / (512 cs)
+      // When a k-step takes two stages (the generated tiles then live in stages 0 and 2) and a cluster shares them, the
+      // sixteen warps work as two halves, one per stage: a half builds every other tile, two tasks per thread, and its
+      // fence, arrival and wait for the stage overlap the other half's arithmetic.  A half meets every use of its stage.
+      const bool halves = t.nst == 2 && cs == 2;
+      const int my_half = (warp - (THREADS_BASE >> 5)) >> 3;
+      const int ntask = halves ? 2 : (2 >> csh);        // tasks per thread and tile
       // the plain instantiation's only generated problem is problem 0: constant-bank operands
       const Problem& gp = kGroup ? p : prm.prob[0];
       const int ik = gen_at ? 1 : 0, jk = 1 - ik;       // which index of P advances with k
@@ -950,7 +955,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
       uint32_t t_off[2];
 #pragma unroll
       for (int u = 0; u < 2; ++u) {
-        const int id = gtid + u * GSTRIDE;
+        const int id = halves ? (gtid & (GSTRIDE / 2 - 1)) + u * (GSTRIDE / 2) : gtid + u * GSTRIDE;
         if (gen_at) {
           const int c = id & 15, kr = (int)crank * (BK >> csh) + (id >> 4);
           t_i[u] = kr; t_j[u] = t.m0 + c * 8;
@@ -968,22 +973,27 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         if (t.nst > 1) ring_next(r, ns);            // a k-step takes one or two stages
         const uint32_t stage_off = (uint32_t)s * (geo ? STAGE1_BYTES : STAGE0_BYTES);
         const uint32_t full_off = full_bar(geo, s) - bars;
-        const bool w = mbar_wait(empty_bar(geo, s), eph, abort_flag, prm.status);
         const int k0 = ks * BK;
         if (gp.pp_sparse_s > 0) {
-          // Sparse projection: the tile holds the integer counts.  All generator threads clear it, then one
-          // thread per row of P adds the signs of that row's terms that fall into the tile's columns (a row
-          // has one writer, so colliding terms add without a race).  Every CTA writes the whole tile.
+          // Sparse projection: the tile holds the integer counts and every CTA writes the whole of it.  The
+          // sixteen warps work as four groups of four; the group whose number is the stage's builds the tile, so
+          // that up to four tiles are under construction at once (one tile is a chain of waits -- free stage,
+          // clear, Philox, scatter, fence -- far longer than its arithmetic) and a group meets every use of its
+          // stage.  The group's threads clear the tile, then one thread per row of P adds the signs of the row's
+          // terms that fall into the tile's columns (a row has one writer: colliding terms add without a race).
+          const int grp = (warp - (THREADS_BASE >> 5)) >> 2, gt = gtid & 127;
+          if (grp != s) continue;
+          const bool w = mbar_wait(empty_bar(geo, s), eph, abort_flag, prm.status);
           uint8_t* tile = smem_gen + stage_off + STAGE_A0_OFF;
           if (w) {
-            reinterpret_cast<uint4*>(tile)[gtid] = make_uint4(0u, 0u, 0u, 0u);
-            reinterpret_cast<uint4*>(tile)[gtid + GSTRIDE] = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+            for (int x = 0; x < A_BYTES / 16 / 128; ++x) reinterpret_cast<uint4*>(tile)[gt + 128 * x] = make_uint4(0u, 0u, 0u, 0u);
           }
-          named_barrier(2, GSTRIDE);
+          named_barrier(2 + grp, 128);
           const int nrows = gen_at ? BK : BM;
-          const int i = gen_at ? k0 + gtid : t.m0 + gtid;              // the row of P this thread owns
+          const int i = gen_at ? k0 + gt : t.m0 + gt;                  // the row of P this thread owns
           const int c_first = gen_at ? t.m0 : k0, c_count = gen_at ? BM : BK;
-          if (w && gtid < nrows && i < gp.pp_n) {
+          if (w && gt < nrows && i < gp.pp_n) {
             for (int q = 0; 4 * q < gp.pp_sparse_s; ++q) {
               const uint4 x = sparse_words4((uint32_t)q, (uint32_t)i, gp.pp_epoch, gp.pp_layer_hi, gp.pp_layer_lo, prm.key);
               const uint32_t wd[4] = {x.x, x.y, x.z, x.w};
@@ -991,7 +1001,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
               for (int l = 0; l < 4; ++l) {
                 const int c = sparse_col(wd[l], gp.pp_r) - c_first;
                 if (4 * q + l < gp.pp_sparse_s && c >= 0 && c < c_count) {
-                  const int rr = gtid;
+                  const int rr = gt;
                   const uint32_t off = gen_at ? (uint32_t)((c >> 6) * 8192 + rr * 128 + ((((c >> 3) & 7) ^ (rr & 7)) << 4) + (c & 7) * 2)
                                               : (uint32_t)(rr * 128 + (((c >> 3) ^ (rr & 7)) << 4) + (c & 7) * 2);
                   __nv_bfloat16* e = reinterpret_cast<__nv_bfloat16*>(tile + off);
@@ -1000,10 +1010,16 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
               }
             }
           }
+          fence_proxy_async_smem();
+          ok = __all_sync(0xffffffffu, w);
+          if (ok && lane == 0) mbar_arrive_n(full_bar(geo, s), NUM_GEN_WARPS / 4);     // four warps stand in for the sixteen
+          continue;
         }
+        if (halves && ((s >> 1) & 1) != my_half) continue;
+        const bool w = mbar_wait(empty_bar(geo, s), eph, abort_flag, prm.status);
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
-          if (u < ntask && w && gp.pp_sparse_s == 0) {
+          if (u < ntask && w) {
             const uint4 val = projection8_bf16(prm.key, gp.pp_layer_hi, gp.pp_layer_lo, gp.pp_epoch, gp.pp_n, gp.pp_r,
                                                gp.pp_scale, t_i[u] + ik * k0, t_j[u] + jk * k0);
             const uint32_t off = stage_off + t_off[u];
@@ -1013,7 +1029,7 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
         }
         fence_proxy_async_smem();
         ok = __all_sync(0xffffffffu, w);
-        if (ok && lane == 0) mbar_arrive(full_bar(geo, s));
+        if (ok && lane == 0) mbar_arrive_n(full_bar(geo, s), halves ? 2 : 1);     // a half's eight warps stand in for the sixteen
         // later stages of the k-step hold no generated data: the stage owner arrives for the generators there
       }
       if (geo) r1 = r; else r0 = r;
