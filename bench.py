@@ -257,10 +257,12 @@ class LayerBuffers:
 
 
 # DRAM traffic per launch from the committed ncu captures (profiles/): bytes per algorithmic flop of the forward and
-# backward launches of the C5 q_proj layer, and bytes per algorithmic byte of one update launch whose W does not
-# sit in L2 beforehand.  Scaled to the benchmarked launches by their algorithmic work.
-NCU_GEMM_DRAM_BYTES_PER_FLOP = (578.9e6 + 629.6e6) / 1236.95e9
-NCU_UPDATE_DRAM_BYTES_PER_ALG_BYTE = None
+# backward launches of the C5 q_proj layer (compact_gemm_kernel_c5_qproj_full.md: 441.1 + 132.9 and 425.9 + 160.5 MB
+# for 2 x 618.5 GFLOP), and bytes per algorithmic byte of one update launch whose W does not sit in L2 beforehand
+# (compact_update_kernel_c5_gate_proj.md: 169.6 + 97.4 MB for 293.1 MB).  Scaled to the benchmarked launches by
+# their algorithmic work.
+NCU_GEMM_DRAM_BYTES_PER_FLOP = (441.1e6 + 132.9e6 + 425.9e6 + 160.5e6) / 1236.95e9
+NCU_UPDATE_DRAM_BYTES_PER_ALG_BYTE = (169.6e6 + 97.4e6) / 293.1e6
 
 
 def must_spawn(gpus: int, environ) -> bool:
