@@ -257,10 +257,12 @@ compact_status_t compact_debug_projection(const compact_layer_t* layer, uint32_t
                                           void* P_dev, void* stream);
 
 /* Selects the kernel family: 0 = automatic (tensor-core kernels for bf16 where
- * the shape allows, SIMT otherwise), 1 = force the SIMT kernels, 2 = tensor-core
- * kernels in which every CTA generates its own tiles of P instead of sharing
- * them across a thread-block cluster (1 and 2 are used by the tests as on-device
- * cross-checks).  Returns the previous value. */
+ * the shape allows -- pairs of SMs for the TMA-fed products, a cluster that shares
+ * every generated tile of P, the one-launch update --, SIMT otherwise), 1 = force
+ * the SIMT kernels, 2 = tensor-core kernels that work one SM at a time: every CTA
+ * computes its own tiles and generates its own tiles of P, and the update is the
+ * Adam kernel followed by the streaming GEMM (1 and 2 are used by the tests as
+ * on-device cross-checks).  Returns the previous value. */
 int compact_set_kernel_family(int family);
 
 /* Number of kernels this library has launched since it was loaded. */

@@ -15,6 +15,7 @@
 #include "simt_kernels.cuh"
 #include "tc_kernels.cuh"
 #include "update_kernel.cuh"
+#include "gemm2_kernel.cuh"
 
 using namespace compact;
 
@@ -297,9 +298,24 @@ compact_status_t compact_linear_fwd(compact_layer_t* L, int64_t tokens, const vo
     typedef __nv_bfloat16 T;
     if (g_family.load() != 1) {
       tc::LaunchInfo li{g_family.load() == 2 ? 1 : CFG_CS, st, status_word(L), sched_words(L), &g_launches};
-      s = tc::forward(li, make_pp(L, L->epoch), tokens, L->cfg.m, (const T*)X, ldx, (const T*)W, ldw, (T*)Y, ldy, (T*)Z, ldz,
-                      (int)compact_z_ld(L));
-      if (s != COMPACT_ERR_SHAPE) return s;   // SHAPE: the tensor-core kernel does not take it
+      // Two routes with the same bits.  One launch: the Z items, then the Y items as 256 x 256 tiles on single SMs,
+      // which also fill the SMs the Z items leave idle.  Two launches: Z alone, then Y on pairs of SMs, whose
+      // epilogues run under the next tile's MMAs (about 3 % on Y).  The second pays when that gain outweighs the
+      // idle tail of a launch that holds nothing but Z items.
+      bool split = false;
+      if (g_family.load() == 0 && Z && tokens >= 2 * tc::BN_MAX) {
+        const double z_rounds = (double)((compact_z_ld(L) + tc::BM - 1) / tc::BM) * (double)((tokens + 511) / 512) / tc::NUM_SMS;
+        const double y_rounds = (double)((tokens + 255) / 256) * (double)((L->cfg.m + 255) / 256) / tc::NUM_SMS;
+        split = (ceil(z_rounds) - z_rounds) < 0.03 * y_rounds;
+      }
+      if (split) {
+        s = tc::forward(li, make_pp(L, L->epoch), tokens, L->cfg.m, (const T*)X, ldx, nullptr, 0, nullptr, 0, (T*)Z, ldz, (int)compact_z_ld(L));
+        if (s == COMPACT_OK) s = g2::g2_forward_y(li, tokens, L->cfg.n, L->cfg.m, (const T*)X, ldx, (const T*)W, ldw, (T*)Y, ldy);
+      } else {
+        s = tc::forward(li, make_pp(L, L->epoch), tokens, L->cfg.m, (const T*)X, ldx, (const T*)W, ldw, (T*)Y, ldy, (T*)Z, ldz,
+                        (int)compact_z_ld(L));
+      }
+      if (s != COMPACT_ERR_SHAPE) return s;   // SHAPE: the tensor-core kernels do not take it
     }
     return fwd_simt<T>(L, tokens, (const T*)X, ldx, (const T*)W, ldw, (T*)Y, ldy, (T*)Z, ldz, st);
   }
@@ -339,8 +355,13 @@ compact_status_t compact_linear_bwd(compact_layer_t* L, int64_t tokens, const vo
     typedef __nv_bfloat16 T;
     if (g_family.load() != 1) {
       tc::LaunchInfo li{g_family.load() == 2 ? 1 : CFG_CS, st, status_word(L), sched_words(L), &g_launches};
-      s = tc::backward(li, tokens, L->cfg.n, L->cfg.m, L->cfg.r, (int)compact_z_ld(L), (const T*)dY, lddy, (const T*)Z, ldz, (const T*)W,
-                       ldw, (T*)dX, lddx, Gc, ldg, accumulate, workspace, workspace_bytes);
+      // both products on pairs of SMs (family 2: on single SMs, the cross-check)
+      if (g_family.load() == 0)
+        s = g2::g2_backward(li, tokens, L->cfg.n, L->cfg.m, L->cfg.r, (int)compact_z_ld(L), (const T*)dY, lddy, (const T*)Z, ldz, (const T*)W,
+                            ldw, (T*)dX, lddx, Gc, ldg, accumulate, workspace, workspace_bytes);
+      else
+        s = tc::backward(li, tokens, L->cfg.n, L->cfg.m, L->cfg.r, (int)compact_z_ld(L), (const T*)dY, lddy, (const T*)Z, ldz, (const T*)W,
+                         ldw, (T*)dX, lddx, Gc, ldg, accumulate, workspace, workspace_bytes);
       if (s != COMPACT_ERR_SHAPE) return s;
     }
     return bwd_simt<T>(L, tokens, (const T*)dY, lddy, (const T*)Z, ldz, (const T*)W, ldw, (T*)dX, lddx, Gc, ldg,

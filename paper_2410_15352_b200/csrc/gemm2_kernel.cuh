@@ -1,0 +1,451 @@
+// The TMA-fed products of the CompAct layer on pairs of SMs:
+//   Y = X W              (Algorithm 1 line 3)
+//   dX = dY W^T          (Algorithm 2 line 2)
+//   Gc = Z^T dY          (Algorithm 2 line 1; split over tokens)
+// A cluster of two CTAs computes one 256 x 256 tile with tcgen05.mma.cta_group::2: each CTA holds 128 rows of A, half
+// (128 columns) of B and 128 rows of the accumulator, and the leader CTA (rank 0) issues the MMAs for both.  Against a
+// 256 x 256 tile per single CTA this moves the same bytes per flop into each SM, but the tile takes only 256 of a
+// CTA's 512 TMEM columns, so the accumulator is double-buffered and a tile's epilogue runs under the next tile's MMAs;
+// and a stage is 32 KB, so six of them (six k-steps) are in flight.
+//
+// Protocol (per stage s, per accumulator slot a; every barrier exists in both CTAs at the same offset):
+//   empty[s]   each CTA's loader waits on its own; the leader's tcgen05.commit arrives on both (multicast)
+//   full[s]    only the leader's is used: its loader declares the bytes of both CTAs' copies, and every copy (the
+//              neighbour's too) completes on it
+//   tfull[a]   each CTA's epilogue waits on its own; the leader's commit arrives on both
+//   tempty[a]  only the leader's is used: the epilogue warps of both CTAs arrive on it
+// Items are dealt statically: pair p takes items p, p + pairs, ... (both CTAs walk the same list).
+#pragma once
+#include "tc_kernels.cuh"
+
+namespace compact {
+namespace g2 {
+
+using namespace tc;
+
+constexpr int G2_NS = 6;
+constexpr int G2_HALF = 128;                         // rows of A, and columns of B, that one CTA holds
+constexpr int G2_A_BYTES = G2_HALF * BK * 2;         // 16 KB
+constexpr int G2_STAGE_BYTES = 2 * G2_A_BYTES;       // [A | B]
+constexpr int G2_RING_BYTES = G2_NS * G2_STAGE_BYTES;
+constexpr int G2_EPI_WARPS = 8;
+constexpr int G2_THREADS = 32 * (2 + G2_EPI_WARPS);
+constexpr int G2_STAGING_OFF = G2_RING_BYTES;
+constexpr int G2_BARS_OFF = G2_STAGING_OFF + G2_EPI_WARPS * STAGING_BYTES;
+constexpr int G2_NUM_BARS = 2 * G2_NS + 4;
+constexpr int G2_SMEM_BYTES = 1024 + G2_BARS_OFF + 8 * G2_NUM_BARS + 32;
+static_assert(G2_SMEM_BYTES <= 232448, "shared memory budget");
+constexpr int G2_MAXP = 2;
+
+struct G2Problem {
+  int M, N, K;                 // C[M x N] = A[M x K] B[K x N]
+  int tiles_m, tiles_n, splits, ksteps_total, ksteps_per_split;
+  int a_mode, b_mode;          // TMA_KMAJOR or TMA_MNMAJOR
+  int a_blocked, b_blocked;    // MN-major operand read through the blocked map (column count a multiple of 64)
+  int epi_mode;                // EPI_BF16 or EPI_F32 (3-D map [split][M][N])
+  int tile_begin;
+};
+
+struct alignas(64) G2Params {
+  CUtensorMap tmA[G2_MAXP];
+  CUtensorMap tmB[G2_MAXP];
+  CUtensorMap tmC[G2_MAXP];
+  G2Problem prob[G2_MAXP];
+  int num_problems;
+  int total_tiles;
+  unsigned int* status;
+};
+
+// Copy of a tile into this CTA's shared memory whose bytes complete on a barrier of the pair's leader CTA.
+__device__ __forceinline__ void tma2_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t leader_bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+      "l"(map), "r"(leader_bar), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tma2_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t leader_bar, int x, int y, int z) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(dst),
+      "l"(map), "r"(leader_bar), "r"(x), "r"(y), "r"(z)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc2(uint32_t dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish2() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// D[256 x N] (+)= A[256 x 16] B[16 x N] over the pair: both CTAs' operands sit at these offsets of their shared memory
+__device__ __forceinline__ void umma2_bf16(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                           uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %2};\n\t"
+      "mov.b64 db, {%3, %4};\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrives, once the pair's MMAs issued so far are done, on the barrier at this offset in every CTA of `mask`
+__device__ __forceinline__ void umma2_commit_mc(uint32_t bar, uint16_t mask) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+               "h"(mask)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+
+struct G2Tile {
+  int prob, m0, n0, k_begin, k_end, split;
+};
+
+__device__ __forceinline__ G2Tile g2_decode(const G2Params& prm, int tile) {
+  G2Tile t;
+  t.prob = (prm.num_problems > 1 && tile >= prm.prob[1].tile_begin) ? 1 : 0;
+  const G2Problem& p = prm.prob[t.prob];
+  int local = tile - p.tile_begin;
+  const int nb = local % p.tiles_n;
+  local /= p.tiles_n;
+  const int mb = local % p.tiles_m;
+  t.split = local / p.tiles_m;
+  t.m0 = mb * 2 * G2_HALF;
+  t.n0 = nb * 2 * G2_HALF;
+  t.k_begin = t.split * p.ksteps_per_split;
+  t.k_end = min(p.ksteps_total, t.k_begin + p.ksteps_per_split);
+  return t;
+}
+
+// Warp roles (in each CTA of the pair): 0 = loader of this CTA's A rows and B columns; 1 = owner of TMEM, and in the
+// leader CTA the MMA issuer; 2..9 = epilogue of this CTA's 128 rows of the tile.
+__global__ void __launch_bounds__(G2_THREADS, 1) compact_gemm2_kernel(const __grid_constant__ G2Params prm) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t staging = smem_base + G2_STAGING_OFF;
+  const uint32_t bars = smem_base + G2_BARS_OFF;
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (G2_NS + s); };
+  auto tfull_bar = [&](int a) { return bars + 8u * (2 * G2_NS + a); };
+  auto tempty_bar = [&](int a) { return bars + 8u * (2 * G2_NS + 2 + a); };
+  uint8_t* tail = smem_gen + G2_BARS_OFF + 8 * G2_NUM_BARS;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(tail);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 8);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint32_t crank = cluster_ctarank();
+  const bool leader = crank == 0;
+  const int pair_id = (int)(blockIdx.x >> 1);
+  const int npairs = (int)(gridDim.x >> 1);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < G2_NS; ++s) {
+      mbar_init(full_bar(s), 1);          // the leader's loader
+      mbar_init(empty_bar(s), 1);         // the leader's commit
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(tfull_bar(a), 1);                     // the leader's commit
+      mbar_init(tempty_bar(a), 2 * G2_EPI_WARPS);     // the epilogue warps of both CTAs
+    }
+    *abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async_smem();
+  }
+  if (warp == 1) {
+    tmem_alloc2(smem_u32((const void*)tmem_slot), 512);
+    tmem_relinquish2();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  cluster_sync_all();                     // both CTAs' barriers and TMEM exist before anything crosses
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t leader_bars = map_to_cta(bars, 0u);
+
+  if (warp == 0) {
+    // ------------------------------ loader ---------------------------------------
+    Ring r = {0, 0u};
+    bool ok = true;
+    for (int tile = pair_id; tile < prm.total_tiles && ok; tile += npairs) {
+      const G2Tile t = g2_decode(prm, tile);
+      const G2Problem& p = prm.prob[t.prob];
+      const CUtensorMap* mapA = &prm.tmA[t.prob];
+      const CUtensorMap* mapB = &prm.tmB[t.prob];
+      const int m0 = t.m0 + (int)crank * G2_HALF, n0 = t.n0 + (int)crank * G2_HALF;
+      for (int ks = t.k_begin; ks < t.k_end; ++ks, ring_next(r, G2_NS)) {
+        if (!(ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(r.s), r.ph ^ 1u, abort_flag, prm.status)))) break;
+        if (elect_one()) {
+          const int k0 = ks * BK;
+          const uint32_t fb = leader_bars + 8u * r.s;                      // the leader's full barrier of this stage
+          if (leader) mbar_arrive_expect_tx(full_bar(r.s), 2 * G2_STAGE_BYTES);
+          const uint32_t dstA = smem_base + (uint32_t)r.s * G2_STAGE_BYTES, dstB = dstA + G2_A_BYTES;
+          if (p.a_mode == TMA_KMAJOR) {
+            tma2_load_2d(dstA, mapA, fb, k0, m0);
+          } else if (p.a_blocked) {
+            tma2_load_3d(dstA, mapA, fb, 0, k0, m0 >> 6);
+          } else {
+            tma2_load_2d(dstA, mapA, fb, m0, k0);
+            tma2_load_2d(dstA + 8192, mapA, fb, m0 + 64, k0);
+          }
+          if (p.b_mode == TMA_KMAJOR) {
+            tma2_load_2d(dstB, mapB, fb, k0, n0);
+          } else if (p.b_blocked) {
+            tma2_load_3d(dstB, mapB, fb, 0, k0, n0 >> 6);
+          } else {
+            tma2_load_2d(dstB, mapB, fb, n0, k0);
+            tma2_load_2d(dstB + 8192, mapB, fb, n0 + 64, k0);
+          }
+        }
+        __syncwarp();
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer (leader CTA) ----------------------
+    if (leader) {
+      Ring r = {0, 0u};
+      bool ok = true;
+      int slot = 0;
+      uint32_t slot_phase = 0;
+      const uint32_t ring_lo = (smem_base >> 4) & 0x3FFFu;
+      const uint32_t lbo = (8192u >> 4) << 16, one = 1u << 16;
+      for (int tile = pair_id; tile < prm.total_tiles && ok; tile += npairs) {
+        const G2Tile t = g2_decode(prm, tile);
+        const G2Problem& p = prm.prob[t.prob];
+        const bool a_mn = p.a_mode == TMA_MNMAJOR, b_mn = p.b_mode == TMA_MNMAJOR;
+        // M = 256 over the pair, N = 256
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+                               ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+        const uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4), b_step = b_mn ? (2048u >> 4) : (32u >> 4);
+        const uint32_t a_flags = a_mn ? lbo : one, b_flags = b_mn ? lbo : one;
+        if (!(ok = __all_sync(0xffffffffu, mbar_wait(tempty_bar(slot), slot_phase ^ 1u, abort_flag, prm.status)))) break;
+        tc_fence_after();
+        const uint32_t d = tmem_base + (uint32_t)slot * 256;
+        for (int ks = t.k_begin; ks < t.k_end && ok; ++ks, ring_next(r, G2_NS)) {
+          if (!(ok = __all_sync(0xffffffffu, mbar_wait(full_bar(r.s), r.ph, abort_flag, prm.status)))) break;
+          tc_fence_after();
+          if (elect_one()) {
+            const uint32_t base = ring_lo + (((uint32_t)r.s * G2_STAGE_BYTES) >> 4);
+            const uint32_t a_lo = base | a_flags, b_lo = (base + (G2_A_BYTES >> 4)) | b_flags;
+            umma2_bf16(d, a_lo, DESC_HI, b_lo, DESC_HI, idesc, ks > t.k_begin ? 1u : 0u);
+            umma2_bf16(d, a_lo + a_step, DESC_HI, b_lo + b_step, DESC_HI, idesc, 1u);
+            umma2_bf16(d, a_lo + 2 * a_step, DESC_HI, b_lo + 2 * b_step, DESC_HI, idesc, 1u);
+            umma2_bf16(d, a_lo + 3 * a_step, DESC_HI, b_lo + 3 * b_step, DESC_HI, idesc, 1u);
+            umma2_commit_mc(empty_bar(r.s), (uint16_t)3);          // the stage goes back to both loaders
+          }
+          __syncwarp();
+        }
+        if (!ok) break;
+        if (elect_one()) umma2_commit_mc(tfull_bar(slot), (uint16_t)3);   // the accumulator is complete in both CTAs
+        __syncwarp();
+        if (++slot == 2) { slot = 0; slot_phase ^= 1u; }
+      }
+    }
+  } else {
+    // ------------------------------ epilogue ------------------------------------
+    // This CTA's 128 rows of the tile: TMEM -> registers -> 128B-swizzled staging tile -> TMA store.
+    const int q = warp & 3;                 // TMEM lane quarter this warp may read
+    const int eset = (warp - 2) >> 2;       // the two sets take alternate chunks
+    const uint32_t stg = staging + (warp - 2) * STAGING_BYTES;
+    uint8_t* stg_gen = smem_gen + G2_STAGING_OFF + (warp - 2) * STAGING_BYTES;
+    const uint32_t leader_tempty = leader_bars + 8u * (2 * G2_NS + 2);
+    const int sw = lane & 7;
+    int slot = 0;
+    uint32_t slot_phase = 0;
+    bool ok = true;
+    for (int tile = pair_id; tile < prm.total_tiles && ok; tile += npairs) {
+      const G2Tile t = g2_decode(prm, tile);
+      const G2Problem& p = prm.prob[t.prob];
+      const CUtensorMap* mapC = &prm.tmC[t.prob];
+      if (!(ok = mbar_wait(tfull_bar(slot), slot_phase, abort_flag, prm.status))) break;
+      tc_fence_after();
+      const int row0 = t.m0 + (int)crank * G2_HALF + q * 32;
+      const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)slot * 256;
+      const int cw = p.epi_mode == EPI_F32 ? 32 : 64;
+      for (int ci = eset; ci < 256 / cw && row0 < p.M; ci += 2) {
+        const int col = t.n0 + ci * cw;
+        if (col >= p.N) break;
+        if (p.epi_mode == EPI_BF16) {
+          uint32_t o[32];
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            uint32_t v[32];
+            tmem_ld32(tcol + ci * cw + 32 * h, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 16; ++j) o[16 * h + j] = pack_bf16x2(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+          }
+          if (lane == 0) tma_store_wait_read();          // the previous store has read the staging tile
+          __syncwarp();
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            *reinterpret_cast<uint4*>(stg_gen + lane * 128 + ((j ^ sw) << 4)) = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_2d(mapC, stg, col, row0);
+            tma_store_commit();
+          }
+        } else {
+          uint32_t v[32];
+          tmem_ld32(tcol + ci * cw, v);
+          tmem_ld_wait();
+          if (lane == 0) tma_store_wait_read();
+          __syncwarp();
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            *reinterpret_cast<uint4*>(stg_gen + lane * 128 + ((j ^ sw) << 4)) = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_3d(mapC, stg, col, row0, t.split);
+            tma_store_commit();
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        if (leader) mbar_arrive(tempty_bar(slot));
+        else mbar_arrive_cluster(leader_tempty + 8u * slot);
+      }
+      if (++slot == 2) { slot = 0; slot_phase ^= 1u; }
+    }
+    if (lane == 0) tma_store_wait_all();
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                     // neither CTA frees TMEM, or leaves, while the pair may still use or signal it
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc2(tmem_base, 512);
+  }
+}
+
+// --------------------------------------------------------------------------------------
+// Host side
+// --------------------------------------------------------------------------------------
+inline void g2_finish(G2Problem& p, int splits_wanted) {
+  p.tiles_m = (p.M + 2 * G2_HALF - 1) / (2 * G2_HALF);
+  p.tiles_n = (p.N + 2 * G2_HALF - 1) / (2 * G2_HALF);
+  p.ksteps_total = (p.K + BK - 1) / BK;
+  int s = splits_wanted < 1 ? 1 : splits_wanted;
+  if (s > p.ksteps_total) s = p.ksteps_total;
+  p.ksteps_per_split = (p.ksteps_total + s - 1) / s;
+  p.splits = (p.ksteps_total + p.ksteps_per_split - 1) / p.ksteps_per_split;
+}
+
+inline compact_status_t g2_launch(const LaunchInfo& li, G2Params& prm) {
+  static std::atomic<bool> attr_set[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return COMPACT_ERR_CUDA; }
+  if (!attr_set[dev].load(std::memory_order_acquire)) {
+    if (cudaFuncSetAttribute(compact_gemm2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, G2_SMEM_BYTES) != cudaSuccess) {
+      cudaGetLastError();
+      return COMPACT_ERR_CUDA;
+    }
+    attr_set[dev].store(true, std::memory_order_release);
+  }
+  int t = 0;
+  for (int i = 0; i < prm.num_problems; ++i) {
+    prm.prob[i].tile_begin = t;
+    t += prm.prob[i].tiles_m * prm.prob[i].tiles_n * prm.prob[i].splits;
+  }
+  prm.total_tiles = t;
+  prm.status = li.status;
+  const int pairs = t < NUM_SMS / 2 ? t : NUM_SMS / 2;
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
+  cfg.blockDim = dim3((unsigned)G2_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = G2_SMEM_BYTES;
+  cfg.stream = li.stream;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = 2;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, compact_gemm2_kernel, prm);
+  (*li.launches)++;
+  if (e != cudaSuccess) { cudaGetLastError(); return COMPACT_ERR_CUDA; }
+  return cudaGetLastError() == cudaSuccess ? COMPACT_OK : COMPACT_ERR_CUDA;
+}
+
+// Y = X W (Algorithm 1 line 3): A = X (K-major), B = W (MN-major).
+inline compact_status_t g2_forward_y(const LaunchInfo& li, int64_t tokens, int n, int m, const __nv_bfloat16* X, int64_t ldx,
+                                     const __nv_bfloat16* W, int64_t ldw, __nv_bfloat16* Y, int64_t ldy) {
+  if (!tc_shape_ok(tokens, n, m)) return COMPACT_ERR_SHAPE;
+  if (!li.status) return COMPACT_ERR_CUDA;
+  G2Params prm;
+  memset(&prm, 0, sizeof(prm));
+  prm.num_problems = 1;
+  G2Problem& py = prm.prob[0];
+  py.M = (int)tokens; py.N = m; py.K = n;
+  py.a_mode = TMA_KMAJOR; py.b_mode = TMA_MNMAJOR; py.epi_mode = EPI_BF16;
+  py.b_blocked = m % 64 == 0;
+  g2_finish(py, 1);
+  if (!make_map(&prm.tmA[0], X, n, tokens, ldx, BK, G2_HALF)) return COMPACT_ERR_CUDA;
+  if (py.b_blocked ? !make_map_blocked(&prm.tmB[0], W, m, n, ldw, BK, G2_HALF / 64) : !make_map(&prm.tmB[0], W, m, n, ldw, 64, BK))
+    return COMPACT_ERR_CUDA;
+  if (!make_map(&prm.tmC[0], Y, m, tokens, ldy, 64, 32)) return COMPACT_ERR_CUDA;
+  return g2_launch(li, prm);
+}
+
+// Algorithm 2: problem 0 = Gc = Z^T dY (both operands MN-major, split over tokens), problem 1 = dX = dY W^T.
+inline compact_status_t g2_backward(const LaunchInfo& li, int64_t tokens, int n, int m, int r, int zcols,
+                                    const __nv_bfloat16* dY, int64_t lddy, const __nv_bfloat16* Z, int64_t ldz,
+                                    const __nv_bfloat16* W, int64_t ldw, __nv_bfloat16* dX, int64_t lddx, float* Gc,
+                                    int64_t ldg, int accumulate, void* workspace, size_t workspace_bytes) {
+  if (!tc_shape_ok(tokens, n, m)) return COMPACT_ERR_SHAPE;
+  if (!li.status) return COMPACT_ERR_CUDA;
+  G2Params prm;
+  memset(&prm, 0, sizeof(prm));
+  prm.num_problems = dX ? 2 : 1;
+  const int splits = plan_gc_splits(tokens, r, m);
+  const bool staged = splits > 1 || accumulate;
+  if (staged && workspace_bytes < (size_t)splits * r * m * sizeof(float)) return COMPACT_ERR_WORKSPACE;
+  G2Problem& pg = prm.prob[0];
+  pg.M = r; pg.N = m; pg.K = (int)tokens;
+  pg.a_mode = TMA_MNMAJOR; pg.b_mode = TMA_MNMAJOR; pg.epi_mode = EPI_F32;
+  pg.a_blocked = zcols % 64 == 0;
+  pg.b_blocked = m % 64 == 0;
+  g2_finish(pg, splits);
+  if (staged) {
+    if (!make_map_f32_3d(&prm.tmC[0], workspace, m, r, pg.splits, m, (int64_t)r * m)) return COMPACT_ERR_CUDA;
+  } else {
+    if (!make_map_f32_3d(&prm.tmC[0], Gc, m, r, 1, ldg, (int64_t)r * ldg)) return COMPACT_ERR_CUDA;
+  }
+  if (pg.a_blocked ? !make_map_blocked(&prm.tmA[0], Z, zcols, tokens, ldz, BK, G2_HALF / 64) : !make_map(&prm.tmA[0], Z, zcols, tokens, ldz, 64, BK))
+    return COMPACT_ERR_CUDA;
+  if (pg.b_blocked ? !make_map_blocked(&prm.tmB[0], dY, m, tokens, lddy, BK, G2_HALF / 64) : !make_map(&prm.tmB[0], dY, m, tokens, lddy, 64, BK))
+    return COMPACT_ERR_CUDA;
+  if (dX) {
+    G2Problem& px = prm.prob[1];
+    px.M = (int)tokens; px.N = n; px.K = m;
+    px.a_mode = TMA_KMAJOR; px.b_mode = TMA_KMAJOR; px.epi_mode = EPI_BF16;
+    g2_finish(px, 1);
+    if (!make_map(&prm.tmA[1], dY, m, tokens, lddy, BK, G2_HALF)) return COMPACT_ERR_CUDA;
+    if (!make_map(&prm.tmB[1], W, m, n, ldw, BK, G2_HALF)) return COMPACT_ERR_CUDA;
+    if (!make_map(&prm.tmC[1], dX, n, tokens, lddx, 64, 32)) return COMPACT_ERR_CUDA;
+  }
+  compact_status_t s = g2_launch(li, prm);
+  if (s != COMPACT_OK) return s;
+  if (staged) {
+    const long long cnt = (long long)r * (m / 4);
+    reduce_partials_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, li.stream>>>(
+        (const float*)workspace, (long long)r * m, pg.splits, Gc, ldg, r, m, accumulate);
+    (*li.launches)++;
+    if (cudaGetLastError() != cudaSuccess) return COMPACT_ERR_CUDA;
+  }
+  return COMPACT_OK;
+}
+
+}  // namespace g2
+}  // namespace compact
