@@ -256,12 +256,12 @@ class LayerBuffers:
         self.lay.workspace(tokens)
 
 
-# DRAM traffic per launch from the committed ncu captures (profiles/): bytes per algorithmic flop of the forward and
-# backward launches of the C5 q_proj layer (compact_gemm_kernel_c5_qproj_full.md: 441.1 + 132.9 and 425.9 + 160.5 MB
-# for 2 x 618.5 GFLOP), and bytes per algorithmic byte of one update launch whose W does not sit in L2 beforehand
-# (compact_update_kernel_c5_gate_proj.md: 169.6 + 97.4 MB for 293.1 MB).  Scaled to the benchmarked launches by
-# their algorithmic work.
-NCU_GEMM_DRAM_BYTES_PER_FLOP = (441.1e6 + 132.9e6 + 425.9e6 + 160.5e6) / 1236.95e9
+# DRAM traffic from the committed ncu captures (profiles/): bytes per algorithmic flop of the forward (Z launch + Y
+# launch) and backward launches of the C5 q_proj layer (compact_gemm_kernel_c5_qproj_full.md: 134.3 + 5.0, 203.0 + 117.8
+# and 401.6 + 159.6 MB for 2 x 618.5 GFLOP), and bytes per algorithmic byte of one update launch whose W does not sit in
+# L2 beforehand (compact_update_kernel_c5_gate_proj.md: 169.6 + 97.4 MB for 293.1 MB).  Scaled to the benchmarked
+# launches by their algorithmic work.
+NCU_GEMM_DRAM_BYTES_PER_FLOP = (134.3e6 + 5.0e6 + 203.0e6 + 117.8e6 + 401.6e6 + 159.6e6) / 1236.95e9
 NCU_UPDATE_DRAM_BYTES_PER_ALG_BYTE = (169.6e6 + 97.4e6) / 293.1e6
 
 
@@ -429,13 +429,13 @@ def run_ours(args):
     traffic_gemm = NCU_GEMM_DRAM_BYTES_PER_FLOP * gemm_flops / gemm_launches
     traffic_upd = (NCU_UPDATE_DRAM_BYTES_PER_ALG_BYTE * upd_bytes / len(wl.layers)
                    if NCU_UPDATE_DRAM_BYTES_PER_ALG_BYTE is not None else None)
-    roofline = {"kernel": "compact_gemm_kernel (forward and backward launches)", "bound": "tensor",
+    roofline = {"kernel": "compact_gemm2_kernel + compact_gemm_kernel (the forward and backward calls: Y, dX, Gc on pairs of SMs; Z with its generated operand)", "bound": "tensor",
                 "achieved": gemm_tflops, "peak": tens_peak, "unit": "TFLOP/s", "frac": gemm_tflops / tens_peak,
                 "peak_kind": f"{peak_kind} bf16 sustained (the kernel is timed inside a long step)",
                 "frac_of_measured_burst": gemm_tflops / tens_burst, "frac_of_nominal_2250": gemm_tflops / NOMINAL_BF16_TFLOPS,
-                "avg_launch_ms": gemm_ms / gemm_launches, "launches_per_step": gemm_launches,
+                "avg_launch_ms": gemm_ms / gemm_launches, "calls_per_step": gemm_launches,
                 "algorithmic_flops_per_launch": gemm_flops / gemm_launches, "traffic": traffic_gemm,
-                "traffic_note": "DRAM bytes per launch, scaled by flops from the ncu capture of the C5 q_proj forward and backward launches"}
+                "traffic_note": "DRAM bytes per forward or backward call, scaled by flops from the ncu capture of the C5 q_proj calls"}
     # each layer's update against the roofline that bounds it: HBM below the ridge n r / (2 n + 10 r) flop/byte, tensor above
     ridge = tens_peak * 1e12 / (hbm_peak * 1e9)
     upd_layers = {}
