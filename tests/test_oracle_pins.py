@@ -44,38 +44,53 @@ def test_philox_vectorised_equals_scalar_calls():
 
 
 def test_projection_words_counter_layout():
-    # word (i, 4q+w) is word w of philox(ctr=(q, i, layer, epoch), key=(seed_lo, seed_hi))
+    # word (i, 4q+w) is word w of philox(ctr=(q, i, layer, epoch), key=(seed_lo, seed_hi)); call q covers columns 8q .. 8q+7
     seed, layer, epoch = (0x1234 << 32) | 0x89ABCDEF, 5, 3
-    words = co.projection_words(seed, layer, epoch, 9, 10)
+    words = co.projection_words(seed, layer, epoch, 9, 18)
     assert words.shape == (9, 12)
     for i, q in [(0, 0), (8, 2), (4, 1)]:
         ref = co.philox4x32_10(np.array([q, i, layer, epoch]), np.array([0x89ABCDEF, 0x1234]))
         assert (words[i, 4 * q:4 * q + 4] == ref).all()
     # the all-zero call is the first published vector
-    w0 = co.projection_words(0, 0, 0, 1, 4)
+    w0 = co.projection_words(0, 0, 0, 1, 8)
     assert [int(x) for x in w0[0]] == _kat_rows()[0][2]
+    # entry (i, j) comes from word (j >> 1) & 3 of call j >> 3: the cos of the word's pair for even j, the sin for odd j
+    r = 18
+    P = co.projection(seed, layer, epoch, 9, r) * math.sqrt(r)
+    for i, j in [(0, 0), (3, 5), (8, 17), (4, 10)]:
+        w = int(words[i, 4 * (j >> 3) + ((j >> 1) & 3)])
+        rad = math.sqrt(-2 * math.log(((w & 0xFFFF) + 0.5) / 65536))
+        ang = 2 * math.pi * (w >> 16) / 65536
+        assert P[i, j] == pytest.approx(rad * (math.sin(ang) if j & 1 else math.cos(ang)), rel=1e-12, abs=1e-15)
 
 
 # --- Box-Muller closed forms and distribution -----------------------------------
 def test_box_muller_closed_forms():
-    # u2 = 0 -> (rad, 0); u2 = 1/4 -> (0, rad)
-    w = np.array([[0x80000000, 0, 0x80000000, 1 << 30]], dtype=np.uint32)
+    # a word's high half is the angle, its low half the radius
+    lo = 0x8000
+    rad = math.sqrt(-2 * math.log((lo + 0.5) / 65536))
+    # u2 = 0 -> (rad, 0); u2 = 1/4 -> (0, rad); u2 = 1/2 -> (-rad, 0); u2 = 3/4 -> (0, -rad)
+    w = np.array([[lo, (0x4000 << 16) | lo, (0x8000 << 16) | lo, (0xC000 << 16) | lo]], dtype=np.uint32)
     g = co.box_muller_from_words(w)[0]
-    u1 = ((0x80000000 >> 9) + 0.5) * 2.0 ** -23
-    rad = math.sqrt(-2 * math.log(u1))
+    assert g.shape == (8,)
     assert g[0] == pytest.approx(rad, rel=1e-15) and g[1] == 0.0
     assert abs(g[2]) < 1e-15 and g[3] == pytest.approx(rad, rel=1e-15)
-    # extreme radii: u1 = 1 - 2^-24 and u1 = 2^-24
-    w = np.array([[0xFFFFFFFF, 0, 0x00000000, 0]], dtype=np.uint32)
+    assert g[4] == pytest.approx(-rad, rel=1e-15) and abs(g[5]) < 1e-15
+    assert abs(g[6]) < 1e-15 and g[7] == pytest.approx(-rad, rel=1e-15)
+    # extreme radii: u1 = 1 - 2^-17 and u1 = 2^-17
+    w = np.array([[0x0000FFFF, 0x00000000]], dtype=np.uint32)
     g = co.box_muller_from_words(w)[0]
-    assert g[0] == pytest.approx(math.sqrt(-2 * math.log1p(-2.0 ** -24)), rel=1e-9)
-    assert g[0] == pytest.approx(3.4527e-4, rel=1e-4)
-    assert g[2] == pytest.approx(math.sqrt(48 * math.log(2)), rel=1e-15)
-    # u2 = 1/2 -> (-rad, ~0): sign of cos
-    w = np.array([[0, 1 << 31, 0, 3 << 30]], dtype=np.uint32)
-    g = co.box_muller_from_words(w)[0]
-    assert g[0] == pytest.approx(-math.sqrt(48 * math.log(2)), rel=1e-15)
-    assert g[3] == pytest.approx(-math.sqrt(48 * math.log(2)), rel=1e-15)  # sin(3pi/2) = -1
+    assert g[0] == pytest.approx(math.sqrt(-2 * math.log1p(-2.0 ** -17)), rel=1e-9)
+    assert g[0] == pytest.approx(3.9063e-3, rel=1e-4)
+    assert g[2] == pytest.approx(math.sqrt(34 * math.log(2)), rel=1e-15)      # the largest radius: 4.8546
+    assert g[2] == pytest.approx(4.8546, rel=1e-4)
+    # the two halves do not leak into one another
+    a = co.box_muller_from_words(np.array([[0x12345678]], dtype=np.uint32))[0]
+    b = co.box_muller_from_words(np.array([[0x12340000 | 0x5678]], dtype=np.uint32))[0]
+    assert np.array_equal(a, b)
+    rad = math.sqrt(-2 * math.log((0x5678 + 0.5) / 65536))
+    assert math.hypot(a[0], a[1]) == pytest.approx(rad, rel=1e-14)
+    assert math.atan2(a[1], a[0]) == pytest.approx(2 * math.pi * 0x1234 / 65536, rel=1e-13)
 
 
 def test_projection_distribution():
