@@ -239,8 +239,8 @@ compact_status_t compact_layer_status(compact_layer_t* layer);
 compact_status_t compact_debug_wait_that_runs_out(compact_layer_t* layer, void* stream);
 
 /* Test hooks that make the in-kernel generator observable.
- * compact_debug_philox_u32: out_dev[n x 4*ceil(r/4)] receives the raw Philox
- * words behind P (Algorithm 1 lines 1-2), from the generic ten-round function.
+ * compact_debug_philox_u32: out_dev[n x 4*ceil(r/8)] receives the raw Philox
+ * words behind P (one call of four words per eight columns) (Algorithm 1 lines 1-2), from the generic ten-round function.
  * compact_debug_philox_layer_u32: the same words from the form the GEMM kernels'
  * generators call (first round partly precomputed on the host per layer).
  * compact_debug_projection: P_dev[n x r] (layer dtype, pitch r) receives P at

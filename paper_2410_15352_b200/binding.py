@@ -132,7 +132,7 @@ def kernel_launch_count() -> int:
 
 def debug_philox_u32(seed: int, layer_id: int, epoch: int, n: int, r: int, stream=None, layer_form: bool = False) -> torch.Tensor:
     """Raw Philox words behind P; layer_form=True takes them from the function the GEMM kernels' generators call."""
-    out = torch.empty((n, 4 * ((r + 3) // 4)), dtype=torch.int32, device="cuda")
+    out = torch.empty((n, 4 * ((r + 7) // 8)), dtype=torch.int32, device="cuda")
     fn = lib().compact_debug_philox_layer_u32 if layer_form else lib().compact_debug_philox_u32
     _check(fn(seed, layer_id, epoch, n, r, _ptr(out), _stream(stream)), "debug_philox_u32")
     return out

@@ -682,7 +682,7 @@ compact_status_t compact_debug_philox_u32(uint64_t seed, uint32_t layer_id, uint
                                           uint32_t* out_dev, void* stream) {
   if (n < 1 || r < 1 || !out_dev) return COMPACT_ERR_INVALID_ARG;
   if (!aligned16(out_dev)) return COMPACT_ERR_ALIGNMENT;
-  const int groups = (r + 3) / 4;
+  const int groups = (r + 7) / 8;
   const int64_t cnt = (int64_t)n * groups;
   debug_philox_words_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
       make_philox_key(seed), layer_id, epoch, n, groups, out_dev);
@@ -694,7 +694,7 @@ compact_status_t compact_debug_philox_layer_u32(uint64_t seed, uint32_t layer_id
                                                 uint32_t* out_dev, void* stream) {
   if (n < 1 || r < 1 || !out_dev) return COMPACT_ERR_INVALID_ARG;
   if (!aligned16(out_dev)) return COMPACT_ERR_ALIGNMENT;
-  const int groups = (r + 3) / 4;
+  const int groups = (r + 7) / 8;
   const int64_t cnt = (int64_t)n * groups;
   const uint64_t pl = (uint64_t)0xCD9E8D57u * (uint64_t)layer_id;
   debug_philox_layer_words_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
@@ -715,7 +715,7 @@ compact_status_t compact_debug_sparse_terms(const compact_layer_t* L, uint32_t e
 compact_status_t compact_debug_projection(const compact_layer_t* L, uint32_t epoch, void* P_dev, void* stream) {
   if (!L || !P_dev) return COMPACT_ERR_INVALID_ARG;
   const ProjectionParams pp = make_pp(L, epoch);
-  const int64_t cnt = (int64_t)pp.n * ((pp.r + 3) / 4);
+  const int64_t cnt = (int64_t)pp.n * pp.r;
   const unsigned blocks = (unsigned)((cnt + 255) / 256);
   if (L->cfg.dtype == COMPACT_BF16)
     debug_projection_kernel<__nv_bfloat16><<<blocks, 256, 0, (cudaStream_t)stream>>>(pp, (__nv_bfloat16*)P_dev);

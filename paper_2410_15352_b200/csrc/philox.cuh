@@ -1,6 +1,7 @@
 // Device-side generator of the projection P (Algorithm 1 lines 1-2, Algorithm 3
 // lines 6-7, Section 3.3): Philox4x32-10 keyed by the 64-bit layer seed with
-// counter (column group, row, layer_id, epoch), followed by Box-Muller.
+// counter (column group j >> 3, row, layer_id, epoch), followed by Box-Muller with
+// 16 bits per uniform: one call yields the eight entries P[i, 8q .. 8q+7].
 // Entry (i, j) of P is a pure function of (seed, layer_id, epoch, i, j).
 #pragma once
 #include <cuda_bf16.h>
@@ -59,26 +60,24 @@ __device__ __forceinline__ uint4 philox4x32_10_layer(uint32_t q, uint32_t i, uin
   return philox_rounds<1>(c0, c1, c2, c3, key);
 }
 
-// Four consecutive entries P[i, 4q .. 4q+3] before the 1/sqrt(r) scale.
-// Words (0,1) make the (cos, sin) pair of columns 4q, 4q+1; words (2,3) that of 4q+2, 4q+3.
-__device__ __forceinline__ float4 gaussian4(uint4 x) {
-  const float u1a = ((float)(x.x >> 9) + 0.5f) * 1.1920928955078125e-07f;   // 2^-23, in (0,1)
-  const float u2a = (float)(x.y >> 8) * 5.9604644775390625e-08f;            // 2^-24, in [0,1)
-  const float u1b = ((float)(x.z >> 9) + 0.5f) * 1.1920928955078125e-07f;
-  const float u2b = (float)(x.w >> 8) * 5.9604644775390625e-08f;
-  const float ra = sqrtf(-2.0f * logf(u1a));
-  const float rb = sqrtf(-2.0f * logf(u1b));
-  float sa, ca, sb, cb;
-  sincospif(2.0f * u2a, &sa, &ca);
-  sincospif(2.0f * u2b, &sb, &cb);
-  return make_float4(ra * ca, ra * sa, rb * cb, rb * sb);
+// One word makes a pair of standard normals: its low half is the radius' uniform u1 = ((x & 0xffff) + 0.5) 2^-16 in
+// (0,1), its high half the angle's u2 = (x >> 16) 2^-16 in [0,1); the pair is (rad cos(2 pi u2), rad sin(2 pi u2)).
+// Word w of the call for column group q makes columns 8q + 2w and 8q + 2w + 1.
+__device__ __forceinline__ void box_muller(uint32_t x, float& c, float& s) {
+  const float u1 = ((float)(x & 0xFFFFu) + 0.5f) * 1.52587890625e-05f;     // 2^-16
+  const float u2 = (float)(x >> 16) * 1.52587890625e-05f;
+  const float rad = sqrtf(-2.0f * logf(u1));
+  float sn, cs;
+  sincospif(2.0f * u2, &sn, &cs);
+  c = rad * cs;
+  s = rad * sn;
 }
 
-// Same four values already scaled by 1/sqrt(r), built from the hardware
+// The same pair already scaled by 1/sqrt(r), built from the hardware
 // approximations (lg2/sqrt/sin/cos) and bit tricks instead of int->float
 // conversions.  Used where P is rounded to bf16 anyway.
-//   u1 = ((x>>9)+0.5) 2^-23 = float(1.m) - (1 - 2^-24)            (exact)
-//   2 pi u2 = pi*[x>>31] + pi * ((x>>8) & 0x7fffff) 2^-23: the top bit of u2
+//   u1 = float(1.m) - 1 with mantissa m = (x & 0xffff) << 7 | 0x40      (exact)
+//   2 pi u2 = pi*[x>>31] + pi * ((x>>16) & 0x7fff) 2^-15: the top bit of u2
 //   adds pi to the angle, which flips the sign of both cos and sin.
 // neg2ln2_over_r = -2 ln(2) / r, so sqrt(lg2(u1) * neg2ln2_over_r) = sqrt(-2 ln u1) / sqrt(r).
 __device__ __forceinline__ float sqrt_approx(float x) {
@@ -103,19 +102,13 @@ __device__ __forceinline__ float cos_approx(float x) {
   asm("cos.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ void box_muller_fast(uint32_t xa, uint32_t xb, float neg2ln2_over_r, float& c, float& s) {
-  const float u1 = __uint_as_float((xa >> 9) | 0x3F800000u) - 0.99999994f;
-  const float rad = sqrt_approx(fmaxf(lg2_approx(u1) * neg2ln2_over_r, 0.0f));
-  const float th = (__uint_as_float(((xb >> 8) & 0x007FFFFFu) | 0x3F800000u) - 1.0f) * 3.14159265358979f;
-  const float rs = __uint_as_float(__float_as_uint(rad) ^ (xb & 0x80000000u));
+__device__ __forceinline__ void box_muller_fast(uint32_t x, float neg2ln2_over_r, float& c, float& s) {
+  const float u1 = __uint_as_float(((x << 7) & 0x007FFF80u) | 0x3F800040u) - 1.0f;     // at most 1 - 2^-17: lg2 < 0
+  const float rad = sqrt_approx(lg2_approx(u1) * neg2ln2_over_r);
+  const float th = (__uint_as_float(((x >> 8) & 0x007FFF00u) | 0x3F800000u) - 1.0f) * 3.14159265358979f;
+  const float rs = __uint_as_float(__float_as_uint(rad) ^ (x & 0x80000000u));
   c = rs * cos_approx(th);
   s = rs * sin_approx(th);
-}
-__device__ __forceinline__ float4 gaussian4_fast_scaled(uint4 x, float neg2ln2_over_r) {
-  float4 g;
-  box_muller_fast(x.x, x.y, neg2ln2_over_r, g.x, g.y);
-  box_muller_fast(x.z, x.w, neg2ln2_over_r, g.z, g.w);
-  return g;
 }
 
 struct ProjectionParams {
@@ -156,33 +149,24 @@ __device__ __forceinline__ float sparse_count(const ProjectionParams& pp, int i,
   return k;
 }
 
-// P[i, 4q .. 4q+3] in fp32; columns >= r are zero, rows >= n are zero.
+// Entry (i, j) of P in fp32; zero outside n x r.
 // kFast selects the approximate Box-Muller (bf16 layers); fp32 layers use the accurate one.
 template <bool kFast>
-__device__ __forceinline__ float4 projection4(const ProjectionParams& pp, int i, int q) {
-  if (i >= pp.n || 4 * q >= pp.r) return make_float4(0.f, 0.f, 0.f, 0.f);
-  const uint4 x = philox4x32_10_layer((uint32_t)q, (uint32_t)i, pp.epoch, pp.layer_hi, pp.layer_lo, pp.key);
-  float4 g;
-  if (kFast) {
-    g = gaussian4_fast_scaled(x, pp.neg2ln2_over_r);
-  } else {
-    g = gaussian4(x);
-    g.x *= pp.inv_sqrt_r; g.y *= pp.inv_sqrt_r; g.z *= pp.inv_sqrt_r; g.w *= pp.inv_sqrt_r;
-  }
-  if (4 * q + 4 > pp.r) {
-    if (4 * q + 1 >= pp.r) g.y = 0.f;
-    if (4 * q + 2 >= pp.r) g.z = 0.f;
-    if (4 * q + 3 >= pp.r) g.w = 0.f;
-  }
-  return g;
-}
-
-template <bool kFast>
 __device__ __forceinline__ float projection1(const ProjectionParams& pp, int i, int j) {
-  if (pp.sparse_s > 0) return (i < pp.n && j < pp.r) ? sparse_count(pp, i, j) * pp.inv_sqrt_s : 0.f;
-  const float4 g = projection4<kFast>(pp, i, j >> 2);
-  const int l = j & 3;
-  return l == 0 ? g.x : (l == 1 ? g.y : (l == 2 ? g.z : g.w));
+  if (i >= pp.n || j >= pp.r) return 0.f;
+  if (pp.sparse_s > 0) return sparse_count(pp, i, j) * pp.inv_sqrt_s;
+  const uint4 x = philox4x32_10_layer((uint32_t)(j >> 3), (uint32_t)i, pp.epoch, pp.layer_hi, pp.layer_lo, pp.key);
+  const int w = (j >> 1) & 3;
+  const uint32_t word = w == 0 ? x.x : (w == 1 ? x.y : (w == 2 ? x.z : x.w));
+  float c, s;
+  if (kFast) {
+    box_muller_fast(word, pp.neg2ln2_over_r, c, s);
+  } else {
+    box_muller(word, c, s);
+    c *= pp.inv_sqrt_r;
+    s *= pp.inv_sqrt_r;
+  }
+  return (j & 1) ? s : c;
 }
 
 }  // namespace compact

@@ -175,19 +175,10 @@ __global__ void debug_sparse_terms_kernel(ProjectionParams pp, uint32_t* out) {
 
 template <typename T>
 __global__ void debug_projection_kernel(ProjectionParams pp, T* P) {
-  const int groups = (pp.r + 3) / 4;
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (idx >= (int64_t)pp.n * groups) return;
-  const int i = (int)(idx / groups), q = (int)(idx % groups);
-  float v[4];
-  if (pp.sparse_s > 0) {
-    for (int l = 0; l < 4; ++l) v[l] = projection1<sizeof(T) == 2>(pp, i, 4 * q + l);
-  } else {
-    const float4 g = projection4<sizeof(T) == 2>(pp, i, q);
-    v[0] = g.x; v[1] = g.y; v[2] = g.z; v[3] = g.w;
-  }
-  for (int l = 0; l < 4; ++l)
-    if (4 * q + l < pp.r) P[(int64_t)i * pp.r + 4 * q + l] = simt::from_f32<T>(v[l]);
+  if (idx >= (int64_t)pp.n * pp.r) return;
+  const int i = (int)(idx / pp.r), j = (int)(idx % pp.r);
+  P[idx] = simt::from_f32<T>(projection1<sizeof(T) == 2>(pp, i, j));
 }
 
 }  // namespace compact

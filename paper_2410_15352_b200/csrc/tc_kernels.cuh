@@ -322,21 +322,22 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 
-// Eight consecutive entries P[i, j0 .. j0+7] (j0 a multiple of 8) of a problem's projection as packed bf16;
-// entries outside n x r are zero.
+// Eight consecutive entries P[i, j0 .. j0+7] (j0 a multiple of 8) of a problem's projection as packed bf16: the
+// four words of one Philox call, a Box-Muller pair each; entries outside n x r are zero.
 __device__ __forceinline__ uint4 projection8_bf16(const PhiloxKey& key, uint32_t layer_hi, uint32_t layer_lo, uint32_t epoch,
                                                   int n, int r, float neg2ln2_over_r, int i, int j0) {
-  const uint32_t q = (uint32_t)(j0 >> 2);
-  const uint4 xa = philox4x32_10_layer(q, (uint32_t)i, epoch, layer_hi, layer_lo, key);
-  const uint4 xb = philox4x32_10_layer(q + 1, (uint32_t)i, epoch, layer_hi, layer_lo, key);
-  float4 a = gaussian4_fast_scaled(xa, neg2ln2_over_r);
-  float4 b = gaussian4_fast_scaled(xb, neg2ln2_over_r);
+  const uint4 x = philox4x32_10_layer((uint32_t)(j0 >> 3), (uint32_t)i, epoch, layer_hi, layer_lo, key);
+  float g[8];
+  box_muller_fast(x.x, neg2ln2_over_r, g[0], g[1]);
+  box_muller_fast(x.y, neg2ln2_over_r, g[2], g[3]);
+  box_muller_fast(x.z, neg2ln2_over_r, g[4], g[5]);
+  box_muller_fast(x.w, neg2ln2_over_r, g[6], g[7]);
   const int left = i < n ? r - j0 : 0;      // valid entries among the eight
   if (left < 8) {
-    a.x = left > 0 ? a.x : 0.f; a.y = left > 1 ? a.y : 0.f; a.z = left > 2 ? a.z : 0.f; a.w = left > 3 ? a.w : 0.f;
-    b.x = left > 4 ? b.x : 0.f; b.y = left > 5 ? b.y : 0.f; b.z = left > 6 ? b.z : 0.f; b.w = left > 7 ? b.w : 0.f;
+#pragma unroll
+    for (int l = 0; l < 8; ++l) g[l] = left > l ? g[l] : 0.f;
   }
-  return make_uint4(pack_bf16x2(a.x, a.y), pack_bf16x2(a.z, a.w), pack_bf16x2(b.x, b.y), pack_bf16x2(b.z, b.w));
+  return make_uint4(pack_bf16x2(g[0], g[1]), pack_bf16x2(g[2], g[3]), pack_bf16x2(g[4], g[5]), pack_bf16x2(g[6], g[7]));
 }
 
 // Test hook: one CTA waits, with a small limit, on a barrier that nothing will ever arrive at.  The wait gives

@@ -63,15 +63,18 @@ def test_projection_fp32_entries():
 def test_projection_bf16_entries():
     # bf16 layers use the hardware lg2/sqrt/sin/cos approximations in fp32 and round once;
     # the oracle computes in fp64 and rounds once.  Bound: one bf16 ulp of the value plus
-    # the absolute error of the approximations, 2e-5/sqrt(r) (sin/cos: 2^-20.9 * rad <= 3e-6/sqrt(r);
-    # lg2 near u1 = 1: up to 1.7e-5/sqrt(r) on radii below 0.01/sqrt(r)).
+    # the absolute error of the approximations, 5e-5/sqrt(r) (sin/cos: 2^-20.9 * rad <= 3e-6/sqrt(r);
+    # lg2.approx has absolute error 2^-22, and with 16-bit uniforms lg2(u1) comes as close to zero as
+    # -2.2e-5 at u1 = 1 - 2^-17 + 2^-17/2: the smallest radii, 3.9e-3/sqrt(r), are then off by up to
+    # 1.1 %, 4.3e-5/sqrt(r); that concerns the few entries in 10^5 whose radius is below 0.01/sqrt(r)).
+    # The hard part is the count: fewer than 0.5 % of the entries may differ at all.
     n, r = 1376, 344
     lay = cb.CompactLinear(n, 64, r, dtype=torch.bfloat16, seed=9, layer_id=1)
     P = to64(lay.debug_projection(epoch=0))
     want = co.projection(9, 1, 0, n, r, mode="bf16")
     assert (P != want).mean() < 5e-3
     ulp = np.maximum(np.abs(want), 2.0 ** -126) * 2.0 ** -7
-    assert np.all(np.abs(P - want) <= ulp * 1.001 + 2e-5 / math.sqrt(r))
+    assert np.all(np.abs(P - want) <= ulp * 1.001 + 5e-5 / math.sqrt(r))
     assert co.rel_frobenius(P, want) < 1e-3
 
 
@@ -158,7 +161,11 @@ def test_z_token_indexing_bit_exact(family):
     _, Z, _ = lay.forward(X.cuda(), W)
     want = Pb[torch.from_numpy(rows).cuda()].clone()
     want[::7] = 0
-    assert torch.equal(Z[:, :r].view(torch.int16), want.view(torch.int16))
+    # exact equality of values; the one thing bits may differ in is the sign of a zero: an entry of P that is
+    # -0 (the sine at an angle of exactly pi, one pair in 2^15) comes out of the sum 1 * (-0) + 0 + ... as +0
+    assert torch.equal(Z[:, :r].float(), want.float())
+    nz = want != 0
+    assert torch.equal(Z[:, :r][nz].view(torch.int16), want[nz].view(torch.int16))
     assert not Z[:, r:].any()
     # permuting tokens permutes rows of Z bitwise
     Xr = torch.randn((tokens, n), generator=torch.Generator().manual_seed(1)).to(torch.bfloat16).cuda()
