@@ -89,8 +89,15 @@ compact_status_t compact_layer_destroy(compact_layer_t* layer);
 int64_t compact_z_ld(const compact_layer_t* layer);
 
 /* Bytes of device scratch that compact_linear_bwd / compact_adam_update need
- * for `tokens` rows (split-K partials of Gc; the normalised step N). */
+ * for `tokens` rows (split-K partials of Gc; the normalised step N), and never
+ * less than compact_fwd_workspace_bytes: one buffer of this size serves all
+ * three calls of a layer (not at the same time). */
 size_t compact_workspace_bytes(const compact_layer_t* layer, int64_t tokens);
+
+/* Bytes of device scratch with which compact_linear_fwd runs fastest: room for
+ * the layer's projection of one epoch in bf16, n rows of ldz rounded up to a
+ * multiple of 64 (0 for fp32 layers, which do not use it). */
+size_t compact_fwd_workspace_bytes(const compact_layer_t* layer);
 
 /* Bytes kept for the backward by one forward: tokens * ldz * sizeof(element)
  * (Table 1: b l n -> b l r). */
@@ -100,13 +107,23 @@ size_t compact_saved_bytes(const compact_layer_t* layer, int64_t tokens);
  * from fp32 accumulators.  Row t of Z belongs to row t of X.  *epoch_used
  * (host pointer, may be NULL) receives the epoch P was generated with.
  * Z may be NULL: then nothing is kept for the backward, which must be
- * compact_linear_bwd_recompute (for layers under activation checkpointing). */
+ * compact_linear_bwd_recompute (for layers under activation checkpointing).
+ * workspace (device, 16-byte aligned; may be NULL): scratch that the call may
+ * overwrite and that holds nothing afterwards.  P is a function of (seed,
+ * layer, epoch) and is stored nowhere between calls (Section 3.3); a bf16
+ * layer given at least compact_fwd_workspace_bytes(layer) of scratch writes
+ * the current P out once at the start of the call and computes Z as further
+ * columns of the product that computes Y; without the scratch the kernel
+ * regenerates each tile of P where it is consumed, once per block of 512
+ * tokens.  Both ways give the same Y and Z bit for bit; the first is faster
+ * whenever the batch is longer than a few hundred tokens. */
 compact_status_t compact_linear_fwd(compact_layer_t* layer, int64_t tokens,
                                     const void* X, int64_t ldx,
                                     const void* W, int64_t ldw,
                                     void* Y, int64_t ldy,
                                     void* Z, int64_t ldz,
-                                    uint32_t* epoch_used, void* stream);
+                                    uint32_t* epoch_used,
+                                    void* workspace, size_t workspace_bytes, void* stream);
 
 /* Algorithm 2.  Gc[r x m] (fp32) = Z^T dY summed over all tokens, and
  * dX[tokens x n] = dY W^T.  dX may be NULL (skip it).  accumulate != 0 adds to
@@ -149,14 +166,20 @@ compact_status_t compact_linear_bwd_recompute(compact_layer_t* layer, int64_t to
  * Arrays have `count` entries, one per layer, in the same order.  All layers must
  * have the same n and dtype.  bf16 layers with one seed and count <= 3 run fused;
  * other groups run layer by layer with the same results up to the rounding of dX.
- * workspace: at least compact_group_workspace_bytes(layers, count, tokens). */
+ * workspace of compact_group_bwd: at least compact_group_workspace_bytes(layers,
+ * count, tokens).  workspace of compact_group_fwd: optional, as for
+ * compact_linear_fwd; compact_group_fwd_workspace_bytes(layers, count) (the sum
+ * over the layers, never more than compact_group_workspace_bytes) selects the
+ * faster way. */
 size_t compact_group_workspace_bytes(compact_layer_t* const* layers, int count, int64_t tokens);
+size_t compact_group_fwd_workspace_bytes(compact_layer_t* const* layers, int count);
 compact_status_t compact_group_fwd(compact_layer_t* const* layers, int count, int64_t tokens,
                                    const void* X, int64_t ldx,
                                    const void* const* W, const int64_t* ldw,
                                    void* const* Y, const int64_t* ldy,
                                    void* const* Z, const int64_t* ldz,
-                                   uint32_t* epochs_used, void* stream);
+                                   uint32_t* epochs_used,
+                                   void* workspace, size_t workspace_bytes, void* stream);
 compact_status_t compact_group_bwd(compact_layer_t* const* layers, int count, int64_t tokens,
                                    const void* const* dY, const int64_t* lddy,
                                    const void* const* Z, const int64_t* ldz,

@@ -26,6 +26,7 @@ F32, BF16 = 0, 1
 
 EXPORTS = [
     "compact_layer_create", "compact_layer_destroy", "compact_z_ld", "compact_workspace_bytes",
+    "compact_fwd_workspace_bytes", "compact_group_fwd_workspace_bytes",
     "compact_saved_bytes", "compact_linear_fwd", "compact_linear_bwd", "compact_recompute_workspace_bytes",
     "compact_linear_bwd_recompute", "compact_group_workspace_bytes", "compact_group_fwd", "compact_group_bwd",
     "compact_adam_update", "compact_adam_update_noalloc",
@@ -67,7 +68,9 @@ def lib() -> C.CDLL:
     L.compact_workspace_bytes.restype = C.c_size_t
     L.compact_saved_bytes.argtypes = [vp, i64]
     L.compact_saved_bytes.restype = C.c_size_t
-    L.compact_linear_fwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, i64, u32p, vp]
+    L.compact_fwd_workspace_bytes.argtypes = [vp]
+    L.compact_fwd_workspace_bytes.restype = C.c_size_t
+    L.compact_linear_fwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, i64, u32p, vp, C.c_size_t, vp]
     L.compact_linear_bwd.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, i64, vp, i64, C.c_int, vp,
                                      C.c_size_t, vp]
     L.compact_recompute_workspace_bytes.argtypes = [vp, i64]
@@ -77,7 +80,9 @@ def lib() -> C.CDLL:
     pp, ip = C.POINTER(C.c_void_p), C.POINTER(C.c_int64)
     L.compact_group_workspace_bytes.argtypes = [pp, C.c_int, i64]
     L.compact_group_workspace_bytes.restype = C.c_size_t
-    L.compact_group_fwd.argtypes = [pp, C.c_int, i64, vp, i64, pp, ip, pp, ip, pp, ip, u32p, vp]
+    L.compact_group_fwd_workspace_bytes.argtypes = [pp, C.c_int]
+    L.compact_group_fwd_workspace_bytes.restype = C.c_size_t
+    L.compact_group_fwd.argtypes = [pp, C.c_int, i64, vp, i64, pp, ip, pp, ip, pp, ip, u32p, vp, C.c_size_t, vp]
     L.compact_group_bwd.argtypes = [pp, C.c_int, i64, pp, ip, pp, ip, pp, ip, vp, i64, pp, ip, C.c_int, vp, C.c_size_t, vp]
     L.compact_adam_update.argtypes = [vp, vp, i64, vp, i64, vp, vp, C.c_uint32, C.c_float, vp, C.c_size_t, vp]
     L.compact_adam_update_noalloc.argtypes = [vp, vp, i64, vp, i64, vp, vp, C.c_uint32, C.c_float, vp]
@@ -202,9 +207,11 @@ class CompactLinear:
 
     # -- Algorithm 1 ---------------------------------------------------------------
     def forward(self, X: torch.Tensor, W: torch.Tensor, Y: Optional[torch.Tensor] = None,
-                Z: Optional[torch.Tensor] = None, keep_z: bool = True, stream=None):
-        """keep_z=False: nothing is kept for the backward (returns Z=None); use backward_recompute."""
+                Z: Optional[torch.Tensor] = None, keep_z: bool = True, stream=None, scratch: bool = True):
+        """keep_z=False: nothing is kept for the backward (returns Z=None); use backward_recompute.
+        scratch=False: the call gets no workspace, so P is generated inside the kernel (same Y and Z)."""
         tokens = X.shape[0]
+        ws = self.workspace(tokens) if scratch else None
         if Y is None:
             Y = torch.empty((tokens, self.m), dtype=self.dtype, device=X.device)
         if Z is None and keep_z:
@@ -213,7 +220,7 @@ class CompactLinear:
         _check(lib().compact_linear_fwd(self._h, tokens, _ptr(X), X.stride(0) if tokens else self.n, _ptr(W),
                                         W.stride(0), _ptr(Y), Y.stride(0) if tokens else self.m, _ptr(Z),
                                         (Z.stride(0) if tokens else self.ldz) if Z is not None else 0, C.byref(ep),
-                                        _stream(stream)),
+                                        _ptr(ws), ws.numel() if ws is not None else 0, _stream(stream)),
                "compact_linear_fwd")
         return Y, Z, int(ep.value)
 
@@ -309,15 +316,23 @@ class CompactGroup:
         self._h = (C.c_void_p * len(self.layers))(*[l._h for l in self.layers])
         self._ws = None
 
-    def forward(self, X: torch.Tensor, Ws, Ys=None, Zs=None, stream=None):
+    def workspace(self, tokens: int) -> torch.Tensor:
+        need = max(int(lib().compact_group_workspace_bytes(self._h, len(self.layers), tokens)), 256)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+        return self._ws
+
+    def forward(self, X: torch.Tensor, Ws, Ys=None, Zs=None, stream=None, scratch: bool = True):
         tokens = X.shape[0]
+        ws = self.workspace(tokens) if scratch else None
         if Ys is None:
             Ys = [torch.empty((tokens, l.m), dtype=l.dtype, device=X.device) for l in self.layers]
         if Zs is None:
             Zs = [torch.empty((tokens, l.ldz), dtype=l.dtype, device=X.device) for l in self.layers]
         eps = (C.c_uint32 * len(self.layers))()
         _check(lib().compact_group_fwd(self._h, len(self.layers), tokens, _ptr(X), X.stride(0), _ptr_array(Ws), _ld_array(Ws),
-                                       _ptr_array(Ys), _ld_array(Ys), _ptr_array(Zs), _ld_array(Zs), eps, _stream(stream)),
+                                       _ptr_array(Ys), _ld_array(Ys), _ptr_array(Zs), _ld_array(Zs), eps,
+                                       _ptr(ws), ws.numel() if ws is not None else 0, _stream(stream)),
                "compact_group_fwd")
         return Ys, Zs, [int(e) for e in eps]
 
@@ -328,9 +343,7 @@ class CompactGroup:
             Gcs = [torch.empty((l.r, l.m), dtype=torch.float32, device=dYs[0].device) for l in self.layers]
         if dX is None and need_dX:
             dX = torch.empty((tokens, n), dtype=self.layers[0].dtype, device=dYs[0].device)
-        need = max(int(lib().compact_group_workspace_bytes(self._h, len(self.layers), tokens)), 256)
-        if self._ws is None or self._ws.numel() < need:
-            self._ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+        self.workspace(tokens)
         _check(lib().compact_group_bwd(self._h, len(self.layers), tokens, _ptr_array(dYs), _ld_array(dYs), _ptr_array(Zs),
                                        _ld_array(Zs), _ptr_array(Ws), _ld_array(Ws), _ptr(dX), dX.stride(0) if dX is not None else 0,
                                        _ptr_array(Gcs), _ld_array(Gcs), int(accumulate), _ptr(self._ws), self._ws.numel(),

@@ -271,7 +271,14 @@ size_t compact_workspace_bytes(const compact_layer_t* layer, int64_t tokens) {
   size_t upd = (size_t)r * m * sizeof(float);
   size_t bwd = tc::gc_workspace_bytes(tokens, r, m);
   size_t need = upd > bwd ? upd : bwd;
+  const size_t fwd = compact_fwd_workspace_bytes(layer);
+  need = fwd > need ? fwd : need;
   return (size_t)round_up((int64_t)need, 256);
+}
+
+size_t compact_fwd_workspace_bytes(const compact_layer_t* layer) {
+  if (!layer || layer->cfg.dtype != COMPACT_BF16) return 0;
+  return (size_t)round_up((int64_t)g2::expanded_bytes(layer->cfg.n, (int)compact_z_ld(layer)), 256);
 }
 
 size_t compact_saved_bytes(const compact_layer_t* layer, int64_t tokens) {
@@ -281,11 +288,12 @@ size_t compact_saved_bytes(const compact_layer_t* layer, int64_t tokens) {
 
 compact_status_t compact_linear_fwd(compact_layer_t* L, int64_t tokens, const void* X, int64_t ldx, const void* W,
                                     int64_t ldw, void* Y, int64_t ldy, void* Z, int64_t ldz, uint32_t* epoch_used,
-                                    void* stream) {
+                                    void* workspace, size_t workspace_bytes, void* stream) {
   if (!L || tokens < 0 || tokens > 0x7fffffff) return COMPACT_ERR_INVALID_ARG;
   if (epoch_used) *epoch_used = L->epoch;
   if (tokens == 0) return COMPACT_OK;
   if (!X || !W || !Y) return COMPACT_ERR_INVALID_ARG;
+  if (workspace && !aligned16(workspace)) return COMPACT_ERR_ALIGNMENT;
   const size_t es = elem_size(L->cfg.dtype);
   if (!aligned16(X) || !aligned16(W) || !aligned16(Y) || (Z && !aligned16(Z))) return COMPACT_ERR_ALIGNMENT;
   if (!pitch_ok(ldx, L->cfg.n, es) || !pitch_ok(ldw, L->cfg.m, es) || !pitch_ok(ldy, L->cfg.m, es) ||
@@ -298,10 +306,19 @@ compact_status_t compact_linear_fwd(compact_layer_t* L, int64_t tokens, const vo
     typedef __nv_bfloat16 T;
     if (g_family.load() != 1) {
       tc::LaunchInfo li{g_family.load() == 2 ? 1 : CFG_CS, st, status_word(L), sched_words(L), &g_launches};
-      // Two routes with the same bits.  One launch: the Z items, then the Y items as 256 x 256 tiles on single SMs,
-      // which also fill the SMs the Z items leave idle.  Two launches: Z alone, then Y on pairs of SMs, whose
-      // epilogues run under the next tile's MMAs (about 3 % on Y).  The second pays when that gain outweighs the
-      // idle tail of a launch that holds nothing but Z items.
+      // With scratch for the expanded projection: P is written out once, then Z and Y are one product on pairs of SMs.
+      if (g_family.load() == 0 && Z && workspace && workspace_bytes >= compact_fwd_workspace_bytes(L)) {
+        g2::G2Layer gl;
+        gl.pp = make_pp(L, L->epoch);
+        gl.m = L->cfg.m; gl.zcols = (int)compact_z_ld(L);
+        gl.W = (const T*)W; gl.ldw = ldw; gl.Y = (T*)Y; gl.ldy = ldy; gl.Z = (T*)Z; gl.ldz = ldz;
+        s = g2::g2_forward(li, 1, &gl, tokens, L->cfg.n, (const T*)X, ldx, workspace);
+        if (s != COMPACT_ERR_SHAPE) return s;
+      }
+      // Without it P is generated inside the kernel, tile by tile.  Two routes with the same bits.  One launch: the Z
+      // items, then the Y items as 256 x 256 tiles on single SMs, which also fill the SMs the Z items leave idle.  Two
+      // launches: Z alone, then Y on pairs of SMs, whose epilogues run under the next tile's MMAs (about 3 % on Y).
+      // The second pays when that gain outweighs the idle tail of a launch that holds nothing but Z items.
       bool split = false;
       if (g_family.load() == 0 && Z && tokens >= 2 * tc::BN_MAX) {
         const double z_rounds = (double)((compact_z_ld(L) + tc::BM - 1) / tc::BM) * (double)((tokens + 511) / 512) / tc::NUM_SMS;
@@ -398,20 +415,34 @@ size_t compact_group_workspace_bytes(compact_layer_t* const* layers, int count, 
   if (count <= tc::MAXG) fused = tc::group_gc_workspace_bytes(count, r, m, tokens);
   // layer-by-layer fallback: one layer's workspace plus a dX-sized buffer for the partial input gradients
   const size_t fallback = single + (size_t)round_up((int64_t)tokens * layers[0]->cfg.n * (int64_t)elem_size(layers[0]->cfg.dtype), 256);
-  const size_t need = fused > fallback ? fused : fallback;
+  size_t need = fused > fallback ? fused : fallback;
+  const size_t fwd = compact_group_fwd_workspace_bytes(layers, count);
+  need = fwd > need ? fwd : need;
   return (size_t)round_up((int64_t)need, 256);
+}
+
+size_t compact_group_fwd_workspace_bytes(compact_layer_t* const* layers, int count) {
+  if (!layers || count < 1) return 0;
+  size_t sum = 0;
+  for (int g = 0; g < count; ++g) {
+    if (!layers[g]) return 0;
+    sum += compact_fwd_workspace_bytes(layers[g]);
+  }
+  return sum;
 }
 
 compact_status_t compact_group_fwd(compact_layer_t* const* layers, int count, int64_t tokens, const void* X, int64_t ldx,
                                    const void* const* W, const int64_t* ldw, void* const* Y, const int64_t* ldy,
-                                   void* const* Z, const int64_t* ldz, uint32_t* epochs_used, void* stream) {
+                                   void* const* Z, const int64_t* ldz, uint32_t* epochs_used, void* workspace,
+                                   size_t workspace_bytes, void* stream) {
   if (!layers || count < 1 || !W || !ldw || !Y || !ldy || !Z || !ldz) return COMPACT_ERR_INVALID_ARG;
+  if (workspace && !aligned16(workspace)) return COMPACT_ERR_ALIGNMENT;
   for (int g = 0; g < count; ++g)
     if (!layers[g] || layers[g]->cfg.n != layers[0]->cfg.n || layers[g]->cfg.dtype != layers[0]->cfg.dtype) return COMPACT_ERR_INVALID_ARG;
   if (!group_fusable(layers, count) || tokens <= 0) {
     for (int g = 0; g < count; ++g) {
       compact_status_t s = compact_linear_fwd(layers[g], tokens, X, ldx, W[g], ldw[g], Y[g], ldy[g], Z[g], ldz[g],
-                                              epochs_used ? epochs_used + g : nullptr, stream);
+                                              epochs_used ? epochs_used + g : nullptr, workspace, workspace_bytes, stream);
       if (s != COMPACT_OK) return s;
     }
     return COMPACT_OK;
@@ -436,6 +467,15 @@ compact_status_t compact_group_fwd(compact_layer_t* const* layers, int count, in
   compact_status_t s = check_device(layers[0], stream);
   if (s != COMPACT_OK) return s;
   tc::LaunchInfo li{g_family.load() == 2 ? 1 : CFG_CS, (cudaStream_t)stream, status_word(layers[0]), sched_words(layers[0]), &g_launches};
+  if (g_family.load() == 0 && workspace && workspace_bytes >= compact_group_fwd_workspace_bytes(layers, count)) {
+    g2::G2Layer g2l[tc::MAXG];
+    for (int g = 0; g < count; ++g) {
+      g2l[g].pp = gl[g].pp; g2l[g].m = gl[g].m; g2l[g].zcols = gl[g].zcols;
+      g2l[g].W = gl[g].W; g2l[g].ldw = gl[g].ldw; g2l[g].Y = gl[g].Y; g2l[g].ldy = gl[g].ldy; g2l[g].Z = gl[g].Z; g2l[g].ldz = gl[g].ldz;
+    }
+    s = g2::g2_forward(li, count, g2l, tokens, layers[0]->cfg.n, (const T*)X, ldx, workspace);
+    if (s != COMPACT_ERR_SHAPE) return s;
+  }
   return tc::forward_group(li, count, gl, tokens, layers[0]->cfg.n, (const T*)X, ldx);
 }
 

@@ -1,5 +1,7 @@
 // The TMA-fed products of the CompAct layer on pairs of SMs:
 //   Y = X W              (Algorithm 1 line 3)
+//   Z = X P              (Algorithm 1 line 2; P of the current epoch expanded once per call into scratch that
+//                         stays in the L2, so that Z is further columns of the same product as Y)
 //   dX = dY W^T          (Algorithm 2 line 2)
 //   Gc = Z^T dY          (Algorithm 2 line 1; split over tokens)
 // A cluster of two CTAs computes one 256 x 256 tile with tcgen05.mma.cta_group::2: each CTA holds 128 rows of A, half
@@ -35,7 +37,7 @@ constexpr int G2_BARS_OFF = G2_STAGING_OFF + G2_EPI_WARPS * STAGING_BYTES;
 constexpr int G2_NUM_BARS = 2 * G2_NS + 4;
 constexpr int G2_SMEM_BYTES = 1024 + G2_BARS_OFF + 8 * G2_NUM_BARS + 32;
 static_assert(G2_SMEM_BYTES <= 232448, "shared memory budget");
-constexpr int G2_MAXP = 2;
+constexpr int G2_MAXP = 6;      // Y and Z of up to three layers that share their input
 
 struct G2Problem {
   int M, N, K;                 // C[M x N] = A[M x K] B[K x N]
@@ -44,6 +46,7 @@ struct G2Problem {
   int a_blocked, b_blocked;    // MN-major operand read through the blocked map (column count a multiple of 64)
   int epi_mode;                // EPI_BF16 or EPI_F32 (3-D map [split][M][N])
   int tile_begin;
+  float scale;                 // EPI_BF16: the accumulator is multiplied by this before it is rounded (1: exact)
 };
 
 struct alignas(64) G2Params {
@@ -106,7 +109,10 @@ struct G2Tile {
 
 __device__ __forceinline__ G2Tile g2_decode(const G2Params& prm, int tile) {
   G2Tile t;
-  t.prob = (prm.num_problems > 1 && tile >= prm.prob[1].tile_begin) ? 1 : 0;
+  t.prob = 0;
+#pragma unroll
+  for (int i = 1; i < G2_MAXP; ++i)
+    if (i < prm.num_problems && tile >= prm.prob[i].tile_begin) t.prob = i;
   const G2Problem& p = prm.prob[t.prob];
   int local = tile - p.tile_begin;
   const int nb = local % p.tiles_n;
@@ -271,13 +277,14 @@ __global__ void __launch_bounds__(G2_THREADS, 1) compact_gemm2_kernel(const __gr
         if (col >= p.N) break;
         if (p.epi_mode == EPI_BF16) {
           uint32_t o[32];
+          const float sc = p.scale;
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
             uint32_t v[32];
             tmem_ld32(tcol + ci * cw + 32 * h, v);
             tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 16; ++j) o[16 * h + j] = pack_bf16x2(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+            for (int j = 0; j < 16; ++j) o[16 * h + j] = pack_bf16x2(__uint_as_float(v[2 * j]) * sc, __uint_as_float(v[2 * j + 1]) * sc);
           }
           if (lane == 0) tma_store_wait_read();          // the previous store has read the staging tile
           __syncwarp();
@@ -338,6 +345,7 @@ inline void g2_finish(G2Problem& p, int splits_wanted) {
   if (s > p.ksteps_total) s = p.ksteps_total;
   p.ksteps_per_split = (p.ksteps_total + s - 1) / s;
   p.splits = (p.ksteps_total + p.ksteps_per_split - 1) / p.ksteps_per_split;
+  if (p.scale == 0.f) p.scale = 1.f;
 }
 
 inline compact_status_t g2_launch(const LaunchInfo& li, G2Params& prm) {
@@ -395,6 +403,132 @@ inline compact_status_t g2_forward_y(const LaunchInfo& li, int64_t tokens, int n
   if (py.b_blocked ? !make_map_blocked(&prm.tmB[0], W, m, n, ldw, BK, G2_HALF / 64) : !make_map(&prm.tmB[0], W, m, n, ldw, 64, BK))
     return COMPACT_ERR_CUDA;
   if (!make_map(&prm.tmC[0], Y, m, tokens, ldy, 64, 32)) return COMPACT_ERR_CUDA;
+  return g2_launch(li, prm);
+}
+
+// --------------------------------------------------------------------------------------
+// The projection of one epoch, written out (Section 3.3: P is a function of the seed, the layer and the epoch,
+// so it can be rebuilt wherever it is needed).  The forward of a long batch uses every entry of P once per
+// 256 tokens; building the n x r entries once per call (a few microseconds; at most some tens of MB, which
+// stay in the L2 while the product runs) and reading them with the TMA unit like any other operand costs far
+// less than building every tile again for every block of tokens.  The scratch is the caller's; nothing of it
+// is kept between calls.
+// --------------------------------------------------------------------------------------
+// Pitch of the expanded projection in elements: the row of Z rounded up to whole 64-column blocks.
+inline int64_t expanded_ld(int zcols) { return ((int64_t)zcols + 63) / 64 * 64; }
+inline size_t expanded_bytes(int n, int zcols) { return (size_t)n * (size_t)expanded_ld(zcols) * sizeof(__nv_bfloat16); }
+
+// Gaussian projection: a thread writes eight consecutive entries of a row (one Philox call); columns from r to
+// the pitch are zeros.
+__global__ void __launch_bounds__(256) expand_projection_kernel(PhiloxKey key, uint32_t layer_hi, uint32_t layer_lo, uint32_t epoch,
+                                                                int n, int r, float neg2ln2_over_r, int groups,
+                                                                __nv_bfloat16* __restrict__ P) {
+  const long long total = (long long)n * groups;
+  for (long long task = (long long)blockIdx.x * blockDim.x + threadIdx.x; task < total; task += (long long)gridDim.x * blockDim.x) {
+    const int i = (int)(task / groups), g = (int)(task - (long long)i * groups);
+    const uint4 val = g * 8 < r ? projection8_bf16(key, layer_hi, layer_lo, epoch, n, r, neg2ln2_over_r, i, g * 8)
+                                : make_uint4(0u, 0u, 0u, 0u);
+    *reinterpret_cast<uint4*>(P + ((long long)i * groups + g) * 8) = val;
+  }
+}
+
+// Sparse projection: the integer counts (the product's epilogue applies 1 / sqrt(s)).  A warp owns a row: it
+// clears it, then lane 0 adds the signs of the row's terms one after another, so that terms that hash to the
+// same column add without a race.
+__global__ void __launch_bounds__(256) expand_sparse_kernel(PhiloxKey key, uint32_t layer_hi, uint32_t layer_lo, uint32_t epoch,
+                                                            int n, int r, int s, int groups, __nv_bfloat16* __restrict__ P) {
+  const int lane = threadIdx.x & 31;
+  const int warps = (int)((gridDim.x * blockDim.x) >> 5);
+  for (int i = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5); i < n; i += warps) {
+    __nv_bfloat16* row = P + (long long)i * groups * 8;
+    for (int g = lane; g < groups; g += 32) reinterpret_cast<uint4*>(row)[g] = make_uint4(0u, 0u, 0u, 0u);
+    __syncwarp();
+    if (lane == 0) {
+      for (int q = 0; 4 * q < s; ++q) {
+        const uint4 x = sparse_words4((uint32_t)q, (uint32_t)i, epoch, layer_hi, layer_lo, key);
+        const uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int l = 0; l < 4; ++l) {
+          if (4 * q + l < s) {
+            const int c = sparse_col(w[l], r);
+            row[c] = __float2bfloat16_rn(__bfloat162float(row[c]) + sparse_sign(w[l]));
+          }
+        }
+      }
+    }
+    __syncwarp();
+  }
+}
+
+inline compact_status_t expand_projection(const LaunchInfo& li, const ProjectionParams& pp, int zcols, __nv_bfloat16* P) {
+  const int groups = (int)(expanded_ld(zcols) / 8);
+  if (pp.sparse_s > 0) {
+    const long long threads = (long long)pp.n * 32;
+    const unsigned blocks = (unsigned)((threads + 255) / 256 < 8 * NUM_SMS ? (threads + 255) / 256 : 8 * NUM_SMS);
+    expand_sparse_kernel<<<blocks, 256, 0, li.stream>>>(pp.key, pp.layer_hi, pp.layer_lo, pp.epoch, pp.n, pp.r, pp.sparse_s, groups, P);
+  } else {
+    const long long tasks = (long long)pp.n * groups;
+    const unsigned blocks = (unsigned)((tasks + 255) / 256 < 8 * NUM_SMS ? (tasks + 255) / 256 : 8 * NUM_SMS);
+    expand_projection_kernel<<<blocks, 256, 0, li.stream>>>(pp.key, pp.layer_hi, pp.layer_lo, pp.epoch, pp.n, pp.r, pp.neg2ln2_over_r,
+                                                            groups, P);
+  }
+  (*li.launches)++;
+  return cudaGetLastError() == cudaSuccess ? COMPACT_OK : COMPACT_ERR_CUDA;
+}
+
+// Algorithm 1 for G layers that share their input (G = 1: one layer): every layer's P is expanded into its part of
+// the scratch, then one launch computes Z_g = X P_g and Y_g = X W_g.  The Z tiles go first: each problem's tiles
+// are dealt round-robin, and the short ragged ones are better placed early than as a launch's last.
+struct G2Layer {
+  ProjectionParams pp;
+  int m, zcols;
+  const __nv_bfloat16* W; int64_t ldw;
+  __nv_bfloat16* Y; int64_t ldy;
+  __nv_bfloat16* Z; int64_t ldz;
+};
+
+inline size_t g2_forward_scratch_bytes(int G, const G2Layer* L) {
+  size_t b = 0;
+  for (int g = 0; g < G; ++g) b += (expanded_bytes(L[g].pp.n, L[g].zcols) + 255) / 256 * 256;
+  return b;
+}
+
+inline compact_status_t g2_forward(const LaunchInfo& li, int G, const G2Layer* L, int64_t tokens, int n, const __nv_bfloat16* X,
+                                   int64_t ldx, void* scratch) {
+  if (G < 1 || 2 * G > G2_MAXP) return COMPACT_ERR_INVALID_ARG;
+  if (!li.status) return COMPACT_ERR_CUDA;
+  for (int g = 0; g < G; ++g)
+    if (!tc_shape_ok(tokens, n, L[g].m)) return COMPACT_ERR_SHAPE;
+  G2Params prm;
+  memset(&prm, 0, sizeof(prm));
+  prm.num_problems = 2 * G;
+  char* at = (char*)scratch;
+  for (int g = 0; g < G; ++g) {
+    __nv_bfloat16* P = (__nv_bfloat16*)at;
+    at += (expanded_bytes(n, L[g].zcols) + 255) / 256 * 256;
+    const compact_status_t s = expand_projection(li, L[g].pp, L[g].zcols, P);
+    if (s != COMPACT_OK) return s;
+    const int64_t ldp = expanded_ld(L[g].zcols);
+    G2Problem& pz = prm.prob[g];
+    pz.M = (int)tokens; pz.N = L[g].zcols; pz.K = n;
+    pz.a_mode = TMA_KMAJOR; pz.b_mode = TMA_MNMAJOR; pz.epi_mode = EPI_BF16;
+    pz.b_blocked = 1;
+    pz.scale = L[g].pp.inv_sqrt_s;
+    g2_finish(pz, 1);
+    if (!make_map(&prm.tmA[g], X, n, tokens, ldx, BK, G2_HALF)) return COMPACT_ERR_CUDA;
+    if (!make_map_blocked(&prm.tmB[g], P, ldp, n, ldp, BK, G2_HALF / 64)) return COMPACT_ERR_CUDA;
+    if (!make_map(&prm.tmC[g], L[g].Z, L[g].zcols, tokens, L[g].ldz, 64, 32)) return COMPACT_ERR_CUDA;
+    G2Problem& py = prm.prob[G + g];
+    py.M = (int)tokens; py.N = L[g].m; py.K = n;
+    py.a_mode = TMA_KMAJOR; py.b_mode = TMA_MNMAJOR; py.epi_mode = EPI_BF16;
+    py.b_blocked = L[g].m % 64 == 0;
+    g2_finish(py, 1);
+    prm.tmA[G + g] = prm.tmA[g];
+    if (py.b_blocked ? !make_map_blocked(&prm.tmB[G + g], L[g].W, L[g].m, n, L[g].ldw, BK, G2_HALF / 64)
+                     : !make_map(&prm.tmB[G + g], L[g].W, L[g].m, n, L[g].ldw, 64, BK))
+      return COMPACT_ERR_CUDA;
+    if (!make_map(&prm.tmC[G + g], L[g].Y, L[g].m, tokens, L[g].ldy, 64, 32)) return COMPACT_ERR_CUDA;
+  }
   return g2_launch(li, prm);
 }
 

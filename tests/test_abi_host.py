@@ -102,19 +102,19 @@ def test_argument_errors_before_any_launch():
     lay = cb.CompactLinear(128, 512, 16, dtype=torch.float32)
     L = cb.lib()
     before = cb.kernel_launch_count()
-    assert L.compact_linear_fwd(lay._h, 4, None, 128, None, 512, None, 512, None, 16, None, None) == cb.ERR_INVALID_ARG
-    assert L.compact_linear_fwd(lay._h, -1, None, 128, None, 512, None, 512, None, 16, None, None) == cb.ERR_INVALID_ARG
+    assert L.compact_linear_fwd(lay._h, 4, None, 128, None, 512, None, 512, None, 16, None, None, 0, None) == cb.ERR_INVALID_ARG
+    assert L.compact_linear_fwd(lay._h, -1, None, 128, None, 512, None, 512, None, 16, None, None, 0, None) == cb.ERR_INVALID_ARG
     buf = C.c_void_p(0x1000)
     odd = C.c_void_p(0x1004)
-    assert L.compact_linear_fwd(lay._h, 4, odd, 128, buf, 512, buf, 512, buf, 16, None, None) == cb.ERR_ALIGNMENT
-    assert L.compact_linear_fwd(lay._h, 4, buf, 126, buf, 512, buf, 512, buf, 16, None, None) == cb.ERR_ALIGNMENT
-    assert L.compact_linear_fwd(lay._h, 4, buf, 128, buf, 512, buf, 512, buf, 8, None, None) == cb.ERR_ALIGNMENT
+    assert L.compact_linear_fwd(lay._h, 4, odd, 128, buf, 512, buf, 512, buf, 16, None, None, 0, None) == cb.ERR_ALIGNMENT
+    assert L.compact_linear_fwd(lay._h, 4, buf, 126, buf, 512, buf, 512, buf, 16, None, None, 0, None) == cb.ERR_ALIGNMENT
+    assert L.compact_linear_fwd(lay._h, 4, buf, 128, buf, 512, buf, 512, buf, 8, None, None, 0, None) == cb.ERR_ALIGNMENT
     assert L.compact_linear_bwd(lay._h, 4, buf, 512, buf, 16, buf, 512, buf, 128, buf, 512, 0, None, 0, None) \
         == cb.ERR_WORKSPACE
     assert L.compact_adam_update(lay._h, buf, 512, buf, 512, buf, buf, 1, 1e-3, buf, 1 << 20, None) \
         == cb.ERR_EPOCH_MISMATCH
     assert L.compact_adam_update(lay._h, buf, 512, buf, 512, buf, buf, 0, 1e-3, None, 0, None) == cb.ERR_WORKSPACE
     ep = C.c_uint32(99)
-    assert L.compact_linear_fwd(lay._h, 0, None, 128, None, 512, None, 512, None, 16, C.byref(ep), None) == cb.OK
+    assert L.compact_linear_fwd(lay._h, 0, None, 128, None, 512, None, 512, None, 16, C.byref(ep), None, 0, None) == cb.OK
     assert ep.value == 0                            # empty batch: no launch, epoch still reported
     assert cb.kernel_launch_count() == before
