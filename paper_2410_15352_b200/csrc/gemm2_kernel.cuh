@@ -56,6 +56,8 @@ struct alignas(64) G2Params {
   G2Problem prob[G2_MAXP];
   int num_problems;
   int total_tiles;
+  int by_rows;                 // all problems share A and M: tiles are numbered row block by row block, across the problems
+  int cols_total;              // by_rows: column tiles of all problems together (tile_begin is then a problem's first)
   unsigned int* status;
 };
 
@@ -110,6 +112,20 @@ struct G2Tile {
 __device__ __forceinline__ G2Tile g2_decode(const G2Params& prm, int tile) {
   G2Tile t;
   t.prob = 0;
+  if (prm.by_rows) {
+    // consecutive tiles read the same rows of A: (row block, column tile over the problems side by side)
+    const int mb = tile / prm.cols_total, c = tile - mb * prm.cols_total;
+#pragma unroll
+    for (int i = 1; i < G2_MAXP; ++i)
+      if (i < prm.num_problems && c >= prm.prob[i].tile_begin) t.prob = i;
+    const G2Problem& p = prm.prob[t.prob];
+    t.split = 0;
+    t.m0 = mb * 2 * G2_HALF;
+    t.n0 = (c - p.tile_begin) * 2 * G2_HALF;
+    t.k_begin = 0;
+    t.k_end = p.ksteps_total;
+    return t;
+  }
 #pragma unroll
   for (int i = 1; i < G2_MAXP; ++i)
     if (i < prm.num_problems && tile >= prm.prob[i].tile_begin) t.prob = i;
@@ -360,9 +376,18 @@ inline compact_status_t g2_launch(const LaunchInfo& li, G2Params& prm) {
     attr_set[dev].store(true, std::memory_order_release);
   }
   int t = 0;
-  for (int i = 0; i < prm.num_problems; ++i) {
-    prm.prob[i].tile_begin = t;
-    t += prm.prob[i].tiles_m * prm.prob[i].tiles_n * prm.prob[i].splits;
+  if (prm.by_rows) {
+    for (int i = 0; i < prm.num_problems; ++i) {
+      prm.prob[i].tile_begin = t;
+      t += prm.prob[i].tiles_n;
+    }
+    prm.cols_total = t;
+    t *= prm.prob[0].tiles_m;
+  } else {
+    for (int i = 0; i < prm.num_problems; ++i) {
+      prm.prob[i].tile_begin = t;
+      t += prm.prob[i].tiles_m * prm.prob[i].tiles_n * prm.prob[i].splits;
+    }
   }
   prm.total_tiles = t;
   prm.status = li.status;
@@ -477,8 +502,7 @@ inline compact_status_t expand_projection(const LaunchInfo& li, const Projection
 }
 
 // Algorithm 1 for G layers that share their input (G = 1: one layer): every layer's P is expanded into its part of
-// the scratch, then one launch computes Z_g = X P_g and Y_g = X W_g.  The Z tiles go first: each problem's tiles
-// are dealt round-robin, and the short ragged ones are better placed early than as a launch's last.
+// the scratch, then one launch computes Z_g = X P_g and Y_g = X W_g, row block by row block of X.
 struct G2Layer {
   ProjectionParams pp;
   int m, zcols;
@@ -529,6 +553,13 @@ inline compact_status_t g2_forward(const LaunchInfo& li, int G, const G2Layer* L
       return COMPACT_ERR_CUDA;
     if (!make_map(&prm.tmC[G + g], L[g].Y, L[g].m, tokens, L[g].ldy, 64, 32)) return COMPACT_ERR_CUDA;
   }
+  // Row block by row block, X is read from DRAM once instead of once per problem -- as long as the B operands
+  // (every W and P of the launch, which each round of tiles walks in full) stay in the 126 MB L2 beside it.
+  // Measured on 16384 tokens: 4096 x (4096 + 512) -2.3 %, 4096 x (11008 + 512) (94 MB) -1.2 %,
+  // 11008 x (4096 + 1408) (121 MB) +2 %.
+  size_t b_bytes = 0;
+  for (int g = 0; g < G; ++g) b_bytes += (size_t)n * (size_t)(L[g].m + expanded_ld(L[g].zcols)) * sizeof(__nv_bfloat16);
+  prm.by_rows = b_bytes <= ((size_t)100 << 20) ? 1 : 0;
   return g2_launch(li, prm);
 }
 

@@ -70,6 +70,24 @@ def test_z_pitch_and_saved_bytes():
     assert abs(comp / dense - 1964 / 4784) < 2e-3   # the 684 -> 688 pad shifts it slightly
 
 
+def test_forward_scratch_accounting():
+    # room for P of one epoch in bf16: n rows of ldz rounded up to whole 64-column blocks; one workspace of
+    # compact_workspace_bytes serves forward, backward and update; a group's is the sum over its layers
+    L = cb.lib()
+    for n, m, r, cols in ((4096, 4096, 512, 512), (11008, 4096, 1376, 1408), (2736, 1024, 342, 384), (64, 64, 1, 64)):
+        lay = cb.CompactLinear(n, m, r)
+        assert L.compact_fwd_workspace_bytes(lay._h) == n * cols * 2
+        for tokens in (0, 1, 16384):
+            assert lay.workspace_bytes(tokens) >= n * cols * 2
+    assert L.compact_fwd_workspace_bytes(cb.CompactLinear(128, 512, 16, dtype=torch.float32)._h) == 0
+    lays = [cb.CompactLinear(4096, 4096, 512), cb.CompactLinear(4096, 1024, 512), cb.CompactLinear(4096, 1024, 100)]
+    h = (C.c_void_p * 3)(*[l._h for l in lays])
+    total = sum(L.compact_fwd_workspace_bytes(l._h) for l in lays)
+    assert L.compact_group_fwd_workspace_bytes(h, 3) == total
+    assert L.compact_group_workspace_bytes(h, 3, 16) >= total
+    assert L.compact_group_fwd_workspace_bytes(None, 3) == 0
+
+
 def test_refresh_schedule_is_host_only():
     lay = cb.CompactLinear(128, 512, 16, dtype=torch.float32, refresh_T=2)
     before = cb.kernel_launch_count()

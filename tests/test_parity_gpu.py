@@ -176,24 +176,25 @@ def test_z_token_indexing_bit_exact(family):
 
 
 def test_cluster_and_single_cta_generation_agree_bitwise():
-    # sharing generated tiles across a cluster changes who computes an entry of P, not its value, and leaves the
-    # accumulation order of every output alone
+    # sharing generated tiles across a cluster, or writing P out before the product, changes who computes an entry
+    # of P, not its value, and leaves the accumulation order of every output alone
     tokens, n, m, r = 1300, 320, 1096, 200
     wl = wlm.Workload("clu", 99, "bf16", tokens, [wlm.LayerShape("l", n, m, r)], x_scale_inv_sqrt_n=True)
     X, dY = wlm.draw_X(wl, 0, 0).cuda(), wlm.draw_dY(wl, 0, 0).cuda()
     out = []
-    for fam in (0, 2):
+    for fam, scratch in ((0, True), (0, False), (2, False)):
         cb.set_kernel_family(fam)
         gpu, _, W0 = make_pair(wl, 0)
         W = W0.cuda()
-        Y, Z, ep = gpu.forward(X, W)
+        Y, Z, ep = gpu.forward(X, W, scratch=scratch)
         dX, Gc = gpu.backward(dY, Z, W)
         M, V = torch.zeros_like(Gc), torch.zeros_like(Gc)
         gpu.adam_update(W, Gc, M, V, ep)
         out.append((Y, Z, dX, Gc, W))
     cb.set_kernel_family(0)
-    for a, b in zip(*out):
-        assert torch.equal(a.view(torch.int16) if a.dtype == torch.bfloat16 else a, b.view(torch.int16) if b.dtype == torch.bfloat16 else b)
+    for other in out[1:]:
+        for a, b in zip(out[0], other):
+            assert torch.equal(a.view(torch.int16) if a.dtype == torch.bfloat16 else a, b.view(torch.int16) if b.dtype == torch.bfloat16 else b)
 
 
 # ---- determinism, accumulation, empty input, epoch guard -----------------------------------
