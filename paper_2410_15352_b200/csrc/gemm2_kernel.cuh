@@ -56,8 +56,10 @@ struct alignas(64) G2Params {
   G2Problem prob[G2_MAXP];
   int num_problems;
   int total_tiles;
-  int by_rows;                 // all problems share A and M: tiles are numbered row block by row block, across the problems
-  int cols_total;              // by_rows: column tiles of all problems together (tile_begin is then a problem's first)
+  int by_rows;                 // > 0: the problems share A and M, and every run of this many problems is numbered row
+                               // block by row block across its problems (tile_begin: a problem's first column tile in its run)
+  int run_begin[G2_MAXP / 2 + 1];   // by_rows: first tile of each run
+  int run_cols[G2_MAXP / 2];        // by_rows: column tiles of a run's problems together
   unsigned int* status;
 };
 
@@ -114,10 +116,16 @@ __device__ __forceinline__ G2Tile g2_decode(const G2Params& prm, int tile) {
   t.prob = 0;
   if (prm.by_rows) {
     // consecutive tiles read the same rows of A: (row block, column tile over the problems side by side)
-    const int mb = tile / prm.cols_total, c = tile - mb * prm.cols_total;
+    int q = 0;
+#pragma unroll
+    for (int i = 1; i < G2_MAXP / 2; ++i)
+      if (i * prm.by_rows < prm.num_problems && tile >= prm.run_begin[i]) q = i;
+    const int local = tile - prm.run_begin[q];
+    const int mb = local / prm.run_cols[q], c = local - mb * prm.run_cols[q];
+    t.prob = q * prm.by_rows;
 #pragma unroll
     for (int i = 1; i < G2_MAXP; ++i)
-      if (i < prm.num_problems && c >= prm.prob[i].tile_begin) t.prob = i;
+      if (i < prm.by_rows && c >= prm.prob[q * prm.by_rows + i].tile_begin) t.prob = q * prm.by_rows + i;
     const G2Problem& p = prm.prob[t.prob];
     t.split = 0;
     t.m0 = mb * 2 * G2_HALF;
@@ -377,12 +385,16 @@ inline compact_status_t g2_launch(const LaunchInfo& li, G2Params& prm) {
   }
   int t = 0;
   if (prm.by_rows) {
-    for (int i = 0; i < prm.num_problems; ++i) {
-      prm.prob[i].tile_begin = t;
-      t += prm.prob[i].tiles_n;
+    for (int q = 0; q * prm.by_rows < prm.num_problems; ++q) {
+      int cols = 0;
+      for (int i = q * prm.by_rows; i < (q + 1) * prm.by_rows && i < prm.num_problems; ++i) {
+        prm.prob[i].tile_begin = cols;
+        cols += prm.prob[i].tiles_n;
+      }
+      prm.run_begin[q] = t;
+      prm.run_cols[q] = cols;
+      t += cols * prm.prob[0].tiles_m;
     }
-    prm.cols_total = t;
-    t *= prm.prob[0].tiles_m;
   } else {
     for (int i = 0; i < prm.num_problems; ++i) {
       prm.prob[i].tile_begin = t;
@@ -533,33 +545,40 @@ inline compact_status_t g2_forward(const LaunchInfo& li, int G, const G2Layer* L
     const compact_status_t s = expand_projection(li, L[g].pp, L[g].zcols, P);
     if (s != COMPACT_OK) return s;
     const int64_t ldp = expanded_ld(L[g].zcols);
-    G2Problem& pz = prm.prob[g];
+    const int iz = 2 * g, iy = 2 * g + 1;
+    G2Problem& pz = prm.prob[iz];
     pz.M = (int)tokens; pz.N = L[g].zcols; pz.K = n;
     pz.a_mode = TMA_KMAJOR; pz.b_mode = TMA_MNMAJOR; pz.epi_mode = EPI_BF16;
     pz.b_blocked = 1;
     pz.scale = L[g].pp.inv_sqrt_s;
     g2_finish(pz, 1);
-    if (!make_map(&prm.tmA[g], X, n, tokens, ldx, BK, G2_HALF)) return COMPACT_ERR_CUDA;
-    if (!make_map_blocked(&prm.tmB[g], P, ldp, n, ldp, BK, G2_HALF / 64)) return COMPACT_ERR_CUDA;
-    if (!make_map(&prm.tmC[g], L[g].Z, L[g].zcols, tokens, L[g].ldz, 64, 32)) return COMPACT_ERR_CUDA;
-    G2Problem& py = prm.prob[G + g];
+    if (!make_map(&prm.tmA[iz], X, n, tokens, ldx, BK, G2_HALF)) return COMPACT_ERR_CUDA;
+    if (!make_map_blocked(&prm.tmB[iz], P, ldp, n, ldp, BK, G2_HALF / 64)) return COMPACT_ERR_CUDA;
+    if (!make_map(&prm.tmC[iz], L[g].Z, L[g].zcols, tokens, L[g].ldz, 64, 32)) return COMPACT_ERR_CUDA;
+    G2Problem& py = prm.prob[iy];
     py.M = (int)tokens; py.N = L[g].m; py.K = n;
     py.a_mode = TMA_KMAJOR; py.b_mode = TMA_MNMAJOR; py.epi_mode = EPI_BF16;
     py.b_blocked = L[g].m % 64 == 0;
     g2_finish(py, 1);
-    prm.tmA[G + g] = prm.tmA[g];
-    if (py.b_blocked ? !make_map_blocked(&prm.tmB[G + g], L[g].W, L[g].m, n, L[g].ldw, BK, G2_HALF / 64)
-                     : !make_map(&prm.tmB[G + g], L[g].W, L[g].m, n, L[g].ldw, 64, BK))
+    prm.tmA[iy] = prm.tmA[iz];
+    if (py.b_blocked ? !make_map_blocked(&prm.tmB[iy], L[g].W, L[g].m, n, L[g].ldw, BK, G2_HALF / 64)
+                     : !make_map(&prm.tmB[iy], L[g].W, L[g].m, n, L[g].ldw, 64, BK))
       return COMPACT_ERR_CUDA;
-    if (!make_map(&prm.tmC[G + g], L[g].Y, L[g].m, tokens, L[g].ldy, 64, 32)) return COMPACT_ERR_CUDA;
+    if (!make_map(&prm.tmC[iy], L[g].Y, L[g].m, tokens, L[g].ldy, 64, 32)) return COMPACT_ERR_CUDA;
   }
   // Row block by row block, X is read from DRAM once instead of once per problem -- as long as the B operands
   // (every W and P of the launch, which each round of tiles walks in full) stay in the 126 MB L2 beside it.
   // Measured on 16384 tokens: 4096 x (4096 + 512) -2.3 %, 4096 x (11008 + 512) (94 MB) -1.2 %,
   // 11008 x (4096 + 1408) (121 MB) +2 %.
-  size_t b_bytes = 0;
-  for (int g = 0; g < G; ++g) b_bytes += (size_t)n * (size_t)(L[g].m + expanded_ld(L[g].zcols)) * sizeof(__nv_bfloat16);
-  prm.by_rows = b_bytes <= ((size_t)100 << 20) ? 1 : 0;
+  // A group of layers whose operands together are too large runs layer after layer, each by rows if it fits.
+  const size_t fits = (size_t)100 << 20;
+  size_t all = 0, largest = 0;
+  for (int g = 0; g < G; ++g) {
+    const size_t b = (size_t)n * (size_t)(L[g].m + expanded_ld(L[g].zcols)) * sizeof(__nv_bfloat16);
+    all += b;
+    largest = b > largest ? b : largest;
+  }
+  prm.by_rows = all <= fits ? 2 * G : (largest <= fits ? 2 : 0);
   return g2_launch(li, prm);
 }
 
