@@ -195,7 +195,12 @@ compact_status_t compact_group_bwd(compact_layer_t* const* layers, int count, in
  * Increments the layer's step.  bf16 layers on the tensor-core path form the
  * increment -eta * alpha * (P N) in fp32, round it to bf16 and add it to W with
  * one more rounding (the add is done by the TMA unit at the L2, so W makes one
- * trip instead of two); fp32 layers and the SIMT path round W once. */
+ * trip instead of two); fp32 layers and the SIMT path round W once.
+ * workspace: at least r * m * 4 bytes (rounded up to 256).  With
+ * compact_workspace_bytes(layer, 0) bytes a bf16 layer whose rank is beyond
+ * the 512 columns of P that the one-launch update keeps on chip also has room
+ * for P written out next to N, and its product runs on pairs of SMs; with
+ * less, P is regenerated tile by tile.  Same W, M, V bit for bit. */
 compact_status_t compact_adam_update(compact_layer_t* layer,
                                      void* W, int64_t ldw,
                                      const float* Gc, int64_t ldg,

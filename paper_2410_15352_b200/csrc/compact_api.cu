@@ -120,6 +120,9 @@ unsigned int* sched_words(const compact_layer_t*) {
   return base ? base + 4 * (g_sched_seq.fetch_add(1) % kSchedRing) : nullptr;
 }
 
+// What every route of the update can work with: N as fp32 r x m (the tensor-core routes keep it in bf16).
+size_t update_min_bytes(const compact_layer_t* L) { return (size_t)round_up((int64_t)L->cfg.r * L->cfg.m * (int64_t)sizeof(float), 256); }
+
 ProjectionParams make_pp(const compact_layer_t* L, uint32_t epoch) {
   ProjectionParams pp;
   pp.key = make_philox_key(L->cfg.seed);
@@ -273,6 +276,11 @@ size_t compact_workspace_bytes(const compact_layer_t* layer, int64_t tokens) {
   size_t need = upd > bwd ? upd : bwd;
   const size_t fwd = compact_fwd_workspace_bytes(layer);
   need = fwd > need ? fwd : need;
+  // layers beyond the one-launch update's panel: N and the expanded P side by side
+  if (layer->cfg.dtype == COMPACT_BF16 && !upd::fused_update_ok(layer->cfg.n, m, r)) {
+    const size_t u2 = g2::g2_update_scratch_bytes(layer->cfg.n, m, r, (int)compact_z_ld(layer));
+    need = u2 > need ? u2 : need;
+  }
   return (size_t)round_up((int64_t)need, 256);
 }
 
@@ -586,7 +594,7 @@ compact_status_t compact_adam_update(compact_layer_t* L, void* W, int64_t ldw, c
   const size_t es = elem_size(L->cfg.dtype);
   if (!aligned16(W) || !aligned16(Gc) || !aligned16(M) || !aligned16(V)) return COMPACT_ERR_ALIGNMENT;
   if (!pitch_ok(ldw, L->cfg.m, es) || !pitch_ok(ldg, L->cfg.m, 4)) return COMPACT_ERR_ALIGNMENT;
-  if (!workspace || workspace_bytes < compact_workspace_bytes(L, 0)) return COMPACT_ERR_WORKSPACE;
+  if (!workspace || workspace_bytes < update_min_bytes(L)) return COMPACT_ERR_WORKSPACE;
   if (!aligned16(workspace)) return COMPACT_ERR_ALIGNMENT;
   compact_status_t s = check_device(L, stream);
   if (s != COMPACT_OK) return s;
@@ -605,6 +613,10 @@ compact_status_t compact_adam_update(compact_layer_t* L, void* W, int64_t ldw, c
       if (g_family.load() == 0 && upd::fused_update_ok(L->cfg.n, L->cfg.m, L->cfg.r))
         s = upd::fused_update(li, pp, adam_scalars(L, L->step + 1), L->cfg.n, L->cfg.m, L->cfg.r, (T*)W, ldw,
                               Gc, ldg, M, V, step_scale, workspace, workspace_bytes);
+      else if (g_family.load() == 0 &&
+               workspace_bytes >= g2::g2_update_scratch_bytes(L->cfg.n, L->cfg.m, L->cfg.r, (int)compact_z_ld(L)))
+        s = g2::g2_update(li, pp, adam_scalars(L, L->step + 1), L->cfg.n, L->cfg.m, L->cfg.r, (int)compact_z_ld(L), (T*)W, ldw,
+                          Gc, ldg, M, V, step_scale, workspace, workspace_bytes);
       else
         s = tc::update(li, pp, adam_scalars(L, L->step + 1), L->cfg.n, L->cfg.m, L->cfg.r, (T*)W, ldw,
                        Gc, ldg, M, V, step_scale, workspace, workspace_bytes);
@@ -646,7 +658,7 @@ compact_status_t compact_adam_update_noalloc(compact_layer_t* L, void* W, int64_
                                              float* M, float* V, uint32_t epoch_of_Gc, float lr, void* stream) {
   if (!L) return COMPACT_ERR_INVALID_ARG;
   // the update needs r x m scratch entries (fp32 in the plain kernels, bf16 in the tensor-core ones)
-  if (compact_workspace_bytes(L, 0) > (size_t)COMPACT_NOALLOC_SCRATCH_BYTES) return COMPACT_ERR_SCRATCH_LIMIT;
+  if (update_min_bytes(L) > (size_t)COMPACT_NOALLOC_SCRATCH_BYTES) return COMPACT_ERR_SCRATCH_LIMIT;
   compact_status_t s = check_device(L, stream);
   if (s != COMPACT_OK) return s;
   void* scratch = nullptr;

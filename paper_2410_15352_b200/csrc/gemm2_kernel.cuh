@@ -44,9 +44,9 @@ struct G2Problem {
   int tiles_m, tiles_n, splits, ksteps_total, ksteps_per_split;
   int a_mode, b_mode;          // TMA_KMAJOR or TMA_MNMAJOR
   int a_blocked, b_blocked;    // MN-major operand read through the blocked map (column count a multiple of 64)
-  int epi_mode;                // EPI_BF16 or EPI_F32 (3-D map [split][M][N])
+  int epi_mode;                // EPI_BF16, EPI_UPDATE_W (C += -scale * acc) or EPI_F32 (3-D map [split][M][N])
   int tile_begin;
-  float scale;                 // EPI_BF16: the accumulator is multiplied by this before it is rounded (1: exact)
+  float scale;                 // bf16 epilogues: the accumulator is multiplied by this before it is rounded (1: exact)
 };
 
 struct alignas(64) G2Params {
@@ -299,9 +299,10 @@ __global__ void __launch_bounds__(G2_THREADS, 1) compact_gemm2_kernel(const __gr
       for (int ci = eset; ci < 256 / cw && row0 < p.M; ci += 2) {
         const int col = t.n0 + ci * cw;
         if (col >= p.N) break;
-        if (p.epi_mode == EPI_BF16) {
+        if (p.epi_mode == EPI_BF16 || p.epi_mode == EPI_UPDATE_W) {
+          // The update stages -(eta alpha) (P N) and lets the TMA unit add it to W (Algorithm 3 line 9).
           uint32_t o[32];
-          const float sc = p.scale;
+          const float sc = p.epi_mode == EPI_UPDATE_W ? -p.scale : p.scale;
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
             uint32_t v[32];
@@ -318,7 +319,8 @@ __global__ void __launch_bounds__(G2_THREADS, 1) compact_gemm2_kernel(const __gr
           fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) {
-            tma_store_2d(mapC, stg, col, row0);
+            if (p.epi_mode == EPI_UPDATE_W) tma_reduce_add_2d(mapC, stg, col, row0);
+            else tma_store_2d(mapC, stg, col, row0);
             tma_store_commit();
           }
         } else {
@@ -579,6 +581,45 @@ inline compact_status_t g2_forward(const LaunchInfo& li, int G, const G2Layer* L
     largest = b > largest ? b : largest;
   }
   prm.by_rows = all <= fits ? 2 * G : (largest <= fits ? 2 : 0);
+  return g2_launch(li, prm);
+}
+
+// Algorithm 3 for layers whose rank does not fit the one-launch update's resident panel: Adam moments -> N (bf16, front
+// of the scratch), P written out behind it, then W <- W - scale * P N as one product on pairs of SMs whose epilogue
+// adds the increment to W.  Same N, same entries of P, same order of accumulation and the same roundings as the
+// streaming update on single SMs (which needs no room for P and remains the route when the scratch is small).
+inline size_t g2_update_scratch_bytes(int n, int m, int r, int zcols) {
+  return ((size_t)r * m * sizeof(__nv_bfloat16) + 255) / 256 * 256 + expanded_bytes(n, zcols);
+}
+
+inline compact_status_t g2_update(const LaunchInfo& li, const ProjectionParams& pp, const simt::AdamScalars& as, int n, int m, int r,
+                                  int zcols, __nv_bfloat16* W, int64_t ldw, const float* Gc, int64_t ldg, float* M, float* V,
+                                  float scale, void* workspace, size_t workspace_bytes) {
+  if (!tc_shape_ok(1, n, m)) return COMPACT_ERR_SHAPE;
+  if (!li.status) return COMPACT_ERR_CUDA;
+  if (workspace_bytes < g2_update_scratch_bytes(n, m, r, zcols)) return COMPACT_ERR_WORKSPACE;
+  __nv_bfloat16* Nbuf = (__nv_bfloat16*)workspace;
+  __nv_bfloat16* P = (__nv_bfloat16*)((char*)workspace + ((size_t)r * m * sizeof(__nv_bfloat16) + 255) / 256 * 256);
+  const long long cnt = (long long)r * (m / 4);
+  adam_moments_bf16_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, li.stream>>>(Gc, ldg, M, V, Nbuf, r, m, as);
+  (*li.launches)++;
+  if (cudaGetLastError() != cudaSuccess) return COMPACT_ERR_CUDA;
+  compact_status_t s = expand_projection(li, pp, zcols, P);
+  if (s != COMPACT_OK) return s;
+  const int64_t ldp = expanded_ld(zcols);
+  G2Params prm;
+  memset(&prm, 0, sizeof(prm));
+  prm.num_problems = 1;
+  G2Problem& pu = prm.prob[0];
+  pu.M = n; pu.N = m; pu.K = r;
+  pu.a_mode = TMA_KMAJOR; pu.b_mode = TMA_MNMAJOR; pu.epi_mode = EPI_UPDATE_W;
+  pu.b_blocked = m % 64 == 0;
+  pu.scale = scale;
+  g2_finish(pu, 1);
+  if (!make_map(&prm.tmA[0], P, ldp, n, ldp, BK, G2_HALF)) return COMPACT_ERR_CUDA;
+  if (pu.b_blocked ? !make_map_blocked(&prm.tmB[0], Nbuf, m, r, m, BK, G2_HALF / 64) : !make_map(&prm.tmB[0], Nbuf, m, r, m, 64, BK))
+    return COMPACT_ERR_CUDA;
+  if (!make_map(&prm.tmC[0], W, m, n, ldw, 64, 32)) return COMPACT_ERR_CUDA;
   return g2_launch(li, prm);
 }
 

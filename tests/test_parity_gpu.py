@@ -2,9 +2,11 @@
 oracle on the same seeded inputs.  Integer streams must match bit for bit;
 floating-point tensors within the stated relative Frobenius tolerance
 (1e-5 in fp32, 2e-2 in bf16 with fp32 accumulation)."""
+import ctypes as C
 import math
 
 import numpy as np
+
 import pytest
 import torch
 
@@ -487,6 +489,46 @@ def test_one_launch_update_equals_two_kernel_update_bitwise(n, m, r):
     cb.set_kernel_family(0)
     assert torch.equal(out[0][0].view(torch.int16), out[1][0].view(torch.int16))
     assert torch.equal(out[0][1], out[1][1]) and torch.equal(out[0][2], out[1][2])
+    assert not torch.equal(out[0][0].view(torch.int16), W0.view(torch.int16))
+
+
+@pytest.mark.parametrize("n,m,r,s", [
+    (4000, 1344, 600, 0),      # rank beyond the resident panel; ragged row panel and column block; r not a multiple of 64
+    (2048, 520, 100, 0),       # m not a multiple of 64: the one-launch update does not take it
+    (11008, 1024, 1376, 0),    # the LLaMA-7B down_proj rank and row count
+    (4000, 1344, 600, 8),      # sparse projection: integer counts in scratch, 1 / sqrt(s) on the step size
+])
+def test_pair_of_sms_update_equals_streaming_update_bitwise(n, m, r, s):
+    # Layers the one-launch update does not take: with room for P in the workspace the product runs on pairs of SMs
+    # from the written-out P; with a workspace that only holds N (and in the single-SM family) the streaming kernel
+    # regenerates P tile by tile.  Same N, same entries of P, same accumulation order, same roundings.
+    g = torch.Generator().manual_seed(n + m + r)
+    Gc = (torch.randn((r, m), generator=g) * 1e-3).cuda()
+    W0 = (torch.randn((n, m), generator=g) * 0.02).to(torch.bfloat16).cuda()
+    out = []
+    for fam, small in ((0, False), (0, True), (2, False)):
+        cb.set_kernel_family(fam)
+        lay = cb.CompactLinear(n, m, r, seed=11, layer_id=3, lr=2e-3, alpha=0.5, sparse_s=s)
+        W, M, V = W0.clone(), torch.full((r, m), 1e-4, device="cuda"), torch.full((r, m), 1e-7, device="cuda")
+        before = cb.kernel_launch_count()
+        for _ in range(2):
+            if small:
+                # the documented minimum: less than N and P side by side
+                ws = torch.empty(-(-r * m * 4 // 256) * 256, dtype=torch.uint8, device="cuda")
+                assert ws.numel() < lay.workspace_bytes(0)
+                st = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+                code = cb.lib().compact_adam_update(lay._h, W.data_ptr(), W.stride(0), Gc.data_ptr(), Gc.stride(0), M.data_ptr(),
+                                                    V.data_ptr(), 0, float("nan"), ws.data_ptr(), ws.numel(), st)
+                assert code == cb.OK
+            else:
+                lay.adam_update(W, Gc, M, V, 0)
+        assert lay.status() == cb.OK
+        assert cb.kernel_launch_count() - before == (6 if (fam == 0 and not small) else 4)
+        out.append((W, M, V))
+    cb.set_kernel_family(0)
+    for o in out[1:]:
+        assert torch.equal(out[0][0].view(torch.int16), o[0].view(torch.int16))
+        assert torch.equal(out[0][1], o[1]) and torch.equal(out[0][2], o[2])
     assert not torch.equal(out[0][0].view(torch.int16), W0.view(torch.int16))
 
 
