@@ -197,10 +197,9 @@ compact_status_t compact_group_bwd(compact_layer_t* const* layers, int count, in
  * one more rounding (the add is done by the TMA unit at the L2, so W makes one
  * trip instead of two); fp32 layers and the SIMT path round W once.
  * workspace: at least r * m * 4 bytes (rounded up to 256).  With
- * compact_workspace_bytes(layer, 0) bytes a bf16 layer whose rank is beyond
- * the 512 columns of P that the one-launch update keeps on chip also has room
- * for P written out next to N, and its product runs on pairs of SMs; with
- * less, P is regenerated tile by tile.  Same W, M, V bit for bit. */
+ * compact_workspace_bytes(layer, 0) bytes a bf16 layer has room for P written
+ * out next to N, and the product P N runs on pairs of SMs like the forward's;
+ * with less, the kernel regenerates P tile by tile.  Same W, M, V bit for bit. */
 compact_status_t compact_adam_update(compact_layer_t* layer,
                                      void* W, int64_t ldw,
                                      const float* Gc, int64_t ldg,
@@ -285,11 +284,11 @@ compact_status_t compact_debug_projection(const compact_layer_t* layer, uint32_t
                                           void* P_dev, void* stream);
 
 /* Selects the kernel family: 0 = automatic (tensor-core kernels for bf16 where
- * the shape allows -- pairs of SMs for the TMA-fed products, a cluster that shares
- * every generated tile of P, the one-launch update --, SIMT otherwise), 1 = force
- * the SIMT kernels, 2 = tensor-core kernels that work one SM at a time: every CTA
- * computes its own tiles and generates its own tiles of P, and the update is the
- * Adam kernel followed by the streaming GEMM (1 and 2 are used by the tests as
+ * the shape allows -- every product on pairs of SMs, with P written out into the
+ * workspace where the call has one; without, a cluster of two CTAs shares every
+ * tile of P it generates --, SIMT otherwise), 1 = force the SIMT kernels,
+ * 2 = tensor-core kernels that work one SM at a time: every CTA computes its
+ * own tiles and generates its own tiles of P (1 and 2 are used by the tests as
  * on-device cross-checks).  Returns the previous value. */
 int compact_set_kernel_family(int family);
 

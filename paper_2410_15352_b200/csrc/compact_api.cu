@@ -14,7 +14,6 @@
 #include "philox.cuh"
 #include "simt_kernels.cuh"
 #include "tc_kernels.cuh"
-#include "update_kernel.cuh"
 #include "gemm2_kernel.cuh"
 
 using namespace compact;
@@ -276,8 +275,8 @@ size_t compact_workspace_bytes(const compact_layer_t* layer, int64_t tokens) {
   size_t need = upd > bwd ? upd : bwd;
   const size_t fwd = compact_fwd_workspace_bytes(layer);
   need = fwd > need ? fwd : need;
-  // layers beyond the one-launch update's panel: N and the expanded P side by side
-  if (layer->cfg.dtype == COMPACT_BF16 && !upd::fused_update_ok(layer->cfg.n, m, r)) {
+  // the update's fastest route: N and the expanded P side by side
+  if (layer->cfg.dtype == COMPACT_BF16) {
     const size_t u2 = g2::g2_update_scratch_bytes(layer->cfg.n, m, r, (int)compact_z_ld(layer));
     need = u2 > need ? u2 : need;
   }
@@ -605,16 +604,13 @@ compact_status_t compact_adam_update(compact_layer_t* L, void* W, int64_t ldw, c
     s = COMPACT_ERR_SHAPE;
     if (g_family.load() != 1) {
       tc::LaunchInfo li{g_family.load() == 2 ? 1 : CFG_CS, st, status_word(L), sched_words(L), &g_launches};
-      // one launch (Adam, resident panel of P, sweep over W) where the rank fits the panel; otherwise the Adam
-      // kernel followed by the streaming GEMM
+      // Two routes with the same bits.  With room for P next to N: the Adam kernel, P written out, and the product on
+      // pairs of SMs.  Without: the Adam kernel followed by the streaming GEMM that regenerates P tile by tile.
       // (the tiles of a sparse projection hold integer counts: its 1/sqrt(s) rides on the step size)
       const ProjectionParams pp = make_pp(L, L->epoch);
       const float step_scale = lr * L->cfg.alpha * pp.inv_sqrt_s;
-      if (g_family.load() == 0 && upd::fused_update_ok(L->cfg.n, L->cfg.m, L->cfg.r))
-        s = upd::fused_update(li, pp, adam_scalars(L, L->step + 1), L->cfg.n, L->cfg.m, L->cfg.r, (T*)W, ldw,
-                              Gc, ldg, M, V, step_scale, workspace, workspace_bytes);
-      else if (g_family.load() == 0 &&
-               workspace_bytes >= g2::g2_update_scratch_bytes(L->cfg.n, L->cfg.m, L->cfg.r, (int)compact_z_ld(L)))
+      if (g_family.load() == 0 &&
+          workspace_bytes >= g2::g2_update_scratch_bytes(L->cfg.n, L->cfg.m, L->cfg.r, (int)compact_z_ld(L)))
         s = g2::g2_update(li, pp, adam_scalars(L, L->step + 1), L->cfg.n, L->cfg.m, L->cfg.r, (int)compact_z_ld(L), (T*)W, ldw,
                           Gc, ldg, M, V, step_scale, workspace, workspace_bytes);
       else

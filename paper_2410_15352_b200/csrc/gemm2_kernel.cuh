@@ -584,9 +584,8 @@ inline compact_status_t g2_forward(const LaunchInfo& li, int G, const G2Layer* L
   return g2_launch(li, prm);
 }
 
-// Algorithm 3 for layers whose rank does not fit the one-launch update's resident panel: Adam moments -> N (bf16, front
-// of the scratch), P written out behind it, then W <- W - scale * P N as one product on pairs of SMs whose epilogue
-// adds the increment to W.  Same N, same entries of P, same order of accumulation and the same roundings as the
+// Algorithm 3: Adam moments -> N (bf16, front of the scratch), P written out behind it, then W <- W - scale * P N as
+// one product on pairs of SMs whose epilogue adds the increment to W.  Same N, same entries of P, same order of accumulation and the same roundings as the
 // streaming update on single SMs (which needs no room for P and remains the route when the scratch is small).
 inline size_t g2_update_scratch_bytes(int n, int m, int r, int zcols) {
   return ((size_t)r * m * sizeof(__nv_bfloat16) + 255) / 256 * 256 + expanded_bytes(n, zcols);

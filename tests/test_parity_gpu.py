@@ -464,66 +464,40 @@ def test_many_layers_on_two_streams_match_one_stream():
     assert len({lay._h.value for lay in layers}) == 300
 
 
-@pytest.mark.parametrize("n,m,r", [
-    (4096, 4096, 512),        # the LLaMA-7B attention shape: 64 jobs, two column ranges per row panel
-    (1000, 1344, 200),        # ragged last row panel, a ragged last column block, rank short of a k-tile
-    (9736, 128, 24),          # more row panels than clusters: a cluster generates a second panel
-    (128, 64, 8),             # one panel, one block: the neighbour CTA has no block of its own
-    (640, 2752, 512),         # full panel, eleven column blocks over several ranges
-])
-def test_one_launch_update_equals_two_kernel_update_bitwise(n, m, r):
-    # The update that keeps a panel of P resident (one launch: Adam, barrier, sweep) and the update made of the
-    # Adam kernel followed by the streaming GEMM produce N, the products and the roundings in the same order.
-    g = torch.Generator().manual_seed(n + m + r)
-    Gc = (torch.randn((r, m), generator=g) * 1e-3).cuda()
-    W0 = (torch.randn((n, m), generator=g) * 0.02).to(torch.bfloat16).cuda()
-    out = []
-    for fam in (0, 2):
-        cb.set_kernel_family(fam)
-        lay = cb.CompactLinear(n, m, r, seed=11, layer_id=3, lr=2e-3, alpha=0.5)
-        W, M, V = W0.clone(), torch.full((r, m), 1e-4, device="cuda"), torch.full((r, m), 1e-7, device="cuda")
-        for _ in range(2):
-            lay.adam_update(W, Gc, M, V, 0)
-        assert lay.status() == cb.OK
-        out.append((W, M, V))
-    cb.set_kernel_family(0)
-    assert torch.equal(out[0][0].view(torch.int16), out[1][0].view(torch.int16))
-    assert torch.equal(out[0][1], out[1][1]) and torch.equal(out[0][2], out[1][2])
-    assert not torch.equal(out[0][0].view(torch.int16), W0.view(torch.int16))
-
-
 @pytest.mark.parametrize("n,m,r,s", [
-    (4000, 1344, 600, 0),      # rank beyond the resident panel; ragged row panel and column block; r not a multiple of 64
-    (2048, 520, 100, 0),       # m not a multiple of 64: the one-launch update does not take it
+    (4096, 4096, 512, 0),      # the LLaMA-7B attention shape
+    (1000, 1344, 200, 0),      # ragged last row tile and column tile, rank short of a k-step
+    (9736, 128, 24, 0),        # many row tiles, half a column tile
+    (128, 64, 8, 0),           # a single tile, mostly padding
+    (4000, 1344, 600, 0),      # r not a multiple of 64
+    (2048, 520, 100, 0),       # m not a multiple of 64: W and N through the unblocked tensor maps
     (11008, 1024, 1376, 0),    # the LLaMA-7B down_proj rank and row count
     (4000, 1344, 600, 8),      # sparse projection: integer counts in scratch, 1 / sqrt(s) on the step size
 ])
-def test_pair_of_sms_update_equals_streaming_update_bitwise(n, m, r, s):
-    # Layers the one-launch update does not take: with room for P in the workspace the product runs on pairs of SMs
-    # from the written-out P; with a workspace that only holds N (and in the single-SM family) the streaming kernel
-    # regenerates P tile by tile.  Same N, same entries of P, same accumulation order, same roundings.
+def test_update_routes_agree_bitwise(n, m, r, s):
+    # With room for P in the workspace (the size compact_workspace_bytes reports) the product P N runs on pairs of
+    # SMs from the written-out P; with the documented minimum (r * m * 4 bytes) -- where that is less -- and in the
+    # single-SM family the streaming kernel regenerates P tile by tile.  Same N, same entries of P, same accumulation
+    # order, same roundings.
     g = torch.Generator().manual_seed(n + m + r)
     Gc = (torch.randn((r, m), generator=g) * 1e-3).cuda()
     W0 = (torch.randn((n, m), generator=g) * 0.02).to(torch.bfloat16).cuda()
+    st = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    small_bytes = -(-r * m * 4 // 256) * 256
     out = []
     for fam, small in ((0, False), (0, True), (2, False)):
         cb.set_kernel_family(fam)
         lay = cb.CompactLinear(n, m, r, seed=11, layer_id=3, lr=2e-3, alpha=0.5, sparse_s=s)
+        ws = torch.empty(small_bytes if small else lay.workspace_bytes(0), dtype=torch.uint8, device="cuda")
+        room_for_p = ws.numel() >= r * m * 2 + n * (-(-lay.ldz // 64) * 64) * 2
         W, M, V = W0.clone(), torch.full((r, m), 1e-4, device="cuda"), torch.full((r, m), 1e-7, device="cuda")
         before = cb.kernel_launch_count()
         for _ in range(2):
-            if small:
-                # the documented minimum: less than N and P side by side
-                ws = torch.empty(-(-r * m * 4 // 256) * 256, dtype=torch.uint8, device="cuda")
-                assert ws.numel() < lay.workspace_bytes(0)
-                st = C.c_void_p(torch.cuda.current_stream().cuda_stream)
-                code = cb.lib().compact_adam_update(lay._h, W.data_ptr(), W.stride(0), Gc.data_ptr(), Gc.stride(0), M.data_ptr(),
-                                                    V.data_ptr(), 0, float("nan"), ws.data_ptr(), ws.numel(), st)
-                assert code == cb.OK
-            else:
-                lay.adam_update(W, Gc, M, V, 0)
+            assert cb.lib().compact_adam_update(lay._h, W.data_ptr(), W.stride(0), Gc.data_ptr(), Gc.stride(0), M.data_ptr(),
+                                                V.data_ptr(), 0, float("nan"), ws.data_ptr(), ws.numel(), st) == cb.OK
         assert lay.status() == cb.OK
-        assert cb.kernel_launch_count() - before == (6 if (fam == 0 and not small) else 4)
+        assert small or room_for_p
+        assert cb.kernel_launch_count() - before == (6 if (fam == 0 and room_for_p) else 4)
         out.append((W, M, V))
     cb.set_kernel_family(0)
     for o in out[1:]:
