@@ -37,6 +37,16 @@ constexpr int G2_BARS_OFF = G2_STAGING_OFF + G2_EPI_WARPS * STAGING_BYTES;
 constexpr int G2_NUM_BARS = 2 * G2_NS + 4;
 constexpr int G2_SMEM_BYTES = 1024 + G2_BARS_OFF + 8 * G2_NUM_BARS + 32;
 static_assert(G2_SMEM_BYTES <= 232448, "shared memory budget");
+// Tile order and the L2.  A round of 74 tiles reads its row blocks of A and its column tiles of B; what the next
+// round reads again should still be in the L2, which holds 126 MB in two halves and behaves, for data that all SMs
+// read, like about half of that.  A problem whose B operand is larger than G2_PANEL_BYTES is walked in column panels
+// of at most that size (row block by row block inside a panel: the panel stays, A streams once per panel); the
+// forward numbers the Z and Y tiles of a row block together (X is read once for both) while every B operand of
+// the run fits G2_ROWS_BYTES.  Measured on 16384 tokens with 48 MB for both: 4096 x 11008 forward 1.242 -> 1.150 ms,
+// 11008 x 4096 backward 1.385 -> 1.283 ms (its launch read 2.7 GB from DRAM for 0.6 GB of operands), 4096 x 11008
+// backward 1.307 -> 1.292; sizes from 24 to 80 MB give the same within 1 %.
+constexpr long long G2_PANEL_BYTES = 48ll << 20;
+constexpr long long G2_ROWS_BYTES = 48ll << 20;
 constexpr int G2_MAXP = 6;      // Y and Z of up to three layers that share their input
 
 struct G2Problem {
@@ -46,6 +56,8 @@ struct G2Problem {
   int a_blocked, b_blocked;    // MN-major operand read through the blocked map (column count a multiple of 64)
   int epi_mode;                // EPI_BF16, EPI_UPDATE_W (C += -scale * acc) or EPI_F32 (3-D map [split][M][N])
   int tile_begin;
+  int panel_cols;              // > 0 (and splits == 1): tiles are numbered panel by panel of this many column tiles, and
+                               // row block by row block inside a panel, so that a panel of B stays in the L2
   float scale;                 // bf16 epilogues: the accumulator is multiplied by this before it is rounded (1: exact)
 };
 
@@ -139,6 +151,19 @@ __device__ __forceinline__ G2Tile g2_decode(const G2Params& prm, int tile) {
     if (i < prm.num_problems && tile >= prm.prob[i].tile_begin) t.prob = i;
   const G2Problem& p = prm.prob[t.prob];
   int local = tile - p.tile_begin;
+  if (p.panel_cols > 0) {
+    const int per_panel = p.tiles_m * p.panel_cols;
+    const int panel = local / per_panel;
+    local -= panel * per_panel;
+    const int pc = min(p.panel_cols, p.tiles_n - panel * p.panel_cols);
+    const int mb = local / pc;
+    t.split = 0;
+    t.m0 = mb * 2 * G2_HALF;
+    t.n0 = (panel * p.panel_cols + (local - mb * pc)) * 2 * G2_HALF;
+    t.k_begin = 0;
+    t.k_end = p.ksteps_total;
+    return t;
+  }
   const int nb = local % p.tiles_n;
   local /= p.tiles_n;
   const int mb = local % p.tiles_m;
@@ -372,6 +397,13 @@ inline void g2_finish(G2Problem& p, int splits_wanted) {
   p.ksteps_per_split = (p.ksteps_total + s - 1) / s;
   p.splits = (p.ksteps_total + p.ksteps_per_split - 1) / p.ksteps_per_split;
   if (p.scale == 0.f) p.scale = 1.f;
+  // A B operand that does not fit the L2 next to the stream of A goes through it panel by panel.
+  p.panel_cols = 0;
+  const size_t b_bytes = (size_t)p.K * (size_t)p.N * sizeof(__nv_bfloat16);
+  if (p.splits == 1 && b_bytes > (size_t)G2_PANEL_BYTES) {
+    const int npanels = (int)((b_bytes + G2_PANEL_BYTES - 1) / G2_PANEL_BYTES);
+    p.panel_cols = (p.tiles_n + npanels - 1) / npanels;
+  }
 }
 
 inline compact_status_t g2_launch(const LaunchInfo& li, G2Params& prm) {
@@ -569,11 +601,9 @@ inline compact_status_t g2_forward(const LaunchInfo& li, int G, const G2Layer* L
     if (!make_map(&prm.tmC[iy], L[g].Y, L[g].m, tokens, L[g].ldy, 64, 32)) return COMPACT_ERR_CUDA;
   }
   // Row block by row block, X is read from DRAM once instead of once per problem -- as long as the B operands
-  // (every W and P of the launch, which each round of tiles walks in full) stay in the 126 MB L2 beside it.
-  // Measured on 16384 tokens: 4096 x (4096 + 512) -2.3 %, 4096 x (11008 + 512) (94 MB) -1.2 %,
-  // 11008 x (4096 + 1408) (121 MB) +2 %.
+  // (every W and P of the run, which each round of tiles walks in full) stay in the L2 beside it.
   // A group of layers whose operands together are too large runs layer after layer, each by rows if it fits.
-  const size_t fits = (size_t)100 << 20;
+  const size_t fits = (size_t)G2_ROWS_BYTES;
   size_t all = 0, largest = 0;
   for (int g = 0; g < G; ++g) {
     const size_t b = (size_t)n * (size_t)(L[g].m + expanded_ld(L[g].zcols)) * sizeof(__nv_bfloat16);

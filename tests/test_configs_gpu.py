@@ -51,6 +51,28 @@ def test_full_size_two_steps(cfg, li):
     assert_parity(errs, dW, dW_tile, "bf16", (cfg, li))
 
 
+@pytest.mark.parametrize("li", [4, 6])
+def test_full_size_tile_orders_same_bits(li):
+    # At the LLaMA-7B MLP shapes the pair-of-SMs launches walk operands larger than the L2 in column panels (and the
+    # forward numbers Z and Y tiles in its own order).  Every tile of every output against the single-SM family,
+    # which numbers its items differently and generates P on chip: all outputs bit for bit, full size.
+    wl = wlm.config5()
+    X, dY = wlm.draw_X(wl, li, 0).cuda(), wlm.draw_dY(wl, li, 0).cuda()
+    out = []
+    for fam in (0, 2):
+        cb.set_kernel_family(fam)
+        gpu, _, W0 = make_pair(wl, li)
+        W = W0.cuda()
+        Y, Z, _ = gpu.forward(X, W)
+        dX, Gc = gpu.backward(dY, Z, W)
+        assert gpu.status() == cb.OK
+        out.append((Y, Z, dX, Gc))
+        del gpu
+    cb.set_kernel_family(0)
+    for a, b in zip(*out):
+        assert torch.equal(a.view(torch.int16) if a.dtype == torch.bfloat16 else a, b.view(torch.int16) if b.dtype == torch.bfloat16 else b)
+
+
 # ---- configs 3 and 4 at their stated step counts and refresh periods -----------------------------------
 # The attention shapes run at the full token count; the wide shapes (whose oracle step costs seconds) at a
 # quarter of it, which leaves every tile shape, the ragged ranks and the schedule as they are.
