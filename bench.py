@@ -256,13 +256,29 @@ class LayerBuffers:
         self.lay.workspace(tokens)
 
 
-# DRAM traffic from the committed ncu captures (profiles/): bytes per algorithmic flop of the forward (Z launch + Y
-# launch) and backward launches of the C5 q_proj layer (compact_gemm_kernel_c5_qproj_full.md: 134.3 + 5.0, 203.0 + 117.8
-# and 401.6 + 159.6 MB for 2 x 618.5 GFLOP), and bytes per algorithmic byte of one update launch whose W does not sit in
-# L2 beforehand (compact_update_kernel_c5_gate_proj.md: 169.6 + 97.4 MB for 293.1 MB).  Scaled to the benchmarked
-# launches by their algorithmic work.
-NCU_GEMM_DRAM_BYTES_PER_FLOP = (134.3e6 + 5.0e6 + 203.0e6 + 117.8e6 + 401.6e6 + 159.6e6) / 1236.95e9
-NCU_UPDATE_DRAM_BYTES_PER_ALG_BYTE = (169.6e6 + 97.4e6) / 293.1e6
+# DRAM traffic from the committed ncu captures (profiles/compact_gemm2_kernel_c5_*.md): dram__bytes_read.sum +
+# dram__bytes_write.sum of all launches of one forward call (expansion of P, product), one backward call (product,
+# reduction of the Gc partials) and one update call (Adam kernel, expansion, product) of the three distinct C5 shapes,
+# every launch from cold caches.  Other shapes are scaled from the q_proj figures by flops (forward, backward) and by
+# algorithmic bytes (update).  The update's reduce-adds leave W dirty in the L2: its write-back happens after the
+# kernel and is not in these figures.
+NCU_DRAM_BYTES_PER_CALL = {
+    (4096, 4096, 512): (397.0e6, 601.7e6, 67.2e6),
+    (4096, 11008, 512): (1370.9e6, 2577.6e6, 209.9e6),
+    (11008, 4096, 1376): (3122.4e6, 1666.6e6, 238.7e6),
+}
+
+
+def ncu_dram_bytes(L, tokens: int, eb: int):
+    """(forward, backward, update) DRAM bytes of one layer's calls, from the captures or scaled from q_proj's."""
+    key = (L.n, L.m, L.r)
+    if key in NCU_DRAM_BYTES_PER_CALL and tokens == 16384:
+        return NCU_DRAM_BYTES_PER_CALL[key]
+    f0, b0, u0 = NCU_DRAM_BYTES_PER_CALL[(4096, 4096, 512)]
+    qn, qm, qr, qt = 4096, 4096, 512, 16384
+    return (f0 * (tokens * L.n * (L.m + L.r)) / (qt * qn * (qm + qr)),
+            b0 * (tokens * L.m * (L.n + L.r)) / (qt * qm * (qn + qr)),
+            u0 * wlm.update_bytes(L.n, L.m, L.r, eb) / wlm.update_bytes(qn, qm, qr, 2))
 
 
 def must_spawn(gpus: int, environ) -> bool:
@@ -426,16 +442,17 @@ def run_ours(args):
     upd_ms = t_upd / nrec
     upd_gbs = upd_bytes / (upd_ms * 1e-3) / 1e9
     gemm_launches = 2 * len(wl.layers)
-    traffic_gemm = NCU_GEMM_DRAM_BYTES_PER_FLOP * gemm_flops / gemm_launches
-    traffic_upd = (NCU_UPDATE_DRAM_BYTES_PER_ALG_BYTE * upd_bytes / len(wl.layers)
-                   if NCU_UPDATE_DRAM_BYTES_PER_ALG_BYTE is not None else None)
-    roofline = {"kernel": "compact_gemm2_kernel + compact_gemm_kernel (the forward and backward calls: Y, dX, Gc on pairs of SMs; Z with its generated operand)", "bound": "tensor",
+    dram = [ncu_dram_bytes(L, tokens, eb) for L in wl.layers]
+    traffic_gemm = sum(d[0] + d[1] for d in dram) / gemm_launches
+    traffic_upd = sum(d[2] for d in dram) / len(wl.layers)
+    roofline = {"kernel": "compact_gemm2_kernel (the forward and backward calls: Z, Y, Gc, dX on pairs of SMs; with them the expansion of P "
+                          "and the reduction of the Gc partials, 2 % of their time)", "bound": "tensor",
                 "achieved": gemm_tflops, "peak": tens_peak, "unit": "TFLOP/s", "frac": gemm_tflops / tens_peak,
                 "peak_kind": f"{peak_kind} bf16 sustained (the kernel is timed inside a long step)",
                 "frac_of_measured_burst": gemm_tflops / tens_burst, "frac_of_nominal_2250": gemm_tflops / NOMINAL_BF16_TFLOPS,
                 "avg_launch_ms": gemm_ms / gemm_launches, "calls_per_step": gemm_launches,
                 "algorithmic_flops_per_launch": gemm_flops / gemm_launches, "traffic": traffic_gemm,
-                "traffic_note": "DRAM bytes per forward or backward call, scaled by flops from the ncu capture of the C5 q_proj calls"}
+                "traffic_note": "DRAM bytes per forward or backward call: the ncu captures of the three C5 shapes, averaged over the step's 14 calls"}
     # each layer's update against the roofline that bounds it: HBM below the ridge n r / (2 n + 10 r) flop/byte, tensor above
     ridge = tens_peak * 1e12 / (hbm_peak * 1e9)
     upd_layers = {}
@@ -448,7 +465,7 @@ def run_ours(args):
         if ent["bound"] == "tensor":
             ent["frac_of_measured_bf16_sustained"] = ent["TFLOP/s"] / tens_peak
         upd_layers[f"{L.name}#{i}"] = ent
-    roofline_update = {"kernel": "compact update launches (Adam moments, regenerated P, W -= lr alpha P N)", "bound": "hbm",
+    roofline_update = {"kernel": "update calls (adam_moments_bf16_kernel, expand_projection_kernel, compact_gemm2_kernel with W -= lr alpha P N in its epilogue)", "bound": "hbm",
                        "achieved": upd_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": upd_gbs / hbm_peak,
                        "peak_kind": f"{peak_kind} copy", "frac_of_nominal_8000": upd_gbs / NOMINAL_HBM_GBS,
                        "avg_launch_ms": upd_ms / len(wl.layers), "algorithmic_bytes_per_launch": upd_bytes / len(wl.layers),

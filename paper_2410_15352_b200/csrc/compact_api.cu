@@ -539,6 +539,11 @@ compact_status_t compact_group_bwd(compact_layer_t* const* layers, int count, in
   compact_status_t s = check_device(layers[0], stream);
   if (s != COMPACT_OK) return s;
   tc::LaunchInfo li{1, (cudaStream_t)stream, status_word(layers[0]), sched_words(layers[0]), &g_launches};
+  // on pairs of SMs (family 2: on single SMs, the cross-check); same bits
+  if (g_family.load() == 0) {
+    s = g2::g2_backward_group(li, count, gl, tokens, n, (T*)dX, lddx, accumulate, workspace, workspace_bytes);
+    if (s != COMPACT_ERR_SHAPE) return s;
+  }
   return tc::backward_group(li, count, gl, tokens, n, (T*)dX, lddx, accumulate, workspace, workspace_bytes);
 }
 

@@ -55,6 +55,9 @@ struct G2Problem {
   int a_mode, b_mode;          // TMA_KMAJOR or TMA_MNMAJOR
   int a_blocked, b_blocked;    // MN-major operand read through the blocked map (column count a multiple of 64)
   int epi_mode;                // EPI_BF16, EPI_UPDATE_W (C += -scale * acc) or EPI_F32 (3-D map [split][M][N])
+  int map_base;                // index of the problem's tensor maps (A and B: + segment; C: this one)
+  int nseg;                    // > 1: K runs over this many operand pairs laid end to end (dX of a group of layers)
+  int seg_begin[4];            // first k-step of each segment
   int tile_begin;
   int panel_cols;              // > 0 (and splits == 1): tiles are numbered panel by panel of this many column tiles, and
                                // row block by row block inside a panel, so that a panel of B stays in the L2
@@ -229,27 +232,34 @@ __global__ void __launch_bounds__(G2_THREADS, 1) compact_gemm2_kernel(const __gr
     for (int tile = pair_id; tile < prm.total_tiles && ok; tile += npairs) {
       const G2Tile t = g2_decode(prm, tile);
       const G2Problem& p = prm.prob[t.prob];
-      const CUtensorMap* mapA = &prm.tmA[t.prob];
-      const CUtensorMap* mapB = &prm.tmB[t.prob];
       const int m0 = t.m0 + (int)crank * G2_HALF, n0 = t.n0 + (int)crank * G2_HALF;
+      // everything the k loop needs sits in registers before it starts: the loop is one wait and two copies
+      const bool multi = p.nseg > 1;
+      const int a_mode = p.a_mode, b_mode = p.b_mode, a_blocked = p.a_blocked, b_blocked = p.b_blocked;
+      const int seg1 = multi ? p.seg_begin[1] : 0x7fffffff, seg2 = multi ? p.seg_begin[2] : 0x7fffffff;
+      const CUtensorMap* const mapA0 = &prm.tmA[p.map_base];
+      const CUtensorMap* const mapB0 = &prm.tmB[p.map_base];
       for (int ks = t.k_begin; ks < t.k_end; ++ks, ring_next(r, G2_NS)) {
         if (!(ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(r.s), r.ph ^ 1u, abort_flag, prm.status)))) break;
         if (elect_one()) {
-          const int k0 = ks * BK;
+          const int seg = (ks >= seg1) + (ks >= seg2);
+          const CUtensorMap* mapA = mapA0 + seg;
+          const CUtensorMap* mapB = mapB0 + seg;
+          const int k0 = (ks - (seg == 0 ? 0 : (seg == 1 ? seg1 : seg2))) * BK;
           const uint32_t fb = leader_bars + 8u * r.s;                      // the leader's full barrier of this stage
           if (leader) mbar_arrive_expect_tx(full_bar(r.s), 2 * G2_STAGE_BYTES);
           const uint32_t dstA = smem_base + (uint32_t)r.s * G2_STAGE_BYTES, dstB = dstA + G2_A_BYTES;
-          if (p.a_mode == TMA_KMAJOR) {
+          if (a_mode == TMA_KMAJOR) {
             tma2_load_2d(dstA, mapA, fb, k0, m0);
-          } else if (p.a_blocked) {
+          } else if (a_blocked) {
             tma2_load_3d(dstA, mapA, fb, 0, k0, m0 >> 6);
           } else {
             tma2_load_2d(dstA, mapA, fb, m0, k0);
             tma2_load_2d(dstA + 8192, mapA, fb, m0 + 64, k0);
           }
-          if (p.b_mode == TMA_KMAJOR) {
+          if (b_mode == TMA_KMAJOR) {
             tma2_load_2d(dstB, mapB, fb, k0, n0);
-          } else if (p.b_blocked) {
+          } else if (b_blocked) {
             tma2_load_3d(dstB, mapB, fb, 0, k0, n0 >> 6);
           } else {
             tma2_load_2d(dstB, mapB, fb, n0, k0);
@@ -315,19 +325,20 @@ __global__ void __launch_bounds__(G2_THREADS, 1) compact_gemm2_kernel(const __gr
     for (int tile = pair_id; tile < prm.total_tiles && ok; tile += npairs) {
       const G2Tile t = g2_decode(prm, tile);
       const G2Problem& p = prm.prob[t.prob];
-      const CUtensorMap* mapC = &prm.tmC[t.prob];
+      const CUtensorMap* mapC = &prm.tmC[p.map_base];
       if (!(ok = mbar_wait(tfull_bar(slot), slot_phase, abort_flag, prm.status))) break;
       tc_fence_after();
       const int row0 = t.m0 + (int)crank * G2_HALF + q * 32;
       const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)slot * 256;
-      const int cw = p.epi_mode == EPI_F32 ? 32 : 64;
-      for (int ci = eset; ci < 256 / cw && row0 < p.M; ci += 2) {
+      const int epi_mode = p.epi_mode, pM = p.M, pN = p.N;
+      const float sc = epi_mode == EPI_UPDATE_W ? -p.scale : p.scale;
+      const int cw = epi_mode == EPI_F32 ? 32 : 64;
+      for (int ci = eset; ci < 256 / cw && row0 < pM; ci += 2) {
         const int col = t.n0 + ci * cw;
-        if (col >= p.N) break;
-        if (p.epi_mode == EPI_BF16 || p.epi_mode == EPI_UPDATE_W) {
+        if (col >= pN) break;
+        if (epi_mode == EPI_BF16 || epi_mode == EPI_UPDATE_W) {
           // The update stages -(eta alpha) (P N) and lets the TMA unit add it to W (Algorithm 3 line 9).
           uint32_t o[32];
-          const float sc = p.epi_mode == EPI_UPDATE_W ? -p.scale : p.scale;
 #pragma unroll
           for (int h = 0; h < 2; ++h) {
             uint32_t v[32];
@@ -344,7 +355,7 @@ __global__ void __launch_bounds__(G2_THREADS, 1) compact_gemm2_kernel(const __gr
           fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) {
-            if (p.epi_mode == EPI_UPDATE_W) tma_reduce_add_2d(mapC, stg, col, row0);
+            if (epi_mode == EPI_UPDATE_W) tma_reduce_add_2d(mapC, stg, col, row0);
             else tma_store_2d(mapC, stg, col, row0);
             tma_store_commit();
           }
@@ -403,6 +414,11 @@ inline void g2_finish(G2Problem& p, int splits_wanted) {
   if (p.splits == 1 && b_bytes > (size_t)G2_PANEL_BYTES) {
     const int npanels = (int)((b_bytes + G2_PANEL_BYTES - 1) / G2_PANEL_BYTES);
     p.panel_cols = (p.tiles_n + npanels - 1) / npanels;
+    // never narrower than a round of tiles is tall (74 tiles = 9 x 8): with a long K even such a panel exceeds the
+    // L2, and a narrower one only streams A more often (dX of the gate/up group, K = 22016: 2.67 ms with panels of
+    // four column tiles against 2.56 without panels)
+    if (p.panel_cols < 8) p.panel_cols = 8;
+    if (p.panel_cols >= p.tiles_n) p.panel_cols = 0;
   }
 }
 
@@ -416,6 +432,10 @@ inline compact_status_t g2_launch(const LaunchInfo& li, G2Params& prm) {
       return COMPACT_ERR_CUDA;
     }
     attr_set[dev].store(true, std::memory_order_release);
+  }
+  for (int i = 0; i < prm.num_problems; ++i) {
+    G2Problem& p = prm.prob[i];
+    if (p.nseg < 1) { p.nseg = 1; p.map_base = i; }      // a plain problem: its own maps, one segment
   }
   int t = 0;
   if (prm.by_rows) {
@@ -652,7 +672,7 @@ inline compact_status_t g2_update(const LaunchInfo& li, const ProjectionParams& 
   return g2_launch(li, prm);
 }
 
-// Algorithm 2: problem 0 = Gc = Z^T dY (both operands MN-major, split over tokens), problem 1 = dX = dY W^T.
+// Algorithm 2: dX = dY W^T, and Gc = Z^T dY (both operands MN-major, split over tokens).
 inline compact_status_t g2_backward(const LaunchInfo& li, int64_t tokens, int n, int m, int r, int zcols,
                                     const __nv_bfloat16* dY, int64_t lddy, const __nv_bfloat16* Z, int64_t ldz,
                                     const __nv_bfloat16* W, int64_t ldw, __nv_bfloat16* dX, int64_t lddx, float* Gc,
@@ -665,29 +685,31 @@ inline compact_status_t g2_backward(const LaunchInfo& li, int64_t tokens, int n,
   const int splits = plan_gc_splits(tokens, r, m);
   const bool staged = splits > 1 || accumulate;
   if (staged && workspace_bytes < (size_t)splits * r * m * sizeof(float)) return COMPACT_ERR_WORKSPACE;
-  G2Problem& pg = prm.prob[0];
+  // dX first, Gc after: a launch that ends on the shorter tiles has the shorter tail (0.3-0.5 % on the backward)
+  const int ig = dX ? 1 : 0, ix = 1 - ig;
+  G2Problem& pg = prm.prob[ig];
   pg.M = r; pg.N = m; pg.K = (int)tokens;
   pg.a_mode = TMA_MNMAJOR; pg.b_mode = TMA_MNMAJOR; pg.epi_mode = EPI_F32;
   pg.a_blocked = zcols % 64 == 0;
   pg.b_blocked = m % 64 == 0;
   g2_finish(pg, splits);
   if (staged) {
-    if (!make_map_f32_3d(&prm.tmC[0], workspace, m, r, pg.splits, m, (int64_t)r * m)) return COMPACT_ERR_CUDA;
+    if (!make_map_f32_3d(&prm.tmC[ig], workspace, m, r, pg.splits, m, (int64_t)r * m)) return COMPACT_ERR_CUDA;
   } else {
-    if (!make_map_f32_3d(&prm.tmC[0], Gc, m, r, 1, ldg, (int64_t)r * ldg)) return COMPACT_ERR_CUDA;
+    if (!make_map_f32_3d(&prm.tmC[ig], Gc, m, r, 1, ldg, (int64_t)r * ldg)) return COMPACT_ERR_CUDA;
   }
-  if (pg.a_blocked ? !make_map_blocked(&prm.tmA[0], Z, zcols, tokens, ldz, BK, G2_HALF / 64) : !make_map(&prm.tmA[0], Z, zcols, tokens, ldz, 64, BK))
+  if (pg.a_blocked ? !make_map_blocked(&prm.tmA[ig], Z, zcols, tokens, ldz, BK, G2_HALF / 64) : !make_map(&prm.tmA[ig], Z, zcols, tokens, ldz, 64, BK))
     return COMPACT_ERR_CUDA;
-  if (pg.b_blocked ? !make_map_blocked(&prm.tmB[0], dY, m, tokens, lddy, BK, G2_HALF / 64) : !make_map(&prm.tmB[0], dY, m, tokens, lddy, 64, BK))
+  if (pg.b_blocked ? !make_map_blocked(&prm.tmB[ig], dY, m, tokens, lddy, BK, G2_HALF / 64) : !make_map(&prm.tmB[ig], dY, m, tokens, lddy, 64, BK))
     return COMPACT_ERR_CUDA;
   if (dX) {
-    G2Problem& px = prm.prob[1];
+    G2Problem& px = prm.prob[ix];
     px.M = (int)tokens; px.N = n; px.K = m;
     px.a_mode = TMA_KMAJOR; px.b_mode = TMA_KMAJOR; px.epi_mode = EPI_BF16;
     g2_finish(px, 1);
-    if (!make_map(&prm.tmA[1], dY, m, tokens, lddy, BK, G2_HALF)) return COMPACT_ERR_CUDA;
-    if (!make_map(&prm.tmB[1], W, m, n, ldw, BK, G2_HALF)) return COMPACT_ERR_CUDA;
-    if (!make_map(&prm.tmC[1], dX, n, tokens, lddx, 64, 32)) return COMPACT_ERR_CUDA;
+    if (!make_map(&prm.tmA[ix], dY, m, tokens, lddy, BK, G2_HALF)) return COMPACT_ERR_CUDA;
+    if (!make_map(&prm.tmB[ix], W, m, n, ldw, BK, G2_HALF)) return COMPACT_ERR_CUDA;
+    if (!make_map(&prm.tmC[ix], dX, n, tokens, lddx, 64, 32)) return COMPACT_ERR_CUDA;
   }
   compact_status_t s = g2_launch(li, prm);
   if (s != COMPACT_OK) return s;
@@ -695,6 +717,87 @@ inline compact_status_t g2_backward(const LaunchInfo& li, int64_t tokens, int n,
     const long long cnt = (long long)r * (m / 4);
     reduce_partials_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, li.stream>>>(
         (const float*)workspace, (long long)r * m, pg.splits, Gc, ldg, r, m, accumulate);
+    (*li.launches)++;
+    if (cudaGetLastError() != cudaSuccess) return COMPACT_ERR_CUDA;
+  }
+  return COMPACT_OK;
+}
+
+// Algorithm 2 for G layers that share their input: dX = sum_g dY_g W_g^T is ONE problem whose K runs over the
+// layers (segment g reads dY_g and W_g), so the input gradient accumulates in the tensor cores instead of in G
+// tensors added afterwards; the Gc_g are G more problems of the same launch, each split over tokens.
+inline compact_status_t g2_backward_group(const LaunchInfo& li, int G, const GroupLayer* L, int64_t tokens, int n,
+                                          __nv_bfloat16* dX, int64_t lddx, int accumulate, void* workspace,
+                                          size_t workspace_bytes) {
+  if (G < 1 || G > MAXG || 2 * G > G2_MAXP) return COMPACT_ERR_INVALID_ARG;
+  if (!li.status) return COMPACT_ERR_CUDA;
+  for (int g = 0; g < G; ++g)
+    if (!tc_shape_ok(tokens, n, L[g].m)) return COMPACT_ERR_SHAPE;
+  G2Params prm;
+  memset(&prm, 0, sizeof(prm));
+  int np = 0, slot = 0, dx_ksteps = 0;
+  for (int g = 0; g < G; ++g) dx_ksteps += (L[g].m + BK - 1) / BK;
+  // dX first: its tiles are the long ones (K runs over all layers), and the launch should end on short ones
+  if (dX) {
+    G2Problem& px = prm.prob[np++];
+    px.M = (int)tokens; px.N = n; px.K = dx_ksteps * BK;
+    px.a_mode = TMA_KMAJOR; px.b_mode = TMA_KMAJOR; px.epi_mode = EPI_BF16;
+    g2_finish(px, 1);
+    px.nseg = G; px.map_base = slot;
+    int kb = 0;
+    for (int g = 0; g < 4; ++g) {
+      px.seg_begin[g] = kb;
+      if (g < G) kb += (L[g].m + BK - 1) / BK;
+    }
+    for (int g = 0; g < G; ++g) {
+      if (!make_map(&prm.tmA[slot + g], L[g].dY, L[g].m, tokens, L[g].lddy, BK, G2_HALF)) return COMPACT_ERR_CUDA;
+      if (!make_map(&prm.tmB[slot + g], L[g].W, L[g].m, n, L[g].ldw, BK, G2_HALF)) return COMPACT_ERR_CUDA;
+    }
+    if (!make_map(&prm.tmC[slot], dX, n, tokens, lddx, 64, 32)) return COMPACT_ERR_CUDA;
+    slot += G;
+  }
+  size_t ws_off = 0;
+  int splits[MAXG];
+  bool staged[MAXG];
+  size_t part_off[MAXG];
+  for (int g = 0; g < G; ++g) {
+    const int r = L[g].r, m = L[g].m;
+    splits[g] = plan_gc_splits(tokens, r, m, dx_ksteps);
+    staged[g] = splits[g] > 1 || accumulate;
+    part_off[g] = ws_off;
+    ws_off += (size_t)splits[g] * r * m * sizeof(float);
+    if (staged[g] && workspace_bytes < ws_off) return COMPACT_ERR_WORKSPACE;
+    G2Problem& pg = prm.prob[np++];
+    pg.M = r; pg.N = m; pg.K = (int)tokens;
+    pg.a_mode = TMA_MNMAJOR; pg.b_mode = TMA_MNMAJOR; pg.epi_mode = EPI_F32;
+    pg.a_blocked = L[g].zcols % 64 == 0;
+    pg.b_blocked = m % 64 == 0;
+    g2_finish(pg, splits[g]);
+    splits[g] = pg.splits;
+    pg.nseg = 1; pg.map_base = slot;
+    float* part = (float*)((char*)workspace + part_off[g]);
+    if (staged[g]) {
+      if (!make_map_f32_3d(&prm.tmC[slot], part, m, r, pg.splits, m, (int64_t)r * m)) return COMPACT_ERR_CUDA;
+    } else {
+      if (!make_map_f32_3d(&prm.tmC[slot], L[g].Gc, m, r, 1, L[g].ldg, (int64_t)r * L[g].ldg)) return COMPACT_ERR_CUDA;
+    }
+    if (pg.a_blocked ? !make_map_blocked(&prm.tmA[slot], L[g].Z, L[g].zcols, tokens, L[g].ldz, BK, G2_HALF / 64)
+                     : !make_map(&prm.tmA[slot], L[g].Z, L[g].zcols, tokens, L[g].ldz, 64, BK))
+      return COMPACT_ERR_CUDA;
+    if (pg.b_blocked ? !make_map_blocked(&prm.tmB[slot], L[g].dY, m, tokens, L[g].lddy, BK, G2_HALF / 64)
+                     : !make_map(&prm.tmB[slot], L[g].dY, m, tokens, L[g].lddy, 64, BK))
+      return COMPACT_ERR_CUDA;
+    ++slot;
+  }
+  prm.num_problems = np;
+  compact_status_t s = g2_launch(li, prm);
+  if (s != COMPACT_OK) return s;
+  for (int g = 0; g < G; ++g) {
+    if (!staged[g]) continue;
+    const int r = L[g].r, m = L[g].m;
+    const long long cnt = (long long)r * (m / 4);
+    reduce_partials_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, li.stream>>>(
+        (const float*)((char*)workspace + part_off[g]), (long long)r * m, splits[g], L[g].Gc, L[g].ldg, r, m, accumulate);
     (*li.launches)++;
     if (cudaGetLastError() != cudaSuccess) return COMPACT_ERR_CUDA;
   }

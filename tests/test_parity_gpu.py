@@ -354,6 +354,34 @@ def test_repeated_launches_bitwise_stable(tokens, n, m, r):
     assert gpu.status() == cb.OK
 
 
+@pytest.mark.parametrize("tokens,n,shapes", [
+    (1100, 320, [(512, 72), (520, 72), (1096, 40)]),      # segment lengths 512, 520 (ragged k-step), 1096
+    (700, 4096, [(11008, 512), (11008, 512)]),            # gate/up of LLaMA-7B: operands beyond the L2, column panels
+    (300, 192, [(200, 24)]),
+])
+def test_group_calls_on_pairs_of_sms_and_on_single_sms_same_bits(tokens, n, shapes):
+    # The group forward (Z and Y of every layer in one launch) and the group backward (dX with K running over the
+    # layers, every Gc) give the same bits on pairs of SMs, with P written out, as on single SMs with P generated
+    # on chip.
+    wl = wlm.Workload("grp2", 96, "bf16", tokens, [wlm.LayerShape(f"l{g}", n, m, r) for g, (m, r) in enumerate(shapes)],
+                      x_scale_inv_sqrt_n=True)
+    X = wlm.draw_X(wl, 0, 0).cuda()
+    dYs = [wlm.draw_dY(wl, g, 0).cuda() for g in range(len(shapes))]
+    out = []
+    for fam in (0, 2):
+        cb.set_kernel_family(fam)
+        pairs = [make_pair(wl, g) for g in range(len(shapes))]
+        grp = cb.CompactGroup([p[0] for p in pairs])
+        Ws = [p[2].cuda() for p in pairs]
+        Ys, Zs, _ = grp.forward(X, Ws)
+        dX, Gcs = grp.backward(dYs, Zs, Ws)
+        assert all(p[0].status() == cb.OK for p in pairs)
+        out.append(Ys + Zs + [dX] + Gcs)
+    cb.set_kernel_family(0)
+    for a, b in zip(*out):
+        assert torch.equal(a.view(torch.int16) if a.dtype == torch.bfloat16 else a, b.view(torch.int16) if b.dtype == torch.bfloat16 else b)
+
+
 def test_group_of_four_runs_layer_by_layer_and_empty_group_call():
     # more than three layers (or mixed seeds, fp32, the SIMT family) take the layer-by-layer route with the same results
     tokens, n = 260, 128
