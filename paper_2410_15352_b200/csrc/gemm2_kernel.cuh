@@ -509,13 +509,24 @@ inline compact_status_t g2_forward_y(const LaunchInfo& li, int64_t tokens, int n
 inline int64_t expanded_ld(int zcols) { return ((int64_t)zcols + 63) / 64 * 64; }
 inline size_t expanded_bytes(int n, int zcols) { return (size_t)n * (size_t)expanded_ld(zcols) * sizeof(__nv_bfloat16); }
 
+struct ExpandArgs {
+  PhiloxKey key;
+  uint32_t layer_hi, layer_lo, epoch;
+  int n, r, sparse_s, groups;      // groups: eight-entry groups per row of the scratch (its pitch / 8)
+  float neg2ln2_over_r;
+  __nv_bfloat16* P;
+};
+
 // Gaussian projection: a thread writes eight consecutive entries of a row (one Philox call); columns from r to
-// the pitch are zeros.
-__global__ void __launch_bounds__(256) expand_projection_kernel(PhiloxKey key, uint32_t layer_hi, uint32_t layer_lo, uint32_t epoch,
-                                                                int n, int r, float neg2ln2_over_r, int groups,
-                                                                __nv_bfloat16* __restrict__ P) {
+// the pitch are zeros.  This is block `block` of `nblocks` blocks of 256 threads.
+__device__ __forceinline__ void expand_gaussian_blocks(const ExpandArgs& a, int block, int nblocks) {
+  const PhiloxKey& key = a.key;
+  const uint32_t layer_hi = a.layer_hi, layer_lo = a.layer_lo, epoch = a.epoch;
+  const int n = a.n, r = a.r, groups = a.groups;
+  const float neg2ln2_over_r = a.neg2ln2_over_r;
+  __nv_bfloat16* __restrict__ P = a.P;
   const long long total = (long long)n * groups;
-  for (long long task = (long long)blockIdx.x * blockDim.x + threadIdx.x; task < total; task += (long long)gridDim.x * blockDim.x) {
+  for (long long task = (long long)block * 256 + threadIdx.x; task < total; task += (long long)nblocks * 256) {
     const int i = (int)(task / groups), g = (int)(task - (long long)i * groups);
     const uint4 val = g * 8 < r ? projection8_bf16(key, layer_hi, layer_lo, epoch, n, r, neg2ln2_over_r, i, g * 8)
                                 : make_uint4(0u, 0u, 0u, 0u);
@@ -526,11 +537,14 @@ __global__ void __launch_bounds__(256) expand_projection_kernel(PhiloxKey key, u
 // Sparse projection: the integer counts (the product's epilogue applies 1 / sqrt(s)).  A warp owns a row: it
 // clears it, then lane 0 adds the signs of the row's terms one after another, so that terms that hash to the
 // same column add without a race.
-__global__ void __launch_bounds__(256) expand_sparse_kernel(PhiloxKey key, uint32_t layer_hi, uint32_t layer_lo, uint32_t epoch,
-                                                            int n, int r, int s, int groups, __nv_bfloat16* __restrict__ P) {
+__device__ __forceinline__ void expand_sparse_blocks(const ExpandArgs& a, int block, int nblocks) {
+  const PhiloxKey& key = a.key;
+  const uint32_t layer_hi = a.layer_hi, layer_lo = a.layer_lo, epoch = a.epoch;
+  const int n = a.n, r = a.r, s = a.sparse_s, groups = a.groups;
+  __nv_bfloat16* __restrict__ P = a.P;
   const int lane = threadIdx.x & 31;
-  const int warps = (int)((gridDim.x * blockDim.x) >> 5);
-  for (int i = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5); i < n; i += warps) {
+  const int warps = nblocks * 8;
+  for (int i = block * 8 + (int)(threadIdx.x >> 5); i < n; i += warps) {
     __nv_bfloat16* row = P + (long long)i * groups * 8;
     for (int g = lane; g < groups; g += 32) reinterpret_cast<uint4*>(row)[g] = make_uint4(0u, 0u, 0u, 0u);
     __syncwarp();
@@ -551,18 +565,45 @@ __global__ void __launch_bounds__(256) expand_sparse_kernel(PhiloxKey key, uint3
   }
 }
 
+__global__ void __launch_bounds__(256) expand_projection_kernel(const __grid_constant__ ExpandArgs a) {
+  if (a.sparse_s > 0) expand_sparse_blocks(a, (int)blockIdx.x, (int)gridDim.x);
+  else expand_gaussian_blocks(a, (int)blockIdx.x, (int)gridDim.x);
+}
+
+// The update's two preparations in one launch: Algorithm 3 lines 1-5 (moments in place, N in bf16) and P written out.
+// Neither reads what the other writes; the Adam blocks are bound by memory, the expansion by instruction issue, so
+// their blocks alternate and the two run side by side.
+__global__ void __launch_bounds__(256) adam_and_expand_kernel(const float* __restrict__ Gc, long long ldg, float* __restrict__ Mo,
+                                                              float* __restrict__ Vo, __nv_bfloat16* __restrict__ Nout, int r, int m,
+                                                              const __grid_constant__ simt::AdamScalars as, int adam_blocks,
+                                                              const __grid_constant__ ExpandArgs a) {
+  const int b = (int)blockIdx.x, expand_blocks = (int)gridDim.x - adam_blocks;
+  const int paired = 2 * (adam_blocks < expand_blocks ? adam_blocks : expand_blocks);
+  bool is_adam;
+  int idx;
+  if (b < paired) { is_adam = (b & 1) == 0; idx = b >> 1; }
+  else { is_adam = adam_blocks > expand_blocks; idx = b - paired / 2; }
+  if (is_adam) adam_moments_bf16_at((long long)idx * 256 + threadIdx.x, Gc, ldg, Mo, Vo, Nout, r, m, as);
+  else if (a.sparse_s > 0) expand_sparse_blocks(a, idx, expand_blocks);
+  else expand_gaussian_blocks(a, idx, expand_blocks);
+}
+
+inline ExpandArgs make_expand_args(const ProjectionParams& pp, int zcols, __nv_bfloat16* P) {
+  ExpandArgs a;
+  a.key = pp.key; a.layer_hi = pp.layer_hi; a.layer_lo = pp.layer_lo; a.epoch = pp.epoch;
+  a.n = pp.n; a.r = pp.r; a.sparse_s = pp.sparse_s; a.groups = (int)(expanded_ld(zcols) / 8);
+  a.neg2ln2_over_r = pp.neg2ln2_over_r; a.P = P;
+  return a;
+}
+inline unsigned expand_blocks_for(const ExpandArgs& a) {
+  const long long threads = a.sparse_s > 0 ? (long long)a.n * 32 : (long long)a.n * a.groups;
+  const long long blocks = (threads + 255) / 256;
+  return (unsigned)(blocks < 8 * NUM_SMS ? blocks : 8 * NUM_SMS);
+}
+
 inline compact_status_t expand_projection(const LaunchInfo& li, const ProjectionParams& pp, int zcols, __nv_bfloat16* P) {
-  const int groups = (int)(expanded_ld(zcols) / 8);
-  if (pp.sparse_s > 0) {
-    const long long threads = (long long)pp.n * 32;
-    const unsigned blocks = (unsigned)((threads + 255) / 256 < 8 * NUM_SMS ? (threads + 255) / 256 : 8 * NUM_SMS);
-    expand_sparse_kernel<<<blocks, 256, 0, li.stream>>>(pp.key, pp.layer_hi, pp.layer_lo, pp.epoch, pp.n, pp.r, pp.sparse_s, groups, P);
-  } else {
-    const long long tasks = (long long)pp.n * groups;
-    const unsigned blocks = (unsigned)((tasks + 255) / 256 < 8 * NUM_SMS ? (tasks + 255) / 256 : 8 * NUM_SMS);
-    expand_projection_kernel<<<blocks, 256, 0, li.stream>>>(pp.key, pp.layer_hi, pp.layer_lo, pp.epoch, pp.n, pp.r, pp.neg2ln2_over_r,
-                                                            groups, P);
-  }
+  const ExpandArgs a = make_expand_args(pp, zcols, P);
+  expand_projection_kernel<<<expand_blocks_for(a), 256, 0, li.stream>>>(a);
   (*li.launches)++;
   return cudaGetLastError() == cudaSuccess ? COMPACT_OK : COMPACT_ERR_CUDA;
 }
@@ -650,11 +691,11 @@ inline compact_status_t g2_update(const LaunchInfo& li, const ProjectionParams& 
   __nv_bfloat16* Nbuf = (__nv_bfloat16*)workspace;
   __nv_bfloat16* P = (__nv_bfloat16*)((char*)workspace + ((size_t)r * m * sizeof(__nv_bfloat16) + 255) / 256 * 256);
   const long long cnt = (long long)r * (m / 4);
-  adam_moments_bf16_kernel<<<(unsigned)((cnt + 255) / 256), 256, 0, li.stream>>>(Gc, ldg, M, V, Nbuf, r, m, as);
+  const unsigned adam_blocks = (unsigned)((cnt + 255) / 256);
+  const ExpandArgs ea = make_expand_args(pp, zcols, P);
+  adam_and_expand_kernel<<<adam_blocks + expand_blocks_for(ea), 256, 0, li.stream>>>(Gc, ldg, M, V, Nbuf, r, m, as, (int)adam_blocks, ea);
   (*li.launches)++;
   if (cudaGetLastError() != cudaSuccess) return COMPACT_ERR_CUDA;
-  compact_status_t s = expand_projection(li, pp, zcols, P);
-  if (s != COMPACT_OK) return s;
   const int64_t ldp = expanded_ld(zcols);
   G2Params prm;
   memset(&prm, 0, sizeof(prm));

@@ -1060,11 +1060,11 @@ __global__ void __launch_bounds__(THREADS_GEN, 1) compact_gemm_kernel(const __gr
 // Element-wise kernels around the GEMMs
 // --------------------------------------------------------------------------------------
 // Algorithm 3 lines 1-5: moments in place, N rounded to bf16 into scratch (pitch m).
-__global__ void adam_moments_bf16_kernel(const float* __restrict__ Gc, long long ldg, float* __restrict__ Mo,
-                                         float* __restrict__ Vo, __nv_bfloat16* __restrict__ Nout, int r, int m,
-                                         simt::AdamScalars s) {
+__device__ __forceinline__ void adam_moments_bf16_at(long long idx, const float* __restrict__ Gc, long long ldg,
+                                                     float* __restrict__ Mo, float* __restrict__ Vo,
+                                                     __nv_bfloat16* __restrict__ Nout, int r, int m,
+                                                     const simt::AdamScalars& s) {
   const int m4 = m >> 2;
-  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (long long)r * m4) return;
   const int j = (int)(idx / m4), c = (int)(idx % m4) * 4;
   const long long off = (long long)j * ldg + c;
@@ -1087,6 +1087,11 @@ __global__ void adam_moments_bf16_kernel(const float* __restrict__ Gc, long long
   const float n3 = (mm.w * s.inv_bias1) / (sqrtf(vv.w * s.inv_bias2) + s.eps);
   uint2 o = make_uint2(pack_bf16x2(n0, n1), pack_bf16x2(n2, n3));
   *reinterpret_cast<uint2*>(Nout + (long long)j * m + c) = o;
+}
+__global__ void adam_moments_bf16_kernel(const float* __restrict__ Gc, long long ldg, float* __restrict__ Mo,
+                                         float* __restrict__ Vo, __nv_bfloat16* __restrict__ Nout, int r, int m,
+                                         simt::AdamScalars s) {
+  adam_moments_bf16_at((long long)blockIdx.x * blockDim.x + threadIdx.x, Gc, ldg, Mo, Vo, Nout, r, m, s);
 }
 
 // Deterministic reduction of the split-K partials of Gc, in split order.

@@ -516,8 +516,9 @@ def test_update_routes_agree_bitwise(n, m, r, s):
     for fam, small in ((0, False), (0, True), (2, False)):
         cb.set_kernel_family(fam)
         lay = cb.CompactLinear(n, m, r, seed=11, layer_id=3, lr=2e-3, alpha=0.5, sparse_s=s)
-        ws = torch.empty(small_bytes if small else lay.workspace_bytes(0), dtype=torch.uint8, device="cuda")
-        room_for_p = ws.numel() >= r * m * 2 + n * (-(-lay.ldz // 64) * 64) * 2
+        ws = torch.full((small_bytes if small else lay.workspace_bytes(0),), 0x5A, dtype=torch.uint8, device="cuda")
+        n_bytes = -(-r * m * 2 // 256) * 256                      # N in bf16 at the front; P, if written out, behind it
+        room_for_p = ws.numel() >= n_bytes + n * (-(-lay.ldz // 64) * 64) * 2
         W, M, V = W0.clone(), torch.full((r, m), 1e-4, device="cuda"), torch.full((r, m), 1e-7, device="cuda")
         before = cb.kernel_launch_count()
         for _ in range(2):
@@ -525,7 +526,9 @@ def test_update_routes_agree_bitwise(n, m, r, s):
                                                 V.data_ptr(), 0, float("nan"), ws.data_ptr(), ws.numel(), st) == cb.OK
         assert lay.status() == cb.OK
         assert small or room_for_p
-        assert cb.kernel_launch_count() - before == (6 if (fam == 0 and room_for_p) else 4)
+        assert cb.kernel_launch_count() - before == 4             # per update: Adam (with the expansion), product
+        wrote_p = bool((ws[n_bytes:n_bytes + 4096] != 0x5A).any())
+        assert wrote_p == (fam == 0 and room_for_p)               # which route ran
         out.append((W, M, V))
     cb.set_kernel_family(0)
     for o in out[1:]:
