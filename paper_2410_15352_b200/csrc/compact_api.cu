@@ -575,8 +575,12 @@ compact_status_t compact_linear_bwd_recompute(compact_layer_t* L, int64_t tokens
       s = COMPACT_ERR_SHAPE;
       if (g_family.load() != 1) {
         tc::LaunchInfo li{g_family.load() == 2 ? 1 : CFG_CS, st, status_word(L), sched_words(L), &g_launches};
-        s = tc::forward(li, make_pp(L, L->epoch), tokens, L->cfg.m, (const T*)X, ldx, nullptr, 0, nullptr, 0, (T*)workspace, ldz,
-                        (int)ldz);
+        // P goes, for the duration of this product, where the backward will put its partials afterwards
+        if (g_family.load() == 0 && workspace_bytes - zbytes >= compact_fwd_workspace_bytes(L))
+          s = g2::g2_project(li, make_pp(L, L->epoch), tokens, (const T*)X, ldx, (T*)workspace, ldz, (int)ldz, (char*)workspace + zbytes);
+        if (s == COMPACT_ERR_SHAPE)
+          s = tc::forward(li, make_pp(L, L->epoch), tokens, L->cfg.m, (const T*)X, ldx, nullptr, 0, nullptr, 0, (T*)workspace, ldz,
+                          (int)ldz);
       }
       if (s == COMPACT_ERR_SHAPE)
         s = fwd_simt<T>(L, tokens, (const T*)X, ldx, nullptr, 0, nullptr, 0, (T*)workspace, ldz, st);

@@ -675,6 +675,32 @@ inline compact_status_t g2_forward(const LaunchInfo& li, int G, const G2Layer* L
   return g2_launch(li, prm);
 }
 
+// Z = X P alone (Algorithm 1 line 2, for the backward that recomputes it): P written out into `scratch`
+// (expanded_bytes(n, zcols)), then one product.
+inline compact_status_t g2_project(const LaunchInfo& li, const ProjectionParams& pp, int64_t tokens, const __nv_bfloat16* X,
+                                   int64_t ldx, __nv_bfloat16* Z, int64_t ldz, int zcols, void* scratch) {
+  const int n = pp.n;
+  if (!tc_shape_ok(tokens, n, 8)) return COMPACT_ERR_SHAPE;
+  if (!li.status) return COMPACT_ERR_CUDA;
+  __nv_bfloat16* P = (__nv_bfloat16*)scratch;
+  const compact_status_t s = expand_projection(li, pp, zcols, P);
+  if (s != COMPACT_OK) return s;
+  const int64_t ldp = expanded_ld(zcols);
+  G2Params prm;
+  memset(&prm, 0, sizeof(prm));
+  prm.num_problems = 1;
+  G2Problem& pz = prm.prob[0];
+  pz.M = (int)tokens; pz.N = zcols; pz.K = n;
+  pz.a_mode = TMA_KMAJOR; pz.b_mode = TMA_MNMAJOR; pz.epi_mode = EPI_BF16;
+  pz.b_blocked = 1;
+  pz.scale = pp.inv_sqrt_s;
+  g2_finish(pz, 1);
+  if (!make_map(&prm.tmA[0], X, n, tokens, ldx, BK, G2_HALF)) return COMPACT_ERR_CUDA;
+  if (!make_map_blocked(&prm.tmB[0], P, ldp, n, ldp, BK, G2_HALF / 64)) return COMPACT_ERR_CUDA;
+  if (!make_map(&prm.tmC[0], Z, zcols, tokens, ldz, 64, 32)) return COMPACT_ERR_CUDA;
+  return g2_launch(li, prm);
+}
+
 // Algorithm 3: Adam moments -> N (bf16, front of the scratch), P written out behind it, then W <- W - scale * P N as
 // one product on pairs of SMs whose epilogue adds the increment to W.  Same N, same entries of P, same order of accumulation and the same roundings as the
 // streaming update on single SMs (which needs no room for P and remains the route when the scratch is small).
