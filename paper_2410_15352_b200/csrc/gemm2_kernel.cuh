@@ -64,6 +64,10 @@ struct G2Problem {
   float scale;                 // bf16 epilogues: the accumulator is multiplied by this before it is rounded (1: exact)
 };
 
+#ifndef G2_PDL
+#define G2_PDL 1
+#endif
+
 struct alignas(64) G2Params {
   CUtensorMap tmA[G2_MAXP];
   CUtensorMap tmB[G2_MAXP];
@@ -75,6 +79,7 @@ struct alignas(64) G2Params {
                                // block by row block across its problems (tile_begin: a problem's first column tile in its run)
   int run_begin[G2_MAXP / 2 + 1];   // by_rows: first tile of each run
   int run_cols[G2_MAXP / 2];        // by_rows: column tiles of a run's problems together
+  int early;                   // host only: launch behind the previous kernel of the stream without waiting for its end
   unsigned int* status;
 };
 
@@ -222,6 +227,11 @@ __global__ void __launch_bounds__(G2_THREADS, 1) compact_gemm2_kernel(const __gr
   __syncthreads();
   tc_fence_after();
   cluster_sync_all();                     // both CTAs' barriers and TMEM exist before anything crosses
+#if G2_PDL
+  // Launched early (programmatic stream serialization) behind the small kernel that prepares an operand: everything
+  // above ran while that kernel was finishing; nothing below touches global memory before it has completed.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+#endif
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t leader_bars = map_to_cta(bars, 0u);
 
@@ -469,8 +479,17 @@ inline compact_status_t g2_launch(const LaunchInfo& li, G2Params& prm) {
   attr.val.clusterDim.x = 2;
   attr.val.clusterDim.y = 1;
   attr.val.clusterDim.z = 1;
-  cfg.attrs = &attr;
+  cudaLaunchAttribute attrs[2];
+  attrs[0] = attr;
+  cfg.attrs = attrs;
   cfg.numAttrs = 1;
+#if G2_PDL
+  if (prm.early) {
+    attrs[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attrs[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.numAttrs = 2;
+  }
+#endif
   const cudaError_t e = cudaLaunchKernelEx(&cfg, compact_gemm2_kernel, prm);
   (*li.launches)++;
   if (e != cudaSuccess) { cudaGetLastError(); return COMPACT_ERR_CUDA; }
@@ -566,6 +585,9 @@ __device__ __forceinline__ void expand_sparse_blocks(const ExpandArgs& a, int bl
 }
 
 __global__ void __launch_bounds__(256) expand_projection_kernel(const __grid_constant__ ExpandArgs a) {
+#if G2_PDL
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+#endif
   if (a.sparse_s > 0) expand_sparse_blocks(a, (int)blockIdx.x, (int)gridDim.x);
   else expand_gaussian_blocks(a, (int)blockIdx.x, (int)gridDim.x);
 }
@@ -577,6 +599,9 @@ __global__ void __launch_bounds__(256) adam_and_expand_kernel(const float* __res
                                                               float* __restrict__ Vo, __nv_bfloat16* __restrict__ Nout, int r, int m,
                                                               const __grid_constant__ simt::AdamScalars as, int adam_blocks,
                                                               const __grid_constant__ ExpandArgs a) {
+#if G2_PDL
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+#endif
   const int b = (int)blockIdx.x, expand_blocks = (int)gridDim.x - adam_blocks;
   const int paired = 2 * (adam_blocks < expand_blocks ? adam_blocks : expand_blocks);
   bool is_adam;
@@ -672,6 +697,7 @@ inline compact_status_t g2_forward(const LaunchInfo& li, int G, const G2Layer* L
     largest = b > largest ? b : largest;
   }
   prm.by_rows = all <= fits ? 2 * G : (largest <= fits ? 2 : 0);
+  prm.early = 1;
   return g2_launch(li, prm);
 }
 
@@ -736,6 +762,7 @@ inline compact_status_t g2_update(const LaunchInfo& li, const ProjectionParams& 
   if (pu.b_blocked ? !make_map_blocked(&prm.tmB[0], Nbuf, m, r, m, BK, G2_HALF / 64) : !make_map(&prm.tmB[0], Nbuf, m, r, m, 64, BK))
     return COMPACT_ERR_CUDA;
   if (!make_map(&prm.tmC[0], W, m, n, ldw, 64, 32)) return COMPACT_ERR_CUDA;
+  prm.early = 1;
   return g2_launch(li, prm);
 }
 
