@@ -258,14 +258,14 @@ class LayerBuffers:
 
 # DRAM traffic from the committed ncu captures (profiles/compact_gemm2_kernel_c5_*.md): dram__bytes_read.sum +
 # dram__bytes_write.sum of all launches of one forward call (expansion of P, product), one backward call (product,
-# reduction of the Gc partials) and one update call (Adam kernel, expansion, product) of the three distinct C5 shapes,
+# reduction of the Gc partials) and one update call (Adam + expansion, product) of the three distinct C5 shapes,
 # every launch from cold caches.  Other shapes are scaled from the q_proj figures by flops (forward, backward) and by
 # algorithmic bytes (update).  The update's reduce-adds leave W dirty in the L2: its write-back happens after the
 # kernel and is not in these figures.
 NCU_DRAM_BYTES_PER_CALL = {
-    (4096, 4096, 512): (397.0e6, 601.7e6, 67.2e6),
-    (4096, 11008, 512): (1370.9e6, 2577.6e6, 209.9e6),
-    (11008, 4096, 1376): (3122.4e6, 1666.6e6, 238.7e6),
+    (4096, 4096, 512): (399.6e6, 604.0e6, 67.2e6),
+    (4096, 11008, 512): (1367.5e6, 2629.5e6, 212.3e6),
+    (11008, 4096, 1376): (3038.0e6, 1683.9e6, 267.6e6),
 }
 
 
@@ -465,7 +465,7 @@ def run_ours(args):
         if ent["bound"] == "tensor":
             ent["frac_of_measured_bf16_sustained"] = ent["TFLOP/s"] / tens_peak
         upd_layers[f"{L.name}#{i}"] = ent
-    roofline_update = {"kernel": "update calls (adam_moments_bf16_kernel, expand_projection_kernel, compact_gemm2_kernel with W -= lr alpha P N in its epilogue)", "bound": "hbm",
+    roofline_update = {"kernel": "update calls (adam_and_expand_kernel, compact_gemm2_kernel with W -= lr alpha P N in its epilogue)", "bound": "hbm",
                        "achieved": upd_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": upd_gbs / hbm_peak,
                        "peak_kind": f"{peak_kind} copy", "frac_of_nominal_8000": upd_gbs / NOMINAL_HBM_GBS,
                        "avg_launch_ms": upd_ms / len(wl.layers), "algorithmic_bytes_per_launch": upd_bytes / len(wl.layers),
