@@ -13,7 +13,7 @@ from paper_2410_15352_b200 import binding as cb
 from paper_2410_15352_b200 import workloads as wlm
 from paper_2410_15352_b200.build import build_library
 
-from _harness import TOL, make_pair, to64, worst_tile
+from tests._harness import TOL, make_pair, to64, worst_tile
 
 pytestmark = pytest.mark.gpu
 
@@ -62,6 +62,15 @@ def test_with_and_without_scratch_same_bits_and_oracle(tokens, n, m, r, s):
     for a, b in ((Y1, Yo), (Z1[:, :r], Zo)):
         assert co.rel_frobenius(to64(a), b) <= TOL["bf16"]
         assert worst_tile(to64(a), b) <= TOL["bf16"]
+
+
+def test_empty_batch_with_scratch_launches_nothing():
+    lay = cb.CompactLinear(256, 136, 40)
+    W = torch.zeros((256, 136), dtype=torch.bfloat16, device="cuda")
+    X = torch.zeros((0, 256), dtype=torch.bfloat16, device="cuda")
+    before = cb.kernel_launch_count()
+    Y, Z, ep = lay.forward(X, W)
+    assert cb.kernel_launch_count() == before and Y.shape == (0, 136) and Z.shape == (0, lay.ldz) and ep == 0
 
 
 def test_scratch_holds_the_projection_the_debug_kernel_writes():

@@ -357,6 +357,8 @@ def test_repeated_launches_bitwise_stable(tokens, n, m, r):
 @pytest.mark.parametrize("tokens,n,shapes", [
     (1100, 320, [(512, 72), (520, 72), (1096, 40)]),      # segment lengths 512, 520 (ragged k-step), 1096
     (700, 4096, [(11008, 512), (11008, 512)]),            # gate/up of LLaMA-7B: operands beyond the L2, column panels
+    (700, 4096, [(4096, 512), (4096, 512), (4096, 512)]), # q/k/v of LLaMA-7B: the forward numbers each layer's Z and Y
+                                                          # tiles by rows, layer after layer
     (300, 192, [(200, 24)]),
 ])
 def test_group_calls_on_pairs_of_sms_and_on_single_sms_same_bits(tokens, n, shapes):
