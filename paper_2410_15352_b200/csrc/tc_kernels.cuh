@@ -6,6 +6,9 @@
 //   forward  : [Y | Z] = X [W | P]        (Algorithm 1; Z computed as Z^T = P^T X^T, P tiles generated as A)
 //   backward : dX = dY W^T and Gc = Z^T dY (Algorithm 2; Gc split over tokens)
 //   update   : W <- W - eta alpha P N      (Algorithm 3 lines 6-9; P tiles generated as A)
+// These are the products with P generated on chip: the route of calls that bring no scratch for P, of the
+// cross-check family, and the home of the helpers (barriers, TMA, descriptors, tensor maps) that the pair-of-SMs
+// kernel in gemm2_kernel.cuh shares.  Calls with scratch write P out once and run every product there.
 // Launches with a generated operand run as clusters of two CTAs that share every generated tile.
 // Work items are numbered longest first; those with a generated operand are dealt statically to the
 // clusters, the rest come from one atomic counter per launch.
